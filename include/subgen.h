@@ -1,0 +1,188 @@
+/*
+ * subgen.h - C ABI of the B200 (sm_100a) SubGen streaming-attention library.
+ *
+ * The library keeps, per (sequence, KV head) unit, the sublinear cache of "SubGen: Token
+ * Generation in Sublinear Time and Memory" (Algorithm 1):
+ *   D  - online threshold clustering of the keys: per cluster a representative (its first key),
+ *        a member count and t uniformly sampled member keys (procedure UpdateSoftmaxNormalizer,
+ *        Section 2.3, Lemma 2),
+ *   M  - s (key, value) pairs sampled with probability proportional to ||v||^2, and the running
+ *        mu = sum ||v||^2 (procedure UpdateMatrixProduct, Section 2.2, Lemma 1),
+ *   a ring buffer with the most recent `window` tokens kept verbatim (the sliding window of
+ *        Section 3.2),
+ * and answers every stream step with the estimator z / tau of procedure QueryStreamAttn.
+ *
+ * Conventions
+ *  - "device" pointers are CUDA device pointers owned by the caller; they must stay valid until
+ *    the handle's stream has executed the call. "host" pointers are ordinary host memory.
+ *  - Tensors are dense row-major; element type is the handle's dtype (fp32 or bf16), also for
+ *    outputs.
+ *  - Calls are asynchronous on the handle's stream unless stated otherwise. One handle is used by
+ *    one host thread at a time.
+ *  - Return value: 0 (SUBGEN_OK) or a negative SUBGEN_E* code for a host-side error;
+ *    subgen_last_error() then gives a text. Problems found on the device (cluster capacity
+ *    exhausted, non-finite or out-of-range input) never trap: they set sticky per-unit status
+ *    bits, the unit's output becomes NaN, and subgen_status() reports the OR of all bits.
+ *  - There is no CPU fallback. Every entry point fails if no CUDA device is usable.
+ *
+ * Arithmetic that decides an integer (which cluster a key joins, whether it opens one, every
+ * sampling coin) is done in order-independent integer arithmetic so that the result is unique:
+ *   D2(x,k) = sum_j floor(fl32(fl32(x_j-k_j)^2) * 2^32),  join <=> D2 <= floor(delta^2 * 2^32)
+ *   W(v)    = sum_j floor(fl32(v_j*v_j) * 2^24),           mu = sum of W
+ *   cluster coin (prob 1/n):      u * n        < 2^32
+ *   value coin  (prob W/(mu+W)):  u * (mu + W) < W * 2^32
+ * with u a 32-bit word of Philox4x32-10, key = seed, counter = (token index, unit index,
+ * slot / 4, domain), word = slot % 4, domain 0 = cluster slots, 1 = value slots, unit index =
+ * seq * Hkv + kvhead. Inputs must be finite with |x| <= 32768.
+ */
+#ifndef SUBGEN_H_
+#define SUBGEN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SUBGEN_OK 0
+#define SUBGEN_EINVAL (-1)  /* bad argument */
+#define SUBGEN_ENOMEM (-2)  /* allocation failed or workspace too small */
+#define SUBGEN_ESTATE (-3)  /* call not valid in the handle's state */
+#define SUBGEN_ECUDA (-4)   /* a CUDA runtime call failed */
+
+#define SUBGEN_DTYPE_FP32 0
+#define SUBGEN_DTYPE_BF16 1
+
+/* sticky per-unit status bits */
+#define SUBGEN_ST_CAPACITY 1 /* a key had to open a cluster but m_max clusters exist */
+#define SUBGEN_ST_RANGE 2    /* non-finite input, or |x| > 32768 */
+
+typedef struct subgen subgen_t;
+typedef struct subgen_exact subgen_exact_t;
+
+typedef struct subgen_config {
+    int B;          /* sequences */
+    int H;          /* query heads per sequence */
+    int Hkv;        /* KV heads per sequence; H % Hkv == 0, H / Hkv in {1,2,4,8}; 0 means Hkv = H */
+    int d;          /* head dimension: 64 or 128 */
+    float delta;    /* cluster radius (Algorithm 1 input delta), >= 0 */
+    int t;          /* key samples per cluster (Algorithm 1 input t), 1..64 */
+    int s;          /* value samples (Algorithm 1 input s), 1..65536 */
+    int window;     /* recent tokens kept verbatim (Section 3.2), >= 0 */
+    uint64_t seed;  /* Philox key */
+    int dtype;      /* SUBGEN_DTYPE_* */
+    int m_max;      /* cluster capacity per unit; 0 = 8192 */
+    int splits;     /* thread blocks that share one unit in the step kernels; 0 = chosen from B*Hkv */
+    void* workspace;        /* device, >= subgen_workspace_bytes(), 256-byte aligned, or NULL: the library allocates */
+    size_t workspace_bytes;
+    void* stream;           /* cudaStream_t, or NULL for the default stream */
+} subgen_config;
+
+/* Bytes of device memory a handle of this configuration needs (0 on invalid configuration). */
+size_t subgen_workspace_bytes(const subgen_config* cfg);
+
+/* Create a handle: bf16, Hkv = H, default capacity, library-owned memory, default stream.
+ * Parameter names follow Algorithm 1 (delta, t, s) and Section 3.2 (window). NULL on error. */
+subgen_t* subgen_create(int B, int H, int d, float delta, int t, int s, int window, uint64_t seed);
+subgen_t* subgen_create_ex(const subgen_config* cfg);
+void subgen_destroy(subgen_t* h);
+
+/* Append n tokens per sequence to every unit's stream WITHOUT producing outputs. The resulting
+ * state equals that of n update passes of the main loop of Algorithm 1 (UpdateSoftmaxNormalizer,
+ * UpdateMatrixProduct, mu update) applied token by token to the tokens that leave the window.
+ * K, V: device [B, Hkv, n, d]. May be called repeatedly. n = 0 is a no-op. */
+int subgen_prefill(subgen_t* h, const void* K, const void* V, int n);
+
+/* Same with one length per sequence. K, V: device [Hkv, total, d] with the sequences packed along
+ * the token axis; cu_seqlens: HOST array of B+1 non-decreasing offsets, cu_seqlens[0] = 0,
+ * cu_seqlens[B] = total. */
+int subgen_prefill_varlen(subgen_t* h, const void* K, const void* V, const int* cu_seqlens);
+
+/* One pass of the main loop of Algorithm 1 for every unit: the new token (k, v) enters the
+ * window, the token it pushes out is inserted into D and M (old mu in the coin, then mu grows),
+ * and the query q is answered from the updated state:
+ *   z   = sum_{(k,v) in M} mu/(s ||v||^2) exp<q,k> v  +  sum_{window} exp<q,k> v
+ *   tau = sum_{(x,S,n') in D} n'/t sum_{k in S} exp<q,k>  +  sum_{window} exp<q,k>
+ *   out = z / tau                       (no 1/sqrt(d): Eq. 1 has none)
+ * q, out: device [B, H, d]; k, v: device [B, Hkv, d]. Query head h uses KV head h / (H/Hkv). */
+int subgen_step(subgen_t* h, const void* q, const void* k, const void* v, void* out);
+
+/* subgen_step with HOST buffers: copies q, k, v to the device, runs the step, copies out back and
+ * waits for it. Pinned host memory makes the copies asynchronous to the host until the final wait. */
+int subgen_step_host(subgen_t* h, const void* q, const void* k, const void* v, void* out);
+
+/* Waits for the stream, returns the OR of all units' status bits (>= 0) or a negative error. */
+int subgen_status(subgen_t* h);
+
+typedef struct subgen_state_view {
+    int n;             /* tokens seen by this unit */
+    int inserted;      /* tokens that have left the window = tokens represented by D and M */
+    int m;             /* clusters */
+    int status;        /* SUBGEN_ST_* bits */
+    uint64_t mu;       /* fixed-point sum of W over inserted tokens */
+    int last_cluster;  /* cluster joined or opened by the most recent insertion, -1 if none yet */
+    int last_opened;   /* 1 if that insertion opened a cluster */
+    uint64_t last_d2;  /* its D2 to the nearest earlier representative, UINT64_MAX if there was none */
+    /* caller-allocated HOST arrays, any may be NULL */
+    int* counts;       /* [m_max]      n_i */
+    int* centre_tok;   /* [m_max]      token index of representative x_i */
+    int* slot_tok;     /* [m_max * t]  token index held by S_i(j) */
+    int* m_tok;        /* [s]          token index held by M(j), -1 = null */
+    uint64_t* m_w;     /* [s]          W of that token, 0 = null */
+} subgen_state_view;
+
+/* Synchronous copy of one unit's bookkeeping to the host (waits for the stream). */
+int subgen_export_state(subgen_t* h, int seq, int kvhead, subgen_state_view* view);
+
+/* Synchronous copy of one unit's stored vectors to the host. which: 0 representatives [m_max,d],
+ * 1 cluster samples [m_max,t,d] (rows of a cluster with n_i = 1 are not materialised: such a
+ * cluster's samples all equal its representative), 2 M keys [s,d], 3 M values [s,d],
+ * 4 window keys [window,d], 5 window values [window,d] (token j sits in row j % window). */
+int subgen_export_rows(subgen_t* h, int seq, int kvhead, int which, void* host, size_t bytes);
+
+typedef struct subgen_stats {
+    uint64_t units;
+    uint64_t clusters;           /* sum of m */
+    uint64_t singleton_clusters; /* clusters with n_i = 1 (read as one row, not t) */
+    uint64_t m_filled;           /* non-null M slots */
+    uint64_t window_rows;        /* tokens currently in the windows */
+    uint64_t tokens;             /* sum of n */
+    uint64_t insert_bytes;       /* bytes one step must read to place a key: the representatives */
+    uint64_t query_bytes;        /* bytes one step must read to answer the queries: samples, M, window */
+} subgen_stats;
+
+/* Synchronous. Sums over all units, from the current state. */
+int subgen_cache_stats(subgen_t* h, subgen_stats* out);
+
+/* Kernel timing with CUDA events on the handle's stream. While enabled every subgen_step records
+ * events around its two kernels; subgen_profile_read waits, adds up the elapsed times since the last
+ * read and resets. */
+int subgen_profile_enable(subgen_t* h, int on);
+int subgen_profile_read(subgen_t* h, double* insert_ms, double* query_ms, int* steps);
+
+/* Number of kernels this handle has launched so far. */
+uint64_t subgen_launch_count(const subgen_t* h);
+
+/* Text of the calling thread's most recent error. */
+const char* subgen_last_error(void);
+
+/* ---- exact dense decode attention over a full KV cache: the comparison point (Eq. 1) ---------- */
+
+/* Cache of up to n_max tokens per unit, K and V device [B*Hkv, n_max, d], owned by the library. */
+subgen_exact_t* subgen_exact_create(int B, int H, int Hkv, int d, int n_max, int dtype, void* stream);
+void subgen_exact_destroy(subgen_exact_t* h);
+/* Append n tokens per sequence; K, V device [B, Hkv, n, d]. */
+int subgen_exact_append(subgen_exact_t* h, const void* K, const void* V, int n);
+/* Packed variant, layout and cu_seqlens as subgen_prefill_varlen. */
+int subgen_exact_append_varlen(subgen_exact_t* h, const void* K, const void* V, const int* cu_seqlens);
+/* Append (k, v), then out = softmax(K q)^T V over all cached tokens. Shapes as subgen_step. */
+int subgen_exact_step(subgen_exact_t* h, const void* q, const void* k, const void* v, void* out);
+/* Bytes one exact step must read (all cached keys and values), from the current lengths. Synchronous. */
+int subgen_exact_bytes(subgen_exact_t* h, uint64_t* bytes);
+uint64_t subgen_exact_launch_count(const subgen_exact_t* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SUBGEN_H_ */

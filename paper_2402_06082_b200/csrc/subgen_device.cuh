@@ -1,0 +1,431 @@
+// Device-side building blocks of the SubGen kernels (sm_100a).
+//
+// Row geometry: every cached vector is one row of D elements (D*sizeof(T) = 128..512 bytes). A row is
+// read by LPR = D/EPL consecutive lanes with one 16-byte load each (EPL = elements per 16 bytes), so a
+// warp covers RPW = 32/LPR rows per load instruction ("row groups").
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace subgen {
+
+constexpr uint32_t kPhiloxM0 = 0xD2511F53u, kPhiloxM1 = 0xCD9E8D57u;
+constexpr uint32_t kPhiloxW0 = 0x9E3779B9u, kPhiloxW1 = 0xBB67AE85u;
+constexpr float kMaxAbsInput = 32768.0f;
+
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies, key bumped by the
+// Weyl constants between rounds.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(kPhiloxM0, c.x), lo0 = kPhiloxM0 * c.x;
+        const uint32_t hi1 = __umulhi(kPhiloxM1, c.z), lo1 = kPhiloxM1 * c.z;
+        c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+        k0 += kPhiloxW0;
+        k1 += kPhiloxW1;
+    }
+    return c;
+}
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int EPL = 4;
+    static __device__ __forceinline__ void unpack(const uint4& r, float* f) {
+        f[0] = __uint_as_float(r.x); f[1] = __uint_as_float(r.y);
+        f[2] = __uint_as_float(r.z); f[3] = __uint_as_float(r.w);
+    }
+    static __device__ __forceinline__ float to_out(float x) { return x; }
+};
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int EPL = 8;
+    // bf16 -> fp32 is a 16-bit shift of the pattern
+    static __device__ __forceinline__ void unpack(const uint4& r, float* f) {
+        f[0] = __uint_as_float(r.x << 16); f[1] = __uint_as_float(r.x & 0xffff0000u);
+        f[2] = __uint_as_float(r.y << 16); f[3] = __uint_as_float(r.y & 0xffff0000u);
+        f[4] = __uint_as_float(r.z << 16); f[5] = __uint_as_float(r.z & 0xffff0000u);
+        f[6] = __uint_as_float(r.w << 16); f[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+    static __device__ __forceinline__ __nv_bfloat16 to_out(float x) { return __float2bfloat16_rn(x); }
+};
+
+// Fixed-point terms: single binary32 operations, never contracted, truncated to integers.
+__device__ __forceinline__ uint64_t fx_sqdiff(float a, float b) {
+    const float df = __fsub_rn(a, b);
+    return __float2ull_rz(__fmul_rn(__fmul_rn(df, df), 4294967296.0f));
+}
+__device__ __forceinline__ uint64_t fx_sq(float a) {
+    return __float2ull_rz(__fmul_rn(__fmul_rn(a, a), 16777216.0f));
+}
+
+// Cluster coin: probability 1/n.
+__device__ __forceinline__ bool coin_cluster(uint32_t u, uint32_t n) {
+    return (uint64_t)u * (uint64_t)n < 4294967296ull;
+}
+// Value coin: u * tot < W * 2^32 in 128-bit integers, tot = mu_old + W.
+__device__ __forceinline__ bool coin_value(uint32_t u, uint64_t tot, uint64_t W) {
+    const uint64_t lhs_lo = (uint64_t)u * tot, lhs_hi = __umul64hi((uint64_t)u, tot);
+    const uint64_t rhs_lo = W << 32, rhs_hi = W >> 32;
+    return lhs_hi < rhs_hi || (lhs_hi == rhs_hi && lhs_lo < rhs_lo);
+}
+
+struct Best {          // (D2, index) ordered lexicographically: nearest, then lowest index
+    unsigned long long d2;
+    int idx;
+    int pad;
+};
+__device__ __forceinline__ bool better(unsigned long long d2, int idx, const Best& b) {
+    return d2 < b.d2 || (d2 == b.d2 && idx < b.idx);
+}
+
+// Pointers into the per-unit cache arrays (all device memory). Unit u = seq * Hkv + kvhead.
+template <typename T> struct Cache {
+    int B, H, Hkv, G, t, s, w, m_max;
+    unsigned long long delta2_fx;
+    uint32_t key0, key1;
+    T* X;            // [U, m_max, D]     representatives x_i
+    T* S;            // [U, m_max, t, D]  cluster samples S_i (materialised once n_i >= 2)
+    int* cnt;        // [U, m_max]        n_i
+    int* ctok;       // [U, m_max]        token index of x_i
+    int* stok;       // [U, m_max, t]     token index in S_i(j)
+    T* Mk;           // [U, s, D]
+    T* Mv;           // [U, s, D]
+    unsigned long long* MW;    // [U, s]  W of the sampled token, 0 = null
+    int* Mtok;       // [U, s]
+    T* ringK;        // [U, w, D]         token j in row j % w
+    T* ringV;
+    int* n_unit;     // [U] tokens seen
+    int* m_unit;     // [U] clusters
+    unsigned long long* mu;    // [U]
+    int* status;     // [U]
+    int* last_cid;   // [U]
+    int* last_open;  // [U]
+    unsigned long long* last_d2;   // [U]
+    // scratch of the step kernels
+    Best* part1;     // [U, splits]
+    float* part2;    // [U, splits, G, D + 2]
+    unsigned* ticket1;   // [U]
+    unsigned* ticket2;   // [U]
+};
+
+// ---------------------------------------------------------------------------------------------
+// Nearest representative: scan rows [c0, c1) of X_u with `ngroups` row groups, every group keeps its
+// best (D2, idx). kf = this lane's EPL elements of the key. All lanes of a warp must call together.
+template <typename T, int D>
+__device__ __forceinline__ void scan_centres(const T* Xu, int c0, int c1, const float* kf,
+                                             int group, int ngroups, int lr, Best& best) {
+    constexpr int EPL = Elem<T>::EPL, LPR = D / EPL;
+    constexpr int UN = 4;
+    for (int base = c0; base < c1; base += ngroups * UN) {
+        uint4 raw[UN];
+        int row[UN];
+#pragma unroll
+        for (int i = 0; i < UN; ++i) {
+            row[i] = base + i * ngroups + group;
+            raw[i] = make_uint4(0, 0, 0, 0);
+            if (row[i] < c1) raw[i] = *reinterpret_cast<const uint4*>(Xu + (size_t)row[i] * D + lr * EPL);
+        }
+#pragma unroll
+        for (int i = 0; i < UN; ++i) {
+            float xf[EPL];
+            Elem<T>::unpack(raw[i], xf);
+            unsigned long long acc = 0;
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) acc += fx_sqdiff(xf[j], kf[j]);
+#pragma unroll
+            for (int off = 1; off < LPR; off <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            if (row[i] < c1 && better(acc, row[i], best)) { best.d2 = acc; best.idx = row[i]; }
+        }
+    }
+}
+
+// Block-wide lexicographic minimum. sm: shared array of at least 32 Best. Result valid in all threads.
+__device__ __forceinline__ Best block_best(Best b, Best* sm) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const unsigned long long od = __shfl_xor_sync(0xffffffffu, b.d2, off);
+        const int oi = __shfl_xor_sync(0xffffffffu, b.idx, off);
+        if (better(od, oi, b)) { b.d2 = od; b.idx = oi; }
+    }
+    __syncthreads();
+    if (lane == 0) sm[warp] = b;
+    __syncthreads();
+    Best r = sm[0];
+    for (int i = 1; i < nw; ++i) if (better(sm[i].d2, sm[i].idx, r)) r = sm[i];
+    return r;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Insert token e (key/value rows already in shared memory) into D and M of unit u, given the nearest
+// representative. Executed by a whole block; ends with a __syncthreads(). Returns the new m.
+//   UpdateSoftmaxNormalizer: join (count, t coins) or open (representative, count 1; the t copies are
+//   implied while n_i = 1 and written out when the second member arrives);
+//   UpdateMatrixProduct: s coins with the OLD mu; then mu += W.
+template <typename T, int D>
+__device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, const uint4* krow, const uint4* vrow,
+                            unsigned long long* sm_w /* shared, 1 element */) {
+    constexpr int EPL = Elem<T>::EPL, LPR = D / EPL;
+    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5;
+    const int t = C.t, s = C.s;
+
+    // W(v_e) and the input range check, by warp 0
+    if (warp == 0) {
+        unsigned long long acc = 0;
+        bool bad = false;
+        for (int p = lane; p < LPR; p += 32) {
+            float vf[EPL], kf[EPL];
+            Elem<T>::unpack(vrow[p], vf);
+            Elem<T>::unpack(krow[p], kf);
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) {
+                acc += fx_sq(vf[j]);
+                bad |= !(fabsf(vf[j]) <= kMaxAbsInput) || !(fabsf(kf[j]) <= kMaxAbsInput);
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        bad = __any_sync(0xffffffffu, bad);
+        if (lane == 0) {
+            *sm_w = acc;
+            if (bad) atomicOr(&C.status[u], 2);
+        }
+    }
+    __syncthreads();
+    const unsigned long long W = *sm_w;
+    const unsigned long long mu_old = C.mu[u];
+
+    const bool join = (m > 0) && (best.d2 <= C.delta2_fx);
+    const bool full = !join && (m >= C.m_max);
+    T* Xu = C.X + (size_t)u * C.m_max * D;
+    T* Su = C.S + (size_t)u * C.m_max * t * D;
+    int* cntu = C.cnt + (size_t)u * C.m_max;
+    int* stoku = C.stok + (size_t)u * C.m_max * t;
+    int m_new = m;
+    if (join) {
+        const int c = best.idx;
+        const int n_old = cntu[c];
+        const uint32_t n_new = (uint32_t)n_old + 1u;
+        // slot j is written by LPR threads, one 16-byte piece each
+        for (int p = tid; p < t * LPR; p += nt) {
+            const int j = p / LPR, part = p % LPR;
+            const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)(j >> 2), 0u), C.key0, C.key1);
+            const uint32_t word = (j & 3) == 0 ? r.x : (j & 3) == 1 ? r.y : (j & 3) == 2 ? r.z : r.w;
+            uint4* dst = reinterpret_cast<uint4*>(Su + ((size_t)c * t + j) * D) + part;
+            if (coin_cluster(word, n_new)) {
+                *dst = krow[part];
+                if (part == 0) stoku[(size_t)c * t + j] = e;
+            } else if (n_old == 1) {
+                *dst = reinterpret_cast<const uint4*>(Xu + (size_t)c * D)[part];   // write out the implied copy
+            }
+        }
+        __syncthreads();            // n_old was read by everyone before it changes
+        if (tid == 0) cntu[c] = (int)n_new;
+    } else if (!full) {
+        const int c = m;
+        if (tid < LPR) reinterpret_cast<uint4*>(Xu + (size_t)c * D)[tid] = krow[tid];
+        for (int j = tid; j < t; j += nt) stoku[(size_t)c * t + j] = e;
+        if (tid == 0) { cntu[c] = 1; C.ctok[(size_t)u * C.m_max + c] = e; }
+        m_new = m + 1;
+    } else if (tid == 0) {
+        atomicOr(&C.status[u], 1);
+    }
+
+    // UpdateMatrixProduct: slot i flips its own coin; winners copy (k_e, v_e)
+    if (W > 0) {
+        const unsigned long long tot = mu_old + W;
+        T* Mku = C.Mk + (size_t)u * s * D;
+        T* Mvu = C.Mv + (size_t)u * s * D;
+        for (int blk = tid; blk * 4 < s; blk += nt) {
+            const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)blk, 1u), C.key0, C.key1);
+            const uint32_t words[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int i = blk * 4 + q;
+                if (i < s && coin_value(words[q], tot, W)) {
+                    uint4* dk = reinterpret_cast<uint4*>(Mku + (size_t)i * D);
+                    uint4* dv = reinterpret_cast<uint4*>(Mvu + (size_t)i * D);
+                    for (int p = 0; p < LPR; ++p) { dk[p] = krow[p]; dv[p] = vrow[p]; }
+                    C.MW[(size_t)u * s + i] = W;
+                    C.Mtok[(size_t)u * s + i] = e;
+                }
+            }
+        }
+    }
+    __syncthreads();                // every thread has read mu_old
+    if (tid == 0) {
+        C.mu[u] = mu_old + W;
+        C.m_unit[u] = m_new;
+        C.last_cid[u] = join ? best.idx : (full ? -1 : m);
+        C.last_open[u] = join ? 0 : 1;
+        C.last_d2[u] = best.d2;
+    }
+    __syncthreads();
+    return m_new;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Online-softmax accumulators of one row group for G query heads. The d components of z are spread
+// over the group's LPR lanes, EPL each; mx and tau are replicated in the group's lanes.
+template <int G, int EPL> struct Acc {
+    float mx[G], tau[G], z[G][EPL];
+    __device__ __forceinline__ void init() {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            mx[g] = -INFINITY; tau[g] = 0.f;
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) z[g][j] = 0.f;
+        }
+    }
+};
+
+// Scores of UN rows for G heads: dot products reduced over the LPR lanes of the row group.
+template <typename T, int D, int G, int UN>
+__device__ __forceinline__ void scores(const uint4 (&kraw)[UN], const float (&qf)[G][Elem<T>::EPL], float (&sc)[UN][G]) {
+    constexpr int EPL = Elem<T>::EPL, LPR = D / EPL;
+#pragma unroll
+    for (int i = 0; i < UN; ++i) {
+        float kf[EPL];
+        Elem<T>::unpack(kraw[i], kf);
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            float a = 0.f;
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) a = fmaf(qf[g][j], kf[j], a);
+            sc[i][g] = a;
+        }
+    }
+#pragma unroll
+    for (int off = 1; off < LPR; off <<= 1)
+#pragma unroll
+        for (int i = 0; i < UN; ++i)
+#pragma unroll
+            for (int g = 0; g < G; ++g) sc[i][g] += __shfl_xor_sync(0xffffffffu, sc[i][g], off);
+}
+
+// Fold UN scored rows into the accumulators. wt_tau / wt_z: the estimator weights of each row
+// (n'/t and 0 for a cluster sample; 0 and mu/(s W) for a value sample; 1 and 1 for a window token).
+template <typename T, int D, int G, int UN, bool HASV>
+__device__ __forceinline__ void fold(Acc<G, Elem<T>::EPL>& A, const float (&sc)[UN][G], const bool (&valid)[UN],
+                                     const float (&wt_tau)[UN], const float (&wt_z)[UN], const uint4 (&vraw)[UN]) {
+    constexpr int EPL = Elem<T>::EPL;
+    bool any = false;
+#pragma unroll
+    for (int i = 0; i < UN; ++i) any |= valid[i];
+    if (!any) return;
+    float p[UN][G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        float mnew = A.mx[g];
+#pragma unroll
+        for (int i = 0; i < UN; ++i) if (valid[i]) mnew = fmaxf(mnew, sc[i][g]);
+        const float scale = __expf(A.mx[g] - mnew);     // exp(-inf) = 0 on the first rows
+        A.mx[g] = mnew;
+        float tau = A.tau[g] * scale;
+#pragma unroll
+        for (int i = 0; i < UN; ++i) {
+            p[i][g] = valid[i] ? __expf(sc[i][g] - mnew) : 0.f;
+            tau = fmaf(wt_tau[i], p[i][g], tau);
+        }
+        A.tau[g] = tau;
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) A.z[g][j] *= scale;
+    }
+    if (HASV) {
+#pragma unroll
+        for (int i = 0; i < UN; ++i) {
+            float vf[EPL];
+            Elem<T>::unpack(vraw[i], vf);
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const float c = wt_z[i] * p[i][g];
+#pragma unroll
+                for (int j = 0; j < EPL; ++j) A.z[g][j] = fmaf(c, vf[j], A.z[g][j]);
+            }
+        }
+    }
+}
+
+// Merge two accumulator states (mx, tau) -> first; sa, sb are the factors for the two z vectors.
+__device__ __forceinline__ void merge_scalar(float& mx, float& tau, float omx, float otau, float& sa, float& sb) {
+    const float m = fmaxf(mx, omx);
+    sa = (mx == -INFINITY) ? 0.f : __expf(mx - m);
+    sb = (omx == -INFINITY) ? 0.f : __expf(omx - m);
+    tau = tau * sa + otau * sb;
+    mx = m;
+}
+
+// Block-level reduction of the row groups' accumulators and store of the block's partial
+// [G][D+2] = {mx, tau, z[D]} to dst. sm: shared floats, at least (blockDim/32) * G * (D+2).
+template <typename T, int D, int G>
+__device__ __forceinline__ void block_partial(Acc<G, Elem<T>::EPL>& A, float* sm, float* dst) {
+    constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, STR = D + 2;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5, lr = lane % LPR;
+#pragma unroll
+    for (int off = LPR; off < 32; off <<= 1) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const float omx = __shfl_xor_sync(0xffffffffu, A.mx[g], off);
+            const float otau = __shfl_xor_sync(0xffffffffu, A.tau[g], off);
+            float sa, sb;
+            merge_scalar(A.mx[g], A.tau[g], omx, otau, sa, sb);
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) {
+                const float oz = __shfl_xor_sync(0xffffffffu, A.z[g][j], off);
+                A.z[g][j] = A.z[g][j] * sa + oz * sb;
+            }
+        }
+    }
+    if (lane < LPR) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            float* w = sm + ((size_t)warp * G + g) * STR;
+            if (lr == 0) { w[0] = A.mx[g]; w[1] = A.tau[g]; }
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) w[2 + lr * EPL + j] = A.z[g][j];
+        }
+    }
+    __syncthreads();
+    for (int o = tid; o < G * STR; o += blockDim.x) {
+        const int g = o / STR, c = o % STR;
+        float m = -INFINITY;
+        for (int w = 0; w < nw; ++w) m = fmaxf(m, sm[((size_t)w * G + g) * STR]);
+        float r;
+        if (c == 0) r = m;
+        else {
+            r = 0.f;
+            for (int w = 0; w < nw; ++w) {
+                const float wm = sm[((size_t)w * G + g) * STR];
+                if (wm != -INFINITY) r += sm[((size_t)w * G + g) * STR + c] * __expf(wm - m);
+            }
+        }
+        dst[(size_t)g * STR + c] = r;
+    }
+}
+
+// Final merge of `np` block partials and the division z / tau, by a whole block.
+// part: [np][G][D+2]; out rows: out + g * D for g < G. poisoned -> NaN.
+template <typename T, int D, int G>
+__device__ __forceinline__ void final_merge(const float* part, int np, T* out, bool poisoned) {
+    constexpr int STR = D + 2;
+    for (int o = threadIdx.x; o < G * D; o += blockDim.x) {
+        const int g = o / D, c = o % D;
+        float m = -INFINITY;
+        for (int i = 0; i < np; ++i) m = fmaxf(m, __ldcg(part + ((size_t)i * G + g) * STR));
+        float z = 0.f, tau = 0.f;
+        for (int i = 0; i < np; ++i) {
+            const float* pp = part + ((size_t)i * G + g) * STR;
+            const float pm = __ldcg(pp);
+            if (pm != -INFINITY) {
+                const float sc = __expf(pm - m);
+                tau += __ldcg(pp + 1) * sc;
+                z += __ldcg(pp + 2 + c) * sc;
+            }
+        }
+        float r = tau > 0.f ? z / tau : 0.f;
+        if (poisoned) r = __int_as_float(0x7fc00000);
+        out[(size_t)g * D + c] = Elem<T>::to_out(r);
+    }
+}
+
+}  // namespace subgen
