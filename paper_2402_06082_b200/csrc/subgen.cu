@@ -1,0 +1,629 @@
+// Host side of the SubGen library: handles, memory layout, launches, C ABI (see include/subgen.h).
+#include "../../include/subgen.h"
+
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "subgen_kernels.cuh"
+
+using namespace sgk;
+
+namespace {
+
+thread_local std::string g_err;
+
+int fail(int code, const char* fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_err = buf;
+    return code;
+}
+
+#define CUDA_TRY(expr)                                                                      \
+    do {                                                                                    \
+        cudaError_t err__ = (expr);                                                         \
+        if (err__ != cudaSuccess) return fail(SUBGEN_ECUDA, "%s: %s", #expr, cudaGetErrorString(err__)); \
+    } while (0)
+
+constexpr size_t kAlign = 256;
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Layout {
+    size_t X, S, cnt, ctok, stok, Mk, Mv, MW, Mtok, ringK, ringV;
+    size_t n_unit, m_unit, mu, status, last_cid, last_open, last_d2, part1, part2, ticket1, ticket2;
+    size_t stage_q, stage_k, stage_v, stage_out, cu, stats;
+    size_t book_begin, book_end;   // bookkeeping region cleared at creation
+    size_t total;
+};
+
+struct Dims {
+    int B, H, Hkv, G, D, t, s, w, m_max, splits, U;
+    size_t E;   // bytes per element
+};
+
+bool resolve(const subgen_config* c, Dims* o, const char** why) {
+    if (!c) { *why = "config is NULL"; return false; }
+    Dims d;
+    d.B = c->B; d.H = c->H; d.Hkv = c->Hkv ? c->Hkv : c->H; d.D = c->d; d.t = c->t; d.s = c->s; d.w = c->window;
+    d.m_max = c->m_max ? c->m_max : 8192;
+    if (d.B <= 0 || d.H <= 0 || d.Hkv <= 0) { *why = "B, H, Hkv must be positive"; return false; }
+    if (d.H % d.Hkv) { *why = "H must be a multiple of Hkv"; return false; }
+    d.G = d.H / d.Hkv;
+    if (d.G != 1 && d.G != 2 && d.G != 4 && d.G != 8) { *why = "H / Hkv must be 1, 2, 4 or 8"; return false; }
+    if (d.D != 64 && d.D != 128) { *why = "d must be 64 or 128"; return false; }
+    if (d.t < 1 || d.t > 64) { *why = "t must be in 1..64"; return false; }
+    if (d.s < 1 || d.s > 65536) { *why = "s must be in 1..65536"; return false; }
+    if (d.w < 0) { *why = "window must be >= 0"; return false; }
+    if (d.m_max < 1) { *why = "m_max must be positive"; return false; }
+    if (!(c->delta >= 0.f) || !isfinite(c->delta) || c->delta > 32768.f) { *why = "delta must be finite, in [0, 32768]"; return false; }
+    if (c->dtype != SUBGEN_DTYPE_FP32 && c->dtype != SUBGEN_DTYPE_BF16) { *why = "unknown dtype"; return false; }
+    if ((long long)d.B * d.Hkv > 65535) { *why = "B * Hkv must be <= 65535"; return false; }
+    d.E = c->dtype == SUBGEN_DTYPE_FP32 ? 4 : 2;
+    d.U = d.B * d.Hkv;
+    if (c->splits < 0 || c->splits > 128) { *why = "splits must be in 0..128"; return false; }
+    if (c->splits) d.splits = c->splits;
+    else {
+        int sp = (148 * 8 + d.U - 1) / d.U;     // about eight resident blocks per SM over all units
+        d.splits = sp < 1 ? 1 : (sp > 32 ? 32 : sp);
+    }
+    *o = d;
+    return true;
+}
+
+Layout make_layout(const Dims& d) {
+    Layout L;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    const size_t U = d.U, row = (size_t)d.D * d.E;
+    L.X = take(U * d.m_max * row);
+    L.S = take(U * d.m_max * d.t * row);
+    L.Mk = take(U * d.s * row);
+    L.Mv = take(U * d.s * row);
+    L.ringK = take(U * (size_t)d.w * row);
+    L.ringV = take(U * (size_t)d.w * row);
+    L.stage_q = take((size_t)d.B * d.H * row);
+    L.stage_k = take(U * row);
+    L.stage_v = take(U * row);
+    L.stage_out = take((size_t)d.B * d.H * row);
+    L.cu = take(((size_t)d.B + 1) * sizeof(int));
+    L.part1 = take(U * d.splits * sizeof(Best));
+    L.part2 = take(U * d.splits * d.G * (size_t)(d.D + 2) * sizeof(float));
+    L.book_begin = off;
+    L.cnt = take(U * d.m_max * sizeof(int));
+    L.n_unit = take(U * sizeof(int));
+    L.m_unit = take(U * sizeof(int));
+    L.mu = take(U * sizeof(uint64_t));
+    L.status = take(U * sizeof(int));
+    L.last_open = take(U * sizeof(int));
+    L.ticket1 = take(U * sizeof(unsigned));
+    L.ticket2 = take(U * sizeof(unsigned));
+    L.MW = take(U * d.s * sizeof(uint64_t));
+    L.stats = take(8 * sizeof(uint64_t));
+    L.book_end = off;
+    // regions initialised to all-ones (-1 / UINT64_MAX)
+    L.ctok = take(U * d.m_max * sizeof(int));
+    L.stok = take(U * d.m_max * d.t * sizeof(int));
+    L.Mtok = take(U * d.s * sizeof(int));
+    L.last_cid = take(U * sizeof(int));
+    L.last_d2 = take(U * sizeof(uint64_t));
+    L.total = off;
+    return L;
+}
+
+}  // namespace
+
+struct subgen {
+    subgen_config cfg;
+    Dims d;
+    Layout L;
+    char* ws = nullptr;
+    bool owns = false;
+    cudaStream_t st = nullptr;
+    std::vector<int> n_host;     // tokens seen per sequence (mirror of the device counters)
+    uint64_t launches = 0;
+    bool prof = false;
+    std::vector<cudaEvent_t> ev;  // three per profiled step
+    size_t ev_used = 0;
+};
+
+namespace {
+
+template <typename T> Cache<T> make_cache(const subgen* h) {
+    const Dims& d = h->d;
+    const Layout& L = h->L;
+    char* w = h->ws;
+    Cache<T> C;
+    C.B = d.B; C.H = d.H; C.Hkv = d.Hkv; C.G = d.G; C.t = d.t; C.s = d.s; C.w = d.w; C.m_max = d.m_max;
+    C.delta2_fx = (unsigned long long)floor((double)h->cfg.delta * (double)h->cfg.delta * 4294967296.0);
+    C.key0 = (uint32_t)h->cfg.seed; C.key1 = (uint32_t)(h->cfg.seed >> 32);
+    C.X = (T*)(w + L.X); C.S = (T*)(w + L.S);
+    C.cnt = (int*)(w + L.cnt); C.ctok = (int*)(w + L.ctok); C.stok = (int*)(w + L.stok);
+    C.Mk = (T*)(w + L.Mk); C.Mv = (T*)(w + L.Mv);
+    C.MW = (unsigned long long*)(w + L.MW); C.Mtok = (int*)(w + L.Mtok);
+    C.ringK = (T*)(w + L.ringK); C.ringV = (T*)(w + L.ringV);
+    C.n_unit = (int*)(w + L.n_unit); C.m_unit = (int*)(w + L.m_unit);
+    C.mu = (unsigned long long*)(w + L.mu); C.status = (int*)(w + L.status);
+    C.last_cid = (int*)(w + L.last_cid); C.last_open = (int*)(w + L.last_open);
+    C.last_d2 = (unsigned long long*)(w + L.last_d2);
+    C.part1 = (Best*)(w + L.part1); C.part2 = (float*)(w + L.part2);
+    C.ticket1 = (unsigned*)(w + L.ticket1); C.ticket2 = (unsigned*)(w + L.ticket2);
+    return C;
+}
+
+template <typename T, int D>
+int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void* out) {
+    Cache<T> C = make_cache<T>(h);
+    const dim3 grid(h->d.splits, h->d.U);
+    cudaEvent_t* e = nullptr;
+    if (h->prof) {
+        if (h->ev_used + 3 > h->ev.size()) {
+            for (int i = 0; i < 3; ++i) {
+                cudaEvent_t x;
+                CUDA_TRY(cudaEventCreate(&x));
+                h->ev.push_back(x);
+            }
+        }
+        e = &h->ev[h->ev_used];
+        h->ev_used += 3;
+        CUDA_TRY(cudaEventRecord(e[0], h->st));
+    }
+    insert_kernel<T, D><<<grid, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
+    if (e) CUDA_TRY(cudaEventRecord(e[1], h->st));
+    switch (h->d.G) {
+        case 1: query_kernel<T, D, 1><<<grid, kQueryThreads, 0, h->st>>>(C, (const T*)q, (T*)out); break;
+        case 2: query_kernel<T, D, 2><<<grid, kQueryThreads, 0, h->st>>>(C, (const T*)q, (T*)out); break;
+        case 4: query_kernel<T, D, 4><<<grid, kQueryThreads, 0, h->st>>>(C, (const T*)q, (T*)out); break;
+        default: query_kernel<T, D, 8><<<grid, kQueryThreads, 0, h->st>>>(C, (const T*)q, (T*)out); break;
+    }
+    if (e) CUDA_TRY(cudaEventRecord(e[2], h->st));
+    CUDA_TRY(cudaGetLastError());
+    h->launches += 2;
+    return SUBGEN_OK;
+}
+
+int launch_step(subgen* h, const void* q, const void* k, const void* v, void* out) {
+    const bool f32 = h->cfg.dtype == SUBGEN_DTYPE_FP32;
+    if (h->d.D == 64) return f32 ? launch_step_td<float, 64>(h, q, k, v, out) : launch_step_td<__nv_bfloat16, 64>(h, q, k, v, out);
+    return f32 ? launch_step_td<float, 128>(h, q, k, v, out) : launch_step_td<__nv_bfloat16, 128>(h, q, k, v, out);
+}
+
+template <typename T, int D>
+int launch_prefill_td(subgen* h, const void* K, const void* V, int n, const int* cu_dev, int total) {
+    Cache<T> C = make_cache<T>(h);
+    prefill_seq_kernel<T, D><<<h->d.U, kPrefillThreads, 0, h->st>>>(C, (const T*)K, (const T*)V, n, cu_dev, total);
+    CUDA_TRY(cudaGetLastError());
+    h->launches += 1;
+    return SUBGEN_OK;
+}
+
+int launch_prefill(subgen* h, const void* K, const void* V, int n, const int* cu_dev, int total) {
+    const bool f32 = h->cfg.dtype == SUBGEN_DTYPE_FP32;
+    if (h->d.D == 64)
+        return f32 ? launch_prefill_td<float, 64>(h, K, V, n, cu_dev, total)
+                   : launch_prefill_td<__nv_bfloat16, 64>(h, K, V, n, cu_dev, total);
+    return f32 ? launch_prefill_td<float, 128>(h, K, V, n, cu_dev, total)
+               : launch_prefill_td<__nv_bfloat16, 128>(h, K, V, n, cu_dev, total);
+}
+
+int check_device() {
+    int n = 0;
+    cudaError_t e = cudaGetDeviceCount(&n);
+    if (e != cudaSuccess || n <= 0)
+        return fail(SUBGEN_ECUDA, "no usable CUDA device (%s); this library has no CPU path",
+                    e != cudaSuccess ? cudaGetErrorString(e) : "device count is 0");
+    return SUBGEN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* subgen_last_error(void) { return g_err.c_str(); }
+
+size_t subgen_workspace_bytes(const subgen_config* cfg) {
+    Dims d;
+    const char* why = "";
+    if (!resolve(cfg, &d, &why)) { fail(SUBGEN_EINVAL, "subgen_workspace_bytes: %s", why); return 0; }
+    return make_layout(d).total;
+}
+
+subgen_t* subgen_create_ex(const subgen_config* cfg) {
+    Dims d;
+    const char* why = "";
+    if (!resolve(cfg, &d, &why)) { fail(SUBGEN_EINVAL, "subgen_create: %s", why); return nullptr; }
+    if (check_device() != SUBGEN_OK) return nullptr;
+    subgen* h = new subgen();
+    h->cfg = *cfg;
+    h->d = d;
+    h->L = make_layout(d);
+    h->st = (cudaStream_t)cfg->stream;
+    if (cfg->workspace) {
+        if (cfg->workspace_bytes < h->L.total || ((uintptr_t)cfg->workspace % kAlign)) {
+            fail(SUBGEN_ENOMEM, "subgen_create: workspace needs %zu bytes, 256-byte aligned (got %zu)", h->L.total,
+                 cfg->workspace_bytes);
+            delete h;
+            return nullptr;
+        }
+        h->ws = (char*)cfg->workspace;
+    } else {
+        cudaError_t e = cudaMalloc((void**)&h->ws, h->L.total);
+        if (e != cudaSuccess) {
+            fail(SUBGEN_ENOMEM, "subgen_create: cudaMalloc(%zu) failed: %s", h->L.total, cudaGetErrorString(e));
+            delete h;
+            return nullptr;
+        }
+        h->owns = true;
+    }
+    cudaError_t e1 = cudaMemsetAsync(h->ws + h->L.book_begin, 0, h->L.book_end - h->L.book_begin, h->st);
+    cudaError_t e2 = cudaMemsetAsync(h->ws + h->L.book_end, 0xFF, h->L.total - h->L.book_end, h->st);
+    if (e1 != cudaSuccess || e2 != cudaSuccess) {
+        fail(SUBGEN_ECUDA, "subgen_create: cudaMemsetAsync failed: %s", cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
+        if (h->owns) cudaFree(h->ws);
+        delete h;
+        return nullptr;
+    }
+    h->n_host.assign(d.B, 0);
+    return h;
+}
+
+subgen_t* subgen_create(int B, int H, int d, float delta, int t, int s, int window, uint64_t seed) {
+    subgen_config c;
+    memset(&c, 0, sizeof c);
+    c.B = B; c.H = H; c.Hkv = H; c.d = d; c.delta = delta; c.t = t; c.s = s; c.window = window; c.seed = seed;
+    c.dtype = SUBGEN_DTYPE_BF16;
+    return subgen_create_ex(&c);
+}
+
+void subgen_destroy(subgen_t* h) {
+    if (!h) return;
+    cudaStreamSynchronize(h->st);
+    for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
+    if (h->owns) cudaFree(h->ws);
+    delete h;
+}
+
+int subgen_prefill(subgen_t* h, const void* K, const void* V, int n) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_prefill: handle is NULL");
+    if (n < 0) return fail(SUBGEN_EINVAL, "subgen_prefill: n must be >= 0");
+    if (n == 0) return SUBGEN_OK;
+    if (!K || !V) return fail(SUBGEN_EINVAL, "subgen_prefill: K and V must not be NULL");
+    for (int b = 0; b < h->d.B; ++b)
+        if ((long long)h->n_host[b] + n > INT_MAX - 1) return fail(SUBGEN_ESTATE, "subgen_prefill: stream too long");
+    int rc = launch_prefill(h, K, V, n, nullptr, 0);
+    if (rc) return rc;
+    for (int b = 0; b < h->d.B; ++b) h->n_host[b] += n;
+    return SUBGEN_OK;
+}
+
+int subgen_prefill_varlen(subgen_t* h, const void* K, const void* V, const int* cu) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_prefill_varlen: handle is NULL");
+    if (!cu) return fail(SUBGEN_EINVAL, "subgen_prefill_varlen: cu_seqlens is NULL");
+    if (cu[0] != 0) return fail(SUBGEN_EINVAL, "subgen_prefill_varlen: cu_seqlens[0] must be 0");
+    for (int b = 0; b < h->d.B; ++b) {
+        if (cu[b + 1] < cu[b]) return fail(SUBGEN_EINVAL, "subgen_prefill_varlen: cu_seqlens must be non-decreasing");
+        if ((long long)h->n_host[b] + (cu[b + 1] - cu[b]) > INT_MAX - 1)
+            return fail(SUBGEN_ESTATE, "subgen_prefill_varlen: stream too long");
+    }
+    const int total = cu[h->d.B];
+    if (total == 0) return SUBGEN_OK;
+    if (!K || !V) return fail(SUBGEN_EINVAL, "subgen_prefill_varlen: K and V must not be NULL");
+    int* cu_dev = (int*)(h->ws + h->L.cu);
+    // the offsets are consumed by the kernel launched right after, in stream order
+    CUDA_TRY(cudaMemcpyAsync(cu_dev, cu, sizeof(int) * (h->d.B + 1), cudaMemcpyHostToDevice, h->st));
+    CUDA_TRY(cudaStreamSynchronize(h->st));   // cu may be pageable host memory reused by the caller
+    int rc = launch_prefill(h, K, V, 0, cu_dev, total);
+    if (rc) return rc;
+    for (int b = 0; b < h->d.B; ++b) h->n_host[b] += cu[b + 1] - cu[b];
+    return SUBGEN_OK;
+}
+
+int subgen_step(subgen_t* h, const void* q, const void* k, const void* v, void* out) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_step: handle is NULL");
+    if (!q || !k || !v || !out) return fail(SUBGEN_EINVAL, "subgen_step: q, k, v, out must not be NULL");
+    if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15)
+        return fail(SUBGEN_EINVAL, "subgen_step: pointers must be 16-byte aligned");
+    for (int b = 0; b < h->d.B; ++b)
+        if (h->n_host[b] >= INT_MAX - 1) return fail(SUBGEN_ESTATE, "subgen_step: stream too long");
+    int rc = launch_step(h, q, k, v, out);
+    if (rc) return rc;
+    for (int b = 0; b < h->d.B; ++b) h->n_host[b] += 1;
+    return SUBGEN_OK;
+}
+
+int subgen_step_host(subgen_t* h, const void* q, const void* k, const void* v, void* out) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_step_host: handle is NULL");
+    if (!q || !k || !v || !out) return fail(SUBGEN_EINVAL, "subgen_step_host: q, k, v, out must not be NULL");
+    const size_t row = (size_t)h->d.D * h->d.E;
+    const size_t qb = (size_t)h->d.B * h->d.H * row, kb = (size_t)h->d.U * row;
+    char* w = h->ws;
+    CUDA_TRY(cudaMemcpyAsync(w + h->L.stage_q, q, qb, cudaMemcpyHostToDevice, h->st));
+    CUDA_TRY(cudaMemcpyAsync(w + h->L.stage_k, k, kb, cudaMemcpyHostToDevice, h->st));
+    CUDA_TRY(cudaMemcpyAsync(w + h->L.stage_v, v, kb, cudaMemcpyHostToDevice, h->st));
+    int rc = subgen_step(h, w + h->L.stage_q, w + h->L.stage_k, w + h->L.stage_v, w + h->L.stage_out);
+    if (rc) return rc;
+    CUDA_TRY(cudaMemcpyAsync(out, w + h->L.stage_out, qb, cudaMemcpyDeviceToHost, h->st));
+    CUDA_TRY(cudaStreamSynchronize(h->st));
+    return SUBGEN_OK;
+}
+
+int subgen_status(subgen_t* h) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_status: handle is NULL");
+    std::vector<int> st(h->d.U);
+    CUDA_TRY(cudaStreamSynchronize(h->st));
+    CUDA_TRY(cudaMemcpy(st.data(), h->ws + h->L.status, sizeof(int) * h->d.U, cudaMemcpyDeviceToHost));
+    int r = 0;
+    for (int x : st) r |= x;
+    return r;
+}
+
+int subgen_export_state(subgen_t* h, int seq, int kvhead, subgen_state_view* v) {
+    if (!h || !v) return fail(SUBGEN_EINVAL, "subgen_export_state: NULL argument");
+    if (seq < 0 || seq >= h->d.B || kvhead < 0 || kvhead >= h->d.Hkv)
+        return fail(SUBGEN_EINVAL, "subgen_export_state: unit out of range");
+    const size_t u = (size_t)seq * h->d.Hkv + kvhead;
+    const Dims& d = h->d;
+    char* w = h->ws;
+    CUDA_TRY(cudaStreamSynchronize(h->st));
+    auto get = [&](void* dst, size_t off, size_t bytes) { return cudaMemcpy(dst, w + off, bytes, cudaMemcpyDeviceToHost); };
+    CUDA_TRY(get(&v->n, h->L.n_unit + u * 4, 4));
+    CUDA_TRY(get(&v->m, h->L.m_unit + u * 4, 4));
+    CUDA_TRY(get(&v->status, h->L.status + u * 4, 4));
+    CUDA_TRY(get(&v->mu, h->L.mu + u * 8, 8));
+    CUDA_TRY(get(&v->last_cluster, h->L.last_cid + u * 4, 4));
+    CUDA_TRY(get(&v->last_opened, h->L.last_open + u * 4, 4));
+    CUDA_TRY(get(&v->last_d2, h->L.last_d2 + u * 8, 8));
+    v->inserted = v->n > d.w ? v->n - d.w : 0;
+    if (v->counts) CUDA_TRY(get(v->counts, h->L.cnt + u * d.m_max * 4, (size_t)d.m_max * 4));
+    if (v->centre_tok) CUDA_TRY(get(v->centre_tok, h->L.ctok + u * d.m_max * 4, (size_t)d.m_max * 4));
+    if (v->slot_tok) CUDA_TRY(get(v->slot_tok, h->L.stok + u * d.m_max * d.t * 4, (size_t)d.m_max * d.t * 4));
+    if (v->m_tok) CUDA_TRY(get(v->m_tok, h->L.Mtok + u * d.s * 4, (size_t)d.s * 4));
+    if (v->m_w) CUDA_TRY(get(v->m_w, h->L.MW + u * d.s * 8, (size_t)d.s * 8));
+    return SUBGEN_OK;
+}
+
+int subgen_export_rows(subgen_t* h, int seq, int kvhead, int which, void* host, size_t bytes) {
+    if (!h || !host) return fail(SUBGEN_EINVAL, "subgen_export_rows: NULL argument");
+    if (seq < 0 || seq >= h->d.B || kvhead < 0 || kvhead >= h->d.Hkv)
+        return fail(SUBGEN_EINVAL, "subgen_export_rows: unit out of range");
+    const Dims& d = h->d;
+    const size_t u = (size_t)seq * d.Hkv + kvhead, row = (size_t)d.D * d.E;
+    size_t off, need;
+    switch (which) {
+        case 0: need = d.m_max * row; off = h->L.X + u * need; break;
+        case 1: need = (size_t)d.m_max * d.t * row; off = h->L.S + u * need; break;
+        case 2: need = d.s * row; off = h->L.Mk + u * need; break;
+        case 3: need = d.s * row; off = h->L.Mv + u * need; break;
+        case 4: need = d.w * row; off = h->L.ringK + u * need; break;
+        case 5: need = d.w * row; off = h->L.ringV + u * need; break;
+        default: return fail(SUBGEN_EINVAL, "subgen_export_rows: which must be 0..5");
+    }
+    if (bytes < need) return fail(SUBGEN_EINVAL, "subgen_export_rows: buffer needs %zu bytes", need);
+    CUDA_TRY(cudaStreamSynchronize(h->st));
+    if (need) CUDA_TRY(cudaMemcpy(host, h->ws + off, need, cudaMemcpyDeviceToHost));
+    return SUBGEN_OK;
+}
+
+int subgen_cache_stats(subgen_t* h, subgen_stats* out) {
+    if (!h || !out) return fail(SUBGEN_EINVAL, "subgen_cache_stats: NULL argument");
+    unsigned long long* dev = (unsigned long long*)(h->ws + h->L.stats);
+    CUDA_TRY(cudaMemsetAsync(dev, 0, 8 * sizeof(uint64_t), h->st));
+    if (h->cfg.dtype == SUBGEN_DTYPE_FP32) stats_kernel<float><<<h->d.U, 256, 0, h->st>>>(make_cache<float>(h), h->d.U, dev);
+    else stats_kernel<__nv_bfloat16><<<h->d.U, 256, 0, h->st>>>(make_cache<__nv_bfloat16>(h), h->d.U, dev);
+    CUDA_TRY(cudaGetLastError());
+    h->launches += 1;
+    uint64_t r[8];
+    CUDA_TRY(cudaMemcpyAsync(r, dev, sizeof r, cudaMemcpyDeviceToHost, h->st));
+    CUDA_TRY(cudaStreamSynchronize(h->st));
+    const uint64_t row = (uint64_t)h->d.D * h->d.E;
+    out->units = h->d.U;
+    out->clusters = r[0]; out->singleton_clusters = r[1]; out->m_filled = r[2]; out->window_rows = r[3]; out->tokens = r[4];
+    out->insert_bytes = r[0] * row;
+    out->query_bytes = (r[1] + (r[0] - r[1]) * (uint64_t)h->d.t + 2 * r[2] + 2 * r[3]) * row + r[0] * 4 + (uint64_t)h->d.U * h->d.s * 8;
+    return SUBGEN_OK;
+}
+
+int subgen_profile_enable(subgen_t* h, int on) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_profile_enable: handle is NULL");
+    h->prof = on != 0;
+    return SUBGEN_OK;
+}
+
+int subgen_profile_read(subgen_t* h, double* insert_ms, double* query_ms, int* steps) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_profile_read: handle is NULL");
+    CUDA_TRY(cudaStreamSynchronize(h->st));
+    double a = 0, b = 0;
+    for (size_t i = 0; i + 3 <= h->ev_used; i += 3) {
+        float x = 0, y = 0;
+        CUDA_TRY(cudaEventElapsedTime(&x, h->ev[i], h->ev[i + 1]));
+        CUDA_TRY(cudaEventElapsedTime(&y, h->ev[i + 1], h->ev[i + 2]));
+        a += x; b += y;
+    }
+    if (insert_ms) *insert_ms = a;
+    if (query_ms) *query_ms = b;
+    if (steps) *steps = (int)(h->ev_used / 3);
+    h->ev_used = 0;
+    return SUBGEN_OK;
+}
+
+uint64_t subgen_launch_count(const subgen_t* h) { return h ? h->launches : 0; }
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Exact comparison path.
+
+struct subgen_exact {
+    int B, H, Hkv, G, D, n_max, dtype, U, splits;
+    size_t E;
+    char *Kc = nullptr, *Vc = nullptr, *misc = nullptr;
+    size_t off_n, off_part, off_ticket, off_cu, misc_bytes;
+    cudaStream_t st = nullptr;
+    std::vector<int> n_host;
+    uint64_t launches = 0;
+};
+
+namespace {
+
+template <typename T> ExactCache<T> make_exact(const subgen_exact* h) {
+    ExactCache<T> E;
+    E.B = h->B; E.H = h->H; E.Hkv = h->Hkv; E.G = h->G; E.n_max = h->n_max;
+    E.Kc = (T*)h->Kc; E.Vc = (T*)h->Vc;
+    E.n_unit = (int*)(h->misc + h->off_n);
+    E.part = (float*)(h->misc + h->off_part);
+    E.ticket = (unsigned*)(h->misc + h->off_ticket);
+    return E;
+}
+
+template <typename T, int D>
+int exact_append_td(subgen_exact* h, const void* K, const void* V, int n, const int* cu_dev, int total, int longest) {
+    ExactCache<T> E = make_exact<T>(h);
+    int bx = (int)(((size_t)longest * (D / Elem<T>::EPL) + 255) / 256);
+    bx = bx < 1 ? 1 : (bx > 64 ? 64 : bx);
+    exact_append_kernel<T, D><<<dim3(bx, h->U), 256, 0, h->st>>>(E, (const T*)K, (const T*)V, n, cu_dev, total);
+    exact_advance_kernel<T><<<(h->U + 255) / 256, 256, 0, h->st>>>(E, h->U, n, cu_dev);
+    CUDA_TRY(cudaGetLastError());
+    h->launches += 2;
+    return SUBGEN_OK;
+}
+
+int exact_append(subgen_exact* h, const void* K, const void* V, int n, const int* cu_dev, int total, int longest) {
+    const bool f32 = h->dtype == SUBGEN_DTYPE_FP32;
+    if (h->D == 64)
+        return f32 ? exact_append_td<float, 64>(h, K, V, n, cu_dev, total, longest)
+                   : exact_append_td<__nv_bfloat16, 64>(h, K, V, n, cu_dev, total, longest);
+    return f32 ? exact_append_td<float, 128>(h, K, V, n, cu_dev, total, longest)
+               : exact_append_td<__nv_bfloat16, 128>(h, K, V, n, cu_dev, total, longest);
+}
+
+template <typename T, int D>
+int exact_step_td(subgen_exact* h, const void* q, const void* k, const void* v, void* out) {
+    ExactCache<T> E = make_exact<T>(h);
+    const dim3 grid(h->splits, h->U);
+    switch (h->G) {
+        case 1: exact_step_kernel<T, D, 1><<<grid, kQueryThreads, 0, h->st>>>(E, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
+        case 2: exact_step_kernel<T, D, 2><<<grid, kQueryThreads, 0, h->st>>>(E, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
+        case 4: exact_step_kernel<T, D, 4><<<grid, kQueryThreads, 0, h->st>>>(E, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
+        default: exact_step_kernel<T, D, 8><<<grid, kQueryThreads, 0, h->st>>>(E, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
+    }
+    CUDA_TRY(cudaGetLastError());
+    h->launches += 1;
+    return SUBGEN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+subgen_exact_t* subgen_exact_create(int B, int H, int Hkv, int d, int n_max, int dtype, void* stream) {
+    if (Hkv == 0) Hkv = H;
+    if (B <= 0 || H <= 0 || Hkv <= 0 || H % Hkv || n_max <= 0 || (d != 64 && d != 128) ||
+        (dtype != SUBGEN_DTYPE_FP32 && dtype != SUBGEN_DTYPE_BF16) || (long long)B * Hkv > 65535) {
+        fail(SUBGEN_EINVAL, "subgen_exact_create: invalid argument");
+        return nullptr;
+    }
+    const int G = H / Hkv;
+    if (G != 1 && G != 2 && G != 4 && G != 8) { fail(SUBGEN_EINVAL, "subgen_exact_create: H / Hkv must be 1, 2, 4 or 8"); return nullptr; }
+    if (check_device() != SUBGEN_OK) return nullptr;
+    subgen_exact* h = new subgen_exact();
+    h->B = B; h->H = H; h->Hkv = Hkv; h->G = G; h->D = d; h->n_max = n_max; h->dtype = dtype; h->U = B * Hkv;
+    h->E = dtype == SUBGEN_DTYPE_FP32 ? 4 : 2;
+    int sp = (148 * 8 + h->U - 1) / h->U;
+    h->splits = sp < 1 ? 1 : (sp > 32 ? 32 : sp);
+    h->st = (cudaStream_t)stream;
+    const size_t cache = (size_t)h->U * n_max * d * h->E;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    h->off_n = take((size_t)h->U * 4);
+    h->off_ticket = take((size_t)h->U * 4);
+    h->off_cu = take(((size_t)B + 1) * 4);
+    h->off_part = take((size_t)h->U * h->splits * G * (d + 2) * 4);
+    h->misc_bytes = off;
+    if (cudaMalloc((void**)&h->Kc, cache) != cudaSuccess || cudaMalloc((void**)&h->Vc, cache) != cudaSuccess ||
+        cudaMalloc((void**)&h->misc, h->misc_bytes) != cudaSuccess ||
+        cudaMemsetAsync(h->misc, 0, h->misc_bytes, h->st) != cudaSuccess) {
+        fail(SUBGEN_ENOMEM, "subgen_exact_create: allocating 2 x %zu bytes failed: %s", cache, cudaGetErrorString(cudaGetLastError()));
+        cudaFree(h->Kc); cudaFree(h->Vc); cudaFree(h->misc);
+        delete h;
+        return nullptr;
+    }
+    h->n_host.assign(B, 0);
+    return h;
+}
+
+void subgen_exact_destroy(subgen_exact_t* h) {
+    if (!h) return;
+    cudaStreamSynchronize(h->st);
+    cudaFree(h->Kc); cudaFree(h->Vc); cudaFree(h->misc);
+    delete h;
+}
+
+int subgen_exact_append(subgen_exact_t* h, const void* K, const void* V, int n) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_exact_append: handle is NULL");
+    if (n < 0) return fail(SUBGEN_EINVAL, "subgen_exact_append: n must be >= 0");
+    if (n == 0) return SUBGEN_OK;
+    if (!K || !V) return fail(SUBGEN_EINVAL, "subgen_exact_append: K and V must not be NULL");
+    for (int b = 0; b < h->B; ++b)
+        if ((long long)h->n_host[b] + n > h->n_max) return fail(SUBGEN_ESTATE, "subgen_exact_append: cache capacity n_max exceeded");
+    int rc = exact_append(h, K, V, n, nullptr, 0, n);
+    if (rc) return rc;
+    for (int b = 0; b < h->B; ++b) h->n_host[b] += n;
+    return SUBGEN_OK;
+}
+
+int subgen_exact_append_varlen(subgen_exact_t* h, const void* K, const void* V, const int* cu) {
+    if (!h || !cu) return fail(SUBGEN_EINVAL, "subgen_exact_append_varlen: NULL argument");
+    if (cu[0] != 0) return fail(SUBGEN_EINVAL, "subgen_exact_append_varlen: cu_seqlens[0] must be 0");
+    int longest = 0;
+    for (int b = 0; b < h->B; ++b) {
+        const int len = cu[b + 1] - cu[b];
+        if (len < 0) return fail(SUBGEN_EINVAL, "subgen_exact_append_varlen: cu_seqlens must be non-decreasing");
+        if ((long long)h->n_host[b] + len > h->n_max) return fail(SUBGEN_ESTATE, "subgen_exact_append_varlen: cache capacity n_max exceeded");
+        longest = len > longest ? len : longest;
+    }
+    const int total = cu[h->B];
+    if (total == 0) return SUBGEN_OK;
+    if (!K || !V) return fail(SUBGEN_EINVAL, "subgen_exact_append_varlen: K and V must not be NULL");
+    int* cu_dev = (int*)(h->misc + h->off_cu);
+    CUDA_TRY(cudaMemcpyAsync(cu_dev, cu, sizeof(int) * (h->B + 1), cudaMemcpyHostToDevice, h->st));
+    CUDA_TRY(cudaStreamSynchronize(h->st));
+    int rc = exact_append(h, K, V, 0, cu_dev, total, longest);
+    if (rc) return rc;
+    for (int b = 0; b < h->B; ++b) h->n_host[b] += cu[b + 1] - cu[b];
+    return SUBGEN_OK;
+}
+
+int subgen_exact_step(subgen_exact_t* h, const void* q, const void* k, const void* v, void* out) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_exact_step: handle is NULL");
+    if (!q || !k || !v || !out) return fail(SUBGEN_EINVAL, "subgen_exact_step: q, k, v, out must not be NULL");
+    if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15)
+        return fail(SUBGEN_EINVAL, "subgen_exact_step: pointers must be 16-byte aligned");
+    for (int b = 0; b < h->B; ++b)
+        if (h->n_host[b] >= h->n_max) return fail(SUBGEN_ESTATE, "subgen_exact_step: cache capacity n_max exceeded");
+    const bool f32 = h->dtype == SUBGEN_DTYPE_FP32;
+    int rc;
+    if (h->D == 64) rc = f32 ? exact_step_td<float, 64>(h, q, k, v, out) : exact_step_td<__nv_bfloat16, 64>(h, q, k, v, out);
+    else rc = f32 ? exact_step_td<float, 128>(h, q, k, v, out) : exact_step_td<__nv_bfloat16, 128>(h, q, k, v, out);
+    if (rc) return rc;
+    for (int b = 0; b < h->B; ++b) h->n_host[b] += 1;
+    return SUBGEN_OK;
+}
+
+int subgen_exact_bytes(subgen_exact_t* h, uint64_t* bytes) {
+    if (!h || !bytes) return fail(SUBGEN_EINVAL, "subgen_exact_bytes: NULL argument");
+    uint64_t rows = 0;
+    for (int b = 0; b < h->B; ++b) rows += (uint64_t)h->n_host[b] * h->Hkv;
+    *bytes = 2 * rows * (uint64_t)h->D * h->E;
+    return SUBGEN_OK;
+}
+
+uint64_t subgen_exact_launch_count(const subgen_exact_t* h) { return h ? h->launches : 0; }
+
+}  // extern "C"

@@ -8,7 +8,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-namespace subgen {
+namespace sgk {
 
 constexpr uint32_t kPhiloxM0 = 0xD2511F53u, kPhiloxM1 = 0xCD9E8D57u;
 constexpr uint32_t kPhiloxW0 = 0x9E3779B9u, kPhiloxW1 = 0xBB67AE85u;
@@ -428,4 +428,4 @@ __device__ __forceinline__ void final_merge(const float* part, int np, T* out, b
     }
 }
 
-}  // namespace subgen
+}  // namespace sgk
