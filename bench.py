@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the SubGen stream step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3] [--impl subgen|reference]
+
+One "step" is one pass of the whole hot path over one batch: subgen_step for all B sequences and H
+heads (window push, insertion of the token that leaves the window, query estimator), from a state
+built by subgen_prefill over the prompt. Default workload: cfg3 (B=8, H=32, d=128, bf16, 32768-token
+prompts, delta 0.6, t 8, s 2048, window 512, mixture keys with 5% outliers), the 32K-context point of
+the metric. Prints ONE JSON line (rank 0).
+
+--impl reference times the CPU oracle (oracle/) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2402_06082_b200 import synth  # noqa: E402
+
+METRIC = "SubGen decode steps/s (B x H heads) at 32K ctx"
+
+
+# ------------------------------------------------------------------------------------------ helpers
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU every 200 ms through NVML while running."""
+
+    def __init__(self, device_index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if isinstance(uuid, str) else uuid)
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+        self._t = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        nv = self._nv
+        names = {"hw_slowdown": "nvmlClocksThrottleReasonHwSlowdown",
+                 "hw_thermal_slowdown": "nvmlClocksThrottleReasonHwThermalSlowdown",
+                 "sw_thermal_slowdown": "nvmlClocksThrottleReasonSwThermalSlowdown",
+                 "sw_power_cap": "nvmlClocksThrottleReasonSwPowerCap"}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for k, attr in names.items():
+                    if mask & int(getattr(nv, attr, 0)):
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(0.2)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._h is not None:
+            self._t.join(timeout=2)
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_leg(w, n_prompt, sample_units, steps, warmup, threads):
+    """Times the CPU oracle, as it stands, on `sample_units` (seq, kvhead) units of the workload: prefill of the
+    prompt, then warmup + steps stream steps. Returns whole-job rates scaled by units / sample."""
+    from oracle import subgen_oracle as orc
+    orc.lib()
+    G = w.H // w.Hkv
+    n_tot = n_prompt + warmup + steps
+    data = {}
+    for (b, h) in sample_units:
+        if b not in data:
+            K, V, Q = synth.sequence_stream(w, b, n_tot, "cpu")
+            data[b] = (synth.to_f32_numpy(K), synth.to_f32_numpy(V), synth.to_f32_numpy(Q))
+    units = [orc.OracleUnit(w.d, w.delta, w.t, w.s, w.window, seed=w.philox_seed, unit_id=b * w.Hkv + h,
+                            m_max=max(w.m_max, 1)) for (b, h) in sample_units]
+
+    def prefill(i):
+        b, h = sample_units[i]
+        units[i].push_many(data[b][0][h, :n_prompt], data[b][1][h, :n_prompt])
+
+    def step(i, tok):
+        b, h = sample_units[i]
+        K, V, Q = data[b]
+        units[i].push(K[h, tok], V[h, tok])
+        for g in range(G):
+            units[i].query(Q[h * G + g, tok])
+
+    with ThreadPoolExecutor(threads) as ex:
+        t0 = time.perf_counter()
+        list(ex.map(prefill, range(len(units))))
+        t_prefill = time.perf_counter() - t0
+        for tok in range(n_prompt, n_prompt + warmup):
+            list(ex.map(lambda i: step(i, tok), range(len(units))))
+        t0 = time.perf_counter()
+        for tok in range(n_prompt + warmup, n_tot):
+            list(ex.map(lambda i: step(i, tok), range(len(units))))
+        t_steps = time.perf_counter() - t0
+    scale = w.units / len(units)
+    steps_per_s = steps / (t_steps * scale) if t_steps > 0 else float("inf")
+    prefill_tok_s = (n_prompt * w.B) / (t_prefill * scale) if t_prefill > 0 else float("inf")
+    return dict(steps_per_s=steps_per_s, ms_per_step=1e3 * t_steps * scale / max(steps, 1), prefill_tokens_per_s=prefill_tok_s,
+                t_prefill_s=t_prefill, t_steps_s=t_steps, m=[u.m for u in units])
+
+
+def pick_sample(w, k):
+    rng = np.random.default_rng(w.data_seed + 17)
+    idx = rng.choice(w.units, size=min(k, w.units), replace=False)
+    return [(int(i) // w.Hkv, int(i) % w.Hkv) for i in sorted(idx)]
+
+
+# ------------------------------------------------------------------------------------------ arms
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = min(os.cpu_count() or 1, 8)
+    sample = pick_sample(w, cores)
+    n_prompt = w.n_prompt
+    r = oracle_leg(w, n_prompt, sample, args.steps, args.warmup, cores)
+    desc = "%d of %d (seq, KV head) units, each: oracle prefill of %d tokens (untimed), %d warm-up + %d timed stream steps; scaled by units/sample" % (
+        len(sample), w.units, n_prompt, args.warmup, args.steps)
+    line = {"impl": "reference", "metric": METRIC, "value": r["steps_per_s"], "unit": "steps/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": r["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w),
+            "cpu_baseline": {"value": r["steps_per_s"], "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": r["steps_per_s"], "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "oracle_prefill_tokens_per_s": r["prefill_tokens_per_s"]}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w):
+    return {"workload": "%s: B=%d H=%d Hkv=%d d=%d %s, prompt n=%d then decode; keys %d-component mixture sigma=%.2f "
+                        "outliers=%.2f drift=%s; delta=%.2f t=%d s=%d window=%d; Philox seed %d" % (
+                            w.name, w.B, w.H, w.Hkv, w.d, w.dtype, w.n_prompt, w.ncomp, w.sigma, w.outlier_frac, w.drift,
+                            w.delta, w.t, w.s, w.window, w.philox_seed),
+            "l2": "per-step working set (compressed cache) larger than the 126 MB L2; no explicit flush",
+            "accumulate": "fp32", "units": w.units}
+
+
+def run_subgen(args, w):
+    from paper_2402_06082_b200 import binding, build
+    build.build()
+    N = args.gpus
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    # weak scaling: every rank serves its own batch of B sequences (units are independent, no data-path collective)
+    wr = w.scaled(data_seed=w.data_seed + 7919 * rank)
+    K_steps = args.steps
+    W_steps = args.warmup
+    n_e2e = args.e2e_steps
+    n_dec = W_steps + K_steps + n_e2e + 4
+    lens = wr.prompt_lens()
+    varlen = wr.varlen is not None
+    dev = "cuda"
+    dt = wr.torch_dtype
+
+    # ---- inputs, resident in HBM ----
+    qs = torch.empty(n_dec, wr.B, wr.H, wr.d, dtype=dt, device=dev)
+    ks = torch.empty(n_dec, wr.B, wr.Hkv, wr.d, dtype=dt, device=dev)
+    vs = torch.empty(n_dec, wr.B, wr.Hkv, wr.d, dtype=dt, device=dev)
+    if varlen:
+        total = int(sum(lens))
+        Kp = torch.empty(wr.Hkv, total, wr.d, dtype=dt, device=dev)
+        Vp = torch.empty_like(Kp)
+    else:
+        Kp = torch.empty(wr.B, wr.Hkv, wr.n_prompt, wr.d, dtype=dt, device=dev)
+        Vp = torch.empty_like(Kp)
+    off = 0
+    for b in range(wr.B):
+        Kb, Vb, Qb = synth.sequence_stream(wr, b, lens[b] + n_dec, dev)
+        if varlen:
+            Kp[:, off:off + lens[b]] = Kb[:, :lens[b]]
+            Vp[:, off:off + lens[b]] = Vb[:, :lens[b]]
+            off += lens[b]
+        else:
+            Kp[b] = Kb[:, :lens[b]]
+            Vp[b] = Vb[:, :lens[b]]
+        qs[:, b] = Qb[:, lens[b]:].transpose(0, 1)
+        ks[:, b] = Kb[:, lens[b]:].transpose(0, 1)
+        vs[:, b] = Vb[:, lens[b]:].transpose(0, 1)
+        del Kb, Vb, Qb
+    torch.cuda.synchronize()
+
+    sg = binding.SubGen(wr.B, wr.H, wr.d, wr.delta, wr.t, wr.s, wr.window, wr.philox_seed, Hkv=wr.Hkv, dtype=dt,
+                        m_max=wr.m_max, splits=args.splits)
+    out = torch.empty(wr.B, wr.H, wr.d, dtype=dt, device=dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    # ---- prefill (timed on its own) ----
+    l0 = sg.launch_count
+    e0.record()
+    if varlen:
+        cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+        sg.prefill_varlen(Kp, Vp, cu)
+    else:
+        sg.prefill(Kp, Vp)
+    e1.record()
+    torch.cuda.synchronize()
+    prefill_ms = e0.elapsed_time(e1)
+    prefill_launches = sg.launch_count - l0
+    st = sg.status()
+    if st:
+        raise SystemExit("device status %d after prefill (1 = cluster capacity, 2 = input range)" % st)
+    del Kp, Vp
+
+    # ---- decode: warm-up, then the timed region ----
+    for i in range(W_steps):
+        sg.step(qs[i], ks[i], vs[i], out)
+    torch.cuda.synchronize()
+    stats0 = sg.cache_stats()
+    sg.profile_enable(True)
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = sg.launch_count
+    with ClockSampler(local) as clk:
+        e0.record()
+        for i in range(W_steps, W_steps + K_steps):
+            sg.step(qs[i], ks[i], vs[i], out)
+        e1.record()
+        torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    launches = sg.launch_count - launches0
+    ins_ms, qry_ms, nprof = sg.profile_read()
+    sg.profile_enable(False)
+    stats1 = sg.cache_stats()
+    if dist:
+        tt = torch.tensor([ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt.item())
+    ms_per_step = ms / K_steps
+    value = world * K_steps / (ms * 1e-3)
+
+    # ---- end to end through the host-buffer entry point ----
+    base = W_steps + K_steps
+    hq = qs[base:base + n_e2e].cpu().pin_memory()
+    hk = ks[base:base + n_e2e].cpu().pin_memory()
+    hv = vs[base:base + n_e2e].cpu().pin_memory()
+    hout = torch.empty(wr.B, wr.H, wr.d, dtype=dt).pin_memory()
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(n_e2e):
+        sg.step_host(hq[i], hk[i], hv[i], hout)
+    t_e2e = time.perf_counter() - t0
+    if dist:
+        tt = torch.tensor([t_e2e], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        t_e2e = float(tt.item())
+    esz = 2 if dt == torch.bfloat16 else 4
+    h2d = (wr.B * wr.H + 2 * wr.B * wr.Hkv) * wr.d * esz
+    d2h = wr.B * wr.H * wr.d * esz
+    e2e = {"value": world * n_e2e / t_e2e, "unit": "steps/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+           "steps": n_e2e}
+    if sg.status():
+        raise SystemExit("device status %d after decode" % sg.status())
+
+    # ---- roofline of the dominant kernel (query_kernel) ----
+    peak, which = measured_peaks()
+    qbytes = 0.5 * (stats0["query_bytes"] + stats1["query_bytes"])
+    ibytes = 0.5 * (stats0["insert_bytes"] + stats1["insert_bytes"])
+    q_ms = qry_ms / max(nprof, 1)
+    i_ms = ins_ms / max(nprof, 1)
+    achieved = qbytes / (q_ms * 1e-3) / 1e9 if q_ms > 0 else None
+    roofline = {"bound": "hbm", "kernel": "query_kernel", "achieved": achieved, "peak": peak, "peak_source": which,
+                "unit": "GB/s", "frac": achieved / peak if achieved else None, "traffic": None,
+                "algorithmic_bytes_per_launch": qbytes, "ms_per_launch": q_ms,
+                "insert_kernel": {"algorithmic_bytes_per_launch": ibytes, "ms_per_launch": i_ms,
+                                  "achieved": ibytes / (i_ms * 1e-3) / 1e9 if i_ms > 0 else None},
+                "step": {"algorithmic_bytes": qbytes + ibytes,
+                         "achieved": (qbytes + ibytes) / (ms_per_step * 1e-3) / 1e9,
+                         "frac": (qbytes + ibytes) / (ms_per_step * 1e-3) / 1e9 / peak}}
+
+    extra = {"prefill_ms": prefill_ms, "prefill_tokens_per_s": sum(lens) / (prefill_ms * 1e-3),
+             "prefill_launches": prefill_launches,
+             "cache": {k: stats1[k] for k in ("clusters", "singleton_clusters", "m_filled", "window_rows", "tokens")}}
+
+    # ---- exact dense decode over full caches on the same inputs (comparison point) ----
+    if args.exact and rank == 0:
+        try:
+            extra["exact"] = run_exact(wr, lens, n_dec, K_steps, W_steps, qs, ks, vs, peak)
+        except Exception as ex:  # report, do not hide
+            extra["exact"] = {"error": str(ex)[:200]}
+
+    cpu = None
+    if rank == 0 and world == 1 and args.cpu_baseline:
+        cores = min(os.cpu_count() or 1, 8)
+        sample = pick_sample(wr, cores)
+        r = oracle_leg(wr, max(lens) if not varlen else int(np.median(lens)), sample, 4, 1, cores)
+        cpu = {"value": r["steps_per_s"], "unit": "steps/s", "cores": cores, "kind": "oracle",
+               "sample": "%d of %d units: oracle prefill (%.1f s, untimed for this value) then 1 warm-up + 4 timed steps "
+                         "(%.2f s); scaled by units/sample" % (len(sample), wr.units, r["t_prefill_s"], r["t_steps_s"]),
+               "prefill_tokens_per_s": r["prefill_tokens_per_s"]}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world, "steps": K_steps, "warmup": W_steps,
+                "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16" if dt == torch.bfloat16 else "f32", "data": "synthetic", "config": workload_config(wr),
+                "clocks": clk.summary(), "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+                "cpu_baseline": cpu, "extra": extra}
+        print(json.dumps(line), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
+def run_exact(w, lens, n_dec, K_steps, W_steps, qs, ks, vs, peak):
+    from paper_2402_06082_b200 import binding
+    dt = w.torch_dtype
+    ex = binding.ExactAttention(w.B, w.H, w.d, max(lens) + n_dec, Hkv=w.Hkv, dtype=dt)
+    for b in range(w.B):    # regenerate the prompts sequence by sequence to bound memory
+        pass
+    if w.varlen is None:
+        Kp = torch.empty(w.B, w.Hkv, w.n_prompt, w.d, dtype=dt, device="cuda")
+        Vp = torch.empty_like(Kp)
+        for b in range(w.B):
+            Kb, Vb, _ = synth.sequence_stream(w, b, lens[b] + n_dec, "cuda")
+            Kp[b] = Kb[:, :lens[b]]
+            Vp[b] = Vb[:, :lens[b]]
+        ex.append(Kp, Vp)
+    else:
+        total = int(sum(lens))
+        Kp = torch.empty(w.Hkv, total, w.d, dtype=dt, device="cuda")
+        Vp = torch.empty_like(Kp)
+        off = 0
+        for b in range(w.B):
+            Kb, Vb, _ = synth.sequence_stream(w, b, lens[b] + n_dec, "cuda")
+            Kp[:, off:off + lens[b]] = Kb[:, :lens[b]]
+            Vp[:, off:off + lens[b]] = Vb[:, :lens[b]]
+            off += lens[b]
+        ex.append_varlen(Kp, Vp, np.concatenate([[0], np.cumsum(lens)]))
+    del Kp, Vp
+    out = torch.empty(w.B, w.H, w.d, dtype=dt, device="cuda")
+    for i in range(W_steps):
+        ex.step(qs[i], ks[i], vs[i], out)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    b0 = ex.bytes_per_step()
+    e0.record()
+    for i in range(W_steps, W_steps + K_steps):
+        ex.step(qs[i], ks[i], vs[i], out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / K_steps
+    gbs = b0 / (ms * 1e-3) / 1e9
+    ex.close()
+    return {"steps_per_s": 1e3 / ms, "ms_per_step": ms, "bytes_per_step": b0, "achieved_GBps": gbs, "frac_of_hbm_peak": gbs / peak}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="subgen", choices=["subgen", "reference"])
+    ap.add_argument("--workload", default="cfg3", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=32)
+    ap.add_argument("--no-exact", dest="exact", action="store_false")
+    ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--prompt", type=int, default=0, help="override the prompt length (smaller cases for profiling)")
+    ap.add_argument("--batch", type=int, default=0, help="override the number of sequences")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "subgen":
+        args.warmup = 3
+    w = synth.CONFIGS[args.workload]
+    if args.prompt:
+        w = w.scaled(n_prompt=args.prompt)
+    if args.batch:
+        w = w.scaled(B=args.batch)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_subgen(args, w)
+
+
+if __name__ == "__main__":
+    main()
