@@ -27,7 +27,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2402_06082_b200 import synth  # noqa: E402
+from paper_2402_06082_b200 import sharding, synth  # noqa: E402
 
 METRIC = "SubGen decode steps/s (B x H heads) at 32K ctx"
 
@@ -42,7 +42,7 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU every 200 ms through NVML while running."""
+    """Samples SM clock and throttle reasons of one GPU every 50 ms through NVML while running."""
 
     def __init__(self, device_index: int):
         self.samples, self.reasons, self.max_mhz = [], set(), None
@@ -77,7 +77,7 @@ class ClockSampler:
                         self.reasons.add(k)
             except Exception:
                 pass
-            self._stop.wait(0.2)
+            self._stop.wait(0.05)
 
     def __enter__(self):
         if self._h is not None:
@@ -102,23 +102,25 @@ def oracle_leg(w, n_prompt, sample_units, steps, warmup, threads):
     G = w.H // w.Hkv
     n_tot = n_prompt + warmup + steps
     data = {}
-    for (b, h) in sample_units:
-        if b not in data:
-            K, V, Q = synth.sequence_stream(w, b, n_tot, "cpu")
-            data[b] = (synth.to_f32_numpy(K), synth.to_f32_numpy(V), synth.to_f32_numpy(Q))
+    for b in sorted({b for b, _ in sample_units}):
+        K, V, Q = synth.sequence_stream(w, b, n_tot, "cpu")
+        for (bb, h) in sample_units:            # keep only the sampled heads' rows
+            if bb == b:
+                data[(b, h)] = (synth.to_f32_numpy(K[h]), synth.to_f32_numpy(V[h]),
+                                synth.to_f32_numpy(Q[h * G:(h + 1) * G]))
+        del K, V, Q
     units = [orc.OracleUnit(w.d, w.delta, w.t, w.s, w.window, seed=w.philox_seed, unit_id=b * w.Hkv + h,
                             m_max=max(w.m_max, 1)) for (b, h) in sample_units]
 
     def prefill(i):
-        b, h = sample_units[i]
-        units[i].push_many(data[b][0][h, :n_prompt], data[b][1][h, :n_prompt])
+        K, V, _ = data[sample_units[i]]
+        units[i].push_many(K[:n_prompt], V[:n_prompt])
 
     def step(i, tok):
-        b, h = sample_units[i]
-        K, V, Q = data[b]
-        units[i].push(K[h, tok], V[h, tok])
+        K, V, Q = data[sample_units[i]]
+        units[i].push(K[tok], V[tok])
         for g in range(G):
-            units[i].query(Q[h * G + g, tok])
+            units[i].query(Q[g, tok])
 
     with ThreadPoolExecutor(threads) as ex:
         t0 = time.perf_counter()
@@ -138,9 +140,12 @@ def oracle_leg(w, n_prompt, sample_units, steps, warmup, threads):
 
 
 def pick_sample(w, k):
+    """k seeded (seq, kvhead) units drawn from at most two sequences (input generation is per sequence)."""
     rng = np.random.default_rng(w.data_seed + 17)
-    idx = rng.choice(w.units, size=min(k, w.units), replace=False)
-    return [(int(i) // w.Hkv, int(i) % w.Hkv) for i in sorted(idx)]
+    seqs = rng.permutation(w.B)[:2]
+    cand = [(int(b), h) for b in seqs for h in range(w.Hkv)]
+    idx = rng.choice(len(cand), size=min(k, len(cand)), replace=False)
+    return sorted(cand[i] for i in idx)
 
 
 # ------------------------------------------------------------------------------------------ arms
@@ -188,7 +193,7 @@ def run_subgen(args, w):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     # weak scaling: every rank serves its own batch of B sequences (units are independent, no data-path collective)
-    wr = w.scaled(data_seed=w.data_seed + 7919 * rank)
+    wr = sharding.rank_workload(w, rank)
     K_steps = args.steps
     W_steps = args.warmup
     n_e2e = args.e2e_steps
@@ -270,12 +275,9 @@ def run_subgen(args, w):
     ins_ms, qry_ms, nprof = sg.profile_read()
     sg.profile_enable(False)
     stats1 = sg.cache_stats()
-    if dist:
-        tt = torch.tensor([ms], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms = float(tt.item())
+    ms = sharding.max_over_ranks(ms, dist, dev)
     ms_per_step = ms / K_steps
-    value = world * K_steps / (ms * 1e-3)
+    value = sharding.job_steps_per_s(world, K_steps, ms)
 
     # ---- end to end through the host-buffer entry point ----
     base = W_steps + K_steps
@@ -290,10 +292,7 @@ def run_subgen(args, w):
     for i in range(n_e2e):
         sg.step_host(hq[i], hk[i], hv[i], hout)
     t_e2e = time.perf_counter() - t0
-    if dist:
-        tt = torch.tensor([t_e2e], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        t_e2e = float(tt.item())
+    t_e2e = sharding.max_over_ranks(t_e2e, dist, dev)
     esz = 2 if dt == torch.bfloat16 else 4
     h2d = (wr.B * wr.H + 2 * wr.B * wr.Hkv) * wr.d * esz
     d2h = wr.B * wr.H * wr.d * esz
@@ -354,8 +353,6 @@ def run_exact(w, lens, n_dec, K_steps, W_steps, qs, ks, vs, peak):
     from paper_2402_06082_b200 import binding
     dt = w.torch_dtype
     ex = binding.ExactAttention(w.B, w.H, w.d, max(lens) + n_dec, Hkv=w.Hkv, dtype=dt)
-    for b in range(w.B):    # regenerate the prompts sequence by sequence to bound memory
-        pass
     if w.varlen is None:
         Kp = torch.empty(w.B, w.Hkv, w.n_prompt, w.d, dtype=dt, device="cuda")
         Vp = torch.empty_like(Kp)
@@ -396,7 +393,7 @@ def run_exact(w, lens, n_dec, K_steps, W_steps, qs, ks, vs, peak):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="subgen", choices=["subgen", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=sorted(synth.CONFIGS))
