@@ -182,6 +182,40 @@ int subgen_exact_step(subgen_exact_t* h, const void* q, const void* k, const voi
 int subgen_exact_bytes(subgen_exact_t* h, uint64_t* bytes);
 uint64_t subgen_exact_launch_count(const subgen_exact_t* h);
 
+/* ---- exact attention without any allocation -------------------------------------------------- */
+
+/* The paper has no counterpart for this entry point; it exists for integration reasons only.
+ *
+ * Some callers must not call cudaMalloc, directly or through a library: a plugin running inside a
+ * serving process whose own allocator claimed the device memory at start-up (a raw cudaMalloc
+ * there fails or takes memory behind the allocator's back), or request-path code that cannot
+ * afford the device-wide synchronisation an allocation or a free can cause. The handle-based
+ * functions above allocate in their create call; this one needs no handle and allocates nothing,
+ * neither with cudaMalloc/cudaFree nor through any allocating library routine.
+ *
+ * out = softmax(K q)^T V (Eq. 1, no scaling) for every head: q, out device [B, H, d]; K, V device
+ * [B, Hkv, n, d], n >= 1; dtype, d and the H/Hkv rule as for subgen_exact_create; stream is a
+ * cudaStream_t or NULL. The work of one (sequence, KV head) is split over several thread blocks;
+ * their partial results and the arrival counters live in ONE fixed array of
+ * SUBGEN_NOALLOC_SCRATCH_BYTES that is part of the library image: every GPU that loads the library
+ * holds that much memory until the process exits. Shapes that need more than the array for a single
+ * split, B*Hkv*(H/Hkv)*(d+2)*4 + 4*B*Hkv (rounded up to 256) bytes, are rejected with
+ * SUBGEN_EINVAL and a message; larger split counts are reduced to fit.
+ *
+ * The first call on each device looks up the array's device address (the device must be current,
+ * as for every call). Make that first call before starting any stream capture.
+ *
+ * All calls on a device share the array, and it keeps whatever the previous call left there. The
+ * function clears the counters it needs on `stream` before the kernel; partial results are always
+ * written before they are read. Two calls whose kernels can overlap on the GPU (different streams
+ * without an ordering between them, or different host threads) race on the array and give wrong
+ * results: order them.
+ *
+ * Returns 0 or a negative SUBGEN_E* code; asynchronous on `stream`. */
+#define SUBGEN_NOALLOC_SCRATCH_BYTES (4u << 20)
+int subgen_exact_attention_noalloc(const void* q, const void* K, const void* V, void* out, int B, int H, int Hkv,
+                                   int d, int n, int dtype, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

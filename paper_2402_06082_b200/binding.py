@@ -25,7 +25,7 @@ EXPORTS = [
     "subgen_export_rows", "subgen_cache_stats", "subgen_profile_enable", "subgen_profile_read",
     "subgen_launch_count", "subgen_last_error", "subgen_exact_create", "subgen_exact_destroy",
     "subgen_exact_append", "subgen_exact_append_varlen", "subgen_exact_step", "subgen_exact_bytes",
-    "subgen_exact_launch_count",
+    "subgen_exact_launch_count", "subgen_exact_attention_noalloc",
 ]
 
 
@@ -92,6 +92,7 @@ def load():
     L.subgen_exact_bytes.argtypes = [vp, C.POINTER(C.c_uint64)]
     L.subgen_exact_launch_count.argtypes = [vp]
     L.subgen_exact_launch_count.restype = C.c_uint64
+    L.subgen_exact_attention_noalloc.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, vp]
     _lib = L
     return L
 
@@ -281,3 +282,26 @@ class ExactAttention:
     @property
     def launch_count(self) -> int:
         return int(self._L.subgen_exact_launch_count(self._h))
+
+
+NOALLOC_SCRATCH_BYTES = 4 << 20
+
+
+def exact_attention_noalloc(q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, out: torch.Tensor,
+                            stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """out = softmax(K q)^T V per head without any device allocation by the library.
+
+    For callers that may not call cudaMalloc (a plugin inside a process whose allocator owns all device
+    memory, or request-path code that cannot take an allocation's synchronisation): the split partials
+    live in a fixed array inside the library image (NOALLOC_SCRATCH_BYTES per GPU, shared by all calls,
+    so calls that can overlap on the GPU must be ordered). q, out: CUDA [B, H, d]; K, V: CUDA [B, Hkv, n, d].
+    The caller supplies `out`; this wrapper creates no tensor.
+    """
+    B, H, d = q.shape
+    Hkv, n = K.shape[1], K.shape[2]
+    dt = q.dtype
+    st = stream or torch.cuda.current_stream()
+    _check(load().subgen_exact_attention_noalloc(
+        _dev(q, dt, (B, H, d), "q"), _dev(K, dt, (B, Hkv, n, d), "K"), _dev(V, dt, (B, Hkv, n, d), "V"),
+        _dev(out, dt, (B, H, d), "out"), B, H, Hkv, d, n, _dtype_code(dt), st.cuda_stream))
+    return out

@@ -627,3 +627,148 @@ int subgen_exact_bytes(subgen_exact_t* h, uint64_t* bytes) {
 uint64_t subgen_exact_launch_count(const subgen_exact_t* h) { return h ? h->launches : 0; }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Exact attention for callers that must not allocate: the split partials live in a fixed array that
+// is part of the loaded module instead of in memory obtained from cudaMalloc.
+
+#include <mutex>
+
+namespace {
+
+// One array per device that loads this library, held until the process exits. The name below is only
+// meaningful to device code; host code must use the address cudaGetSymbolAddress returns.
+static __device__ __align__(256) unsigned char g_static_scratch[SUBGEN_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices] = {nullptr};
+
+// grid (splits, U): softmax(K q)^T V over the n rows of the caller's K, V [B, Hkv, n, D].
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kQueryThreads) attend_static_kernel(const T* __restrict__ q, const T* __restrict__ K,
+                                                                      const T* __restrict__ V, T* __restrict__ out,
+                                                                      int n, int H, int Hkv, float* part, unsigned* ticket) {
+    constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, RPW = 32 / LPR, STR = D + 2, UN = 2;
+    __shared__ float sm[(kQueryThreads / 32) * G * STR];
+    __shared__ int sm_last;
+    const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5, lr = lane % LPR, sub = lane / LPR;
+    const int b = u / Hkv, kvh = u % Hkv;
+    const size_t qrow0 = (size_t)b * H + (size_t)kvh * G;
+    const T* Ku = K + (size_t)u * n * D;
+    const T* Vu = V + (size_t)u * n * D;
+    float qf[G][EPL];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        const uint4 r = *reinterpret_cast<const uint4*>(q + (qrow0 + g) * D + lr * EPL);
+        Elem<T>::unpack(r, qf[g]);
+    }
+    Acc<G, EPL> A;
+    A.init();
+    const int gg = (blockIdx.x * (kQueryThreads / 32) + warp) * RPW + sub;
+    const int GG = splits * (kQueryThreads / 32) * RPW;
+    for (int jb = 0; jb < n; jb += GG * UN) {
+        uint4 kraw[UN], vraw[UN];
+        bool valid[UN];
+        float wt_tau[UN], wt_z[UN];
+#pragma unroll
+        for (int i = 0; i < UN; ++i) {
+            const int idx = jb + i * GG + gg;
+            valid[i] = idx < n;
+            wt_tau[i] = 1.f; wt_z[i] = 1.f;
+            kraw[i] = make_uint4(0, 0, 0, 0);
+            vraw[i] = kraw[i];
+            if (valid[i]) {
+                kraw[i] = *reinterpret_cast<const uint4*>(Ku + (size_t)idx * D + lr * EPL);
+                vraw[i] = *reinterpret_cast<const uint4*>(Vu + (size_t)idx * D + lr * EPL);
+            }
+        }
+        float sc[UN][G];
+        scores<T, D, G, UN>(kraw, qf, sc);
+        fold<T, D, G, UN, true>(A, sc, valid, wt_tau, wt_z, vraw);
+    }
+    float* part_u = part + (size_t)u * splits * G * STR;
+    block_partial<T, D, G>(A, sm, part_u + (size_t)blockIdx.x * G * STR);
+    __threadfence();
+    __syncthreads();
+    if (splits > 1) {
+        if (tid == 0) {
+            __threadfence();
+            sm_last = (atomicAdd(&ticket[u], 1u) == (unsigned)splits - 1u);
+        }
+        __syncthreads();
+        if (!sm_last) return;
+        __threadfence();
+    }
+    final_merge<T, D, G>(part_u, splits, out + qrow0 * D, false);
+}
+
+template <typename T, int D>
+void launch_attend_static(int G, dim3 grid, cudaStream_t st, const void* q, const void* K, const void* V, void* out, int n,
+                          int H, int Hkv, float* part, unsigned* ticket) {
+    switch (G) {
+        case 1: attend_static_kernel<T, D, 1><<<grid, kQueryThreads, 0, st>>>((const T*)q, (const T*)K, (const T*)V, (T*)out, n, H, Hkv, part, ticket); break;
+        case 2: attend_static_kernel<T, D, 2><<<grid, kQueryThreads, 0, st>>>((const T*)q, (const T*)K, (const T*)V, (T*)out, n, H, Hkv, part, ticket); break;
+        case 4: attend_static_kernel<T, D, 4><<<grid, kQueryThreads, 0, st>>>((const T*)q, (const T*)K, (const T*)V, (T*)out, n, H, Hkv, part, ticket); break;
+        default: attend_static_kernel<T, D, 8><<<grid, kQueryThreads, 0, st>>>((const T*)q, (const T*)K, (const T*)V, (T*)out, n, H, Hkv, part, ticket); break;
+    }
+}
+
+}  // namespace
+
+extern "C" int subgen_exact_attention_noalloc(const void* q, const void* K, const void* V, void* out, int B, int H, int Hkv,
+                                              int d, int n, int dtype, void* stream) {
+    if (Hkv == 0) Hkv = H;
+    if (!q || !K || !V || !out) return fail(SUBGEN_EINVAL, "subgen_exact_attention_noalloc: q, K, V, out must not be NULL");
+    if (B <= 0 || H <= 0 || Hkv <= 0 || H % Hkv || n <= 0 || (d != 64 && d != 128) ||
+        (dtype != SUBGEN_DTYPE_FP32 && dtype != SUBGEN_DTYPE_BF16) || (long long)B * Hkv > 65535)
+        return fail(SUBGEN_EINVAL, "subgen_exact_attention_noalloc: invalid shape or dtype");
+    const int G = H / Hkv;
+    if (G != 1 && G != 2 && G != 4 && G != 8) return fail(SUBGEN_EINVAL, "subgen_exact_attention_noalloc: H / Hkv must be 1, 2, 4 or 8");
+    if (((uintptr_t)q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)out) & 15)
+        return fail(SUBGEN_EINVAL, "subgen_exact_attention_noalloc: pointers must be 16-byte aligned");
+    const int U = B * Hkv;
+    // layout of the fixed array: [tickets: U unsigned, rounded up to 256 bytes][partials: U*splits*G*(d+2) floats]
+    const size_t ticket_bytes = align_up((size_t)U * sizeof(unsigned));
+    const size_t per_split = (size_t)U * G * (d + 2) * sizeof(float);
+    if (ticket_bytes + per_split > (size_t)SUBGEN_NOALLOC_SCRATCH_BYTES)
+        return fail(SUBGEN_EINVAL,
+                    "subgen_exact_attention_noalloc: B*Hkv=%d with H/Hkv=%d, d=%d needs %zu bytes of scratch, the fixed array has %zu",
+                    U, G, d, ticket_bytes + per_split, (size_t)SUBGEN_NOALLOC_SCRATCH_BYTES);
+    int splits = (148 * 8 + U - 1) / U;
+    splits = splits < 1 ? 1 : (splits > 32 ? 32 : splits);
+    const int by_rows = (n + 63) / 64;                      // no more blocks than 64-row pieces
+    if (splits > by_rows) splits = by_rows;
+    const size_t fit = ((size_t)SUBGEN_NOALLOC_SCRATCH_BYTES - ticket_bytes) / per_split;
+    if ((size_t)splits > fit) splits = (int)fit;
+
+    int dev = -1;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(SUBGEN_EINVAL, "subgen_exact_attention_noalloc: device index %d not supported", dev);
+    void* base = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (!g_static_ptr[dev]) {                           // first call on this device: resolve the array's device address
+            void* p = nullptr;
+            CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+            g_static_ptr[dev] = p;
+        }
+        base = g_static_ptr[dev];
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned* ticket = (unsigned*)base;
+    float* part = (float*)((char*)base + ticket_bytes);
+    CUDA_TRY(cudaMemsetAsync(ticket, 0, (size_t)U * sizeof(unsigned), st));   // the array keeps the last call's contents
+    const dim3 grid(splits, U);
+    const bool f32 = dtype == SUBGEN_DTYPE_FP32;
+    if (d == 64) {
+        if (f32) launch_attend_static<float, 64>(G, grid, st, q, K, V, out, n, H, Hkv, part, ticket);
+        else launch_attend_static<__nv_bfloat16, 64>(G, grid, st, q, K, V, out, n, H, Hkv, part, ticket);
+    } else {
+        if (f32) launch_attend_static<float, 128>(G, grid, st, q, K, V, out, n, H, Hkv, part, ticket);
+        else launch_attend_static<__nv_bfloat16, 128>(G, grid, st, q, K, V, out, n, H, Hkv, part, ticket);
+    }
+    CUDA_TRY(cudaGetLastError());
+    return SUBGEN_OK;
+}
