@@ -123,7 +123,7 @@ typedef struct subgen_state_view {
     uint64_t mu;       /* fixed-point sum of W over inserted tokens */
     int last_cluster;  /* cluster joined or opened by the most recent insertion, -1 if none yet */
     int last_opened;   /* 1 if that insertion opened a cluster */
-    uint64_t last_d2;  /* its D2 to the nearest earlier representative, UINT64_MAX if there was none */
+    uint64_t last_d2;  /* D2 to the representative it joined; not meaningful when it opened a cluster */
     /* caller-allocated HOST arrays, any may be NULL */
     int* counts;       /* [m_max]      n_i */
     int* centre_tok;   /* [m_max]      token index of representative x_i */

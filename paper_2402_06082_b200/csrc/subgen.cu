@@ -7,9 +7,12 @@
 #include <string.h>
 
 #include <string>
+#include <type_traits>
 #include <vector>
 
 #include "subgen_kernels.cuh"
+#include "subgen_query_mma.cuh"
+#include "subgen_insert_mma.cuh"
 
 using namespace sgk;
 
@@ -37,8 +40,8 @@ constexpr size_t kAlign = 256;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t X, S, cnt, ctok, stok, Mk, Mv, MW, Mtok, ringK, ringV;
-    size_t n_unit, m_unit, mu, status, last_cid, last_open, last_d2, part1, part2, ticket1, ticket2;
+    size_t X, S, xn, cnt, ctok, stok, Mk, Mv, MW, Mtok, ringK, ringV;
+    size_t n_unit, m_unit, mu, status, last_cid, last_open, last_d2, part1, part2, ticket1, ticket2, qnext;
     size_t stage_q, stage_k, stage_v, stage_out, cu, stats;
     size_t book_begin, book_end;   // bookkeeping region cleared at creation
     size_t total;
@@ -98,6 +101,7 @@ Layout make_layout(const Dims& d) {
     L.part2 = take(U * d.splits * d.G * (size_t)(d.D + 2) * sizeof(float));
     L.book_begin = off;
     L.cnt = take(U * d.m_max * sizeof(int));
+    L.xn = take(U * d.m_max * sizeof(float));
     L.n_unit = take(U * sizeof(int));
     L.m_unit = take(U * sizeof(int));
     L.mu = take(U * sizeof(uint64_t));
@@ -105,6 +109,7 @@ Layout make_layout(const Dims& d) {
     L.last_open = take(U * sizeof(int));
     L.ticket1 = take(U * sizeof(unsigned));
     L.ticket2 = take(U * sizeof(unsigned));
+    L.qnext = take(U * sizeof(unsigned));
     L.MW = take(U * d.s * sizeof(uint64_t));
     L.stats = take(8 * sizeof(uint64_t));
     L.book_end = off;
@@ -144,7 +149,7 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
     C.B = d.B; C.H = d.H; C.Hkv = d.Hkv; C.G = d.G; C.t = d.t; C.s = d.s; C.w = d.w; C.m_max = d.m_max;
     C.delta2_fx = (unsigned long long)floor((double)h->cfg.delta * (double)h->cfg.delta * 4294967296.0);
     C.key0 = (uint32_t)h->cfg.seed; C.key1 = (uint32_t)(h->cfg.seed >> 32);
-    C.X = (T*)(w + L.X); C.S = (T*)(w + L.S);
+    C.X = (T*)(w + L.X); C.S = (T*)(w + L.S); C.xn = (float*)(w + L.xn);
     C.cnt = (int*)(w + L.cnt); C.ctok = (int*)(w + L.ctok); C.stok = (int*)(w + L.stok);
     C.Mk = (T*)(w + L.Mk); C.Mv = (T*)(w + L.Mv);
     C.MW = (unsigned long long*)(w + L.MW); C.Mtok = (int*)(w + L.Mtok);
@@ -155,7 +160,28 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
     C.last_d2 = (unsigned long long*)(w + L.last_d2);
     C.part1 = (Best*)(w + L.part1); C.part2 = (float*)(w + L.part2);
     C.ticket1 = (unsigned*)(w + L.ticket1); C.ticket2 = (unsigned*)(w + L.ticket2);
+    C.qnext = (unsigned*)(w + L.qnext);
     return C;
+}
+
+// fp32 caches: CUDA-core dot products (full fp32 products). bf16 caches: tensor-core kernel.
+template <typename T, int D>
+void launch_query(const Cache<T>& C, int G, dim3 grid, cudaStream_t st, const void* q, void* out) {
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        switch (G) {
+            case 1: query_mma_kernel<D, 1><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
+            case 2: query_mma_kernel<D, 2><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
+            case 4: query_mma_kernel<D, 4><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
+            default: query_mma_kernel<D, 8><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
+        }
+    } else {
+        switch (G) {
+            case 1: query_kernel<T, D, 1><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
+            case 2: query_kernel<T, D, 2><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
+            case 4: query_kernel<T, D, 4><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
+            default: query_kernel<T, D, 8><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
+        }
+    }
 }
 
 template <typename T, int D>
@@ -175,14 +201,12 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
         h->ev_used += 3;
         CUDA_TRY(cudaEventRecord(e[0], h->st));
     }
-    insert_kernel<T, D><<<grid, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
+    if constexpr (std::is_same<T, __nv_bfloat16>::value)
+        insert_mma_kernel<D><<<grid, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
+    else
+        insert_kernel<T, D><<<grid, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
     if (e) CUDA_TRY(cudaEventRecord(e[1], h->st));
-    switch (h->d.G) {
-        case 1: query_kernel<T, D, 1><<<grid, kQueryThreads, 0, h->st>>>(C, (const T*)q, (T*)out); break;
-        case 2: query_kernel<T, D, 2><<<grid, kQueryThreads, 0, h->st>>>(C, (const T*)q, (T*)out); break;
-        case 4: query_kernel<T, D, 4><<<grid, kQueryThreads, 0, h->st>>>(C, (const T*)q, (T*)out); break;
-        default: query_kernel<T, D, 8><<<grid, kQueryThreads, 0, h->st>>>(C, (const T*)q, (T*)out); break;
-    }
+    launch_query<T, D>(C, h->d.G, grid, h->st, q, out);
     if (e) CUDA_TRY(cudaEventRecord(e[2], h->st));
     CUDA_TRY(cudaGetLastError());
     h->launches += 2;
@@ -264,6 +288,8 @@ subgen_t* subgen_create_ex(const subgen_config* cfg) {
     }
     cudaError_t e1 = cudaMemsetAsync(h->ws + h->L.book_begin, 0, h->L.book_end - h->L.book_begin, h->st);
     cudaError_t e2 = cudaMemsetAsync(h->ws + h->L.book_end, 0xFF, h->L.total - h->L.book_end, h->st);
+    // rows of M can be read (with weight zero) before their slot is filled: they must hold finite numbers
+    if (e1 == cudaSuccess) e1 = cudaMemsetAsync(h->ws + h->L.Mk, 0, h->L.ringK - h->L.Mk, h->st);
     if (e1 != cudaSuccess || e2 != cudaSuccess) {
         fail(SUBGEN_ECUDA, "subgen_create: cudaMemsetAsync failed: %s", cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
         if (h->owns) cudaFree(h->ws);

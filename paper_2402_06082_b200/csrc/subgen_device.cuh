@@ -85,6 +85,7 @@ template <typename T> struct Cache {
     uint32_t key0, key1;
     T* X;            // [U, m_max, D]     representatives x_i
     T* S;            // [U, m_max, t, D]  cluster samples S_i (materialised once n_i >= 2)
+    float* xn;       // [U, m_max]        ||x_i||^2 in fp32, used only to pre-filter distance candidates
     int* cnt;        // [U, m_max]        n_i
     int* ctok;       // [U, m_max]        token index of x_i
     int* stok;       // [U, m_max, t]     token index in S_i(j)
@@ -106,6 +107,7 @@ template <typename T> struct Cache {
     float* part2;    // [U, splits, G, D + 2]
     unsigned* ticket1;   // [U]
     unsigned* ticket2;   // [U]
+    unsigned* qnext;     // [U] next work item of the query kernel's per-unit queue
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -164,7 +166,7 @@ __device__ __forceinline__ Best block_best(Best b, Best* sm) {
 //   UpdateMatrixProduct: s coins with the OLD mu; then mu += W.
 template <typename T, int D>
 __device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, const uint4* krow, const uint4* vrow,
-                            unsigned long long* sm_w /* shared, 1 element */) {
+                            unsigned long long* sm_w /* shared, 2 elements */) {
     constexpr int EPL = Elem<T>::EPL, LPR = D / EPL;
     const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5;
     const int t = C.t, s = C.s;
@@ -172,6 +174,7 @@ __device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, c
     // W(v_e) and the input range check, by warp 0
     if (warp == 0) {
         unsigned long long acc = 0;
+        float kk = 0.f;
         bool bad = false;
         for (int p = lane; p < LPR; p += 32) {
             float vf[EPL], kf[EPL];
@@ -180,19 +183,24 @@ __device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, c
 #pragma unroll
             for (int j = 0; j < EPL; ++j) {
                 acc += fx_sq(vf[j]);
+                kk = fmaf(kf[j], kf[j], kk);
                 bad |= !(fabsf(vf[j]) <= kMaxAbsInput) || !(fabsf(kf[j]) <= kMaxAbsInput);
             }
         }
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        for (int off = 16; off > 0; off >>= 1) {
+            acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            kk += __shfl_xor_sync(0xffffffffu, kk, off);
+        }
         bad = __any_sync(0xffffffffu, bad);
         if (lane == 0) {
-            *sm_w = acc;
+            sm_w[0] = acc;
+            sm_w[1] = (unsigned long long)__float_as_uint(kk);
             if (bad) atomicOr(&C.status[u], 2);
         }
     }
     __syncthreads();
-    const unsigned long long W = *sm_w;
+    const unsigned long long W = sm_w[0];
     const unsigned long long mu_old = C.mu[u];
 
     const bool join = (m > 0) && (best.d2 <= C.delta2_fx);
@@ -225,7 +233,11 @@ __device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, c
         const int c = m;
         if (tid < LPR) reinterpret_cast<uint4*>(Xu + (size_t)c * D)[tid] = krow[tid];
         for (int j = tid; j < t; j += nt) stoku[(size_t)c * t + j] = e;
-        if (tid == 0) { cntu[c] = 1; C.ctok[(size_t)u * C.m_max + c] = e; }
+        if (tid == 0) {
+            cntu[c] = 1;
+            C.ctok[(size_t)u * C.m_max + c] = e;
+            C.xn[(size_t)u * C.m_max + c] = __uint_as_float((unsigned)sm_w[1]);
+        }
         m_new = m + 1;
     } else if (tid == 0) {
         atomicOr(&C.status[u], 1);
@@ -355,12 +367,36 @@ __device__ __forceinline__ void merge_scalar(float& mx, float& tau, float omx, f
     mx = m;
 }
 
+// Combine the per-warp partials [warp][G][D+2] = {mx, tau, z[D]} in shared memory into the block's
+// partial at dst (global). Starts with a __syncthreads().
+template <int D, int G>
+__device__ __forceinline__ void block_combine(const float* sm, float* dst) {
+    constexpr int STR = D + 2;
+    const int tid = threadIdx.x, nw = blockDim.x >> 5;
+    __syncthreads();
+    for (int o = tid; o < G * STR; o += blockDim.x) {
+        const int g = o / STR, c = o % STR;
+        float m = -INFINITY;
+        for (int w = 0; w < nw; ++w) m = fmaxf(m, sm[((size_t)w * G + g) * STR]);
+        float r;
+        if (c == 0) r = m;
+        else {
+            r = 0.f;
+            for (int w = 0; w < nw; ++w) {
+                const float wm = sm[((size_t)w * G + g) * STR];
+                if (wm != -INFINITY) r += sm[((size_t)w * G + g) * STR + c] * __expf(wm - m);
+            }
+        }
+        dst[(size_t)g * STR + c] = r;
+    }
+}
+
 // Block-level reduction of the row groups' accumulators and store of the block's partial
 // [G][D+2] = {mx, tau, z[D]} to dst. sm: shared floats, at least (blockDim/32) * G * (D+2).
 template <typename T, int D, int G>
 __device__ __forceinline__ void block_partial(Acc<G, Elem<T>::EPL>& A, float* sm, float* dst) {
     constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, STR = D + 2;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5, lr = lane % LPR;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, lr = lane % LPR;
 #pragma unroll
     for (int off = LPR; off < 32; off <<= 1) {
 #pragma unroll
@@ -385,22 +421,7 @@ __device__ __forceinline__ void block_partial(Acc<G, Elem<T>::EPL>& A, float* sm
             for (int j = 0; j < EPL; ++j) w[2 + lr * EPL + j] = A.z[g][j];
         }
     }
-    __syncthreads();
-    for (int o = tid; o < G * STR; o += blockDim.x) {
-        const int g = o / STR, c = o % STR;
-        float m = -INFINITY;
-        for (int w = 0; w < nw; ++w) m = fmaxf(m, sm[((size_t)w * G + g) * STR]);
-        float r;
-        if (c == 0) r = m;
-        else {
-            r = 0.f;
-            for (int w = 0; w < nw; ++w) {
-                const float wm = sm[((size_t)w * G + g) * STR];
-                if (wm != -INFINITY) r += sm[((size_t)w * G + g) * STR + c] * __expf(wm - m);
-            }
-        }
-        dst[(size_t)g * STR + c] = r;
-    }
+    block_combine<D, G>(sm, dst);
 }
 
 // Final merge of `np` block partials and the division z / tau, by a whole block.

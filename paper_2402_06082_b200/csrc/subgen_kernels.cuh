@@ -22,7 +22,7 @@ __global__ void __launch_bounds__(kInsertThreads) insert_kernel(Cache<T> C, cons
     constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, RPW = 32 / LPR;
     __shared__ uint4 krow[LPR], vrow[LPR];
     __shared__ Best smb[32];
-    __shared__ unsigned long long sm_w;
+    __shared__ unsigned long long sm_w[2];
     __shared__ int sm_last;
     const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, lr = lane % LPR, sub = lane / LPR;
@@ -72,7 +72,7 @@ __global__ void __launch_bounds__(kInsertThreads) insert_kernel(Cache<T> C, cons
     }
     if (tid < LPR) vrow[tid] = w ? ringv[tid] : vnew_u[tid];
     __syncthreads();
-    apply_insert<T, D>(C, u, e, b, m, krow, vrow, &sm_w);
+    apply_insert<T, D>(C, u, e, b, m, krow, vrow, sm_w);
     if (w) {
         if (tid < LPR) ringk[tid] = knew_u[tid];
         else if (tid < 2 * LPR) ringv[tid - LPR] = vnew_u[tid - LPR];
@@ -228,7 +228,7 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_seq_kernel(Cache<T> C
     constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, RPW = 32 / LPR;
     __shared__ uint4 krow[LPR], vrow[LPR];
     __shared__ Best smb[32];
-    __shared__ unsigned long long sm_w;
+    __shared__ unsigned long long sm_w[2];
     const int u = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, lr = lane % LPR, sub = lane / LPR;
     const int b = u / C.Hkv, h = u % C.Hkv, w = C.w;
@@ -250,7 +250,7 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_seq_kernel(Cache<T> C
         bst.d2 = ~0ull; bst.idx = INT_MAX; bst.pad = 0;
         scan_centres<T, D>(Xu, 0, m, kf, warp * RPW + sub, (nt >> 5) * RPW, lr, bst);
         bst = block_best(bst, smb);
-        m = apply_insert<T, D>(C, u, e, bst, m, krow, vrow, &sm_w);
+        m = apply_insert<T, D>(C, u, e, bst, m, krow, vrow, sm_w);
     }
     if (w) {
         const int lo = max(n_prev, n_tot - w);

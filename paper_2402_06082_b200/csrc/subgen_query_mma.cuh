@@ -1,0 +1,287 @@
+// Query kernel for bf16 caches with the dot products on the tensor cores.
+//
+// The stream step is bound by HBM: every cached row is read once and used for one dot product with q
+// (and one axpy into z). On CUDA cores the bf16->fp32 conversions, FMAs and lane reductions of those
+// dot products cost more issue slots per byte than the memory system needs time to deliver it, so here
+// both contractions run as warp-level m16n8k16 MMAs fed straight from 16-byte global loads:
+//
+//   scores S[16 rows][8 heads] = K_tile[16 x D] . q^T[D x 8]          (A = keys,   B = q)
+//   z^T   [16 cols][8 heads]  += V_tile^T[16 cols x 16 rows] . P[16 rows x 8 heads]   (A = values^T, B = P)
+//
+// The G <= 8 query heads of a KV head sit in the N dimension, so grouped-query attention costs no extra
+// instructions. A dot product does not depend on the order of its terms, which lets every lane take the
+// 8 consecutive elements of one 16-byte load as its k-slices (q is loaded with the same pattern); the
+// value tile needs rows paired inside a register, done with two byte permutes per register pair.
+// P (estimator weight times exp(score - max)) is rounded to bf16 for the second MMA; the partition
+// function tau is accumulated from the unrounded fp32 values; accumulation is fp32 throughout.
+//
+// Work of one unit is cut into items (16 clusters; 16 M slots; 16 window rows) handed out through a
+// per-unit atomic counter, so warps of all blocks of the unit stay busy until the unit is done. Nothing
+// spins: the counter only hands out indices.
+#pragma once
+#include "subgen_device.cuh"
+
+namespace sgk {
+
+constexpr int kQmThreads = 128;
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__device__ __forceinline__ uint4 ldg16(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+
+// Per-warp running state. Lane = 4*g + tq. The lane keeps the running maxima and partial partition
+// sums of heads 2tq and 2tq+1, and z^T accumulators acc[cc*4+j] = {z[2tq][c], z[2tq+1][c], z[2tq][c+1],
+// z[2tq+1][c+1]} with c = cc*64 + g*8 + 2j.
+template <int D> struct MmaState {
+    float m0, m1, tau0, tau1;
+    float acc[D / 16][4];
+};
+
+// Scores of one 16-row tile against q, then the online-softmax update of the running maxima.
+// pa / pb: this lane's key rows g and g+8 (valid memory even when the row is masked).
+// Returns p[4] = exp(score - max) for (row g, head 2tq), (g, 2tq+1), (g+8, 2tq), (g+8, 2tq+1); 0 if masked.
+template <int D>
+__device__ __forceinline__ void tile_scores(MmaState<D>& S, const __nv_bfloat16* pa, const __nv_bfloat16* pb, bool va,
+                                            bool vb, const uint32_t (&qb)[D / 32][4], int tq, float (&p)[4]) {
+    constexpr int NC = D / 32;
+    uint4 ka[NC], kb[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        ka[c] = ldg16(pa + c * 32 + tq * 8);
+        kb[c] = ldg16(pb + c * 32 + tq * 8);
+    }
+    float sc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        mma_bf16_16816(sc, ka[c].x, kb[c].x, ka[c].y, kb[c].y, qb[c][0], qb[c][1]);
+        mma_bf16_16816(sc, ka[c].z, kb[c].z, ka[c].w, kb[c].w, qb[c][2], qb[c][3]);
+    }
+    const float s0 = va ? sc[0] : -INFINITY, s1 = va ? sc[1] : -INFINITY;
+    const float s2 = vb ? sc[2] : -INFINITY, s3 = vb ? sc[3] : -INFINITY;
+    float t0 = fmaxf(s0, s2), t1 = fmaxf(s1, s3);
+#pragma unroll
+    for (int off = 4; off < 32; off <<= 1) {
+        t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, off));
+        t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, off));
+    }
+    const float n0 = fmaxf(S.m0, t0), n1 = fmaxf(S.m1, t1);
+    if (__any_sync(0xffffffffu, n0 != S.m0 || n1 != S.m1)) {
+        const float f0 = (S.m0 == -INFINITY) ? 0.f : __expf(S.m0 - n0);
+        const float f1 = (S.m1 == -INFINITY) ? 0.f : __expf(S.m1 - n1);
+        S.tau0 *= f0;
+        S.tau1 *= f1;
+#pragma unroll
+        for (int j = 0; j < D / 16; ++j) {
+            S.acc[j][0] *= f0; S.acc[j][2] *= f0;
+            S.acc[j][1] *= f1; S.acc[j][3] *= f1;
+        }
+        S.m0 = n0;
+        S.m1 = n1;
+    }
+    const float r0 = (n0 == -INFINITY) ? 0.f : n0, r1 = (n1 == -INFINITY) ? 0.f : n1;
+    p[0] = __expf(s0 - r0);
+    p[1] = __expf(s1 - r1);
+    p[2] = __expf(s2 - r0);
+    p[3] = __expf(s3 - r1);
+}
+
+// z^T += V_tile^T . P for one 16-row tile. pz[4]: weighted p in the layout tile_scores returns.
+// pv[i]: this lane's value rows 2tq, 2tq+1, 2tq+8, 2tq+9 of the tile (valid memory, finite contents).
+template <int D>
+__device__ __forceinline__ void tile_values(MmaState<D>& S, const float (&pz)[4], const __nv_bfloat16* const (&pv)[4],
+                                            int g, int tq) {
+    constexpr int NV = D / 64;
+    uint4 v[4][NV];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int cc = 0; cc < NV; ++cc) v[i][cc] = ldg16(pv[i] + cc * 64 + g * 8);
+    // B operand: P[rows 2tq, 2tq+1 | 2tq+8, 2tq+9][head g], gathered from the lanes that own those rows
+    const uint32_t p01 = pack_bf16x2(pz[0], pz[1]), p23 = pack_bf16x2(pz[2], pz[3]);
+    const int la = 8 * tq + (g >> 1), lb = la + 4;
+    const uint32_t a01 = __shfl_sync(0xffffffffu, p01, la), b01 = __shfl_sync(0xffffffffu, p01, lb);
+    const uint32_t a23 = __shfl_sync(0xffffffffu, p23, la), b23 = __shfl_sync(0xffffffffu, p23, lb);
+    const uint32_t sel = (g & 1) ? 0x7632u : 0x5410u;
+    const uint32_t B0 = __byte_perm(a01, b01, sel), B1 = __byte_perm(a23, b23, sel);
+#pragma unroll
+    for (int cc = 0; cc < NV; ++cc) {
+        const uint32_t r0[4] = {v[0][cc].x, v[0][cc].y, v[0][cc].z, v[0][cc].w};
+        const uint32_t r1[4] = {v[1][cc].x, v[1][cc].y, v[1][cc].z, v[1][cc].w};
+        const uint32_t r2[4] = {v[2][cc].x, v[2][cc].y, v[2][cc].z, v[2][cc].w};
+        const uint32_t r3[4] = {v[3][cc].x, v[3][cc].y, v[3][cc].z, v[3][cc].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            mma_bf16_16816(S.acc[cc * 4 + j], __byte_perm(r0[j], r1[j], 0x5410u), __byte_perm(r0[j], r1[j], 0x7632u),
+                           __byte_perm(r2[j], r3[j], 0x5410u), __byte_perm(r2[j], r3[j], 0x7632u), B0, B1);
+        }
+    }
+}
+
+template <int D, int G>
+__global__ void __launch_bounds__(kQmThreads, 4) query_mma_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ q,
+                                                                  __nv_bfloat16* __restrict__ out) {
+    typedef __nv_bfloat16 T;
+    constexpr int NC = D / 32, STR = D + 2, NW = kQmThreads / 32;
+    __shared__ float sm[NW * G * STR];
+    __shared__ int lst_s[NW][16], lst_m[NW][16], cnt_m[NW][16];
+    __shared__ int sm_last;
+    const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5, g = lane >> 2, tq = lane & 3;
+    const int b = u / C.Hkv, kvh = u % C.Hkv;
+    const int n = C.n_unit[u], w = C.w, t = C.t, s = C.s;
+    const int wn = min(n + 1, w), m = C.m_unit[u];
+    const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;
+
+    uint32_t qb[NC][4];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        uint4 r = make_uint4(0, 0, 0, 0);
+        if (g < G) r = ldg16(q + (qrow0 + g) * D + c * 32 + tq * 8);
+        qb[c][0] = r.x; qb[c][1] = r.y; qb[c][2] = r.z; qb[c][3] = r.w;
+    }
+    MmaState<D> S;
+    S.m0 = S.m1 = -INFINITY;
+    S.tau0 = S.tau1 = 0.f;
+#pragma unroll
+    for (int j = 0; j < D / 16; ++j) S.acc[j][0] = S.acc[j][1] = S.acc[j][2] = S.acc[j][3] = 0.f;
+
+    const T* Xu = C.X + (size_t)u * C.m_max * D;
+    const T* Su = C.S + (size_t)u * C.m_max * t * D;
+    const int* cntu = C.cnt + (size_t)u * C.m_max;
+    const T* Mku = C.Mk + (size_t)u * s * D;
+    const T* Mvu = C.Mv + (size_t)u * s * D;
+    const unsigned long long* MWu = C.MW + (size_t)u * s;
+    const T* Rk = C.ringK + (size_t)u * w * D;
+    const T* Rv = C.ringV + (size_t)u * w * D;
+    const float mu_over_s = (float)C.mu[u] / (float)s;
+    const float inv_t = 1.f / (float)t;
+
+    const int n_a = (m + 15) >> 4, n_b = (s + 15) >> 4, n_c = (wn + 15) >> 4, total = n_a + n_b + n_c;
+    int item = 0;
+    if (lane == 0) item = (int)atomicAdd(&C.qnext[u], 1u);
+    item = __shfl_sync(0xffffffffu, item, 0);
+    while (item < total) {
+        int next = 0;
+        if (lane == 0) next = (int)atomicAdd(&C.qnext[u], 1u);     // asked for early, needed late
+        if (item < n_a) {
+            // (a) 16 clusters: singletons are read as their representative (weight 1), the others as
+            //     their t samples (weight n'/t)
+            const int c = item * 16 + lane;
+            const int cn = (lane < 16 && c < m) ? cntu[c] : 0;
+            const unsigned ms = __ballot_sync(0xffffffffu, cn == 1), mm = __ballot_sync(0xffffffffu, cn > 1);
+            const unsigned lt = (1u << lane) - 1u;
+            __syncwarp();
+            if (cn == 1) lst_s[warp][__popc(ms & lt)] = c;
+            if (cn > 1) { const int r = __popc(mm & lt); lst_m[warp][r] = c; cnt_m[warp][r] = cn; }
+            __syncwarp();
+            const int ns = __popc(ms), rows_m = __popc(mm) * t;
+            float p[4];
+            if (ns > 0) {
+                const bool va = g < ns, vb = g + 8 < ns;
+                const T* pa = Xu + (size_t)lst_s[warp][va ? g : 0] * D;
+                const T* pb = Xu + (size_t)lst_s[warp][vb ? g + 8 : 0] * D;
+                tile_scores<D>(S, pa, pb, va, vb, qb, tq, p);
+                S.tau0 += p[0] + p[2];
+                S.tau1 += p[1] + p[3];
+            }
+            for (int r0 = 0; r0 < rows_m; r0 += 16) {
+                const int ra = r0 + g, rb = r0 + g + 8;
+                const bool va = ra < rows_m, vb = rb < rows_m;
+                const int ca = va ? ra / t : 0, cb = vb ? rb / t : 0;
+                const int ja = va ? ra - ca * t : 0, jb = vb ? rb - cb * t : 0;
+                const T* pa = Su + ((size_t)lst_m[warp][ca] * t + ja) * D;
+                const T* pb = Su + ((size_t)lst_m[warp][cb] * t + jb) * D;
+                tile_scores<D>(S, pa, pb, va, vb, qb, tq, p);
+                const float wa = (float)cnt_m[warp][ca] * inv_t, wb = (float)cnt_m[warp][cb] * inv_t;
+                S.tau0 += wa * p[0] + wb * p[2];
+                S.tau1 += wa * p[1] + wb * p[3];
+            }
+        } else {
+            // (b) 16 value samples (weight mu/(s W), numerator only) or (c) 16 window rows (weight 1, both sums)
+            const bool isM = item < n_a + n_b;
+            const int base = (isM ? item - n_a : item - n_a - n_b) * 16;
+            const int lim = isM ? s : wn;
+            const T* Kb = isM ? Mku : Rk;
+            const T* Vb = isM ? Mvu : Rv;
+            const int ia = min(base + g, lim - 1), ib = min(base + g + 8, lim - 1);
+            bool va = base + g < lim, vb = base + g + 8 < lim;
+            float wza = 1.f, wzb = 1.f;
+            if (isM) {
+                const unsigned long long Wa = MWu[ia], Wb = MWu[ib];
+                va = va && Wa != 0ull;
+                vb = vb && Wb != 0ull;
+                wza = va ? mu_over_s / (float)Wa : 0.f;
+                wzb = vb ? mu_over_s / (float)Wb : 0.f;
+            }
+            float p[4];
+            tile_scores<D>(S, Kb + (size_t)ia * D, Kb + (size_t)ib * D, va, vb, qb, tq, p);
+            if (!isM) {
+                S.tau0 += p[0] + p[2];
+                S.tau1 += p[1] + p[3];
+            }
+            const float pz[4] = {wza * p[0], wza * p[1], wzb * p[2], wzb * p[3]};
+            const T* pv[4];
+            pv[0] = Vb + (size_t)min(base + 2 * tq, lim - 1) * D;
+            pv[1] = Vb + (size_t)min(base + 2 * tq + 1, lim - 1) * D;
+            pv[2] = Vb + (size_t)min(base + 2 * tq + 8, lim - 1) * D;
+            pv[3] = Vb + (size_t)min(base + 2 * tq + 9, lim - 1) * D;
+            tile_values<D>(S, pz, pv, g, tq);
+        }
+        item = __shfl_sync(0xffffffffu, next, 0);
+    }
+
+    // warp partial -> shared [warp][G][D+2]
+#pragma unroll
+    for (int off = 4; off < 32; off <<= 1) {
+        S.tau0 += __shfl_xor_sync(0xffffffffu, S.tau0, off);
+        S.tau1 += __shfl_xor_sync(0xffffffffu, S.tau1, off);
+    }
+    {
+        const int h0 = 2 * tq, h1 = 2 * tq + 1;
+        float* w0 = sm + ((size_t)warp * G + (h0 < G ? h0 : 0)) * STR;
+        float* w1 = sm + ((size_t)warp * G + (h1 < G ? h1 : 0)) * STR;
+        if (g == 0) {
+            if (h0 < G) { w0[0] = S.m0; w0[1] = S.tau0; }
+            if (h1 < G) { w1[0] = S.m1; w1[1] = S.tau1; }
+        }
+#pragma unroll
+        for (int j = 0; j < D / 16; ++j) {
+            const int col = (j >> 2) * 64 + g * 8 + 2 * (j & 3);
+            if (h0 < G) { w0[2 + col] = S.acc[j][0]; w0[2 + col + 1] = S.acc[j][2]; }
+            if (h1 < G) { w1[2 + col] = S.acc[j][1]; w1[2 + col + 1] = S.acc[j][3]; }
+        }
+    }
+    float* part_u = C.part2 + (size_t)u * splits * G * STR;
+    block_combine<D, G>(sm, part_u + (size_t)blockIdx.x * G * STR);
+    __threadfence();
+    __syncthreads();
+    if (splits > 1) {
+        if (tid == 0) {
+            __threadfence();
+            sm_last = (atomicAdd(&C.ticket2[u], 1u) == (unsigned)splits - 1u);
+        }
+        __syncthreads();
+        if (!sm_last) return;
+        __threadfence();
+    }
+    final_merge<T, D, G>(part_u, splits, out + qrow0 * D, C.status[u] != 0);
+    if (tid == 0) {
+        C.n_unit[u] = n + 1;
+        C.ticket2[u] = 0;
+        C.qnext[u] = 0;
+    }
+}
+
+}  // namespace sgk

@@ -242,7 +242,16 @@ def test_step_host_matches_step():
         o1 = a.step(q, k, v)
         out = torch.empty(o1.shape, dtype=o1.dtype).pin_memory()
         b.step_host(q.cpu().pin_memory(), k.cpu().pin_memory(), v.cpu().pin_memory(), out)
-        assert torch.equal(o1.cpu(), out)
+        # same arithmetic, but the order in which partial sums meet depends on scheduling: compare to rounding
+        err = hp.rel_err(f32(o1).reshape(-1, w.d), f32(out).reshape(-1, w.d))
+        assert err <= 1e-2
+    for bb in range(w.B):
+        for h in range(w.Hkv):
+            s1, s2 = a.export_state(bb, h), b.export_state(bb, h)
+            for key in ("m", "mu", "n"):
+                assert s1[key] == s2[key]
+            for key in ("counts", "centre_tok", "slot_tok", "m_tok"):
+                np.testing.assert_array_equal(s1[key], s2[key])
 
 
 def test_cache_stats_and_profile():
