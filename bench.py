@@ -272,7 +272,7 @@ def run_subgen(args, w):
         dist.barrier()
     ms = e0.elapsed_time(e1)
     launches = sg.launch_count - launches0
-    ins_ms, qry_ms, nprof = sg.profile_read()
+    ins_ms, tau_ms, z_ms, nprof = sg.profile_read()
     sg.profile_enable(False)
     stats1 = sg.cache_stats()
     ms = sharding.max_over_ranks(ms, dist, dev)
@@ -303,19 +303,28 @@ def run_subgen(args, w):
 
     # ---- roofline of the dominant kernel (query_kernel) ----
     peak, which = measured_peaks()
-    qbytes = 0.5 * (stats0["query_bytes"] + stats1["query_bytes"])
-    ibytes = 0.5 * (stats0["insert_bytes"] + stats1["insert_bytes"])
-    q_ms = qry_ms / max(nprof, 1)
-    i_ms = ins_ms / max(nprof, 1)
-    achieved = qbytes / (q_ms * 1e-3) / 1e9 if q_ms > 0 else None
-    roofline = {"bound": "hbm", "kernel": "query_kernel", "achieved": achieved, "peak": peak, "peak_source": which,
+    def avg(key):
+        return 0.5 * (stats0[key] + stats1[key])
+
+    def gbs(nbytes, ms_):
+        return nbytes / (ms_ * 1e-3) / 1e9 if ms_ > 0 else None
+
+    cbytes, vbytes, ibytes = avg("cluster_bytes"), avg("value_bytes"), avg("insert_bytes")
+    c_ms, v_ms, i_ms = tau_ms / max(nprof, 1), z_ms / max(nprof, 1), ins_ms / max(nprof, 1)
+    if v_ms > 0:
+        dom = ("query_tau_kernel", cbytes, c_ms) if c_ms >= v_ms else ("query_z_kernel", vbytes, v_ms)
+    else:
+        dom = ("query_kernel", cbytes + vbytes, c_ms)
+    achieved = gbs(dom[1], dom[2])
+    roofline = {"bound": "hbm", "kernel": dom[0], "achieved": achieved, "peak": peak, "peak_source": which,
                 "unit": "GB/s", "frac": achieved / peak if achieved else None, "traffic": None,
-                "algorithmic_bytes_per_launch": qbytes, "ms_per_launch": q_ms,
-                "insert_kernel": {"algorithmic_bytes_per_launch": ibytes, "ms_per_launch": i_ms,
-                                  "achieved": ibytes / (i_ms * 1e-3) / 1e9 if i_ms > 0 else None},
-                "step": {"algorithmic_bytes": qbytes + ibytes,
-                         "achieved": (qbytes + ibytes) / (ms_per_step * 1e-3) / 1e9,
-                         "frac": (qbytes + ibytes) / (ms_per_step * 1e-3) / 1e9 / peak}}
+                "algorithmic_bytes_per_launch": dom[1], "ms_per_launch": dom[2],
+                "kernels": {"insert": {"algorithmic_bytes_per_launch": ibytes, "ms_per_launch": i_ms, "achieved": gbs(ibytes, i_ms)},
+                            "cluster_scan": {"algorithmic_bytes_per_launch": cbytes, "ms_per_launch": c_ms, "achieved": gbs(cbytes, c_ms)},
+                            "value_scan": {"algorithmic_bytes_per_launch": vbytes, "ms_per_launch": v_ms, "achieved": gbs(vbytes, v_ms)}},
+                "step": {"algorithmic_bytes": cbytes + vbytes + ibytes,
+                         "achieved": gbs(cbytes + vbytes + ibytes, ms_per_step),
+                         "frac": gbs(cbytes + vbytes + ibytes, ms_per_step) / peak}}
 
     extra = {"prefill_ms": prefill_ms, "prefill_tokens_per_s": sum(lens) / (prefill_ms * 1e-3),
              "prefill_launches": prefill_launches,

@@ -149,17 +149,21 @@ typedef struct subgen_stats {
     uint64_t window_rows;        /* tokens currently in the windows */
     uint64_t tokens;             /* sum of n */
     uint64_t insert_bytes;       /* bytes one step must read to place a key: the representatives */
-    uint64_t query_bytes;        /* bytes one step must read to answer the queries: samples, M, window */
+    uint64_t query_bytes;        /* bytes one step must read to answer the queries: cluster_bytes + value_bytes */
+    uint64_t cluster_bytes;      /* cluster samples (t rows, or the representative alone while n_i = 1) and counts */
+    uint64_t value_bytes;        /* M keys and values with their weights, window keys and values */
 } subgen_stats;
 
 /* Synchronous. Sums over all units, from the current state. */
 int subgen_cache_stats(subgen_t* h, subgen_stats* out);
 
 /* Kernel timing with CUDA events on the handle's stream. While enabled every subgen_step records
- * events around its two kernels; subgen_profile_read waits, adds up the elapsed times since the last
- * read and resets. */
+ * events around its kernels; subgen_profile_read waits, adds up the elapsed milliseconds since the last
+ * read and resets. ms[0]: insertion kernel (window push, nearest representative, updates); ms[1]: scan
+ * of the clusters (partition function); ms[2]: scan of M and the window plus the final merge. For fp32
+ * handles the whole query is one kernel, reported in ms[1], and ms[2] is 0. */
 int subgen_profile_enable(subgen_t* h, int on);
-int subgen_profile_read(subgen_t* h, double* insert_ms, double* query_ms, int* steps);
+int subgen_profile_read(subgen_t* h, double ms[3], int* steps);
 
 /* Number of kernels this handle has launched so far. */
 uint64_t subgen_launch_count(const subgen_t* h);

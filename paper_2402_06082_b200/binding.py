@@ -45,7 +45,7 @@ class StateView(C.Structure):
 
 class Stats(C.Structure):
     _fields_ = [(k, C.c_uint64) for k in ("units", "clusters", "singleton_clusters", "m_filled", "window_rows",
-                                           "tokens", "insert_bytes", "query_bytes")]
+                                           "tokens", "insert_bytes", "query_bytes", "cluster_bytes", "value_bytes")]
 
 
 _lib = None
@@ -78,7 +78,7 @@ def load():
     L.subgen_export_rows.argtypes = [vp, C.c_int, C.c_int, C.c_int, vp, C.c_size_t]
     L.subgen_cache_stats.argtypes = [vp, C.POINTER(Stats)]
     L.subgen_profile_enable.argtypes = [vp, C.c_int]
-    L.subgen_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), ip]
+    L.subgen_profile_read.argtypes = [vp, C.POINTER(C.c_double), ip]
     L.subgen_launch_count.argtypes = [vp]
     L.subgen_launch_count.restype = C.c_uint64
     L.subgen_last_error.restype = C.c_char_p
@@ -221,9 +221,10 @@ class SubGen:
         _check(self._L.subgen_profile_enable(self._h, int(on)))
 
     def profile_read(self):
-        a, b, n = C.c_double(), C.c_double(), C.c_int()
-        _check(self._L.subgen_profile_read(self._h, C.byref(a), C.byref(b), C.byref(n)))
-        return a.value, b.value, n.value
+        """(insert_ms, cluster_scan_ms, value_scan_ms, steps) accumulated since the last read."""
+        ms, n = (C.c_double * 3)(), C.c_int()
+        _check(self._L.subgen_profile_read(self._h, ms, C.byref(n)))
+        return ms[0], ms[1], ms[2], n.value
 
     @property
     def launch_count(self) -> int:

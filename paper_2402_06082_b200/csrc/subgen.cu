@@ -41,7 +41,7 @@ size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
     size_t X, S, xn, cnt, ctok, stok, Mk, Mv, MW, Mtok, ringK, ringV;
-    size_t n_unit, m_unit, mu, status, last_cid, last_open, last_d2, part1, part2, ticket1, ticket2, qnext;
+    size_t n_unit, m_unit, mu, status, last_cid, last_open, last_d2, part1, part2, ticket1, ticket2, qnext, qnext2, part_tau, MinvW;
     size_t stage_q, stage_k, stage_v, stage_out, cu, stats;
     size_t book_begin, book_end;   // bookkeeping region cleared at creation
     size_t total;
@@ -99,6 +99,7 @@ Layout make_layout(const Dims& d) {
     L.cu = take(((size_t)d.B + 1) * sizeof(int));
     L.part1 = take(U * d.splits * sizeof(Best));
     L.part2 = take(U * d.splits * d.G * (size_t)(d.D + 2) * sizeof(float));
+    L.part_tau = take(U * d.splits * d.G * 2 * sizeof(float));
     L.book_begin = off;
     L.cnt = take(U * d.m_max * sizeof(int));
     L.xn = take(U * d.m_max * sizeof(float));
@@ -110,6 +111,8 @@ Layout make_layout(const Dims& d) {
     L.ticket1 = take(U * sizeof(unsigned));
     L.ticket2 = take(U * sizeof(unsigned));
     L.qnext = take(U * sizeof(unsigned));
+    L.qnext2 = take(U * sizeof(unsigned));
+    L.MinvW = take(U * d.s * sizeof(float));
     L.MW = take(U * d.s * sizeof(uint64_t));
     L.stats = take(8 * sizeof(uint64_t));
     L.book_end = off;
@@ -135,7 +138,7 @@ struct subgen {
     std::vector<int> n_host;     // tokens seen per sequence (mirror of the device counters)
     uint64_t launches = 0;
     bool prof = false;
-    std::vector<cudaEvent_t> ev;  // three per profiled step
+    std::vector<cudaEvent_t> ev;  // four per profiled step
     size_t ev_used = 0;
 };
 
@@ -160,19 +163,28 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
     C.last_d2 = (unsigned long long*)(w + L.last_d2);
     C.part1 = (Best*)(w + L.part1); C.part2 = (float*)(w + L.part2);
     C.ticket1 = (unsigned*)(w + L.ticket1); C.ticket2 = (unsigned*)(w + L.ticket2);
-    C.qnext = (unsigned*)(w + L.qnext);
+    C.qnext = (unsigned*)(w + L.qnext); C.qnext2 = (unsigned*)(w + L.qnext2);
+    C.part_tau = (float*)(w + L.part_tau); C.MinvW = (float*)(w + L.MinvW);
     return C;
 }
 
 // fp32 caches: CUDA-core dot products (full fp32 products). bf16 caches: tensor-core kernel.
 template <typename T, int D>
-void launch_query(const Cache<T>& C, int G, dim3 grid, cudaStream_t st, const void* q, void* out) {
+void launch_query(const Cache<T>& C, int G, dim3 grid, cudaStream_t st, const void* q, void* out, cudaEvent_t mid) {
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
         switch (G) {
-            case 1: query_mma_kernel<D, 1><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
-            case 2: query_mma_kernel<D, 2><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
-            case 4: query_mma_kernel<D, 4><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
-            default: query_mma_kernel<D, 8><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
+            case 1: query_tau_kernel<D, 1><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
+                    if (mid) cudaEventRecord(mid, st);
+                    query_z_kernel<D, 1><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
+            case 2: query_tau_kernel<D, 2><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
+                    if (mid) cudaEventRecord(mid, st);
+                    query_z_kernel<D, 2><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
+            case 4: query_tau_kernel<D, 4><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
+                    if (mid) cudaEventRecord(mid, st);
+                    query_z_kernel<D, 4><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
+            default: query_tau_kernel<D, 8><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
+                    if (mid) cudaEventRecord(mid, st);
+                     query_z_kernel<D, 8><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
         }
     } else {
         switch (G) {
@@ -181,6 +193,7 @@ void launch_query(const Cache<T>& C, int G, dim3 grid, cudaStream_t st, const vo
             case 4: query_kernel<T, D, 4><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
             default: query_kernel<T, D, 8><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
         }
+        if (mid) cudaEventRecord(mid, st);
     }
 }
 
@@ -190,15 +203,15 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
     const dim3 grid(h->d.splits, h->d.U);
     cudaEvent_t* e = nullptr;
     if (h->prof) {
-        if (h->ev_used + 3 > h->ev.size()) {
-            for (int i = 0; i < 3; ++i) {
+        if (h->ev_used + 4 > h->ev.size()) {
+            for (int i = 0; i < 4; ++i) {
                 cudaEvent_t x;
                 CUDA_TRY(cudaEventCreate(&x));
                 h->ev.push_back(x);
             }
         }
         e = &h->ev[h->ev_used];
-        h->ev_used += 3;
+        h->ev_used += 4;
         CUDA_TRY(cudaEventRecord(e[0], h->st));
     }
     if constexpr (std::is_same<T, __nv_bfloat16>::value)
@@ -206,10 +219,10 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
     else
         insert_kernel<T, D><<<grid, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
     if (e) CUDA_TRY(cudaEventRecord(e[1], h->st));
-    launch_query<T, D>(C, h->d.G, grid, h->st, q, out);
-    if (e) CUDA_TRY(cudaEventRecord(e[2], h->st));
+    launch_query<T, D>(C, h->d.G, grid, h->st, q, out, e ? e[2] : nullptr);
+    if (e) CUDA_TRY(cudaEventRecord(e[3], h->st));
     CUDA_TRY(cudaGetLastError());
-    h->launches += 2;
+    h->launches += std::is_same<T, __nv_bfloat16>::value ? 3 : 2;
     return SUBGEN_OK;
 }
 
@@ -452,7 +465,9 @@ int subgen_cache_stats(subgen_t* h, subgen_stats* out) {
     out->units = h->d.U;
     out->clusters = r[0]; out->singleton_clusters = r[1]; out->m_filled = r[2]; out->window_rows = r[3]; out->tokens = r[4];
     out->insert_bytes = r[0] * row;
-    out->query_bytes = (r[1] + (r[0] - r[1]) * (uint64_t)h->d.t + 2 * r[2] + 2 * r[3]) * row + r[0] * 4 + (uint64_t)h->d.U * h->d.s * 8;
+    out->cluster_bytes = (r[1] + (r[0] - r[1]) * (uint64_t)h->d.t) * row + r[0] * 4;
+    out->value_bytes = (2 * r[2] + 2 * r[3]) * row + (uint64_t)h->d.U * h->d.s * 4;
+    out->query_bytes = out->cluster_bytes + out->value_bytes;
     return SUBGEN_OK;
 }
 
@@ -462,19 +477,19 @@ int subgen_profile_enable(subgen_t* h, int on) {
     return SUBGEN_OK;
 }
 
-int subgen_profile_read(subgen_t* h, double* insert_ms, double* query_ms, int* steps) {
+int subgen_profile_read(subgen_t* h, double* ms, int* steps) {
     if (!h) return fail(SUBGEN_EINVAL, "subgen_profile_read: handle is NULL");
     CUDA_TRY(cudaStreamSynchronize(h->st));
-    double a = 0, b = 0;
-    for (size_t i = 0; i + 3 <= h->ev_used; i += 3) {
-        float x = 0, y = 0;
-        CUDA_TRY(cudaEventElapsedTime(&x, h->ev[i], h->ev[i + 1]));
-        CUDA_TRY(cudaEventElapsedTime(&y, h->ev[i + 1], h->ev[i + 2]));
-        a += x; b += y;
+    double acc[3] = {0, 0, 0};
+    for (size_t i = 0; i + 4 <= h->ev_used; i += 4) {
+        for (int k = 0; k < 3; ++k) {
+            float x = 0;
+            CUDA_TRY(cudaEventElapsedTime(&x, h->ev[i + k], h->ev[i + k + 1]));
+            acc[k] += x;
+        }
     }
-    if (insert_ms) *insert_ms = a;
-    if (query_ms) *query_ms = b;
-    if (steps) *steps = (int)(h->ev_used / 3);
+    if (ms) { ms[0] = acc[0]; ms[1] = acc[1]; ms[2] = acc[2]; }
+    if (steps) *steps = (int)(h->ev_used / 4);
     h->ev_used = 0;
     return SUBGEN_OK;
 }

@@ -93,6 +93,7 @@ template <typename T> struct Cache {
     T* Mv;           // [U, s, D]
     unsigned long long* MW;    // [U, s]  W of the sampled token, 0 = null
     int* Mtok;       // [U, s]
+    float* MinvW;    // [U, s]            1/W in fp32 (0 = null), the query's estimator weight is mu/s times this
     T* ringK;        // [U, w, D]         token j in row j % w
     T* ringV;
     int* n_unit;     // [U] tokens seen
@@ -107,7 +108,9 @@ template <typename T> struct Cache {
     float* part2;    // [U, splits, G, D + 2]
     unsigned* ticket1;   // [U]
     unsigned* ticket2;   // [U]
-    unsigned* qnext;     // [U] next work item of the query kernel's per-unit queue
+    float* part_tau;     // [U, splits, G, 2] cluster partials {max, tau} of the query
+    unsigned* qnext;     // [U] next work item of the cluster scan's per-unit queue
+    unsigned* qnext2;    // [U] same for the scan of M and the window
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -259,6 +262,7 @@ __device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, c
                     uint4* dv = reinterpret_cast<uint4*>(Mvu + (size_t)i * D);
                     for (int p = 0; p < LPR; ++p) { dk[p] = krow[p]; dv[p] = vrow[p]; }
                     C.MW[(size_t)u * s + i] = W;
+                    C.MinvW[(size_t)u * s + i] = 1.f / (float)W;
                     C.Mtok[(size_t)u * s + i] = e;
                 }
             }

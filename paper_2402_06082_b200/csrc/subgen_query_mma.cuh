@@ -15,6 +15,11 @@
 // P (estimator weight times exp(score - max)) is rounded to bf16 for the second MMA; the partition
 // function tau is accumulated from the unrounded fp32 values; accumulation is fp32 throughout.
 //
+// The query runs as two kernels so that each keeps only the registers it needs and many warps stay
+// resident: query_tau_kernel scans the clusters (keys only, partition function), query_z_kernel scans the
+// value samples M and the window (keys and values, numerator and the window's share of tau) and its last
+// block merges everything into out = z / tau.
+//
 // Work of one unit is cut into items (16 clusters; 16 M slots; 16 window rows) handed out through a
 // per-unit atomic counter, so warps of all blocks of the unit stay busy until the unit is done. Nothing
 // spins: the counter only hands out indices.
@@ -52,8 +57,8 @@ template <int D> struct MmaState {
 // Scores of one 16-row tile against q, then the online-softmax update of the running maxima.
 // pa / pb: this lane's key rows g and g+8 (valid memory even when the row is masked).
 // Returns p[4] = exp(score - max) for (row g, head 2tq), (g, 2tq+1), (g+8, 2tq), (g+8, 2tq+1); 0 if masked.
-template <int D>
-__device__ __forceinline__ void tile_scores(MmaState<D>& S, const __nv_bfloat16* pa, const __nv_bfloat16* pb, bool va,
+template <int D, int DA>
+__device__ __forceinline__ void tile_scores(MmaState<DA>& S, const __nv_bfloat16* pa, const __nv_bfloat16* pb, bool va,
                                             bool vb, const uint32_t (&qb)[D / 32][4], int tq, float (&p)[4]) {
     constexpr int NC = D / 32;
     uint4 ka[NC], kb[NC];
@@ -83,9 +88,12 @@ __device__ __forceinline__ void tile_scores(MmaState<D>& S, const __nv_bfloat16*
         S.tau0 *= f0;
         S.tau1 *= f1;
 #pragma unroll
-        for (int j = 0; j < D / 16; ++j) {
-            S.acc[j][0] *= f0; S.acc[j][2] *= f0;
-            S.acc[j][1] *= f1; S.acc[j][3] *= f1;
+        if (DA == D) {                 // DA != D: caller keeps no numerator accumulators
+#pragma unroll
+            for (int j = 0; j < DA / 16; ++j) {
+                S.acc[j][0] *= f0; S.acc[j][2] *= f0;
+                S.acc[j][1] *= f1; S.acc[j][3] *= f1;
+            }
         }
         S.m0 = n0;
         S.m1 = n1;
@@ -129,19 +137,123 @@ __device__ __forceinline__ void tile_values(MmaState<D>& S, const float (&pz)[4]
     }
 }
 
+// floor(r / t) for small r by one multiply-high (t = 1 handled by the caller's magic = 0)
+__device__ __forceinline__ int div_small(int r, unsigned magic) { return magic ? (int)__umulhi((unsigned)r, magic) : r; }
+
+// ---------------------------------------------------------------------------------------------
+// Clusters: tau_D = sum over clusters of n'/t sum over the t samples of exp<q,k>; a cluster with n' = 1
+// is read as its representative with weight 1. Writes per block {max, tau} per head to part_tau.
 template <int D, int G>
-__global__ void __launch_bounds__(kQmThreads, 4) query_mma_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ q,
-                                                                  __nv_bfloat16* __restrict__ out) {
+__global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ q) {
+    typedef __nv_bfloat16 T;
+    constexpr int NC = D / 32, NW = kQmThreads / 32;
+    __shared__ float sm[NW][G][2];
+    __shared__ int lst[NW][16], wcn[NW][16];
+    const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5, g = lane >> 2, tq = lane & 3;
+    const int b = u / C.Hkv, kvh = u % C.Hkv;
+    const int t = C.t, m = C.m_unit[u];
+    const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;
+
+    uint32_t qb[NC][4];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        uint4 r = make_uint4(0, 0, 0, 0);
+        if (g < G) r = ldg16(q + (qrow0 + g) * D + c * 32 + tq * 8);
+        qb[c][0] = r.x; qb[c][1] = r.y; qb[c][2] = r.z; qb[c][3] = r.w;
+    }
+    MmaState<16> S;                       // the accumulators stay untouched here and cost no registers
+    S.m0 = S.m1 = -INFINITY;
+    S.tau0 = S.tau1 = 0.f;
+    S.acc[0][0] = S.acc[0][1] = S.acc[0][2] = S.acc[0][3] = 0.f;
+
+    const T* Xu = C.X + (size_t)u * C.m_max * D;
+    const T* Su = C.S + (size_t)u * C.m_max * t * D;
+    const int* cntu = C.cnt + (size_t)u * C.m_max;
+    const float inv_t = 1.f / (float)t;
+    const unsigned magic = t > 1 ? (unsigned)(4294967296ull / (unsigned)t) + 1u : 0u;
+    const int total = (m + 15) >> 4;
+    int item = 0;
+    if (lane == 0) item = (int)atomicAdd(&C.qnext[u], 1u);
+    item = __shfl_sync(0xffffffffu, item, 0);
+    while (item < total) {
+        int next = 0;
+        if (lane == 0) next = (int)atomicAdd(&C.qnext[u], 1u);     // asked for early, needed late
+        // 16 clusters -> one list of rows: first the t samples of every cluster with n' > 1, then the
+        // representatives of the singletons
+        const int c = item * 16 + lane;
+        const int cn = (lane < 16 && c < m) ? cntu[c] : 0;
+        const unsigned ms = __ballot_sync(0xffffffffu, cn == 1), mm = __ballot_sync(0xffffffffu, cn > 1);
+        const unsigned lt = (1u << lane) - 1u;
+        const int nm = __popc(mm), ns = __popc(ms);
+        __syncwarp();
+        if (cn > 1) { const int r = __popc(mm & lt); lst[warp][r] = c; wcn[warp][r] = cn; }
+        if (cn == 1) lst[warp][nm + __popc(ms & lt)] = c;
+        __syncwarp();
+        const int rows_m = nm * t, rows = rows_m + ns;
+        for (int r0 = 0; r0 < rows; r0 += 16) {
+            const int ra = r0 + g, rb = r0 + g + 8;
+            const bool va = ra < rows, vb = rb < rows;
+            const T *pa = Xu, *pb = Xu;
+            float wa = 1.f, wb = 1.f;
+            if (ra < rows_m) {
+                const int ci = div_small(ra, magic);
+                pa = Su + ((size_t)lst[warp][ci] * t + (ra - ci * t)) * D;
+                wa = (float)wcn[warp][ci] * inv_t;
+            } else if (va) {
+                pa = Xu + (size_t)lst[warp][nm + ra - rows_m] * D;
+            }
+            if (rb < rows_m) {
+                const int ci = div_small(rb, magic);
+                pb = Su + ((size_t)lst[warp][ci] * t + (rb - ci * t)) * D;
+                wb = (float)wcn[warp][ci] * inv_t;
+            } else if (vb) {
+                pb = Xu + (size_t)lst[warp][nm + rb - rows_m] * D;
+            }
+            float p[4];
+            tile_scores<D, 16>(S, pa, pb, va, vb, qb, tq, p);
+            S.tau0 += wa * p[0] + wb * p[2];
+            S.tau1 += wa * p[1] + wb * p[3];
+        }
+        item = __shfl_sync(0xffffffffu, next, 0);
+    }
+#pragma unroll
+    for (int off = 4; off < 32; off <<= 1) {
+        S.tau0 += __shfl_xor_sync(0xffffffffu, S.tau0, off);
+        S.tau1 += __shfl_xor_sync(0xffffffffu, S.tau1, off);
+    }
+    if (g == 0) {
+        if (2 * tq < G) { sm[warp][2 * tq][0] = S.m0; sm[warp][2 * tq][1] = S.tau0; }
+        if (2 * tq + 1 < G) { sm[warp][2 * tq + 1][0] = S.m1; sm[warp][2 * tq + 1][1] = S.tau1; }
+    }
+    __syncthreads();
+    if (tid < G) {
+        float mx = -INFINITY, tau = 0.f;
+        for (int wv = 0; wv < NW; ++wv) mx = fmaxf(mx, sm[wv][tid][0]);
+        for (int wv = 0; wv < NW; ++wv)
+            if (sm[wv][tid][0] != -INFINITY) tau += sm[wv][tid][1] * __expf(sm[wv][tid][0] - mx);
+        float* dst = C.part_tau + (((size_t)u * splits + blockIdx.x) * G + tid) * 2;
+        dst[0] = mx;
+        dst[1] = tau;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Value samples and window: z = sum_M mu/(s W) exp<q,k> v + sum_window exp<q,k> v, tau_window. The block
+// that finishes last merges its siblings' partials with the cluster partials of query_tau_kernel, writes
+// out = z / tau and advances the unit's token count.
+template <int D, int G>
+__global__ void __launch_bounds__(kQmThreads, 4) query_z_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ q,
+                                                                __nv_bfloat16* __restrict__ out, int splits_tau) {
     typedef __nv_bfloat16 T;
     constexpr int NC = D / 32, STR = D + 2, NW = kQmThreads / 32;
     __shared__ float sm[NW * G * STR];
-    __shared__ int lst_s[NW][16], lst_m[NW][16], cnt_m[NW][16];
     __shared__ int sm_last;
     const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5, g = lane >> 2, tq = lane & 3;
     const int b = u / C.Hkv, kvh = u % C.Hkv;
-    const int n = C.n_unit[u], w = C.w, t = C.t, s = C.s;
-    const int wn = min(n + 1, w), m = C.m_unit[u];
+    const int n = C.n_unit[u], w = C.w, s = C.s;
+    const int wn = min(n + 1, w);
     const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;
 
     uint32_t qb[NC][4];
@@ -157,88 +269,48 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_mma_kernel(Cache<__nv_bfl
 #pragma unroll
     for (int j = 0; j < D / 16; ++j) S.acc[j][0] = S.acc[j][1] = S.acc[j][2] = S.acc[j][3] = 0.f;
 
-    const T* Xu = C.X + (size_t)u * C.m_max * D;
-    const T* Su = C.S + (size_t)u * C.m_max * t * D;
-    const int* cntu = C.cnt + (size_t)u * C.m_max;
     const T* Mku = C.Mk + (size_t)u * s * D;
     const T* Mvu = C.Mv + (size_t)u * s * D;
-    const unsigned long long* MWu = C.MW + (size_t)u * s;
+    const float* MiWu = C.MinvW + (size_t)u * s;
     const T* Rk = C.ringK + (size_t)u * w * D;
     const T* Rv = C.ringV + (size_t)u * w * D;
     const float mu_over_s = (float)C.mu[u] / (float)s;
-    const float inv_t = 1.f / (float)t;
-
-    const int n_a = (m + 15) >> 4, n_b = (s + 15) >> 4, n_c = (wn + 15) >> 4, total = n_a + n_b + n_c;
+    const int n_b = (s + 15) >> 4, n_c = (wn + 15) >> 4, total = n_b + n_c;
     int item = 0;
-    if (lane == 0) item = (int)atomicAdd(&C.qnext[u], 1u);
+    if (lane == 0) item = (int)atomicAdd(&C.qnext2[u], 1u);
     item = __shfl_sync(0xffffffffu, item, 0);
     while (item < total) {
         int next = 0;
-        if (lane == 0) next = (int)atomicAdd(&C.qnext[u], 1u);     // asked for early, needed late
-        if (item < n_a) {
-            // (a) 16 clusters: singletons are read as their representative (weight 1), the others as
-            //     their t samples (weight n'/t)
-            const int c = item * 16 + lane;
-            const int cn = (lane < 16 && c < m) ? cntu[c] : 0;
-            const unsigned ms = __ballot_sync(0xffffffffu, cn == 1), mm = __ballot_sync(0xffffffffu, cn > 1);
-            const unsigned lt = (1u << lane) - 1u;
-            __syncwarp();
-            if (cn == 1) lst_s[warp][__popc(ms & lt)] = c;
-            if (cn > 1) { const int r = __popc(mm & lt); lst_m[warp][r] = c; cnt_m[warp][r] = cn; }
-            __syncwarp();
-            const int ns = __popc(ms), rows_m = __popc(mm) * t;
-            float p[4];
-            if (ns > 0) {
-                const bool va = g < ns, vb = g + 8 < ns;
-                const T* pa = Xu + (size_t)lst_s[warp][va ? g : 0] * D;
-                const T* pb = Xu + (size_t)lst_s[warp][vb ? g + 8 : 0] * D;
-                tile_scores<D>(S, pa, pb, va, vb, qb, tq, p);
-                S.tau0 += p[0] + p[2];
-                S.tau1 += p[1] + p[3];
-            }
-            for (int r0 = 0; r0 < rows_m; r0 += 16) {
-                const int ra = r0 + g, rb = r0 + g + 8;
-                const bool va = ra < rows_m, vb = rb < rows_m;
-                const int ca = va ? ra / t : 0, cb = vb ? rb / t : 0;
-                const int ja = va ? ra - ca * t : 0, jb = vb ? rb - cb * t : 0;
-                const T* pa = Su + ((size_t)lst_m[warp][ca] * t + ja) * D;
-                const T* pb = Su + ((size_t)lst_m[warp][cb] * t + jb) * D;
-                tile_scores<D>(S, pa, pb, va, vb, qb, tq, p);
-                const float wa = (float)cnt_m[warp][ca] * inv_t, wb = (float)cnt_m[warp][cb] * inv_t;
-                S.tau0 += wa * p[0] + wb * p[2];
-                S.tau1 += wa * p[1] + wb * p[3];
-            }
-        } else {
-            // (b) 16 value samples (weight mu/(s W), numerator only) or (c) 16 window rows (weight 1, both sums)
-            const bool isM = item < n_a + n_b;
-            const int base = (isM ? item - n_a : item - n_a - n_b) * 16;
-            const int lim = isM ? s : wn;
-            const T* Kb = isM ? Mku : Rk;
-            const T* Vb = isM ? Mvu : Rv;
-            const int ia = min(base + g, lim - 1), ib = min(base + g + 8, lim - 1);
-            bool va = base + g < lim, vb = base + g + 8 < lim;
-            float wza = 1.f, wzb = 1.f;
-            if (isM) {
-                const unsigned long long Wa = MWu[ia], Wb = MWu[ib];
-                va = va && Wa != 0ull;
-                vb = vb && Wb != 0ull;
-                wza = va ? mu_over_s / (float)Wa : 0.f;
-                wzb = vb ? mu_over_s / (float)Wb : 0.f;
-            }
-            float p[4];
-            tile_scores<D>(S, Kb + (size_t)ia * D, Kb + (size_t)ib * D, va, vb, qb, tq, p);
-            if (!isM) {
-                S.tau0 += p[0] + p[2];
-                S.tau1 += p[1] + p[3];
-            }
-            const float pz[4] = {wza * p[0], wza * p[1], wzb * p[2], wzb * p[3]};
-            const T* pv[4];
-            pv[0] = Vb + (size_t)min(base + 2 * tq, lim - 1) * D;
-            pv[1] = Vb + (size_t)min(base + 2 * tq + 1, lim - 1) * D;
-            pv[2] = Vb + (size_t)min(base + 2 * tq + 8, lim - 1) * D;
-            pv[3] = Vb + (size_t)min(base + 2 * tq + 9, lim - 1) * D;
-            tile_values<D>(S, pz, pv, g, tq);
+        if (lane == 0) next = (int)atomicAdd(&C.qnext2[u], 1u);
+        // 16 value samples (weight mu/(s W), numerator only) or 16 window rows (weight 1, both sums)
+        const bool isM = item < n_b;
+        const int base = (isM ? item : item - n_b) * 16;
+        const int lim = isM ? s : wn;
+        const T* Kb = isM ? Mku : Rk;
+        const T* Vb = isM ? Mvu : Rv;
+        const int ia = min(base + g, lim - 1), ib = min(base + g + 8, lim - 1);
+        bool va = base + g < lim, vb = base + g + 8 < lim;
+        float wza = 1.f, wzb = 1.f;
+        if (isM) {
+            const float ia_w = MiWu[ia], ib_w = MiWu[ib];          // 1/W, 0 for a null slot
+            va = va && ia_w != 0.f;
+            vb = vb && ib_w != 0.f;
+            wza = va ? mu_over_s * ia_w : 0.f;
+            wzb = vb ? mu_over_s * ib_w : 0.f;
         }
+        float p[4];
+        tile_scores<D, D>(S, Kb + (size_t)ia * D, Kb + (size_t)ib * D, va, vb, qb, tq, p);
+        if (!isM) {
+            S.tau0 += p[0] + p[2];
+            S.tau1 += p[1] + p[3];
+        }
+        const float pz[4] = {wza * p[0], wza * p[1], wzb * p[2], wzb * p[3]};
+        const T* pv[4];
+        pv[0] = Vb + (size_t)min(base + 2 * tq, lim - 1) * D;
+        pv[1] = Vb + (size_t)min(base + 2 * tq + 1, lim - 1) * D;
+        pv[2] = Vb + (size_t)min(base + 2 * tq + 8, lim - 1) * D;
+        pv[3] = Vb + (size_t)min(base + 2 * tq + 9, lim - 1) * D;
+        tile_values<D>(S, pz, pv, g, tq);
         item = __shfl_sync(0xffffffffu, next, 0);
     }
 
@@ -276,11 +348,38 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_mma_kernel(Cache<__nv_bfl
         if (!sm_last) return;
         __threadfence();
     }
-    final_merge<T, D, G>(part_u, splits, out + qrow0 * D, C.status[u] != 0);
+    // final merge: z partials of this kernel and the cluster partials {max, tau} of query_tau_kernel
+    const float* part_t = C.part_tau + (size_t)u * splits_tau * G * 2;
+    const bool poisoned = C.status[u] != 0;
+    for (int o = tid; o < G * D; o += blockDim.x) {
+        const int hh = o / D, c = o % D;
+        float mx = -INFINITY;
+        for (int i = 0; i < splits; ++i) mx = fmaxf(mx, __ldcg(part_u + ((size_t)i * G + hh) * STR));
+        for (int i = 0; i < splits_tau; ++i) mx = fmaxf(mx, __ldcg(part_t + ((size_t)i * G + hh) * 2));
+        float z = 0.f, tau = 0.f;
+        for (int i = 0; i < splits; ++i) {
+            const float* pp = part_u + ((size_t)i * G + hh) * STR;
+            const float pm = __ldcg(pp);
+            if (pm != -INFINITY) {
+                const float sc = __expf(pm - mx);
+                tau += __ldcg(pp + 1) * sc;
+                z += __ldcg(pp + 2 + c) * sc;
+            }
+        }
+        for (int i = 0; i < splits_tau; ++i) {
+            const float* pp = part_t + ((size_t)i * G + hh) * 2;
+            const float pm = __ldcg(pp);
+            if (pm != -INFINITY) tau += __ldcg(pp + 1) * __expf(pm - mx);
+        }
+        float r = tau > 0.f ? z / tau : 0.f;
+        if (poisoned) r = __int_as_float(0x7fc00000);
+        out[(qrow0 + hh) * D + c] = __float2bfloat16_rn(r);
+    }
     if (tid == 0) {
         C.n_unit[u] = n + 1;
         C.ticket2[u] = 0;
         C.qnext[u] = 0;
+        C.qnext2[u] = 0;
     }
 }
 

@@ -265,14 +265,17 @@ def test_cache_stats_and_profile():
     row = w.d * 2
     assert st["insert_bytes"] == st["clusters"] * row
     rows = st["singleton_clusters"] + (st["clusters"] - st["singleton_clusters"]) * w.t + 2 * st["m_filled"] + 2 * 64
-    assert st["query_bytes"] == rows * row + st["clusters"] * 4 + 2 * w.s * 8
+    crow = st["singleton_clusters"] + (st["clusters"] - st["singleton_clusters"]) * w.t
+    assert st["cluster_bytes"] == crow * row + st["clusters"] * 4
+    assert st["value_bytes"] == (rows - crow) * row + 2 * w.s * 4
+    assert st["query_bytes"] == st["cluster_bytes"] + st["value_bytes"]
     sg.profile_enable(True)
     K, V, Q = synth.batch_stream(w, 3, "cuda")
     before = sg.launch_count
     for i in range(3):
         sg.step(Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous())
-    ins, qry, steps = sg.profile_read()
-    assert steps == 3 and ins > 0 and qry > 0 and sg.launch_count == before + 6
+    ins, tau, zz, steps = sg.profile_read()
+    assert steps == 3 and ins > 0 and tau > 0 and zz > 0 and sg.launch_count == before + 9
 
 
 # ------------------------------------------------------------------------------------------- exact path
