@@ -4,6 +4,7 @@
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <string>
@@ -49,6 +50,7 @@ struct Layout {
 
 struct Dims {
     int B, H, Hkv, G, D, t, s, w, m_max, splits, U;
+    int sp_insert, sp_tau, sp_z;   // blocks per unit of the three step kernels (splits = their maximum)
     size_t E;   // bytes per element
 };
 
@@ -72,11 +74,28 @@ bool resolve(const subgen_config* c, Dims* o, const char** why) {
     d.E = c->dtype == SUBGEN_DTYPE_FP32 ? 4 : 2;
     d.U = d.B * d.Hkv;
     if (c->splits < 0 || c->splits > 128) { *why = "splits must be in 0..128"; return false; }
-    if (c->splits) d.splits = c->splits;
-    else {
-        int sp = (148 * 8 + d.U - 1) / d.U;     // about eight resident blocks per SM over all units
-        d.splits = sp < 1 ? 1 : (sp > 32 ? 32 : sp);
+    const bool bf16 = c->dtype == SUBGEN_DTYPE_BF16;
+    if (c->splits) {
+        d.sp_insert = d.sp_tau = d.sp_z = c->splits;
+    } else {
+        // Aim at one resident wave: the kernels hand out work inside a unit dynamically, so blocks that are all
+        // resident finish together, while a partial second wave leaves most SMs idle at the end.
+        // Resident blocks per SM: insert 3 (256 threads), cluster scan 6, value scan 4 (128 threads).
+        auto fit = [&](int per_sm, int lo) {
+            int sp = (148 * per_sm) / d.U;
+            return sp < lo ? lo : (sp > 32 ? 32 : sp);
+        };
+        if (bf16) { d.sp_insert = fit(3, 1); d.sp_tau = fit(6, 1); d.sp_z = fit(4, 1); }
+        else { d.sp_insert = d.sp_tau = d.sp_z = fit(8, 1); }
     }
+    if (const char* env = getenv("SUBGEN_SPLITS")) {       // tuning aid: "insert,cluster,value"
+        int a = 0, b = 0, e = 0;
+        if (sscanf(env, "%d,%d,%d", &a, &b, &e) == 3 && a > 0 && b > 0 && e > 0 && a <= 128 && b <= 128 && e <= 128) {
+            d.sp_insert = a; d.sp_tau = b; d.sp_z = e;
+        }
+    }
+    d.splits = d.sp_insert > d.sp_tau ? d.sp_insert : d.sp_tau;
+    if (d.sp_z > d.splits) d.splits = d.sp_z;
     *o = d;
     return true;
 }
@@ -170,21 +189,21 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
 
 // fp32 caches: CUDA-core dot products (full fp32 products). bf16 caches: tensor-core kernel.
 template <typename T, int D>
-void launch_query(const Cache<T>& C, int G, dim3 grid, cudaStream_t st, const void* q, void* out, cudaEvent_t mid) {
+void launch_query(const Cache<T>& C, int G, dim3 grid, dim3 grid_z, cudaStream_t st, const void* q, void* out, cudaEvent_t mid) {
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
         switch (G) {
             case 1: query_tau_kernel<D, 1><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                    query_z_kernel<D, 1><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
+                    query_z_kernel<D, 1><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
             case 2: query_tau_kernel<D, 2><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                    query_z_kernel<D, 2><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
+                    query_z_kernel<D, 2><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
             case 4: query_tau_kernel<D, 4><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                    query_z_kernel<D, 4><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
+                    query_z_kernel<D, 4><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
             default: query_tau_kernel<D, 8><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                     query_z_kernel<D, 8><<<grid, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
+                     query_z_kernel<D, 8><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
         }
     } else {
         switch (G) {
@@ -200,7 +219,7 @@ void launch_query(const Cache<T>& C, int G, dim3 grid, cudaStream_t st, const vo
 template <typename T, int D>
 int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void* out) {
     Cache<T> C = make_cache<T>(h);
-    const dim3 grid(h->d.splits, h->d.U);
+    const dim3 grid_i(h->d.sp_insert, h->d.U), grid_t(h->d.sp_tau, h->d.U), grid_z(h->d.sp_z, h->d.U);
     cudaEvent_t* e = nullptr;
     if (h->prof) {
         if (h->ev_used + 4 > h->ev.size()) {
@@ -215,11 +234,11 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
         CUDA_TRY(cudaEventRecord(e[0], h->st));
     }
     if constexpr (std::is_same<T, __nv_bfloat16>::value)
-        insert_mma_kernel<D><<<grid, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
+        insert_mma_kernel<D><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
     else
-        insert_kernel<T, D><<<grid, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
+        insert_kernel<T, D><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
     if (e) CUDA_TRY(cudaEventRecord(e[1], h->st));
-    launch_query<T, D>(C, h->d.G, grid, h->st, q, out, e ? e[2] : nullptr);
+    launch_query<T, D>(C, h->d.G, grid_t, grid_z, h->st, q, out, e ? e[2] : nullptr);
     if (e) CUDA_TRY(cudaEventRecord(e[3], h->st));
     CUDA_TRY(cudaGetLastError());
     h->launches += std::is_same<T, __nv_bfloat16>::value ? 3 : 2;

@@ -68,18 +68,23 @@ __global__ void __launch_bounds__(kInsertThreads) insert_mma_kernel(Cache<__nv_b
     const int c0 = blockIdx.x * per, c1 = min(m, c0 + per);
     Best b;
     b.d2 = ~0ull; b.idx = INT_MAX; b.pad = 0;
-    for (int base = c0 + warp * 16; base < c1; base += nw * 16) {
-        const int ra = base + g, rb = base + g + 8;
-        const bool va = ra < c1, vb = rb < c1;
-        const T* pa = Xu + (size_t)(va ? ra : c1 - 1) * D;
-        const T* pb = Xu + (size_t)(vb ? rb : c1 - 1) * D;
-        uint4 ka[NC], kc[NC];
+    // exact D2 of one flagged row, by the whole warp
+    auto exact_row = [&](int row) {
+        unsigned long long acc = 0;
+        if (lane < LPR) {
+            float xf[8], kf[8];
+            Elem<T>::unpack(*reinterpret_cast<const uint4*>(Xu + (size_t)row * D + lane * 8), xf);
+            Elem<T>::unpack(krow[lane], kf);
 #pragma unroll
-        for (int c = 0; c < NC; ++c) {
-            ka[c] = ldg16(pa + c * 32 + tq * 8);
-            kc[c] = ldg16(pb + c * 32 + tq * 8);
+            for (int j = 0; j < 8; ++j) acc += fx_sqdiff(xf[j], kf[j]);
         }
-        const float xa = va ? xnu[ra] : 0.f, xb = vb ? xnu[rb] : 0.f;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        if (better(acc, row, b)) { b.d2 = acc; b.idx = row; }
+    };
+    // approximate distances of one 16-row tile and the exact follow-up of its flagged rows
+    auto filter_tile = [&](int base, const uint4 (&ka)[NC], const uint4 (&kc)[NC], bool va, bool vb) {
+        const float xa = va ? xnu[base + g] : 0.f, xb = vb ? xnu[base + g + 8] : 0.f;
         float sc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
@@ -91,22 +96,14 @@ __global__ void __launch_bounds__(kInsertThreads) insert_mma_kernel(Cache<__nv_b
         const bool fa = va && tq == 0 && (na - 2.f * sc[0]) <= d2f + 1.220703125e-4f * na;
         const bool fb = vb && tq == 0 && (nb - 2.f * sc[2]) <= d2f + 1.220703125e-4f * nb;
         unsigned ma = __ballot_sync(0xffffffffu, fa), mb = __ballot_sync(0xffffffffu, fb);
-        while (ma | mb) {                                   // rare: exact D2 of one flagged row per turn
-            int row;
-            if (ma) { row = base + ((__ffs(ma) - 1) >> 2); ma &= ma - 1; }
-            else { row = base + 8 + ((__ffs(mb) - 1) >> 2); mb &= mb - 1; }
-            unsigned long long acc = 0;
-            if (lane < LPR) {
-                float xf[8], kf[8];
-                Elem<T>::unpack(*reinterpret_cast<const uint4*>(Xu + (size_t)row * D + lane * 8), xf);
-                Elem<T>::unpack(krow[lane], kf);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) acc += fx_sqdiff(xf[j], kf[j]);
-            }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-            if (better(acc, row, b)) { b.d2 = acc; b.idx = row; }
-        }
+        while (ma) { exact_row(base + ((__ffs(ma) - 1) >> 2)); ma &= ma - 1; }      // rare
+        while (mb) { exact_row(base + 8 + ((__ffs(mb) - 1) >> 2)); mb &= mb - 1; }
+    };
+    for (int base = c0 + warp * 16; base < c1; base += nw * 16) {
+        const bool va = base + g < c1, vb = base + g + 8 < c1;
+        uint4 ka[NC], kc[NC];
+        load_keys<D>(Xu + (size_t)(va ? base + g : c1 - 1) * D, Xu + (size_t)(vb ? base + g + 8 : c1 - 1) * D, tq, ka, kc);
+        filter_tile(base, ka, kc, va, vb);
     }
     b = block_best(b, smb);
     if (splits > 1) {

@@ -55,18 +55,22 @@ template <int D> struct MmaState {
 };
 
 // Scores of one 16-row tile against q, then the online-softmax update of the running maxima.
-// pa / pb: this lane's key rows g and g+8 (valid memory even when the row is masked).
+// ka / kb: this lane's pieces of key rows g and g+8 (load_keys; valid memory even when the row is masked).
 // Returns p[4] = exp(score - max) for (row g, head 2tq), (g, 2tq+1), (g+8, 2tq), (g+8, 2tq+1); 0 if masked.
-template <int D, int DA>
-__device__ __forceinline__ void tile_scores(MmaState<DA>& S, const __nv_bfloat16* pa, const __nv_bfloat16* pb, bool va,
-                                            bool vb, const uint32_t (&qb)[D / 32][4], int tq, float (&p)[4]) {
-    constexpr int NC = D / 32;
-    uint4 ka[NC], kb[NC];
+template <int D>
+__device__ __forceinline__ void load_keys(const __nv_bfloat16* pa, const __nv_bfloat16* pb, int tq, uint4 (&ka)[D / 32],
+                                          uint4 (&kb)[D / 32]) {
 #pragma unroll
-    for (int c = 0; c < NC; ++c) {
+    for (int c = 0; c < D / 32; ++c) {
         ka[c] = ldg16(pa + c * 32 + tq * 8);
         kb[c] = ldg16(pb + c * 32 + tq * 8);
     }
+}
+
+template <int D, int DA>
+__device__ __forceinline__ void tile_scores(MmaState<DA>& S, const uint4 (&ka)[D / 32], const uint4 (&kb)[D / 32], bool va,
+                                            bool vb, const uint32_t (&qb)[D / 32][4], float (&p)[4]) {
+    constexpr int NC = D / 32;
     float sc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
@@ -106,16 +110,18 @@ __device__ __forceinline__ void tile_scores(MmaState<DA>& S, const __nv_bfloat16
 }
 
 // z^T += V_tile^T . P for one 16-row tile. pz[4]: weighted p in the layout tile_scores returns.
-// pv[i]: this lane's value rows 2tq, 2tq+1, 2tq+8, 2tq+9 of the tile (valid memory, finite contents).
+// v: this lane's pieces of value rows 2tq, 2tq+1, 2tq+8, 2tq+9 of the tile (load_values; finite contents).
 template <int D>
-__device__ __forceinline__ void tile_values(MmaState<D>& S, const float (&pz)[4], const __nv_bfloat16* const (&pv)[4],
-                                            int g, int tq) {
-    constexpr int NV = D / 64;
-    uint4 v[4][NV];
+__device__ __forceinline__ void load_values(const __nv_bfloat16* const (&pv)[4], int g, uint4 (&v)[4][D / 64]) {
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int cc = 0; cc < NV; ++cc) v[i][cc] = ldg16(pv[i] + cc * 64 + g * 8);
+        for (int cc = 0; cc < D / 64; ++cc) v[i][cc] = ldg16(pv[i] + cc * 64 + g * 8);
+}
+
+template <int D>
+__device__ __forceinline__ void tile_values(MmaState<D>& S, const float (&pz)[4], const uint4 (&v)[4][D / 64], int g, int tq) {
+    constexpr int NV = D / 64;
     // B operand: P[rows 2tq, 2tq+1 | 2tq+8, 2tq+9][head g], gathered from the lanes that own those rows
     const uint32_t p01 = pack_bf16x2(pz[0], pz[1]), p23 = pack_bf16x2(pz[2], pz[3]);
     const int la = 8 * tq + (g >> 1), lb = la + 4;
@@ -191,27 +197,27 @@ __global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfl
         if (cn == 1) lst[warp][nm + __popc(ms & lt)] = c;
         __syncwarp();
         const int rows_m = nm * t, rows = rows_m + ns;
+        // row r of the list -> pointer, weight, validity
+        auto resolve = [&](int r, const T*& ptr, float& wgt) -> bool {
+            ptr = Xu;
+            wgt = 1.f;
+            if (r < rows_m) {
+                const int ci = div_small(r, magic);
+                ptr = Su + ((size_t)lst[warp][ci] * t + (r - ci * t)) * D;
+                wgt = (float)wcn[warp][ci] * inv_t;
+            } else if (r < rows) {
+                ptr = Xu + (size_t)lst[warp][nm + r - rows_m] * D;
+            }
+            return r < rows;
+        };
         for (int r0 = 0; r0 < rows; r0 += 16) {
-            const int ra = r0 + g, rb = r0 + g + 8;
-            const bool va = ra < rows, vb = rb < rows;
-            const T *pa = Xu, *pb = Xu;
-            float wa = 1.f, wb = 1.f;
-            if (ra < rows_m) {
-                const int ci = div_small(ra, magic);
-                pa = Su + ((size_t)lst[warp][ci] * t + (ra - ci * t)) * D;
-                wa = (float)wcn[warp][ci] * inv_t;
-            } else if (va) {
-                pa = Xu + (size_t)lst[warp][nm + ra - rows_m] * D;
-            }
-            if (rb < rows_m) {
-                const int ci = div_small(rb, magic);
-                pb = Su + ((size_t)lst[warp][ci] * t + (rb - ci * t)) * D;
-                wb = (float)wcn[warp][ci] * inv_t;
-            } else if (vb) {
-                pb = Xu + (size_t)lst[warp][nm + rb - rows_m] * D;
-            }
+            const T *pa, *pb;
+            float wa, wb;
+            const bool va = resolve(r0 + g, pa, wa), vb = resolve(r0 + g + 8, pb, wb);
+            uint4 ka[NC], kb[NC];
+            load_keys<D>(pa, pb, tq, ka, kb);
             float p[4];
-            tile_scores<D, 16>(S, pa, pb, va, vb, qb, tq, p);
+            tile_scores<D, 16>(S, ka, kb, va, vb, qb, p);
             S.tau0 += wa * p[0] + wb * p[2];
             S.tau1 += wa * p[1] + wb * p[3];
         }
@@ -298,19 +304,22 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_kernel(Cache<__nv_bfloa
             wza = va ? mu_over_s * ia_w : 0.f;
             wzb = vb ? mu_over_s * ib_w : 0.f;
         }
-        float p[4];
-        tile_scores<D, D>(S, Kb + (size_t)ia * D, Kb + (size_t)ib * D, va, vb, qb, tq, p);
-        if (!isM) {
-            S.tau0 += p[0] + p[2];
-            S.tau1 += p[1] + p[3];
-        }
-        const float pz[4] = {wza * p[0], wza * p[1], wzb * p[2], wzb * p[3]};
         const T* pv[4];
         pv[0] = Vb + (size_t)min(base + 2 * tq, lim - 1) * D;
         pv[1] = Vb + (size_t)min(base + 2 * tq + 1, lim - 1) * D;
         pv[2] = Vb + (size_t)min(base + 2 * tq + 8, lim - 1) * D;
         pv[3] = Vb + (size_t)min(base + 2 * tq + 9, lim - 1) * D;
-        tile_values<D>(S, pz, pv, g, tq);
+        uint4 ka[NC], kb[NC], v[4][D / 64];
+        load_keys<D>(Kb + (size_t)ia * D, Kb + (size_t)ib * D, tq, ka, kb);      // keys and values in flight together
+        load_values<D>(pv, g, v);
+        float p[4];
+        tile_scores<D, D>(S, ka, kb, va, vb, qb, p);
+        if (!isM) {
+            S.tau0 += p[0] + p[2];
+            S.tau1 += p[1] + p[3];
+        }
+        const float pz[4] = {wza * p[0], wza * p[1], wzb * p[2], wzb * p[3]};
+        tile_values<D>(S, pz, v, g, tq);
         item = __shfl_sync(0xffffffffu, next, 0);
     }
 
