@@ -80,12 +80,12 @@ bool resolve(const subgen_config* c, Dims* o, const char** why) {
     } else {
         // Aim at one resident wave: the kernels hand out work inside a unit dynamically, so blocks that are all
         // resident finish together, while a partial second wave leaves most SMs idle at the end.
-        // Resident blocks per SM: insert 3 (256 threads), cluster scan 6, value scan 4 (128 threads).
+        // Resident blocks per SM (128 threads each): insert 6, cluster scan 6, value scan 4.
         auto fit = [&](int per_sm, int lo) {
             int sp = (148 * per_sm) / d.U;
             return sp < lo ? lo : (sp > 32 ? 32 : sp);
         };
-        if (bf16) { d.sp_insert = fit(3, 1); d.sp_tau = fit(6, 1); d.sp_z = fit(4, 1); }
+        if (bf16) { d.sp_insert = fit(6, 1); d.sp_tau = fit(6, 1); d.sp_z = fit(4, 1); }
         else { d.sp_insert = d.sp_tau = d.sp_z = fit(8, 1); }
     }
     if (const char* env = getenv("SUBGEN_SPLITS")) {       // tuning aid: "insert,cluster,value"
@@ -234,7 +234,7 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
         CUDA_TRY(cudaEventRecord(e[0], h->st));
     }
     if constexpr (std::is_same<T, __nv_bfloat16>::value)
-        insert_mma_kernel<D><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
+        insert_mma_kernel<D><<<grid_i, kInsertMmaThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
     else
         insert_kernel<T, D><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
     if (e) CUDA_TRY(cudaEventRecord(e[1], h->st));

@@ -16,8 +16,10 @@
 
 namespace sgk {
 
+constexpr int kInsertMmaThreads = 128;
+
 template <int D>
-__global__ void __launch_bounds__(kInsertThreads) insert_mma_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ k_new,
+__global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ k_new,
                                                                     const __nv_bfloat16* __restrict__ v_new) {
     typedef __nv_bfloat16 T;
     constexpr int EPL = 8, LPR = D / EPL, NC = D / 32;
