@@ -14,6 +14,7 @@
 #include "subgen_kernels.cuh"
 #include "subgen_query_mma.cuh"
 #include "subgen_insert_mma.cuh"
+#include "subgen_prefill.cuh"
 
 using namespace sgk;
 
@@ -159,6 +160,9 @@ struct subgen {
     bool prof = false;
     std::vector<cudaEvent_t> ev;  // four per profiled step
     size_t ev_used = 0;
+    char* scratch = nullptr;      // prefill scratch (library-owned, grows on demand)
+    size_t scratch_bytes = 0;
+    bool seq_prefill = false;     // SUBGEN_PREFILL=seq: token-by-token prefill also for bf16
 };
 
 namespace {
@@ -260,8 +264,80 @@ int launch_prefill_td(subgen* h, const void* K, const void* V, int n, const int*
     return SUBGEN_OK;
 }
 
-int launch_prefill(subgen* h, const void* K, const void* V, int n, const int* cu_dev, int total) {
+// bf16: values for the whole call at once, keys chunk by chunk (subgen_prefill.cuh).
+// add[b]: tokens appended to sequence b by this call (host copy).
+template <int D>
+int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const int* cu_dev, int total, const int* add) {
+    typedef __nv_bfloat16 T;
+    Cache<T> C = make_cache<T>(h);
+    const Dims& d = h->d;
+    int Lmax = 0;
+    for (int b = 0; b < d.B; ++b) {
+        const int lo = h->n_host[b] > d.w ? h->n_host[b] - d.w : 0;
+        const int hi = h->n_host[b] + add[b] > d.w ? h->n_host[b] + add[b] - d.w : 0;
+        Lmax = hi - lo > Lmax ? hi - lo : Lmax;
+    }
+    int slices = (148 * 4 + d.U - 1) / d.U;
+    slices = slices < 1 ? 1 : (slices > 16 ? 16 : slices);
+    PrefillArgs a;
+    a.K = (const T*)K; a.V = (const T*)V; a.n_uniform = n; a.cu = cu_dev; a.total = total; a.Lmax = Lmax; a.slices = slices;
+    a.Wbuf = nullptr; a.Tot = nullptr; a.Mwin = nullptr; a.pbest = nullptr;
+    int launches = 0;
+    if (Lmax > 0) {
+        const size_t b_w = align_up((size_t)d.U * Lmax * 8), b_m = align_up((size_t)d.U * d.s * 4);
+        const size_t b_p = align_up((size_t)d.U * slices * kChunk * sizeof(Best));
+        const size_t need = 2 * b_w + b_m + b_p;
+        if (need > h->scratch_bytes) {
+            if (h->scratch) { CUDA_TRY(cudaStreamSynchronize(h->st)); CUDA_TRY(cudaFree(h->scratch)); h->scratch = nullptr; h->scratch_bytes = 0; }
+            cudaError_t e = cudaMalloc((void**)&h->scratch, need);
+            if (e != cudaSuccess) return fail(SUBGEN_ENOMEM, "subgen_prefill: cudaMalloc(%zu) for scratch failed: %s", need, cudaGetErrorString(e));
+            h->scratch_bytes = need;
+        }
+        a.Wbuf = (unsigned long long*)h->scratch;
+        a.Tot = (unsigned long long*)(h->scratch + b_w);
+        a.Mwin = (int*)(h->scratch + 2 * b_w);
+        a.pbest = (Best*)(h->scratch + 2 * b_w + b_m);
+        CUDA_TRY(cudaMemsetAsync(a.Mwin, 0xFF, (size_t)d.U * d.s * 4, h->st));
+        constexpr int RPW = 32 / (D / 8);
+        int bx = (Lmax + 8 * RPW - 1) / (8 * RPW);
+        bx = bx > 64 ? 64 : bx;
+        prefill_w_kernel<D><<<dim3(bx, d.U), 256, 0, h->st>>>(C, a);
+        prefill_scan_kernel<<<d.U, 1024, 0, h->st>>>(C, a);
+        const int cbx = ((d.s + 3) / 4 + 127) / 128;
+        long long want = (300000LL + (long long)d.U * cbx * 128 - 1) / ((long long)d.U * cbx * 128);   // fill the GPU about once
+        int segs = (int)(want < 1 ? 1 : want);
+        int seg_len = (Lmax + segs - 1) / segs;
+        seg_len = seg_len < 256 ? 256 : seg_len;
+        segs = (Lmax + seg_len - 1) / seg_len;
+        prefill_coin_kernel<<<dim3(cbx, segs, d.U), 128, 0, h->st>>>(C, a, seg_len);
+        int gx = (d.s + 8 * RPW - 1) / (8 * RPW);
+        gx = gx > 32 ? 32 : gx;
+        prefill_gather_kernel<D><<<dim3(gx, d.U), 256, 0, h->st>>>(C, a);
+        launches += 4;
+        const int nchunks = (Lmax + kChunk - 1) / kChunk;
+        for (int c = 0; c < nchunks; ++c) {
+            prefill_score_kernel<D><<<dim3(slices, d.U), kScoreThreads, 0, h->st>>>(C, a, c);
+            prefill_resolve_kernel<D><<<d.U, kResolveThreads, 0, h->st>>>(C, a, c);
+        }
+        launches += 2 * nchunks;
+    }
+    int longest = 0;
+    for (int b = 0; b < d.B; ++b) longest = add[b] > longest ? add[b] : longest;
+    int fx = (int)(((size_t)(longest < d.w ? longest : d.w) * (D / 8) + 255) / 256);
+    fx = fx < 1 ? 1 : (fx > 16 ? 16 : fx);
+    prefill_finish_kernel<D><<<dim3(fx, d.U), 256, 0, h->st>>>(C, a);
+    prefill_commit_kernel<<<(d.U + 255) / 256, 256, 0, h->st>>>(C, a, d.U);
+    launches += 2;
+    CUDA_TRY(cudaGetLastError());
+    h->launches += launches;
+    return SUBGEN_OK;
+}
+
+int launch_prefill(subgen* h, const void* K, const void* V, int n, const int* cu_dev, int total, const int* add) {
     const bool f32 = h->cfg.dtype == SUBGEN_DTYPE_FP32;
+    if (!f32 && !h->seq_prefill)
+        return h->d.D == 64 ? launch_prefill_chunked<64>(h, K, V, n, cu_dev, total, add)
+                            : launch_prefill_chunked<128>(h, K, V, n, cu_dev, total, add);
     if (h->d.D == 64)
         return f32 ? launch_prefill_td<float, 64>(h, K, V, n, cu_dev, total)
                    : launch_prefill_td<__nv_bfloat16, 64>(h, K, V, n, cu_dev, total);
@@ -329,6 +405,7 @@ subgen_t* subgen_create_ex(const subgen_config* cfg) {
         return nullptr;
     }
     h->n_host.assign(d.B, 0);
+    if (const char* env = getenv("SUBGEN_PREFILL")) h->seq_prefill = strcmp(env, "seq") == 0;
     return h;
 }
 
@@ -345,6 +422,7 @@ void subgen_destroy(subgen_t* h) {
     cudaStreamSynchronize(h->st);
     for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
     if (h->owns) cudaFree(h->ws);
+    if (h->scratch) cudaFree(h->scratch);
     delete h;
 }
 
@@ -355,7 +433,8 @@ int subgen_prefill(subgen_t* h, const void* K, const void* V, int n) {
     if (!K || !V) return fail(SUBGEN_EINVAL, "subgen_prefill: K and V must not be NULL");
     for (int b = 0; b < h->d.B; ++b)
         if ((long long)h->n_host[b] + n > INT_MAX - 1) return fail(SUBGEN_ESTATE, "subgen_prefill: stream too long");
-    int rc = launch_prefill(h, K, V, n, nullptr, 0);
+    std::vector<int> add(h->d.B, n);
+    int rc = launch_prefill(h, K, V, n, nullptr, 0, add.data());
     if (rc) return rc;
     for (int b = 0; b < h->d.B; ++b) h->n_host[b] += n;
     return SUBGEN_OK;
@@ -377,7 +456,9 @@ int subgen_prefill_varlen(subgen_t* h, const void* K, const void* V, const int* 
     // the offsets are consumed by the kernel launched right after, in stream order
     CUDA_TRY(cudaMemcpyAsync(cu_dev, cu, sizeof(int) * (h->d.B + 1), cudaMemcpyHostToDevice, h->st));
     CUDA_TRY(cudaStreamSynchronize(h->st));   // cu may be pageable host memory reused by the caller
-    int rc = launch_prefill(h, K, V, 0, cu_dev, total);
+    std::vector<int> add(h->d.B);
+    for (int b = 0; b < h->d.B; ++b) add[b] = cu[b + 1] - cu[b];
+    int rc = launch_prefill(h, K, V, 0, cu_dev, total, add.data());
     if (rc) return rc;
     for (int b = 0; b < h->d.B; ++b) h->n_host[b] += cu[b + 1] - cu[b];
     return SUBGEN_OK;

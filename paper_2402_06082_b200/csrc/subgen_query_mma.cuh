@@ -91,7 +91,6 @@ __device__ __forceinline__ void tile_scores(MmaState<DA>& S, const uint4 (&ka)[D
         const float f1 = (S.m1 == -INFINITY) ? 0.f : __expf(S.m1 - n1);
         S.tau0 *= f0;
         S.tau1 *= f1;
-#pragma unroll
         if (DA == D) {                 // DA != D: caller keeps no numerator accumulators
 #pragma unroll
             for (int j = 0; j < DA / 16; ++j) {

@@ -278,6 +278,40 @@ def test_cache_stats_and_profile():
     assert steps == 3 and ins > 0 and tau > 0 and zz > 0 and sg.launch_count == before + 9
 
 
+def test_chunked_prefill_equals_token_by_token_prefill(monkeypatch):
+    """bf16 handles prefill chunk by chunk on the tensor cores; SUBGEN_PREFILL=seq selects the token-by-token
+    kernel. Both must leave the same state, also when a call continues a stream whose tail is in the window."""
+    w = synth.CFG3.scaled(B=2, H=4, Hkv=2, n_prompt=1000, ncomp=24, s=96, t=6, window=48, m_max=512)
+    K, V, _ = synth.batch_stream(w, 1000, "cuda")
+    a = _sg(w)
+    monkeypatch.setenv("SUBGEN_PREFILL", "seq")
+    b = _sg(w)
+    monkeypatch.delenv("SUBGEN_PREFILL")
+    for lo, hi in ((0, 7), (7, 300), (300, 301), (301, 1000)):
+        a.prefill(K[:, :, lo:hi].contiguous(), V[:, :, lo:hi].contiguous())
+        b.prefill(K[:, :, lo:hi].contiguous(), V[:, :, lo:hi].contiguous())
+        for bb in range(w.B):
+            for h in range(w.Hkv):
+                s1, s2 = a.export_state(bb, h), b.export_state(bb, h)
+                for key in ("m", "mu", "n", "last_cluster", "last_opened", "status"):
+                    assert s1[key] == s2[key], (key, lo, hi)
+                for key in ("counts", "centre_tok", "slot_tok", "m_tok", "m_w"):
+                    np.testing.assert_array_equal(s1[key], s2[key], err_msg="%s after [%d,%d)" % (key, lo, hi))
+                hp.assert_rows_match_tokens(a, bb, h, s1, K[bb, h], V[bb, h])
+                hp.assert_rows_match_tokens(b, bb, h, s2, K[bb, h], V[bb, h])
+    assert a.launch_count > b.launch_count
+
+
+def test_prefill_capacity_overflow_is_reported():
+    from paper_2402_06082_b200 import binding
+    w = synth.CFG3.scaled(B=1, H=2, Hkv=2, n_prompt=400, ncomp=64, s=32, window=8, m_max=16)
+    K, V, _ = synth.batch_stream(w, 400, "cuda")
+    sg = _sg(w)
+    sg.prefill(K, V)
+    assert sg.status() == binding.ST_CAPACITY
+    assert sg.export_state(0, 0)["m"] == 16
+
+
 # ------------------------------------------------------------------------------------------- exact path
 @pytest.mark.parametrize("dtype,G", [("fp32", 1), ("bf16", 4)])
 def test_exact_attention_matches_eq1(dtype, G):
@@ -323,3 +357,50 @@ def test_exact_varlen_and_short_window_agreement():
                 want = orc.exact_attention(f32(streams[b][0])[hq // 2, : lens[b] + i + 1],
                                            f32(streams[b][1])[hq // 2, : lens[b] + i + 1], f32(q)[b, hq])
                 assert hp.rel_err(a[b, hq], want) <= 2e-2 and hp.rel_err(e[b, hq], want) <= 2e-2
+
+
+# ------------------------------------------------------------------------------------------- full size
+def test_benchmark_workload_full_size_sampled_units():
+    """The benchmark's workload (cfg3: 8 x 32 heads, 32768-token prompts, bf16) in the benchmark's launch
+    configuration; the oracle replays a seeded sample of (sequence, head) units in full."""
+    from concurrent.futures import ThreadPoolExecutor
+    w = synth.CFG3
+    n0, nd = w.n_prompt, 6
+    sg = _sg(w)
+    rng = np.random.default_rng(5)
+    sample = [(int(b), int(h)) for b, h in zip(rng.integers(0, w.B, 3), rng.integers(0, w.Hkv, 3))]
+    Kp = torch.empty(w.B, w.Hkv, n0, w.d, dtype=w.torch_dtype, device="cuda")
+    Vp = torch.empty_like(Kp)
+    dec, host = [], {}
+    for b in range(w.B):
+        K, V, Q = synth.sequence_stream(w, b, n0 + nd, "cuda")
+        Kp[b], Vp[b] = K[:, :n0], V[:, :n0]
+        dec.append((K[:, n0:].clone(), V[:, n0:].clone(), Q[:, n0:].clone()))
+        for (bb, h) in sample:
+            if bb == b:
+                host[(b, h)] = (f32(K[h]), f32(V[h]), f32(Q[h]))
+        del K, V, Q
+    sg.prefill(Kp, Vp)
+    del Kp, Vp
+    orcs = {bh: hp.oracle_unit(w, *bh) for bh in sample}
+
+    def replay(bh):
+        orcs[bh].push_many(host[bh][0][:n0], host[bh][1][:n0])
+    with ThreadPoolExecutor(len(sample)) as ex:
+        list(ex.map(replay, sample))
+    for bh in sample:
+        hp.assert_state_equal(sg.export_state(*bh), orcs[bh], "full-size prefill unit %s" % (bh,))
+        assert orcs[bh].m > 1500
+    for i in range(nd):
+        q = torch.stack([d[2][:, i] for d in dec]).contiguous()
+        k = torch.stack([d[0][:, i] for d in dec]).contiguous()
+        v = torch.stack([d[1][:, i] for d in dec]).contiguous()
+        out = f32(sg.step(q, k, v))
+        for (b, h) in sample:
+            Kh, Vh, Qh = host[(b, h)]
+            orcs[(b, h)].push(Kh[n0 + i], Vh[n0 + i])
+            err = hp.rel_err(out[b, h], orcs[(b, h)].query(Qh[n0 + i]))
+            assert err <= hp.TOL[torch.bfloat16], "step %d unit %s: %.3g" % (i, (b, h), err)
+    for bh in sample:
+        hp.assert_state_equal(sg.export_state(*bh), orcs[bh], "full-size steps unit %s" % (bh,))
+    assert sg.status() == 0
