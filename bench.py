@@ -31,6 +31,11 @@ from paper_2402_06082_b200 import sharding, synth  # noqa: E402
 
 METRIC = "SubGen decode steps/s (B x H heads) at 32K ctx"
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised in
+# profiles/step_kernels_cfg3.md (cfg3 state at 32K tokens, 64 units). Valid for cfg3 only; set an entry to
+# None when its kernel changes.
+NCU_TRAFFIC = {"query_tau_kernel": {"dram_bytes": 157.98e6, "units": 64, "workload": "cfg3"}}
+
 
 # ------------------------------------------------------------------------------------------ helpers
 def measured_peaks():
@@ -316,8 +321,12 @@ def run_subgen(args, w):
     else:
         dom = ("query_kernel", cbytes + vbytes, c_ms)
     achieved = gbs(dom[1], dom[2])
+    traffic = None
+    if NCU_TRAFFIC.get(dom[0]) and NCU_TRAFFIC[dom[0]]["workload"] == wr.name and not args.prompt:          # DRAM bytes of one launch from the ncu capture, scaled by the units processed
+        t = NCU_TRAFFIC[dom[0]]
+        traffic = t["dram_bytes"] * wr.units / t["units"]
     roofline = {"bound": "hbm", "kernel": dom[0], "achieved": achieved, "peak": peak, "peak_source": which,
-                "unit": "GB/s", "frac": achieved / peak if achieved else None, "traffic": None,
+                "unit": "GB/s", "frac": achieved / peak if achieved else None, "traffic": traffic,
                 "algorithmic_bytes_per_launch": dom[1], "ms_per_launch": dom[2],
                 "kernels": {"insert": {"algorithmic_bytes_per_launch": ibytes, "ms_per_launch": i_ms, "achieved": gbs(ibytes, i_ms)},
                             "cluster_scan": {"algorithmic_bytes_per_launch": cbytes, "ms_per_launch": c_ms, "achieved": gbs(cbytes, c_ms)},
