@@ -281,12 +281,12 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
     slices = slices < 1 ? 1 : (slices > 16 ? 16 : slices);
     PrefillArgs a;
     a.K = (const T*)K; a.V = (const T*)V; a.n_uniform = n; a.cu = cu_dev; a.total = total; a.Lmax = Lmax; a.slices = slices;
-    a.Wbuf = nullptr; a.Tot = nullptr; a.Mwin = nullptr; a.pbest = nullptr;
+    a.Wbuf = nullptr; a.Tot = nullptr; a.Thr = nullptr; a.Mwin = nullptr; a.pbest = nullptr;
     int launches = 0;
     if (Lmax > 0) {
         const size_t b_w = align_up((size_t)d.U * Lmax * 8), b_m = align_up((size_t)d.U * d.s * 4);
         const size_t b_p = align_up((size_t)d.U * slices * kChunk * sizeof(Best));
-        const size_t need = 2 * b_w + b_m + b_p;
+        const size_t need = 3 * b_w + b_m + b_p;
         if (need > h->scratch_bytes) {
             if (h->scratch) { CUDA_TRY(cudaStreamSynchronize(h->st)); CUDA_TRY(cudaFree(h->scratch)); h->scratch = nullptr; h->scratch_bytes = 0; }
             cudaError_t e = cudaMalloc((void**)&h->scratch, need);
@@ -295,8 +295,9 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         }
         a.Wbuf = (unsigned long long*)h->scratch;
         a.Tot = (unsigned long long*)(h->scratch + b_w);
-        a.Mwin = (int*)(h->scratch + 2 * b_w);
-        a.pbest = (Best*)(h->scratch + 2 * b_w + b_m);
+        a.Thr = (unsigned long long*)(h->scratch + 2 * b_w);
+        a.Mwin = (int*)(h->scratch + 3 * b_w);
+        a.pbest = (Best*)(h->scratch + 3 * b_w + b_m);
         CUDA_TRY(cudaMemsetAsync(a.Mwin, 0xFF, (size_t)d.U * d.s * 4, h->st));
         constexpr int RPW = 32 / (D / 8);
         int bx = (Lmax + 8 * RPW - 1) / (8 * RPW);

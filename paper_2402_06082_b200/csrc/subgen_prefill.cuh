@@ -8,7 +8,8 @@
 //   values (UpdateMatrixProduct, whole prompt at once)
 //     W kernel      W(v_e) for every inserted token, input range check
 //     scan kernel   tot_e = mu_before + sum_{e' <= e} W_e'   (64-bit integers: any order gives the same bits)
-//     coin kernel   slot i keeps the LAST token whose coin u*(tot_e) < W_e 2^32 succeeds (atomicMax on the index)
+//     coin kernel   slot i keeps the LAST token whose coin u*(tot_e) < W_e 2^32 succeeds (as u < ceil(W_e 2^32 / tot_e);
+//                   atomicMax on the token index)
 //     gather kernel copies the winners' rows into M
 //   keys (UpdateSoftmaxNormalizer), chunk by chunk of kChunk tokens
 //     score kernel  chunk x existing representatives as a dense contraction on the tensor cores
@@ -36,6 +37,7 @@ struct PrefillArgs {
     int Lmax;                          // longest insert range over all units (row stride of the scratch arrays)
     unsigned long long* Wbuf;          // [U, Lmax] W of the e-th inserted token of this call
     unsigned long long* Tot;           // [U, Lmax] inclusive prefix incl. mu_before
+    unsigned long long* Thr;           // [U, Lmax] coin threshold ceil(W 2^32 / tot): the coin succeeds iff u < Thr
     int* Mwin;                         // [U, s] winning token per M slot, -1 none
     Best* pbest;                       // [U, slices, kChunk] partial nearest old representative per chunk token
     int slices;
@@ -123,7 +125,25 @@ __global__ void prefill_scan_kernel(Cache<__nv_bfloat16> C, PrefillArgs a) {
         __syncthreads();
         unsigned long long pre = carry;
         for (int wv = 0; wv < warp; ++wv) pre += wsum[wv];
-        if (i < len) a.Tot[(size_t)u * a.Lmax + i] = pre + x;
+        if (i < len) {
+            const unsigned long long W = a.Wbuf[(size_t)u * a.Lmax + i], tot = pre + x;
+            a.Tot[(size_t)u * a.Lmax + i] = tot;
+            // u * tot < W 2^32  <=>  u < ceil(W 2^32 / tot): one long division per token instead of a 128-bit
+            // product per coin (W <= tot < 2^63, so the shifted remainder never overflows)
+            unsigned long long q = 0, rem = W;
+            if (W) {
+                if (W == tot) q = 1ull << 32;
+                else {
+                    for (int bit = 0; bit < 32; ++bit) {
+                        rem <<= 1;
+                        q <<= 1;
+                        if (rem >= tot) { rem -= tot; q |= 1ull; }
+                    }
+                    if (rem) ++q;
+                }
+            }
+            a.Thr[(size_t)u * a.Lmax + i] = q;
+        }
         __syncthreads();
         if (tid == blockDim.x - 1) {
             unsigned long long tot = carry;
@@ -142,19 +162,17 @@ __global__ void prefill_coin_kernel(Cache<__nv_bfloat16> C, PrefillArgs a, int s
     const int len = r.ins_hi - r.ins_lo;
     const int i0 = blockIdx.y * seg_len, i1 = min(len, i0 + seg_len);
     if (blk * 4 >= C.s || i0 >= i1) return;
-    const unsigned long long* Wb = a.Wbuf + (size_t)u * a.Lmax;
-    const unsigned long long* Tb = a.Tot + (size_t)u * a.Lmax;
+    const unsigned long long* Tb = a.Thr + (size_t)u * a.Lmax;
     int win[4] = {-1, -1, -1, -1};
     for (int i = i0; i < i1; ++i) {
-        const unsigned long long W = Wb[i];
-        if (W == 0ull) continue;
-        const unsigned long long tot = Tb[i];
+        const unsigned long long thr = Tb[i];
+        if (thr == 0ull) continue;                          // W = 0: never sampled
         const int e = r.ins_lo + i;
         const uint4 rr = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)blk, 1u), C.key0, C.key1);
-        if (coin_value(rr.x, tot, W)) win[0] = e;
-        if (coin_value(rr.y, tot, W)) win[1] = e;
-        if (coin_value(rr.z, tot, W)) win[2] = e;
-        if (coin_value(rr.w, tot, W)) win[3] = e;
+        if ((unsigned long long)rr.x < thr) win[0] = e;
+        if ((unsigned long long)rr.y < thr) win[1] = e;
+        if ((unsigned long long)rr.z < thr) win[2] = e;
+        if ((unsigned long long)rr.w < thr) win[3] = e;
     }
 #pragma unroll
     for (int q = 0; q < 4; ++q)
