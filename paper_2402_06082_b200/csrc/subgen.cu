@@ -15,6 +15,7 @@
 #include "subgen_query_mma.cuh"
 #include "subgen_insert_mma.cuh"
 #include "subgen_prefill.cuh"
+#include "subgen_exact_mma.cuh"
 
 using namespace sgk;
 
@@ -84,9 +85,12 @@ bool resolve(const subgen_config* c, Dims* o, const char** why) {
         // Resident blocks per SM (128 threads each): insert 6, cluster scan 6, value scan 4.
         auto fit = [&](int per_sm, int lo) {
             int sp = (148 * per_sm) / d.U;
-            return sp < lo ? lo : (sp > 32 ? 32 : sp);
+            return sp < lo ? lo : (sp > 64 ? 64 : sp);
         };
-        if (bf16) { d.sp_insert = fit(6, 1); d.sp_tau = fit(6, 1); d.sp_z = fit(4, 1); }
+        if (bf16) {
+            d.sp_insert = fit(6, 1); d.sp_tau = fit(6, 1); d.sp_z = fit(4, 1);
+            if (d.sp_z > 16) d.sp_z = 16;      // the last block merges sp_z numerator partials of G*d floats each
+        }
         else { d.sp_insert = d.sp_tau = d.sp_z = fit(8, 1); }
     }
     if (const char* env = getenv("SUBGEN_SPLITS")) {       // tuning aid: "insert,cluster,value"
@@ -606,7 +610,7 @@ struct subgen_exact {
     int B, H, Hkv, G, D, n_max, dtype, U, splits;
     size_t E;
     char *Kc = nullptr, *Vc = nullptr, *misc = nullptr;
-    size_t off_n, off_part, off_ticket, off_cu, misc_bytes;
+    size_t off_n, off_part, off_ticket, off_cu, off_q, misc_bytes;
     cudaStream_t st = nullptr;
     std::vector<int> n_host;
     uint64_t launches = 0;
@@ -621,6 +625,7 @@ template <typename T> ExactCache<T> make_exact(const subgen_exact* h) {
     E.n_unit = (int*)(h->misc + h->off_n);
     E.part = (float*)(h->misc + h->off_part);
     E.ticket = (unsigned*)(h->misc + h->off_ticket);
+    E.qnext = (unsigned*)(h->misc + h->off_q);
     return E;
 }
 
@@ -660,6 +665,25 @@ int exact_step_td(subgen_exact* h, const void* q, const void* k, const void* v, 
     return SUBGEN_OK;
 }
 
+// bf16: append the step's token (k, v are [U, 1, d] in the dense layout), then the tensor-core scan.
+template <int D>
+int exact_step_mma(subgen_exact* h, const void* q, const void* k, const void* v, void* out) {
+    typedef __nv_bfloat16 T;
+    int rc = exact_append_td<T, D>(h, k, v, 1, nullptr, 0, 1);
+    if (rc) return rc;
+    ExactCache<T> E = make_exact<T>(h);
+    const dim3 grid(h->splits, h->U);
+    switch (h->G) {
+        case 1: exact_mma_kernel<D, 1><<<grid, kQmThreads, 0, h->st>>>(E, (const T*)q, (T*)out); break;
+        case 2: exact_mma_kernel<D, 2><<<grid, kQmThreads, 0, h->st>>>(E, (const T*)q, (T*)out); break;
+        case 4: exact_mma_kernel<D, 4><<<grid, kQmThreads, 0, h->st>>>(E, (const T*)q, (T*)out); break;
+        default: exact_mma_kernel<D, 8><<<grid, kQmThreads, 0, h->st>>>(E, (const T*)q, (T*)out); break;
+    }
+    CUDA_TRY(cudaGetLastError());
+    h->launches += 1;
+    return SUBGEN_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -677,14 +701,15 @@ subgen_exact_t* subgen_exact_create(int B, int H, int Hkv, int d, int n_max, int
     subgen_exact* h = new subgen_exact();
     h->B = B; h->H = H; h->Hkv = Hkv; h->G = G; h->D = d; h->n_max = n_max; h->dtype = dtype; h->U = B * Hkv;
     h->E = dtype == SUBGEN_DTYPE_FP32 ? 4 : 2;
-    int sp = (148 * 8 + h->U - 1) / h->U;
-    h->splits = sp < 1 ? 1 : (sp > 32 ? 32 : sp);
+    int sp = dtype == SUBGEN_DTYPE_BF16 ? (148 * 4) / h->U : (148 * 8 + h->U - 1) / h->U;   // bf16: one resident wave of 4 blocks/SM
+    h->splits = sp < 1 ? 1 : (sp > 64 ? 64 : sp);
     h->st = (cudaStream_t)stream;
     const size_t cache = (size_t)h->U * n_max * d * h->E;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
     h->off_n = take((size_t)h->U * 4);
     h->off_ticket = take((size_t)h->U * 4);
+    h->off_q = take((size_t)h->U * 4);
     h->off_cu = take(((size_t)B + 1) * 4);
     h->off_part = take((size_t)h->U * h->splits * G * (d + 2) * 4);
     h->misc_bytes = off;
@@ -751,8 +776,8 @@ int subgen_exact_step(subgen_exact_t* h, const void* q, const void* k, const voi
         if (h->n_host[b] >= h->n_max) return fail(SUBGEN_ESTATE, "subgen_exact_step: cache capacity n_max exceeded");
     const bool f32 = h->dtype == SUBGEN_DTYPE_FP32;
     int rc;
-    if (h->D == 64) rc = f32 ? exact_step_td<float, 64>(h, q, k, v, out) : exact_step_td<__nv_bfloat16, 64>(h, q, k, v, out);
-    else rc = f32 ? exact_step_td<float, 128>(h, q, k, v, out) : exact_step_td<__nv_bfloat16, 128>(h, q, k, v, out);
+    if (h->D == 64) rc = f32 ? exact_step_td<float, 64>(h, q, k, v, out) : exact_step_mma<64>(h, q, k, v, out);
+    else rc = f32 ? exact_step_td<float, 128>(h, q, k, v, out) : exact_step_mma<128>(h, q, k, v, out);
     if (rc) return rc;
     for (int b = 0; b < h->B; ++b) h->n_host[b] += 1;
     return SUBGEN_OK;

@@ -428,29 +428,57 @@ __device__ __forceinline__ void block_partial(Acc<G, Elem<T>::EPL>& A, float* sm
     block_combine<D, G>(sm, dst);
 }
 
-// Final merge of `np` block partials and the division z / tau, by a whole block.
-// part: [np][G][D+2]; out rows: out + g * D for g < G. poisoned -> NaN.
+// Final merge of block partials and the division z / tau, by a whole block (all threads must call).
+// part: [np][G][D+2] = {max, tau, z[D]}; part_t (may be NULL): [np_t][G][2] = {max, tau} partials that carry no
+// numerator; out rows: out + g * D for g < G. poisoned -> NaN. sred: 16 floats of shared memory.
+// The loads of different partials are independent (no branches, unrolled), so their latencies overlap.
 template <typename T, int D, int G>
-__device__ __forceinline__ void final_merge(const float* part, int np, T* out, bool poisoned) {
+__device__ __forceinline__ void merge_partials(const float* part, int np, const float* part_t, int np_t, T* out,
+                                               bool poisoned, float* sred) {
     constexpr int STR = D + 2;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    for (int g = warp; g < G; g += nw) {            // per head: global maximum, then the partition function
+        float m = -INFINITY;
+        for (int i = lane; i < np; i += 32) m = fmaxf(m, __ldcg(part + ((size_t)i * G + g) * STR));
+        for (int i = lane; i < np_t; i += 32) m = fmaxf(m, __ldcg(part_t + ((size_t)i * G + g) * 2));
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+        float tau = 0.f;
+        for (int i = lane; i < np; i += 32) {
+            const float* pp = part + ((size_t)i * G + g) * STR;
+            const float pm = __ldcg(pp), pt = __ldcg(pp + 1);
+            tau += pm == -INFINITY ? 0.f : pt * __expf(pm - m);
+        }
+        for (int i = lane; i < np_t; i += 32) {
+            const float* pp = part_t + ((size_t)i * G + g) * 2;
+            const float pm = __ldcg(pp), pt = __ldcg(pp + 1);
+            tau += pm == -INFINITY ? 0.f : pt * __expf(pm - m);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) tau += __shfl_xor_sync(0xffffffffu, tau, off);
+        if (lane == 0) { sred[g] = m; sred[8 + g] = tau; }
+    }
+    __syncthreads();
     for (int o = threadIdx.x; o < G * D; o += blockDim.x) {
         const int g = o / D, c = o % D;
-        float m = -INFINITY;
-        for (int i = 0; i < np; ++i) m = fmaxf(m, __ldcg(part + ((size_t)i * G + g) * STR));
-        float z = 0.f, tau = 0.f;
+        const float m = sred[g], tau = sred[8 + g];
+        float z = 0.f;
+#pragma unroll 16
         for (int i = 0; i < np; ++i) {
             const float* pp = part + ((size_t)i * G + g) * STR;
-            const float pm = __ldcg(pp);
-            if (pm != -INFINITY) {
-                const float sc = __expf(pm - m);
-                tau += __ldcg(pp + 1) * sc;
-                z += __ldcg(pp + 2 + c) * sc;
-            }
+            const float pm = __ldcg(pp), pz = __ldcg(pp + 2 + c);
+            z += pm == -INFINITY ? 0.f : pz * __expf(pm - m);
         }
         float r = tau > 0.f ? z / tau : 0.f;
         if (poisoned) r = __int_as_float(0x7fc00000);
         out[(size_t)g * D + c] = Elem<T>::to_out(r);
     }
+}
+
+template <typename T, int D, int G>
+__device__ __forceinline__ void final_merge(const float* part, int np, T* out, bool poisoned) {
+    __shared__ float sred[16];
+    merge_partials<T, D, G>(part, np, nullptr, 0, out, poisoned, sred);
 }
 
 }  // namespace sgk

@@ -294,6 +294,7 @@ template <typename T> struct ExactCache {
     int* n_unit;     // [U]
     float* part;     // [U, splits, G, D + 2]
     unsigned* ticket;
+    unsigned* qnext; // [U] work queue of the tensor-core kernel
 };
 
 template <typename T, int D>

@@ -357,32 +357,9 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_kernel(Cache<__nv_bfloa
         __threadfence();
     }
     // final merge: z partials of this kernel and the cluster partials {max, tau} of query_tau_kernel
-    const float* part_t = C.part_tau + (size_t)u * splits_tau * G * 2;
-    const bool poisoned = C.status[u] != 0;
-    for (int o = tid; o < G * D; o += blockDim.x) {
-        const int hh = o / D, c = o % D;
-        float mx = -INFINITY;
-        for (int i = 0; i < splits; ++i) mx = fmaxf(mx, __ldcg(part_u + ((size_t)i * G + hh) * STR));
-        for (int i = 0; i < splits_tau; ++i) mx = fmaxf(mx, __ldcg(part_t + ((size_t)i * G + hh) * 2));
-        float z = 0.f, tau = 0.f;
-        for (int i = 0; i < splits; ++i) {
-            const float* pp = part_u + ((size_t)i * G + hh) * STR;
-            const float pm = __ldcg(pp);
-            if (pm != -INFINITY) {
-                const float sc = __expf(pm - mx);
-                tau += __ldcg(pp + 1) * sc;
-                z += __ldcg(pp + 2 + c) * sc;
-            }
-        }
-        for (int i = 0; i < splits_tau; ++i) {
-            const float* pp = part_t + ((size_t)i * G + hh) * 2;
-            const float pm = __ldcg(pp);
-            if (pm != -INFINITY) tau += __ldcg(pp + 1) * __expf(pm - mx);
-        }
-        float r = tau > 0.f ? z / tau : 0.f;
-        if (poisoned) r = __int_as_float(0x7fc00000);
-        out[(qrow0 + hh) * D + c] = __float2bfloat16_rn(r);
-    }
+    __shared__ float sred[16];
+    merge_partials<T, D, G>(part_u, splits, C.part_tau + (size_t)u * splits_tau * G * 2, splits_tau, out + qrow0 * D,
+                            C.status[u] != 0, sred);
     if (tid == 0) {
         C.n_unit[u] = n + 1;
         C.ticket2[u] = 0;
