@@ -459,19 +459,23 @@ __device__ __forceinline__ void merge_partials(const float* part, int np, const 
         if (lane == 0) { sred[g] = m; sred[8 + g] = tau; }
     }
     __syncthreads();
-    for (int o = threadIdx.x; o < G * D; o += blockDim.x) {
-        const int g = o / D, c = o % D;
+    for (int o = threadIdx.x; o < G * D / 2; o += blockDim.x) {       // two neighbouring columns per thread
+        const int g = (2 * o) / D, c = (2 * o) % D;
         const float m = sred[g], tau = sred[8 + g];
-        float z = 0.f;
+        float z0 = 0.f, z1 = 0.f;
 #pragma unroll 16
         for (int i = 0; i < np; ++i) {
             const float* pp = part + ((size_t)i * G + g) * STR;
-            const float pm = __ldcg(pp), pz = __ldcg(pp + 2 + c);
-            z += pm == -INFINITY ? 0.f : pz * __expf(pm - m);
+            const float pm = __ldcg(pp);
+            const float2 pz = __ldcg(reinterpret_cast<const float2*>(pp + 2 + c));     // rows are 8-byte aligned
+            const float sc = pm == -INFINITY ? 0.f : __expf(pm - m);
+            z0 = fmaf(pz.x, sc, z0);
+            z1 = fmaf(pz.y, sc, z1);
         }
-        float r = tau > 0.f ? z / tau : 0.f;
-        if (poisoned) r = __int_as_float(0x7fc00000);
-        out[(size_t)g * D + c] = Elem<T>::to_out(r);
+        float r0 = tau > 0.f ? z0 / tau : 0.f, r1 = tau > 0.f ? z1 / tau : 0.f;
+        if (poisoned) r0 = r1 = __int_as_float(0x7fc00000);
+        out[(size_t)g * D + c] = Elem<T>::to_out(r0);
+        out[(size_t)g * D + c + 1] = Elem<T>::to_out(r1);
     }
 }
 
