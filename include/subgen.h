@@ -57,6 +57,7 @@ extern "C" {
 /* sticky per-unit status bits */
 #define SUBGEN_ST_CAPACITY 1 /* a key had to open a cluster but m_max clusters exist */
 #define SUBGEN_ST_RANGE 2    /* non-finite input, or |x| > 32768 */
+#define SUBGEN_ST_TIMEOUT 4  /* a bounded wait inside a kernel ran out (not expected; the state is unusable) */
 
 typedef struct subgen subgen_t;
 typedef struct subgen_exact subgen_exact_t;

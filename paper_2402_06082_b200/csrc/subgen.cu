@@ -15,6 +15,7 @@
 #include "subgen_query_mma.cuh"
 #include "subgen_insert_mma.cuh"
 #include "subgen_prefill.cuh"
+#include "subgen_score_tc.cuh"
 #include "subgen_exact_mma.cuh"
 
 using namespace sgk;
@@ -167,6 +168,7 @@ struct subgen {
     char* scratch = nullptr;      // prefill scratch (library-owned, grows on demand)
     size_t scratch_bytes = 0;
     bool seq_prefill = false;     // SUBGEN_PREFILL=seq: token-by-token prefill also for bf16
+    bool tc_score = false;        // SUBGEN_PREFILL=tc: chunk scoring with tcgen05 instead of warp-level MMAs (d = 128)
 };
 
 namespace {
@@ -281,8 +283,9 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         const int hi = h->n_host[b] + add[b] > d.w ? h->n_host[b] + add[b] - d.w : 0;
         Lmax = hi - lo > Lmax ? hi - lo : Lmax;
     }
-    int slices = (148 * 4 + d.U - 1) / d.U;
-    slices = slices < 1 ? 1 : (slices > 16 ? 16 : slices);
+    const bool tc = D == 128 && h->tc_score;             // tcgen05 scoring (d = 128), else warp-level MMAs
+    int slices = tc ? (148 * 2) / d.U : (148 * 4 + d.U - 1) / d.U;
+    slices = slices < 1 ? 1 : (slices > 32 ? 32 : slices);
     PrefillArgs a;
     a.K = (const T*)K; a.V = (const T*)V; a.n_uniform = n; a.cu = cu_dev; a.total = total; a.Lmax = Lmax; a.slices = slices;
     a.Wbuf = nullptr; a.Tot = nullptr; a.Thr = nullptr; a.Mwin = nullptr; a.pbest = nullptr;
@@ -320,8 +323,14 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         prefill_gather_kernel<D><<<dim3(gx, d.U), 256, 0, h->st>>>(C, a);
         launches += 4;
         const int nchunks = (Lmax + kChunk - 1) / kChunk;
+        static bool configured = false;
+        if (tc && !configured) {
+            CUDA_TRY(cudaFuncSetAttribute(prefill_score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes));
+            configured = true;
+        }
         for (int c = 0; c < nchunks; ++c) {
-            prefill_score_kernel<D><<<dim3(slices, d.U), kScoreThreads, 0, h->st>>>(C, a, c);
+            if (tc) prefill_score_tc_kernel<<<dim3(slices, d.U), kTcThreads, kTcSmemBytes, h->st>>>(C, a, c);
+            else prefill_score_kernel<D><<<dim3(slices, d.U), kScoreThreads, 0, h->st>>>(C, a, c);
             prefill_resolve_kernel<D><<<d.U, kResolveThreads, 0, h->st>>>(C, a, c);
         }
         launches += 2 * nchunks;
@@ -410,7 +419,7 @@ subgen_t* subgen_create_ex(const subgen_config* cfg) {
         return nullptr;
     }
     h->n_host.assign(d.B, 0);
-    if (const char* env = getenv("SUBGEN_PREFILL")) h->seq_prefill = strcmp(env, "seq") == 0;
+    if (const char* env = getenv("SUBGEN_PREFILL")) { h->seq_prefill = strcmp(env, "seq") == 0; h->tc_score = strcmp(env, "tc") == 0; }
     return h;
 }
 

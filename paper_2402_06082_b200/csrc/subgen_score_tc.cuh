@@ -1,0 +1,250 @@
+// Prefill score kernel on the 5th-generation tensor cores (tcgen05), d = 128.
+//
+// One chunk of 128 keys (A, M = 128) against tiles of 128 representatives (B, N = 128): D[token][centre] =
+// <k, x> by tcgen05.mma.cta_group::1.kind::f16 (bf16 x bf16 -> fp32), K = 128 in eight K = 16 steps, the
+// accumulator in tensor memory (two buffers of 128 columns, so the MMAs of tile j+1 run while tile j is
+// read back). Operands sit in shared memory in the K-major 128-byte-swizzle layout the MMA descriptors
+// describe: 8-row groups of 128-byte rows (1024 bytes per group, 16-byte pieces XOR-ed with the row index
+// inside the group), one 16 KB block per 64-element half of d. The tiles are gathered with ordinary 16-byte
+// loads and stored straight into that layout (the rows of a unit are contiguous but the chunk may come from
+// the window ring, so no tensor map is involved), followed by a proxy fence before the MMA reads them.
+//
+// The MMA result is only a filter: a pair is flagged when <k,x> >= 1/2[(1-g)(||x||^2+||k||^2) - delta^2]
+// (the guard band of the insert kernel rearranged), and every flagged pair gets its exact fixed-point D2.
+// Each thread owns one token row of the accumulator (tensor-memory lane = row) and scans its 128 columns.
+//
+// Waits: the only wait is on the mbarrier that the MMA commit arrives on; it is bounded, and when the bound is
+// hit the block sets the unit's status bit 4, frees its tensor memory and returns.
+#pragma once
+#include "subgen_prefill.cuh"
+
+namespace sgk {
+
+constexpr int kTcThreads = 128;
+constexpr int kTcTileN = 128;
+constexpr int kTcCand = 1024;                    // flagged pairs kept per tile before the exhaustive fallback
+constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((kTcTileN >> 3) << 17) | ((128u >> 4) << 24);
+constexpr unsigned kTcSpinLimit = 1u << 22;
+
+struct TcSmem {                                  // after a 1024-byte aligned base
+    unsigned char A[2 * 128 * 128];              // chunk keys: [half of d][row][128 B swizzled]
+    unsigned char B[2][2 * kTcTileN * 128];      // two buffers of representatives, same layout
+    float kn[kChunk];                            // 1/2 ((1-g) ||k||^2 - delta^2) per token
+    float xa[2][kTcTileN];                       // 1/2 (1-g) ||x||^2 per representative of the tile (+inf: no row)
+    unsigned long long wb_d2[4][kChunk];         // per warp: best exact (D2, index) per token
+    int wb_idx[4][kChunk];
+    unsigned cand[kTcCand];                      // token | row_in_tile << 8
+    unsigned long long mbar[2];
+    unsigned tmem_base, ncand, failed;
+};
+constexpr size_t kTcSmemBytes = sizeof(TcSmem) + 1024;
+
+__device__ __forceinline__ uint32_t sw128_offset(int row, int piece16) {      // piece16: 0..15 over the 256-byte row
+    return (uint32_t)((piece16 >> 3) * (128 * 128) + row * 128 + (((piece16 & 7) ^ (row & 7)) << 4));
+}
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+    // start address >> 4 | LBO = 1 (16 B) << 16 | SBO = 1024 B >> 4 << 32 | version 1 << 46 | layout SWIZZLE_128B (2) << 61
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+__global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<__nv_bfloat16> C, PrefillArgs a, int chunk) {
+    typedef __nv_bfloat16 T;
+    constexpr int D = 128, LPR = 16;
+    extern __shared__ unsigned char dyn_raw[];
+    TcSmem& sm = *reinterpret_cast<TcSmem*>((reinterpret_cast<uintptr_t>(dyn_raw) + 1023) & ~(uintptr_t)1023);
+    const int u = blockIdx.y, slices = gridDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const Range r = unit_range(C, a, u);
+    const int e0 = r.ins_lo + chunk * kChunk, cl = min(kChunk, r.ins_hi - e0);
+    if (cl <= 0) return;
+    const int m = C.m_unit[u];
+    Best* outp = a.pbest + ((size_t)u * slices + blockIdx.x) * kChunk;
+    const int per = (((m + slices - 1) / slices) + kTcTileN - 1) / kTcTileN * kTcTileN;
+    const int c0 = blockIdx.x * per, c1 = min(m, c0 + per);
+    if (c0 >= c1) {
+        for (int j = tid; j < kChunk; j += kTcThreads) { Best bb; bb.d2 = ~0ull; bb.idx = INT_MAX; bb.pad = 0; outp[j] = bb; }
+        return;
+    }
+    const T* Xu = C.X + (size_t)u * C.m_max * D;
+    const float* xnu = C.xn + (size_t)u * C.m_max;
+    const float d2f = (float)((double)C.delta2_fx * (1.0 / 4294967296.0));
+    constexpr float kOneMinusG = 1.f - 1.220703125e-4f;
+    const uint32_t sA = (uint32_t)__cvta_generic_to_shared(sm.A);
+    const uint32_t sB0 = (uint32_t)__cvta_generic_to_shared(sm.B[0]), sB1 = (uint32_t)__cvta_generic_to_shared(sm.B[1]);
+    const uint32_t sBar0 = (uint32_t)__cvta_generic_to_shared(&sm.mbar[0]), sBar1 = (uint32_t)__cvta_generic_to_shared(&sm.mbar[1]);
+
+    // ---- set-up: tensor memory (256 columns), barriers, the chunk ----
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(&sm.tmem_base)), "r"(256u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sBar0) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sBar1) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        sm.ncand = 0;
+        sm.failed = 0;
+    }
+    for (int p = tid; p < kChunk * LPR; p += kTcThreads) {            // chunk keys -> A (rows beyond cl are zero)
+        const int j = p / LPR, q = p % LPR;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (j < cl) v = reinterpret_cast<const uint4*>(key_row<D>(C, a, r, u, e0 + j))[q];
+        *reinterpret_cast<uint4*>(sm.A + sw128_offset(j, q)) = v;
+    }
+    for (int j = tid; j < 4 * kChunk; j += kTcThreads) { sm.wb_d2[j / kChunk][j % kChunk] = ~0ull; sm.wb_idx[j / kChunk][j % kChunk] = INT_MAX; }
+    __syncthreads();
+    {
+        const int j = tid;                                             // one token per thread
+        float acc = 0.f;
+        for (int q = 0; q < LPR; ++q) {
+            float f[8];
+            Elem<T>::unpack(*reinterpret_cast<const uint4*>(sm.A + sw128_offset(j, q)), f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc = fmaf(f[e], f[e], acc);
+        }
+        sm.kn[j] = 0.5f * (kOneMinusG * acc - d2f);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = sm.tmem_base;
+    const float my_kn = sm.kn[tid];
+    const int ntiles = (c1 - c0 + kTcTileN - 1) / kTcTileN;
+
+    auto load_tile = [&](int j, int buf) {                            // representatives of tile j -> B[buf], xa[buf]
+        const int row0 = c0 + j * kTcTileN;
+        unsigned char* dst = sm.B[buf];
+        for (int p = tid; p < kTcTileN * LPR; p += kTcThreads) {
+            const int rr = p / LPR, q = p % LPR;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (row0 + rr < c1) v = ldg16(Xu + (size_t)(row0 + rr) * D + q * 8);
+            *reinterpret_cast<uint4*>(dst + sw128_offset(rr, q)) = v;
+        }
+        sm.xa[buf][tid] = row0 + tid < c1 ? 0.5f * kOneMinusG * xnu[row0 + tid] : INFINITY;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy stores -> visible to the MMA
+    };
+    auto issue_mma = [&](int buf) {                                    // one thread: 8 MMAs of K = 16, then commit
+        const uint32_t sBb = buf ? sB1 : sB0;
+        const uint32_t dcol = tmem + (uint32_t)(buf * kTcTileN);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t off = (uint32_t)((ks >> 2) * (128 * 128) + (ks & 3) * 32);
+            const uint64_t da = umma_desc_sw128(sA + off), db = umma_desc_sw128(sBb + off);
+            const uint32_t accum = ks ? 1u : 0u;
+            asm volatile(
+                "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
+                ::"r"(dcol), "l"(da), "l"(db), "r"(kTcIdesc), "r"(accum), "r"(0u) : "memory");
+        }
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(buf ? sBar1 : sBar0) : "memory");
+    };
+    // exact D2 of (token tokj, representative row), by one warp; keeps the warp's best per token
+    auto exact_pair = [&](int tokj, int row) {
+        unsigned long long acc = 0;
+        if (lane < LPR) {
+            float xf[8], kf[8];
+            Elem<T>::unpack(*reinterpret_cast<const uint4*>(Xu + (size_t)row * D + lane * 8), xf);
+            Elem<T>::unpack(*reinterpret_cast<const uint4*>(sm.A + sw128_offset(tokj, lane)), kf);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc += fx_sqdiff(xf[e], kf[e]);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        if (lane == 0) {
+            Best cur;
+            cur.d2 = sm.wb_d2[warp][tokj]; cur.idx = sm.wb_idx[warp][tokj];
+            if (better(acc, row, cur)) { sm.wb_d2[warp][tokj] = acc; sm.wb_idx[warp][tokj] = row; }
+        }
+    };
+
+    load_tile(0, 0);
+    __syncthreads();
+    if (tid == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        issue_mma(0);
+    }
+    bool ok = true;
+    for (int j = 0; j < ntiles; ++j) {
+        const int buf = j & 1;
+        if (j + 1 < ntiles) {                                           // next tile: load, then start its MMAs
+            load_tile(j + 1, buf ^ 1);
+            __syncthreads();
+            if (tid == 0) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                issue_mma(buf ^ 1);
+            }
+        }
+        // wait for the MMAs of tile j (bounded)
+        {
+            const uint32_t bar = buf ? sBar1 : sBar0, parity = (uint32_t)((j >> 1) & 1);
+            unsigned done = 0, spins = 0;
+            while (!done && spins < kTcSpinLimit) {
+                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                             : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+                ++spins;
+            }
+            if (!done) sm.failed = 1;
+        }
+        __syncthreads();
+        if (sm.failed) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        // epilogue: this thread's token row, 128 columns in four pieces of 32
+        const float* xat = sm.xa[buf];
+#pragma unroll 1
+        for (int cc = 0; cc < kTcTileN; cc += 32) {
+            uint32_t v[32];
+            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * kTcTileN + cc);
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                  "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+                  "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+                  "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                : "r"(taddr) : "memory");
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (tid < cl) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    if (__uint_as_float(v[i]) >= xat[cc + i] + my_kn) {          // rare
+                        const unsigned slot = atomicAdd(&sm.ncand, 1u);
+                        if (slot < (unsigned)kTcCand) sm.cand[slot] = (unsigned)tid | ((unsigned)(cc + i) << 8);
+                    }
+                }
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        // exact distances of the flagged pairs of this tile
+        const unsigned nc = sm.ncand;
+        const int row0 = c0 + j * kTcTileN;
+        if (nc <= (unsigned)kTcCand) {
+            for (unsigned i = warp; i < nc; i += kTcThreads / 32) {
+                const unsigned cd = sm.cand[i];
+                exact_pair((int)(cd & 255u), row0 + (int)(cd >> 8));
+            }
+        } else {                                                          // too many to list: every pair of the tile
+            const int nrow = min(kTcTileN, c1 - row0);
+            for (int i = warp; i < cl * nrow; i += kTcThreads / 32) exact_pair(i / nrow, row0 + i % nrow);
+        }
+        __syncthreads();
+        if (tid == 0) sm.ncand = 0;
+    }
+    __syncthreads();
+    if (ok) {
+        for (int j = tid; j < kChunk; j += kTcThreads) {
+            Best bb;
+            bb.d2 = sm.wb_d2[0][j]; bb.idx = sm.wb_idx[0][j]; bb.pad = 0;
+            for (int wv = 1; wv < 4; ++wv)
+                if (better(sm.wb_d2[wv][j], sm.wb_idx[wv][j], bb)) { bb.d2 = sm.wb_d2[wv][j]; bb.idx = sm.wb_idx[wv][j]; }
+            outp[j] = bb;
+        }
+    } else {
+        for (int j = tid; j < kChunk; j += kTcThreads) { Best bb; bb.d2 = ~0ull; bb.idx = INT_MAX; bb.pad = 0; outp[j] = bb; }
+        if (tid == 0) atomicOr(&C.status[u], 4);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
+}
+
+}  // namespace sgk
