@@ -168,7 +168,7 @@ struct subgen {
     char* scratch = nullptr;      // prefill scratch (library-owned, grows on demand)
     size_t scratch_bytes = 0;
     bool seq_prefill = false;     // SUBGEN_PREFILL=seq: token-by-token prefill also for bf16
-    bool tc_score = false;        // SUBGEN_PREFILL=tc: chunk scoring with tcgen05 instead of warp-level MMAs (d = 128)
+    bool mma_score = false;       // SUBGEN_PREFILL=mma: chunk scoring with warp-level MMAs instead of tcgen05 (d = 128)
 };
 
 namespace {
@@ -283,7 +283,7 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         const int hi = h->n_host[b] + add[b] > d.w ? h->n_host[b] + add[b] - d.w : 0;
         Lmax = hi - lo > Lmax ? hi - lo : Lmax;
     }
-    const bool tc = D == 128 && h->tc_score;             // tcgen05 scoring (d = 128), else warp-level MMAs
+    const bool tc = D == 128 && !h->mma_score;           // tcgen05 scoring (d = 128), else warp-level MMAs
     int slices = tc ? (148 * 2) / d.U : (148 * 4 + d.U - 1) / d.U;
     slices = slices < 1 ? 1 : (slices > 32 ? 32 : slices);
     PrefillArgs a;
@@ -419,7 +419,7 @@ subgen_t* subgen_create_ex(const subgen_config* cfg) {
         return nullptr;
     }
     h->n_host.assign(d.B, 0);
-    if (const char* env = getenv("SUBGEN_PREFILL")) { h->seq_prefill = strcmp(env, "seq") == 0; h->tc_score = strcmp(env, "tc") == 0; }
+    if (const char* env = getenv("SUBGEN_PREFILL")) { h->seq_prefill = strcmp(env, "seq") == 0; h->mma_score = strcmp(env, "mma") == 0; }
     return h;
 }
 

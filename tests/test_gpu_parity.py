@@ -283,23 +283,37 @@ def test_chunked_prefill_equals_token_by_token_prefill(monkeypatch):
     kernel. Both must leave the same state, also when a call continues a stream whose tail is in the window."""
     w = synth.CFG3.scaled(B=2, H=4, Hkv=2, n_prompt=1000, ncomp=24, s=96, t=6, window=48, m_max=512)
     K, V, _ = synth.batch_stream(w, 1000, "cuda")
-    a = _sg(w)
+    a = _sg(w)                                   # d = 128: chunk scoring with tcgen05
     monkeypatch.setenv("SUBGEN_PREFILL", "seq")
     b = _sg(w)
+    monkeypatch.setenv("SUBGEN_PREFILL", "mma")  # chunk scoring with warp-level MMAs
+    c = _sg(w)
     monkeypatch.delenv("SUBGEN_PREFILL")
     for lo, hi in ((0, 7), (7, 300), (300, 301), (301, 1000)):
-        a.prefill(K[:, :, lo:hi].contiguous(), V[:, :, lo:hi].contiguous())
-        b.prefill(K[:, :, lo:hi].contiguous(), V[:, :, lo:hi].contiguous())
+        for sg in (a, b, c):
+            sg.prefill(K[:, :, lo:hi].contiguous(), V[:, :, lo:hi].contiguous())
         for bb in range(w.B):
             for h in range(w.Hkv):
-                s1, s2 = a.export_state(bb, h), b.export_state(bb, h)
-                for key in ("m", "mu", "n", "last_cluster", "last_opened", "status"):
-                    assert s1[key] == s2[key], (key, lo, hi)
-                for key in ("counts", "centre_tok", "slot_tok", "m_tok", "m_w"):
-                    np.testing.assert_array_equal(s1[key], s2[key], err_msg="%s after [%d,%d)" % (key, lo, hi))
-                hp.assert_rows_match_tokens(a, bb, h, s1, K[bb, h], V[bb, h])
+                s2 = b.export_state(bb, h)
                 hp.assert_rows_match_tokens(b, bb, h, s2, K[bb, h], V[bb, h])
+                for sg in (a, c):
+                    s1 = sg.export_state(bb, h)
+                    for key in ("m", "mu", "n", "last_cluster", "last_opened", "status"):
+                        assert s1[key] == s2[key], (key, lo, hi)
+                    for key in ("counts", "centre_tok", "slot_tok", "m_tok", "m_w"):
+                        np.testing.assert_array_equal(s1[key], s2[key], err_msg="%s after [%d,%d)" % (key, lo, hi))
+                    hp.assert_rows_match_tokens(sg, bb, h, s1, K[bb, h], V[bb, h])
     assert a.launch_count > b.launch_count
+
+
+def test_tcgen05_scoring_many_tiles_and_dense_candidates():
+    """Several 128-representative tiles per chunk, and a radius so large that every pair is inside the guard band
+    (the exhaustive path of the score kernel): state must equal the oracle's."""
+    w = synth.CFG3.scaled(B=1, H=2, Hkv=2, n_prompt=2500, ncomp=400, s=64, t=4, window=16, m_max=1024)
+    _run_stream(w, 2500, 4)
+    w = synth.CFG2.scaled(B=1, H=1, Hkv=1, n_prompt=600, ncomp=4, sigma=0.5, delta=30.0, s=32, t=4, window=8, m_max=64)
+    _, orcs, _ = _run_stream(w, 600, 4)
+    assert orcs[(0, 0)].m == 1
 
 
 def test_prefill_capacity_overflow_is_reported():
