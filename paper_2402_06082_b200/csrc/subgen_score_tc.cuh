@@ -110,16 +110,27 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
     const float my_kn = sm.kn[tid];
     const int ntiles = (c1 - c0 + kTcTileN - 1) / kTcTileN;
 
-    auto load_tile = [&](int j, int buf) {                            // representatives of tile j -> B[buf], xa[buf]
+    // representatives of tile j: global -> registers (tile_fetch), registers -> B[buf], xa[buf] (tile_store)
+    uint4 R[kTcTileN * LPR / kTcThreads];
+    float xr = INFINITY;
+    auto tile_fetch = [&](int j) {
         const int row0 = c0 + j * kTcTileN;
-        unsigned char* dst = sm.B[buf];
-        for (int p = tid; p < kTcTileN * LPR; p += kTcThreads) {
-            const int rr = p / LPR, q = p % LPR;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (row0 + rr < c1) v = ldg16(Xu + (size_t)(row0 + rr) * D + q * 8);
-            *reinterpret_cast<uint4*>(dst + sw128_offset(rr, q)) = v;
+#pragma unroll
+        for (int i = 0; i < kTcTileN * LPR / kTcThreads; ++i) {
+            const int p = i * kTcThreads + tid, rr = p / LPR, q = p % LPR;
+            R[i] = make_uint4(0, 0, 0, 0);
+            if (row0 + rr < c1) R[i] = ldg16(Xu + (size_t)(row0 + rr) * D + q * 8);
         }
-        sm.xa[buf][tid] = row0 + tid < c1 ? 0.5f * kOneMinusG * xnu[row0 + tid] : INFINITY;
+        xr = row0 + tid < c1 ? 0.5f * kOneMinusG * xnu[row0 + tid] : INFINITY;
+    };
+    auto tile_store = [&](int buf) {
+        unsigned char* dst = sm.B[buf];
+#pragma unroll
+        for (int i = 0; i < kTcTileN * LPR / kTcThreads; ++i) {
+            const int p = i * kTcThreads + tid;
+            *reinterpret_cast<uint4*>(dst + sw128_offset(p / LPR, p % LPR)) = R[i];
+        }
+        sm.xa[buf][tid] = xr;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy stores -> visible to the MMA
     };
     auto issue_mma = [&](int buf) {                                    // one thread: 8 MMAs of K = 16, then commit
@@ -156,23 +167,22 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
         }
     };
 
-    load_tile(0, 0);
+    // Pipeline: the MMAs of tile j+1 run while tile j is read back, and the global loads of tile j+2 are in
+    // flight (in registers) during both; they are stored once the MMAs of tile j have released their buffer.
+    tile_fetch(0);
+    tile_store(0);
+    if (ntiles > 1) { tile_fetch(1); tile_store(1); }
     __syncthreads();
     if (tid == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         issue_mma(0);
+        if (ntiles > 1) issue_mma(1);
     }
     bool ok = true;
     for (int j = 0; j < ntiles; ++j) {
         const int buf = j & 1;
-        if (j + 1 < ntiles) {                                           // next tile: load, then start its MMAs
-            load_tile(j + 1, buf ^ 1);
-            __syncthreads();
-            if (tid == 0) {
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                issue_mma(buf ^ 1);
-            }
-        }
+        const bool has2 = j + 2 < ntiles;
+        if (has2) tile_fetch(j + 2);
         // wait for the MMAs of tile j (bounded)
         {
             const uint32_t bar = buf ? sBar1 : sBar0, parity = (uint32_t)((j >> 1) & 1);
@@ -228,6 +238,14 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
         }
         __syncthreads();
         if (tid == 0) sm.ncand = 0;
+        if (has2) {                                                       // buffer and accumulator `buf` are free now
+            tile_store(buf);
+            __syncthreads();
+            if (tid == 0) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                issue_mma(buf);
+            }
+        }
     }
     __syncthreads();
     if (ok) {
