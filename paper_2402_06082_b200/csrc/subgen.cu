@@ -83,13 +83,13 @@ bool resolve(const subgen_config* c, Dims* o, const char** why) {
     } else {
         // Aim at one resident wave: the kernels hand out work inside a unit dynamically, so blocks that are all
         // resident finish together, while a partial second wave leaves most SMs idle at the end.
-        // Resident blocks per SM: insert 6 (128 threads), cluster scan 12 (64 threads), value scan 4 (128 threads).
+        // Resident blocks per SM (128 threads each): insert 6, cluster scan 6, value scan 4.
         auto fit = [&](int per_sm, int lo) {
             int sp = (148 * per_sm) / d.U;
             return sp < lo ? lo : (sp > 64 ? 64 : sp);
         };
         if (bf16) {
-            d.sp_insert = fit(6, 1); d.sp_tau = fit(12, 1); d.sp_z = fit(4, 1);
+            d.sp_insert = fit(6, 1); d.sp_tau = fit(6, 1); d.sp_z = fit(4, 1);
             if (d.sp_z > 16) d.sp_z = 16;      // the last block merges sp_z numerator partials of G*d floats each
         }
         else { d.sp_insert = d.sp_tau = d.sp_z = fit(8, 1); }
@@ -202,16 +202,16 @@ template <typename T, int D>
 void launch_query(const Cache<T>& C, int G, dim3 grid, dim3 grid_z, cudaStream_t st, const void* q, void* out, cudaEvent_t mid) {
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
         switch (G) {
-            case 1: query_tau_kernel<D, 1><<<grid, kTauThreads, 0, st>>>(C, (const T*)q);
+            case 1: query_tau_kernel<D, 1><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
                     query_z_kernel<D, 1><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
-            case 2: query_tau_kernel<D, 2><<<grid, kTauThreads, 0, st>>>(C, (const T*)q);
+            case 2: query_tau_kernel<D, 2><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
                     query_z_kernel<D, 2><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
-            case 4: query_tau_kernel<D, 4><<<grid, kTauThreads, 0, st>>>(C, (const T*)q);
+            case 4: query_tau_kernel<D, 4><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
                     query_z_kernel<D, 4><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
-            default: query_tau_kernel<D, 8><<<grid, kTauThreads, 0, st>>>(C, (const T*)q);
+            default: query_tau_kernel<D, 8><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
                      query_z_kernel<D, 8><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
         }

@@ -29,7 +29,6 @@
 namespace sgk {
 
 constexpr int kQmThreads = 128;
-constexpr int kTauThreads = 64;        // cluster scan: small blocks fill the SMs more evenly (12 resident per SM)
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
@@ -150,9 +149,9 @@ __device__ __forceinline__ int div_small(int r, unsigned magic) { return magic ?
 // Clusters: tau_D = sum over clusters of n'/t sum over the t samples of exp<q,k>; a cluster with n' = 1
 // is read as its representative with weight 1. Writes per block {max, tau} per head to part_tau.
 template <int D, int G>
-__global__ void __launch_bounds__(kTauThreads, 12) query_tau_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ q) {
+__global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ q) {
     typedef __nv_bfloat16 T;
-    constexpr int NC = D / 32, NW = kTauThreads / 32;
+    constexpr int NC = D / 32, NW = kQmThreads / 32;
     __shared__ float sm[NW][G][2];
     __shared__ int lst[NW][16], wcn[NW][16];
     const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
