@@ -46,6 +46,20 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def tensor_roofline(pairs, d, ms):
+    """The prefill's scoring contraction: 2*d flops per (key, representative) pair against the measured bf16 peak."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak, src = 1590.0, "fallback"
+    if os.path.exists(p):
+        with open(p) as f:
+            peak, src = float(json.load(f)["bf16_tflops"]), "measured"
+    if not ms or not pairs:
+        return None
+    tf = 2.0 * d * pairs / (ms * 1e-3) / 1e12
+    return {"bound": "tensor", "flops": 2.0 * d * pairs, "ms": ms, "achieved": tf, "peak": peak, "peak_source": src,
+            "unit": "TFLOP/s", "frac": tf / peak}
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU every 50 ms through NVML while running."""
 
@@ -241,6 +255,7 @@ def run_subgen(args, w):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
     # ---- prefill (timed on its own) ----
+    sg.profile_enable(True)
     l0 = sg.launch_count
     e0.record()
     if varlen:
@@ -252,6 +267,9 @@ def run_subgen(args, w):
     torch.cuda.synchronize()
     prefill_ms = e0.elapsed_time(e1)
     prefill_launches = sg.launch_count - l0
+    pf_values_ms, pf_score_ms, pf_resolve_ms = sg.profile_prefill_read()
+    sg.profile_enable(False)
+    pf_pairs = sg.cache_stats()["prefill_pairs"]
     st = sg.status()
     if st:
         raise SystemExit("device status %d after prefill (1 = cluster capacity, 2 = input range)" % st)
@@ -337,6 +355,8 @@ def run_subgen(args, w):
 
     extra = {"prefill_ms": prefill_ms, "prefill_tokens_per_s": sum(lens) / (prefill_ms * 1e-3),
              "prefill_launches": prefill_launches,
+             "prefill_phases_ms": {"values": pf_values_ms, "score": pf_score_ms, "resolve": pf_resolve_ms},
+             "prefill_score": tensor_roofline(pf_pairs, wr.d, pf_score_ms),
              "cache": {k: stats1[k] for k in ("clusters", "singleton_clusters", "m_filled", "window_rows", "tokens")}}
 
     # ---- exact dense decode over full caches on the same inputs (comparison point) ----

@@ -149,6 +149,7 @@ typedef struct subgen_stats {
     uint64_t m_filled;           /* non-null M slots */
     uint64_t window_rows;        /* tokens currently in the windows */
     uint64_t tokens;             /* sum of n */
+    uint64_t prefill_pairs;      /* (key, representative) pairs the chunked prefill has scored: 2*d flops each */
     uint64_t insert_bytes;       /* bytes one step must read to place a key: the representatives */
     uint64_t query_bytes;        /* bytes one step must read to answer the queries: cluster_bytes + value_bytes */
     uint64_t cluster_bytes;      /* cluster samples (t rows, or the representative alone while n_i = 1) and counts */
@@ -165,6 +166,9 @@ int subgen_cache_stats(subgen_t* h, subgen_stats* out);
  * handles the whole query is one kernel, reported in ms[1], and ms[2] is 0. */
 int subgen_profile_enable(subgen_t* h, int on);
 int subgen_profile_read(subgen_t* h, double ms[3], int* steps);
+/* Phases of the most recent chunked prefill call made while profiling was enabled: ms[0] value phase (W, scan,
+ * coins, gather), ms[1] sum over chunks of the score kernel, ms[2] sum over chunks of the resolve kernel. */
+int subgen_profile_prefill_read(subgen_t* h, double ms[3]);
 
 /* Number of kernels this handle has launched so far. */
 uint64_t subgen_launch_count(const subgen_t* h);

@@ -22,7 +22,7 @@ ST_CAPACITY, ST_RANGE = 1, 2
 EXPORTS = [
     "subgen_workspace_bytes", "subgen_create", "subgen_create_ex", "subgen_destroy", "subgen_prefill",
     "subgen_prefill_varlen", "subgen_step", "subgen_step_host", "subgen_status", "subgen_export_state",
-    "subgen_export_rows", "subgen_cache_stats", "subgen_profile_enable", "subgen_profile_read",
+    "subgen_export_rows", "subgen_cache_stats", "subgen_profile_enable", "subgen_profile_read", "subgen_profile_prefill_read",
     "subgen_launch_count", "subgen_last_error", "subgen_exact_create", "subgen_exact_destroy",
     "subgen_exact_append", "subgen_exact_append_varlen", "subgen_exact_step", "subgen_exact_bytes",
     "subgen_exact_launch_count", "subgen_exact_attention_noalloc",
@@ -45,7 +45,7 @@ class StateView(C.Structure):
 
 class Stats(C.Structure):
     _fields_ = [(k, C.c_uint64) for k in ("units", "clusters", "singleton_clusters", "m_filled", "window_rows",
-                                           "tokens", "insert_bytes", "query_bytes", "cluster_bytes", "value_bytes")]
+                                           "tokens", "prefill_pairs", "insert_bytes", "query_bytes", "cluster_bytes", "value_bytes")]
 
 
 _lib = None
@@ -79,6 +79,7 @@ def load():
     L.subgen_cache_stats.argtypes = [vp, C.POINTER(Stats)]
     L.subgen_profile_enable.argtypes = [vp, C.c_int]
     L.subgen_profile_read.argtypes = [vp, C.POINTER(C.c_double), ip]
+    L.subgen_profile_prefill_read.argtypes = [vp, C.POINTER(C.c_double)]
     L.subgen_launch_count.argtypes = [vp]
     L.subgen_launch_count.restype = C.c_uint64
     L.subgen_last_error.restype = C.c_char_p
@@ -225,6 +226,12 @@ class SubGen:
         ms, n = (C.c_double * 3)(), C.c_int()
         _check(self._L.subgen_profile_read(self._h, ms, C.byref(n)))
         return ms[0], ms[1], ms[2], n.value
+
+    def profile_prefill_read(self):
+        """(value_phase_ms, score_ms, resolve_ms) of the last chunked prefill made with profiling enabled."""
+        ms = (C.c_double * 3)()
+        _check(self._L.subgen_profile_prefill_read(self._h, ms))
+        return ms[0], ms[1], ms[2]
 
     @property
     def launch_count(self) -> int:

@@ -45,7 +45,7 @@ size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
     size_t X, S, xn, cnt, ctok, stok, Mk, Mv, MW, Mtok, ringK, ringV;
-    size_t n_unit, m_unit, mu, status, last_cid, last_open, last_d2, part1, part2, ticket1, ticket2, qnext, qnext2, part_tau, MinvW;
+    size_t n_unit, m_unit, mu, status, last_cid, last_open, last_d2, part1, part2, ticket1, ticket2, qnext, qnext2, part_tau, MinvW, pairs;
     size_t stage_q, stage_k, stage_v, stage_out, cu, stats;
     size_t book_begin, book_end;   // bookkeeping region cleared at creation
     size_t total;
@@ -137,6 +137,7 @@ Layout make_layout(const Dims& d) {
     L.ticket2 = take(U * sizeof(unsigned));
     L.qnext = take(U * sizeof(unsigned));
     L.qnext2 = take(U * sizeof(unsigned));
+    L.pairs = take(U * sizeof(uint64_t));
     L.MinvW = take(U * d.s * sizeof(float));
     L.MW = take(U * d.s * sizeof(uint64_t));
     L.stats = take(8 * sizeof(uint64_t));
@@ -165,6 +166,8 @@ struct subgen {
     bool prof = false;
     std::vector<cudaEvent_t> ev;  // four per profiled step
     size_t ev_used = 0;
+    std::vector<cudaEvent_t> pev; // prefill: start, after the value phase, then (score, resolve) ends per chunk, end
+    size_t pev_used = 0;
     char* scratch = nullptr;      // prefill scratch (library-owned, grows on demand)
     size_t scratch_bytes = 0;
     bool seq_prefill = false;     // SUBGEN_PREFILL=seq: token-by-token prefill also for bf16
@@ -194,6 +197,7 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
     C.ticket1 = (unsigned*)(w + L.ticket1); C.ticket2 = (unsigned*)(w + L.ticket2);
     C.qnext = (unsigned*)(w + L.qnext); C.qnext2 = (unsigned*)(w + L.qnext2);
     C.part_tau = (float*)(w + L.part_tau); C.MinvW = (float*)(w + L.MinvW);
+    C.pairs = (unsigned long long*)(w + L.pairs);
     return C;
 }
 
@@ -305,6 +309,18 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         a.Thr = (unsigned long long*)(h->scratch + 2 * b_w);
         a.Mwin = (int*)(h->scratch + 3 * b_w);
         a.pbest = (Best*)(h->scratch + 3 * b_w + b_m);
+        auto mark = [&]() -> int {                       // profiling: one event on the stream
+            if (!h->prof) return SUBGEN_OK;
+            if (h->pev_used == h->pev.size()) {
+                cudaEvent_t x;
+                CUDA_TRY(cudaEventCreate(&x));
+                h->pev.push_back(x);
+            }
+            CUDA_TRY(cudaEventRecord(h->pev[h->pev_used++], h->st));
+            return SUBGEN_OK;
+        };
+        h->pev_used = 0;
+        if (int rc = mark()) return rc;
         CUDA_TRY(cudaMemsetAsync(a.Mwin, 0xFF, (size_t)d.U * d.s * 4, h->st));
         constexpr int RPW = 32 / (D / 8);
         int bx = (Lmax + 8 * RPW - 1) / (8 * RPW);
@@ -322,6 +338,7 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         gx = gx > 32 ? 32 : gx;
         prefill_gather_kernel<D><<<dim3(gx, d.U), 256, 0, h->st>>>(C, a);
         launches += 4;
+        if (int rc = mark()) return rc;
         const int nchunks = (Lmax + kChunk - 1) / kChunk;
         static bool configured = false;
         if (tc && !configured) {
@@ -331,7 +348,9 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         for (int c = 0; c < nchunks; ++c) {
             if (tc) prefill_score_tc_kernel<<<dim3(slices, d.U), kTcThreads, kTcSmemBytes, h->st>>>(C, a, c);
             else prefill_score_kernel<D><<<dim3(slices, d.U), kScoreThreads, 0, h->st>>>(C, a, c);
+            if (int rc = mark()) return rc;
             prefill_resolve_kernel<D><<<d.U, kResolveThreads, 0, h->st>>>(C, a, c);
+            if (int rc = mark()) return rc;
         }
         launches += 2 * nchunks;
     }
@@ -435,6 +454,7 @@ void subgen_destroy(subgen_t* h) {
     if (!h) return;
     cudaStreamSynchronize(h->st);
     for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
+    for (cudaEvent_t e : h->pev) cudaEventDestroy(e);
     if (h->owns) cudaFree(h->ws);
     if (h->scratch) cudaFree(h->scratch);
     delete h;
@@ -578,6 +598,7 @@ int subgen_cache_stats(subgen_t* h, subgen_stats* out) {
     const uint64_t row = (uint64_t)h->d.D * h->d.E;
     out->units = h->d.U;
     out->clusters = r[0]; out->singleton_clusters = r[1]; out->m_filled = r[2]; out->window_rows = r[3]; out->tokens = r[4];
+    out->prefill_pairs = r[5];
     out->insert_bytes = r[0] * row;
     out->cluster_bytes = (r[1] + (r[0] - r[1]) * (uint64_t)h->d.t) * row + r[0] * 4;
     out->value_bytes = (2 * r[2] + 2 * r[3]) * row + (uint64_t)h->d.U * h->d.s * 4;
@@ -605,6 +626,27 @@ int subgen_profile_read(subgen_t* h, double* ms, int* steps) {
     if (ms) { ms[0] = acc[0]; ms[1] = acc[1]; ms[2] = acc[2]; }
     if (steps) *steps = (int)(h->ev_used / 4);
     h->ev_used = 0;
+    return SUBGEN_OK;
+}
+
+int subgen_profile_prefill_read(subgen_t* h, double* ms) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_profile_prefill_read: handle is NULL");
+    CUDA_TRY(cudaStreamSynchronize(h->st));
+    double acc[3] = {0, 0, 0};
+    if (h->pev_used >= 2) {
+        float x = 0;
+        CUDA_TRY(cudaEventElapsedTime(&x, h->pev[0], h->pev[1]));
+        acc[0] = x;
+        for (size_t i = 1; i + 2 < h->pev_used; i += 2) {       // chunk: events i -> i+1 (score) -> i+2 (resolve)
+            float sc = 0, rs = 0;
+            CUDA_TRY(cudaEventElapsedTime(&sc, h->pev[i], h->pev[i + 1]));
+            CUDA_TRY(cudaEventElapsedTime(&rs, h->pev[i + 1], h->pev[i + 2]));
+            acc[1] += sc;
+            acc[2] += rs;
+        }
+    }
+    if (ms) { ms[0] = acc[0]; ms[1] = acc[1]; ms[2] = acc[2]; }
+    h->pev_used = 0;
     return SUBGEN_OK;
 }
 

@@ -111,6 +111,7 @@ template <typename T> struct Cache {
     float* part_tau;     // [U, splits, G, 2] cluster partials {max, tau} of the query
     unsigned* qnext;     // [U] next work item of the cluster scan's per-unit queue
     unsigned* qnext2;    // [U] same for the scan of M and the window
+    unsigned long long* pairs;   // [U] (key, representative) pairs scored by the chunked prefill so far
 };
 
 // ---------------------------------------------------------------------------------------------

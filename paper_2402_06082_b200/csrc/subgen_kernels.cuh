@@ -282,6 +282,7 @@ __global__ void stats_kernel(Cache<T> C, int U, unsigned long long* out) {
         atomicAdd(&out[0], (unsigned long long)m);
         atomicAdd(&out[3], (unsigned long long)min(n, C.w));
         atomicAdd(&out[4], (unsigned long long)n);
+        atomicAdd(&out[5], C.pairs[u]);
     }
 }
 

@@ -481,6 +481,7 @@ __global__ void __launch_bounds__(kResolveThreads) prefill_resolve_kernel(Cache<
     }
     __syncthreads();
     if (tid == 0) {
+        C.pairs[u] += (unsigned long long)cl * (unsigned long long)m_old;
         C.m_unit[u] = m_old + sm_opened;
         if (sm_full) atomicOr(&C.status[u], 1);
         const int j = cl - 1;
