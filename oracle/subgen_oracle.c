@@ -366,3 +366,39 @@ const uint64_t *oracle_ins_d2(const oracle_unit *u) { return u->ins_d2; }
 const int *oracle_ins_near(const oracle_unit *u) { return u->ins_near; }
 uint64_t oracle_dist2_fx(const float *x, const float *k, int d) { return dist2_fx(x, k, d); }
 uint64_t oracle_norm2_fx(const float *v, int d) { return norm2_fx(v, d); }
+
+/* ------------------------------------------------------------------------ */
+/* Offline greedy k-center compression with a recent-token window: the variant the paper's end-to-end
+ * experiment ran (Section 3.2: keep the most recent r tokens and k centres chosen from the remaining tokens by
+ * the greedy k-center algorithm, applied once to the whole cache).
+ *
+ * Greedy k-center (farthest-point traversal, Dyer and Frieze 1985 / Gonzalez 1985) over the n_old = n - r
+ * oldest keys: the first centre is the first key; every further centre is the key farthest from its nearest
+ * chosen centre. Readings where the paper is silent: distances are the fixed-point D2 above, so the argmax is an
+ * integer decision; ties go to the lowest token index; when n_old <= k every old token is kept. The retained
+ * tokens are then attended exactly (Eq. 1 over centres and window), the same budget semantics as the eviction
+ * baselines it is compared with.
+ *
+ * centres[k_out] receives the chosen token indices in selection order, radius2 (may be NULL) the largest
+ * fixed-point D2 of an old key to its nearest centre after the selection. Returns k_out = min(k, n_old). */
+int oracle_kcenter(const float *K, int n_old, int d, int k, int *centres, uint64_t *radius2) {
+    if (n_old <= 0 || k <= 0) { if (radius2) *radius2 = 0; return 0; }
+    int k_out = k < n_old ? k : n_old;
+    uint64_t *dist = (uint64_t *)malloc(sizeof(uint64_t) * (size_t)n_old);
+    for (int i = 0; i < n_old; ++i) dist[i] = UINT64_MAX;
+    int c = 0;
+    for (int t = 0; t < k_out; ++t) {
+        centres[t] = c;
+        uint64_t far = 0;
+        int far_i = 0;
+        for (int i = 0; i < n_old; ++i) {
+            uint64_t d2 = dist2_fx(K + (size_t)c * d, K + (size_t)i * d, d);
+            if (d2 < dist[i]) dist[i] = d2;
+            if (dist[i] > far) { far = dist[i]; far_i = i; }       /* strict: ties keep the lowest index */
+        }
+        c = far_i;
+        if (radius2) *radius2 = far;
+    }
+    free(dist);
+    return k_out;
+}

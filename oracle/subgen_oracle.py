@@ -73,6 +73,8 @@ def lib():
                 for name in ("oracle_w", "oracle_ins_d2"):
                     getattr(L, name).argtypes = [vp]
                     getattr(L, name).restype = up
+                L.oracle_kcenter.argtypes = [fp, C.c_int, C.c_int, C.c_int, ip, up]
+                L.oracle_kcenter.restype = C.c_int
                 L.oracle_dist2_fx.argtypes = [fp, fp, C.c_int]
                 L.oracle_dist2_fx.restype = C.c_uint64
                 L.oracle_norm2_fx.argtypes = [fp, C.c_int]
@@ -115,6 +117,28 @@ def dist2_fx(x, k) -> int:
 def norm2_fx(v) -> int:
     v = _f32(v)
     return int(lib().oracle_norm2_fx(_fp(v), v.shape[0]))
+
+
+def kcenter(K_old, k):
+    """Greedy k-center over the rows of K_old (first centre = row 0, farthest-point traversal, fixed-point
+    distances, ties to the lowest index). Returns (centres in selection order, covering radius^2 in fixed point)."""
+    K_old = _f32(K_old)
+    n, d = K_old.shape
+    out = np.zeros(max(min(k, n), 1), dtype=np.int32)
+    rad = C.c_uint64(0)
+    kk = lib().oracle_kcenter(_fp(K_old), n, d, int(k), out.ctypes.data_as(C.POINTER(C.c_int)), C.byref(rad))
+    return out[:kk].copy(), int(rad.value)
+
+
+def kcenter_window_attention(K, V, q, k, r):
+    """Section 3.2 variant: exact attention (Eq. 1) over k greedy centres of the n - r oldest tokens plus the r most
+    recent tokens. Returns (out, kept token indices: centres in selection order, then the window)."""
+    K = _f32(K); V = _f32(V)
+    n = K.shape[0]
+    n_old = max(0, n - r)
+    cent, _ = kcenter(K[:n_old], k) if n_old else (np.zeros(0, np.int32), 0)
+    keep = np.concatenate([cent.astype(np.int64), np.arange(n_old, n)])
+    return exact_attention(K[keep], V[keep], q), keep
 
 
 class OracleUnit:
