@@ -191,6 +191,17 @@ int subgen_exact_step(subgen_exact_t* h, const void* q, const void* k, const voi
 int subgen_exact_bytes(subgen_exact_t* h, uint64_t* bytes);
 uint64_t subgen_exact_launch_count(const subgen_exact_t* h);
 
+/* Offline compression of the cache as in the paper's end-to-end experiment (Section 3.2): every unit keeps its r
+ * most recent tokens and k centres chosen among the older ones by the greedy k-center algorithm (farthest-point
+ * traversal: the first centre is the oldest token, each further centre is the token farthest from its nearest
+ * chosen centre; fixed-point distances D2, ties to the lowest token index); with at most k older tokens all are
+ * kept. Kept rows move to the front of the cache (centres in selection order, then the window) and later steps
+ * attend them exactly and keep appending. Synchronous; allocates and frees its own scratch. */
+int subgen_exact_kcenter_compress(subgen_exact_t* h, int k, int r);
+/* Stream positions of the tokens currently cached by one unit, in cache order. tok: host array of n_max ints
+ * (may be NULL to query the count only). Synchronous. */
+int subgen_exact_export_tokens(subgen_exact_t* h, int seq, int kvhead, int* n_out, int* tok);
+
 /* ---- exact attention without any allocation -------------------------------------------------- */
 
 /* The paper has no counterpart for this entry point; it exists for integration reasons only.

@@ -26,6 +26,7 @@ EXPORTS = [
     "subgen_launch_count", "subgen_last_error", "subgen_exact_create", "subgen_exact_destroy",
     "subgen_exact_append", "subgen_exact_append_varlen", "subgen_exact_step", "subgen_exact_bytes",
     "subgen_exact_launch_count", "subgen_exact_attention_noalloc",
+    "subgen_exact_kcenter_compress", "subgen_exact_export_tokens",
 ]
 
 
@@ -93,6 +94,8 @@ def load():
     L.subgen_exact_bytes.argtypes = [vp, C.POINTER(C.c_uint64)]
     L.subgen_exact_launch_count.argtypes = [vp]
     L.subgen_exact_launch_count.restype = C.c_uint64
+    L.subgen_exact_kcenter_compress.argtypes = [vp, C.c_int, C.c_int]
+    L.subgen_exact_export_tokens.argtypes = [vp, C.c_int, C.c_int, ip, ip]
     L.subgen_exact_attention_noalloc.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, vp]
     _lib = L
     return L
@@ -281,6 +284,16 @@ class ExactAttention:
         _check(self._L.subgen_exact_step(self._h, _dev(q, self.dtype, qs, "q"), _dev(k, self.dtype, ks, "k"),
                                          _dev(v, self.dtype, ks, "v"), _dev(out, self.dtype, qs, "out")))
         return out
+
+    def kcenter_compress(self, k: int, r: int):
+        """Keep the r most recent tokens and k greedy k-center centres of the older ones (Section 3.2 variant)."""
+        _check(self._L.subgen_exact_kcenter_compress(self._h, int(k), int(r)))
+
+    def export_tokens(self, seq: int, kvhead: int) -> np.ndarray:
+        n = C.c_int()
+        buf = np.zeros(self.n_max, np.int32)
+        _check(self._L.subgen_exact_export_tokens(self._h, seq, kvhead, C.byref(n), buf.ctypes.data_as(C.POINTER(C.c_int))))
+        return buf[: n.value].copy()
 
     def bytes_per_step(self) -> int:
         b = C.c_uint64()

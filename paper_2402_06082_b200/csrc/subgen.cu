@@ -17,6 +17,7 @@
 #include "subgen_prefill.cuh"
 #include "subgen_score_tc.cuh"
 #include "subgen_exact_mma.cuh"
+#include "subgen_kcenter.cuh"
 
 using namespace sgk;
 
@@ -661,7 +662,7 @@ struct subgen_exact {
     int B, H, Hkv, G, D, n_max, dtype, U, splits;
     size_t E;
     char *Kc = nullptr, *Vc = nullptr, *misc = nullptr;
-    size_t off_n, off_part, off_ticket, off_cu, off_q, misc_bytes;
+    size_t off_n, off_part, off_ticket, off_cu, off_q, off_pos, off_tok, misc_bytes;
     cudaStream_t st = nullptr;
     std::vector<int> n_host;
     uint64_t launches = 0;
@@ -677,6 +678,8 @@ template <typename T> ExactCache<T> make_exact(const subgen_exact* h) {
     E.part = (float*)(h->misc + h->off_part);
     E.ticket = (unsigned*)(h->misc + h->off_ticket);
     E.qnext = (unsigned*)(h->misc + h->off_q);
+    E.pos = (int*)(h->misc + h->off_pos);
+    E.tok = (int*)(h->misc + h->off_tok);
     return E;
 }
 
@@ -761,6 +764,8 @@ subgen_exact_t* subgen_exact_create(int B, int H, int Hkv, int d, int n_max, int
     h->off_n = take((size_t)h->U * 4);
     h->off_ticket = take((size_t)h->U * 4);
     h->off_q = take((size_t)h->U * 4);
+    h->off_pos = take((size_t)h->U * 4);
+    h->off_tok = take((size_t)h->U * n_max * 4);
     h->off_cu = take(((size_t)B + 1) * 4);
     h->off_part = take((size_t)h->U * h->splits * G * (d + 2) * 4);
     h->misc_bytes = off;
@@ -841,6 +846,80 @@ int subgen_exact_bytes(subgen_exact_t* h, uint64_t* bytes) {
     *bytes = 2 * rows * (uint64_t)h->D * h->E;
     return SUBGEN_OK;
 }
+
+}  // extern "C"
+
+namespace {
+
+template <typename T, int D>
+int kcenter_compress_td(subgen_exact* h, int k, int r, int k_iter, int keep_max) {
+    ExactCache<T> E = make_exact<T>(h);
+    int S = (148 * 4 + h->U - 1) / h->U;
+    S = S < 1 ? 1 : (S > 64 ? 64 : S);
+    const size_t b_dist = align_up((size_t)h->U * h->n_max * 8), b_cent = align_up((size_t)h->U * k * 4);
+    const size_t b_part = align_up((size_t)h->U * S * sizeof(Best));
+    const size_t b_rows = align_up((size_t)h->U * keep_max * D * sizeof(T)), b_tok = align_up((size_t)h->U * keep_max * 4);
+    char* scratch = nullptr;
+    cudaError_t e = cudaMalloc((void**)&scratch, b_dist + b_cent + 2 * b_part + 2 * b_rows + b_tok);
+    if (e != cudaSuccess) return fail(SUBGEN_ENOMEM, "subgen_exact_kcenter_compress: scratch allocation failed: %s", cudaGetErrorString(e));
+    unsigned long long* dist = (unsigned long long*)scratch;
+    int* centres = (int*)(scratch + b_dist);
+    Best* part[2] = {(Best*)(scratch + b_dist + b_cent), (Best*)(scratch + b_dist + b_cent + b_part)};
+    T* Kt = (T*)(scratch + b_dist + b_cent + 2 * b_part);
+    T* Vt = (T*)(scratch + b_dist + b_cent + 2 * b_part + b_rows);
+    int* tokt = (int*)(scratch + b_dist + b_cent + 2 * b_part + 2 * b_rows);
+    for (int t = 0; t < k_iter; ++t)
+        kcenter_iter_kernel<T, D><<<dim3(S, h->U), kKcThreads, 0, h->st>>>(E, t, k, r, dist, centres, part[(t + 1) & 1], part[t & 1]);
+    int gx = (int)(((size_t)keep_max * (D / Elem<T>::EPL) + 255) / 256);
+    gx = gx < 1 ? 1 : (gx > 32 ? 32 : gx);
+    kcenter_gather_kernel<T, D><<<dim3(gx, h->U), 256, 0, h->st>>>(E, k, r, centres, Kt, Vt, tokt, keep_max);
+    kcenter_scatter_kernel<T, D><<<dim3(gx, h->U), 256, 0, h->st>>>(E, k, r, Kt, Vt, tokt, keep_max);
+    kcenter_commit_kernel<T><<<(h->U + 255) / 256, 256, 0, h->st>>>(E, h->U, k, r);
+    cudaError_t le = cudaGetLastError();
+    cudaError_t se = cudaStreamSynchronize(h->st);
+    cudaFree(scratch);
+    if (le != cudaSuccess || se != cudaSuccess)
+        return fail(SUBGEN_ECUDA, "subgen_exact_kcenter_compress: %s", cudaGetErrorString(le != cudaSuccess ? le : se));
+    h->launches += (uint64_t)k_iter + 3;
+    return SUBGEN_OK;
+}
+
+}  // namespace
+
+extern "C" int subgen_exact_kcenter_compress(subgen_exact_t* h, int k, int r) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_exact_kcenter_compress: handle is NULL");
+    if (k < 1 || r < 0) return fail(SUBGEN_EINVAL, "subgen_exact_kcenter_compress: k must be >= 1 and r >= 0");
+    int k_iter = 0, keep_max = 0;
+    for (int b = 0; b < h->B; ++b) {
+        const int n = h->n_host[b], n_old = n > r ? n - r : 0, kk = k < n_old ? k : n_old;
+        k_iter = kk > k_iter ? kk : k_iter;
+        keep_max = kk + (n - n_old) > keep_max ? kk + (n - n_old) : keep_max;
+    }
+    if (keep_max == 0) return SUBGEN_OK;
+    const bool f32 = h->dtype == SUBGEN_DTYPE_FP32;
+    int rc;
+    if (h->D == 64) rc = f32 ? kcenter_compress_td<float, 64>(h, k, r, k_iter, keep_max) : kcenter_compress_td<__nv_bfloat16, 64>(h, k, r, k_iter, keep_max);
+    else rc = f32 ? kcenter_compress_td<float, 128>(h, k, r, k_iter, keep_max) : kcenter_compress_td<__nv_bfloat16, 128>(h, k, r, k_iter, keep_max);
+    if (rc) return rc;
+    for (int b = 0; b < h->B; ++b) {
+        const int n = h->n_host[b], n_old = n > r ? n - r : 0;
+        h->n_host[b] = (k < n_old ? k : n_old) + (n - n_old);
+    }
+    return SUBGEN_OK;
+}
+
+extern "C" int subgen_exact_export_tokens(subgen_exact_t* h, int seq, int kvhead, int* n_out, int* tok) {
+    if (!h || !n_out) return fail(SUBGEN_EINVAL, "subgen_exact_export_tokens: NULL argument");
+    if (seq < 0 || seq >= h->B || kvhead < 0 || kvhead >= h->Hkv) return fail(SUBGEN_EINVAL, "subgen_exact_export_tokens: unit out of range");
+    CUDA_TRY(cudaStreamSynchronize(h->st));
+    const size_t u = (size_t)seq * h->Hkv + kvhead;
+    *n_out = h->n_host[seq];
+    if (tok && h->n_host[seq] > 0)
+        CUDA_TRY(cudaMemcpy(tok, h->misc + h->off_tok + u * h->n_max * 4, (size_t)h->n_host[seq] * 4, cudaMemcpyDeviceToHost));
+    return SUBGEN_OK;
+}
+
+extern "C" {
 
 uint64_t subgen_exact_launch_count(const subgen_exact_t* h) { return h ? h->launches : 0; }
 

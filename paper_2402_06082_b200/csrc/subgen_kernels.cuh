@@ -296,6 +296,8 @@ template <typename T> struct ExactCache {
     float* part;     // [U, splits, G, D + 2]
     unsigned* ticket;
     unsigned* qnext; // [U] work queue of the tensor-core kernel
+    int* tok;        // [U, n_max] stream position of the token in each cache row
+    int* pos;        // [U] tokens ever appended (differs from n_unit after a compression)
 };
 
 template <typename T, int D>
@@ -314,6 +316,7 @@ __global__ void exact_append_kernel(ExactCache<T> E, const T* __restrict__ K, co
     for (size_t p = (size_t)blockIdx.x * blockDim.x + threadIdx.x; p < cnt; p += (size_t)gridDim.x * blockDim.x) {
         kd[p] = ks[p];
         vd[p] = vs[p];
+        if (p % LPR == 0) E.tok[(size_t)u * E.n_max + n_prev + p / LPR] = E.pos[u] + (int)(p / LPR);
     }
 }
 
@@ -322,7 +325,9 @@ __global__ void exact_advance_kernel(ExactCache<T> E, int U, int n_uniform, cons
     const int u = blockIdx.x * blockDim.x + threadIdx.x;
     if (u >= U) return;
     const int b = u / E.Hkv;
-    E.n_unit[u] += cu ? cu[b + 1] - cu[b] : n_uniform;
+    const int add = cu ? cu[b + 1] - cu[b] : n_uniform;
+    E.n_unit[u] += add;
+    E.pos[u] += add;
 }
 
 // grid (splits, U): append (k, v) as row n, then softmax(K q)^T V over rows 0..n. The new row is
@@ -347,6 +352,7 @@ __global__ void __launch_bounds__(kQueryThreads) exact_step_kernel(ExactCache<T>
         if (tid < LPR) reinterpret_cast<uint4*>(E.Kc + ((size_t)u * E.n_max + n) * D)[tid] = reinterpret_cast<const uint4*>(kn)[tid];
         else if (tid < 2 * LPR)
             reinterpret_cast<uint4*>(E.Vc + ((size_t)u * E.n_max + n) * D)[tid - LPR] = reinterpret_cast<const uint4*>(vn)[tid - LPR];
+        if (tid == 0) E.tok[(size_t)u * E.n_max + n] = E.pos[u];
     }
     float qf[G][EPL];
 #pragma unroll
@@ -396,6 +402,7 @@ __global__ void __launch_bounds__(kQueryThreads) exact_step_kernel(ExactCache<T>
     final_merge<T, D, G>(part_u, splits, out + qrow0 * D, false);
     if (tid == 0) {
         E.n_unit[u] = n + 1;
+        E.pos[u] = E.pos[u] + 1;
         E.ticket[u] = 0;
     }
 }
