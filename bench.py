@@ -362,7 +362,12 @@ def run_subgen(args, w):
     # ---- exact dense decode over full caches on the same inputs (comparison point) ----
     if args.exact and rank == 0:
         try:
-            extra["exact"] = run_exact(wr, lens, n_dec, K_steps, W_steps, qs, ks, vs, peak)
+            kc = None
+            if args.kcenter:
+                kc = tuple(int(x) for x in args.kcenter.split(","))
+            elif wr.kc_k:
+                kc = (wr.kc_k, wr.kc_r)
+            extra["exact"] = run_exact(wr, lens, n_dec, K_steps, W_steps, qs, ks, vs, peak, kc)
         except Exception as ex:  # report, do not hide
             extra["exact"] = {"error": str(ex)[:200]}
 
@@ -387,7 +392,7 @@ def run_subgen(args, w):
         dist.destroy_process_group()
 
 
-def run_exact(w, lens, n_dec, K_steps, W_steps, qs, ks, vs, peak):
+def run_exact(w, lens, n_dec, K_steps, W_steps, qs, ks, vs, peak, kc=None):
     from paper_2402_06082_b200 import binding
     dt = w.torch_dtype
     ex = binding.ExactAttention(w.B, w.H, w.d, max(lens) + n_dec, Hkv=w.Hkv, dtype=dt)
@@ -424,8 +429,52 @@ def run_exact(w, lens, n_dec, K_steps, W_steps, qs, ks, vs, peak):
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / K_steps
     gbs = b0 / (ms * 1e-3) / 1e9
+    res = {"steps_per_s": 1e3 / ms, "ms_per_step": ms, "bytes_per_step": b0, "achieved_GBps": gbs, "frac_of_hbm_peak": gbs / peak}
+    if kc is not None:
+        res["kcenter"] = run_kcenter(ex, w, [n + W_steps + K_steps for n in lens], kc, qs, ks, vs, out, peak)
     ex.close()
-    return {"steps_per_s": 1e3 / ms, "ms_per_step": ms, "bytes_per_step": b0, "achieved_GBps": gbs, "frac_of_hbm_peak": gbs / peak}
+    return res
+
+
+def run_kcenter(ex, w, n_now, kc, qs, ks, vs, out, peak):
+    """One-shot greedy k-center compression of the full caches (Section 3.2 variant), then decode on what is kept.
+
+    Algorithmic bytes: pass j of a unit reads every older key once (n_old * d * E) and reads and writes the 8-byte
+    running distance of each; a unit takes min(k, n_old) passes.
+    """
+    k, r = kc
+    E = 4 if w.dtype == "fp32" else 2
+    nbytes = 0
+    for n in n_now:
+        n_old = max(0, n - r)
+        nbytes += w.Hkv * min(k, n_old) * n_old * (w.d * E + 16)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = ex.launch_count
+    torch.cuda.synchronize()
+    e0.record()
+    ex.kcenter_compress(k, r)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    launches = ex.launch_count - l0
+    b1 = ex.bytes_per_step()
+    steps = min(64, len(qs))
+    for i in range(3):
+        ex.step(qs[i], ks[i], vs[i], out)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(3, steps):
+        ex.step(qs[i], ks[i], vs[i], out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms_step = e0.elapsed_time(e1) / max(1, steps - 3)
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    looked, full = ex.kcenter_counters()
+    HEAD = 16
+    touched = looked * (HEAD * E + 8) + full * (w.d * E + 8)
+    return {"k": k, "r": r, "tokens_looked_at": looked, "full_rows_read": full, "bytes_touched": touched,
+            "touched_GBps": touched / (ms * 1e-3) / 1e9, "compress_ms": ms, "launches": launches, "algorithmic_bytes": nbytes, "achieved_GBps": gbs,
+            "frac_of_hbm_peak": gbs / peak, "steps_per_s_after": 1e3 / ms_step, "bytes_per_step_after": b1}
 
 
 def main():
@@ -441,6 +490,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--prompt", type=int, default=0, help="override the prompt length (smaller cases for profiling)")
     ap.add_argument("--batch", type=int, default=0, help="override the number of sequences")
+    ap.add_argument("--kcenter", default="", help="k,r: also time the one-shot k-center compression of the exact caches")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "subgen":
         args.warmup = 3

@@ -198,6 +198,11 @@ uint64_t subgen_exact_launch_count(const subgen_exact_t* h);
  * kept. Kept rows move to the front of the cache (centres in selection order, then the window) and later steps
  * attend them exactly and keep appending. Synchronous; allocates and frees its own scratch. */
 int subgen_exact_kcenter_compress(subgen_exact_t* h, int k, int r);
+/* Work done by the last compression, summed over units and passes: tokens_looked_at counts (token, pass) pairs
+ * whose running distance was compared against a new centre; full_rows_read counts those for which the whole key
+ * row had to be read because a lower bound from its first 16 coordinates did not settle the comparison. The
+ * result never depends on which tokens were settled early. Either pointer may be NULL. */
+int subgen_exact_kcenter_counters(const subgen_exact_t* h, uint64_t* tokens_looked_at, uint64_t* full_rows_read);
 /* Stream positions of the tokens currently cached by one unit, in cache order. tok: host array of n_max ints
  * (may be NULL to query the count only). Synchronous. */
 int subgen_exact_export_tokens(subgen_exact_t* h, int seq, int kvhead, int* n_out, int* tok);

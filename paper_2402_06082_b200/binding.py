@@ -26,7 +26,7 @@ EXPORTS = [
     "subgen_launch_count", "subgen_last_error", "subgen_exact_create", "subgen_exact_destroy",
     "subgen_exact_append", "subgen_exact_append_varlen", "subgen_exact_step", "subgen_exact_bytes",
     "subgen_exact_launch_count", "subgen_exact_attention_noalloc",
-    "subgen_exact_kcenter_compress", "subgen_exact_export_tokens",
+    "subgen_exact_kcenter_compress", "subgen_exact_kcenter_counters", "subgen_exact_export_tokens",
 ]
 
 
@@ -95,6 +95,7 @@ def load():
     L.subgen_exact_launch_count.argtypes = [vp]
     L.subgen_exact_launch_count.restype = C.c_uint64
     L.subgen_exact_kcenter_compress.argtypes = [vp, C.c_int, C.c_int]
+    L.subgen_exact_kcenter_counters.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     L.subgen_exact_export_tokens.argtypes = [vp, C.c_int, C.c_int, ip, ip]
     L.subgen_exact_attention_noalloc.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, vp]
     _lib = L
@@ -288,6 +289,12 @@ class ExactAttention:
     def kcenter_compress(self, k: int, r: int):
         """Keep the r most recent tokens and k greedy k-center centres of the older ones (Section 3.2 variant)."""
         _check(self._L.subgen_exact_kcenter_compress(self._h, int(k), int(r)))
+
+    def kcenter_counters(self):
+        """(tokens looked at, full key rows read) of the last compression, summed over units and passes."""
+        a, b = C.c_uint64(), C.c_uint64()
+        _check(self._L.subgen_exact_kcenter_counters(self._h, C.byref(a), C.byref(b)))
+        return int(a.value), int(b.value)
 
     def export_tokens(self, seq: int, kvhead: int) -> np.ndarray:
         n = C.c_int()

@@ -663,6 +663,7 @@ struct subgen_exact {
     size_t E;
     char *Kc = nullptr, *Vc = nullptr, *misc = nullptr;
     size_t off_n, off_part, off_ticket, off_cu, off_q, off_pos, off_tok, misc_bytes;
+    uint64_t kc_counters[2] = {0, 0};   // last compression: tokens looked at, full rows read
     cudaStream_t st = nullptr;
     std::vector<int> n_host;
     uint64_t launches = 0;
@@ -852,15 +853,21 @@ int subgen_exact_bytes(subgen_exact_t* h, uint64_t* bytes) {
 namespace {
 
 template <typename T, int D>
-int kcenter_compress_td(subgen_exact* h, int k, int r, int k_iter, int keep_max) {
+int kcenter_compress_td(subgen_exact* h, int k, int r, int k_iter, int keep_max, int n_old_max) {
     ExactCache<T> E = make_exact<T>(h);
-    int S = (148 * 4 + h->U - 1) / h->U;
+    // one resident wave of 128-thread blocks, and slices short enough for the 16-bit survivor offsets
+    int S = (148 * 8) / h->U;
     S = S < 1 ? 1 : (S > 64 ? 64 : S);
+    const int s_min = (n_old_max + kKcSliceMax - 1) / kKcSliceMax;
+    S = S < s_min ? s_min : S;
+    const size_t smem = (size_t)((n_old_max + S - 1) / S) * sizeof(unsigned short);
+    constexpr int HP = kKcHead / Elem<T>::EPL;
     const size_t b_dist = align_up((size_t)h->U * h->n_max * 8), b_cent = align_up((size_t)h->U * k * 4);
     const size_t b_part = align_up((size_t)h->U * S * sizeof(Best));
     const size_t b_rows = align_up((size_t)h->U * keep_max * D * sizeof(T)), b_tok = align_up((size_t)h->U * keep_max * 4);
+    const size_t b_head = align_up((size_t)h->U * HP * h->n_max * sizeof(uint4)), b_cnt = align_up(16);
     char* scratch = nullptr;
-    cudaError_t e = cudaMalloc((void**)&scratch, b_dist + b_cent + 2 * b_part + 2 * b_rows + b_tok);
+    cudaError_t e = cudaMalloc((void**)&scratch, b_dist + b_cent + 2 * b_part + 2 * b_rows + b_tok + b_head + b_cnt);
     if (e != cudaSuccess) return fail(SUBGEN_ENOMEM, "subgen_exact_kcenter_compress: scratch allocation failed: %s", cudaGetErrorString(e));
     unsigned long long* dist = (unsigned long long*)scratch;
     int* centres = (int*)(scratch + b_dist);
@@ -868,19 +875,26 @@ int kcenter_compress_td(subgen_exact* h, int k, int r, int k_iter, int keep_max)
     T* Kt = (T*)(scratch + b_dist + b_cent + 2 * b_part);
     T* Vt = (T*)(scratch + b_dist + b_cent + 2 * b_part + b_rows);
     int* tokt = (int*)(scratch + b_dist + b_cent + 2 * b_part + 2 * b_rows);
+    uint4* head = (uint4*)(scratch + b_dist + b_cent + 2 * b_part + 2 * b_rows + b_tok);
+    unsigned long long* counters = (unsigned long long*)(scratch + b_dist + b_cent + 2 * b_part + 2 * b_rows + b_tok + b_head);
+    cudaMemsetAsync(counters, 0, 16, h->st);
+    int gi = (h->n_max + 255) / 256;
+    gi = gi > 32 ? 32 : gi;
+    kcenter_init_kernel<T, D><<<dim3(gi, h->U), 256, 0, h->st>>>(E, r, head, dist);
     for (int t = 0; t < k_iter; ++t)
-        kcenter_iter_kernel<T, D><<<dim3(S, h->U), kKcThreads, 0, h->st>>>(E, t, k, r, dist, centres, part[(t + 1) & 1], part[t & 1]);
+        kcenter_iter_kernel<T, D><<<dim3(S, h->U), kKcThreads, smem, h->st>>>(E, t, k, r, head, dist, centres, part[(t + 1) & 1], part[t & 1], counters);
     int gx = (int)(((size_t)keep_max * (D / Elem<T>::EPL) + 255) / 256);
     gx = gx < 1 ? 1 : (gx > 32 ? 32 : gx);
     kcenter_gather_kernel<T, D><<<dim3(gx, h->U), 256, 0, h->st>>>(E, k, r, centres, Kt, Vt, tokt, keep_max);
     kcenter_scatter_kernel<T, D><<<dim3(gx, h->U), 256, 0, h->st>>>(E, k, r, Kt, Vt, tokt, keep_max);
     kcenter_commit_kernel<T><<<(h->U + 255) / 256, 256, 0, h->st>>>(E, h->U, k, r);
     cudaError_t le = cudaGetLastError();
-    cudaError_t se = cudaStreamSynchronize(h->st);
+    cudaError_t se = cudaMemcpyAsync(h->kc_counters, counters, 16, cudaMemcpyDeviceToHost, h->st);
+    if (se == cudaSuccess) se = cudaStreamSynchronize(h->st);
     cudaFree(scratch);
     if (le != cudaSuccess || se != cudaSuccess)
         return fail(SUBGEN_ECUDA, "subgen_exact_kcenter_compress: %s", cudaGetErrorString(le != cudaSuccess ? le : se));
-    h->launches += (uint64_t)k_iter + 3;
+    h->launches += (uint64_t)k_iter + 4;
     return SUBGEN_OK;
 }
 
@@ -889,22 +903,30 @@ int kcenter_compress_td(subgen_exact* h, int k, int r, int k_iter, int keep_max)
 extern "C" int subgen_exact_kcenter_compress(subgen_exact_t* h, int k, int r) {
     if (!h) return fail(SUBGEN_EINVAL, "subgen_exact_kcenter_compress: handle is NULL");
     if (k < 1 || r < 0) return fail(SUBGEN_EINVAL, "subgen_exact_kcenter_compress: k must be >= 1 and r >= 0");
-    int k_iter = 0, keep_max = 0;
+    int k_iter = 0, keep_max = 0, n_old_max = 0;
     for (int b = 0; b < h->B; ++b) {
         const int n = h->n_host[b], n_old = n > r ? n - r : 0, kk = k < n_old ? k : n_old;
+        n_old_max = n_old > n_old_max ? n_old : n_old_max;
         k_iter = kk > k_iter ? kk : k_iter;
         keep_max = kk + (n - n_old) > keep_max ? kk + (n - n_old) : keep_max;
     }
     if (keep_max == 0) return SUBGEN_OK;
     const bool f32 = h->dtype == SUBGEN_DTYPE_FP32;
     int rc;
-    if (h->D == 64) rc = f32 ? kcenter_compress_td<float, 64>(h, k, r, k_iter, keep_max) : kcenter_compress_td<__nv_bfloat16, 64>(h, k, r, k_iter, keep_max);
-    else rc = f32 ? kcenter_compress_td<float, 128>(h, k, r, k_iter, keep_max) : kcenter_compress_td<__nv_bfloat16, 128>(h, k, r, k_iter, keep_max);
+    if (h->D == 64) rc = f32 ? kcenter_compress_td<float, 64>(h, k, r, k_iter, keep_max, n_old_max) : kcenter_compress_td<__nv_bfloat16, 64>(h, k, r, k_iter, keep_max, n_old_max);
+    else rc = f32 ? kcenter_compress_td<float, 128>(h, k, r, k_iter, keep_max, n_old_max) : kcenter_compress_td<__nv_bfloat16, 128>(h, k, r, k_iter, keep_max, n_old_max);
     if (rc) return rc;
     for (int b = 0; b < h->B; ++b) {
         const int n = h->n_host[b], n_old = n > r ? n - r : 0;
         h->n_host[b] = (k < n_old ? k : n_old) + (n - n_old);
     }
+    return SUBGEN_OK;
+}
+
+extern "C" int subgen_exact_kcenter_counters(const subgen_exact_t* h, uint64_t* tokens_looked_at, uint64_t* full_rows_read) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_exact_kcenter_counters: handle is NULL");
+    if (tokens_looked_at) *tokens_looked_at = h->kc_counters[0];
+    if (full_rows_read) *full_rows_read = h->kc_counters[1];
     return SUBGEN_OK;
 }
 

@@ -48,6 +48,8 @@ class Workload:
     philox_seed: int = 0
     data_seed: int = 1000
     m_max: int = 4096
+    kc_k: int = 0                 # offline k-center compression: centres kept among the older tokens
+    kc_r: int = 0                 # ... and most recent tokens kept beside them
 
     @property
     def torch_dtype(self):
@@ -84,7 +86,13 @@ CFG4B = CFG4.scaled(name="cfg4b", drift="emission", m_max=8192)
 CFG5 = Workload("cfg5", B=64, H=32, Hkv=32, d=128, dtype="bf16", n_prompt=65536, n_decode=2048, ncomp=1024, sigma=0.15,
                 weights="dirichlet", value_scale="lognormal", delta=0.6, t=8, s=2048, window=512, outlier_frac=0.05,
                 varlen=(4096, 65536), data_seed=1005, m_max=6144)
-CONFIGS = {w.name: w for w in (CFG1, CFG2, CFG3, CFG4, CFG4B, CFG5)}
+# Shape of the paper's end-to-end experiment (Section 3.2, longest context): a 7B Llama-type model has 32 layers
+# of 32 heads with d = 128, i.e. 1024 independent (layer, head) caches of one 9k-token context, held here as
+# 32 "sequences" of 32 KV heads; the budget r + k is half the context.
+KC9K = Workload("kc9k", B=32, H=32, Hkv=32, d=128, dtype="bf16", n_prompt=9000, n_decode=64, ncomp=256, sigma=0.15,
+                weights="dirichlet", value_scale="lognormal", delta=0.6, t=8, s=1024, window=512, data_seed=1006,
+                m_max=4096, kc_k=3988, kc_r=512)
+CONFIGS = {w.name: w for w in (CFG1, CFG2, CFG3, CFG4, CFG4B, CFG5, KC9K)}
 
 
 def _gen(device, seed: int) -> torch.Generator:

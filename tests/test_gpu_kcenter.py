@@ -87,3 +87,58 @@ def test_kcenter_varlen():
             cent, _ = orc.kcenter(f32(streams[b][0])[h, : n - 25], 40)
             keep = np.concatenate([cent.astype(np.int64), np.arange(n - 25, n)])
             np.testing.assert_array_equal(ex.export_tokens(b, h), keep)
+
+
+def _check_selection(ex, Kn, units, n_old, k, r):
+    for b, h in units:
+        cent, _ = orc.kcenter(Kn[b, h, :n_old], k)
+        keep = np.concatenate([cent.astype(np.int64), np.arange(n_old, n_old + r)])
+        np.testing.assert_array_equal(ex.export_tokens(b, h), keep)
+
+
+def test_kcenter_ties_and_uninformative_heads():
+    """Inputs on which the early lower bound is tight, useless or decides between equal distances.
+
+    Unit 0: a coarse lattice with many duplicates (equal distances everywhere, ties go to the lowest index).
+    Unit 1: keys equal in the first 16 coordinates (the head bound is 0, every comparison needs the full row).
+    Unit 2: keys that differ in the first 16 coordinates only (the head bound is the whole distance).
+    Unit 3: clustered keys plus exact copies of earlier rows.
+    """
+    rng = np.random.default_rng(7)
+    n, d, k, r = 3000, 128, 200, 17
+    K = np.zeros((1, 4, n, d), np.float32)
+    K[0, 0] = rng.integers(-1, 2, (n, d)) * 0.5
+    K[0, 0, :, 4:] = 0.0
+    K[0, 1, :, :16] = 0.25
+    K[0, 1, :, 16:] = rng.normal(size=(n, d - 16))
+    K[0, 2, :, :16] = rng.normal(size=(n, 16))
+    K[0, 2, :, 16:] = -1.5
+    cl = rng.normal(size=(12, d))
+    K[0, 3] = cl[rng.integers(0, 12, n)] + 0.01 * rng.normal(size=(n, d))
+    K[0, 3, 1500:] = K[0, 3, :1500]
+    Kt = torch.tensor(K, dtype=torch.bfloat16, device="cuda")
+    Vt = torch.randn(1, 4, n, d, device="cuda").to(torch.bfloat16)
+    from paper_2402_06082_b200.binding import ExactAttention
+    ex = ExactAttention(1, 4, d, n, Hkv=4, dtype=torch.bfloat16)
+    ex.append(Kt, Vt)
+    ex.kcenter_compress(k, r)
+    _check_selection(ex, f32(Kt), [(0, h) for h in range(4)], n - r, k, r)
+    looked, full = ex.kcenter_counters()
+    assert 0 < full <= looked
+
+
+def test_kcenter_long_slices_many_units():
+    """More units than one wave of blocks and more than 16384 older tokens: every unit is cut into two slices."""
+    w = synth.CFG3.scaled(B=150, H=8, Hkv=8, d=64, n_prompt=16500, ncomp=64)
+    n, k, r = 16500, 24, 50
+    K = torch.empty(w.B, w.Hkv, n, w.d, dtype=torch.bfloat16, device="cuda")
+    for b in range(w.B):
+        K[b] = synth.sequence_stream(w.scaled(data_seed=1003 + b % 3), b, n, "cuda")[0]
+    ex = _exact(w, n)
+    ex.append(K, K)
+    ex.kcenter_compress(k, r)
+    Kn = {b: f32(K[b:b + 1]) for b in (0, 77, 149)}
+    for b, Kb in Kn.items():
+        for h in (0, 7):
+            cent, _ = orc.kcenter(Kb[0, h, : n - r], k)
+            np.testing.assert_array_equal(ex.export_tokens(b, h)[:k], cent.astype(np.int64))
