@@ -173,6 +173,20 @@ int subgen_profile_prefill_read(subgen_t* h, double ms[3]);
 /* Number of kernels this handle has launched so far. */
 uint64_t subgen_launch_count(const subgen_t* h);
 
+/* Checkpoint and resume. The paper describes a stream that never stops; a serving process has to move a
+ * conversation between GPUs or survive a restart, so the state between two calls (D with its samples and counts, M
+ * with its weights, mu, the window ring, the per-unit counters and status bits) can be written to one host blob and
+ * loaded into another handle. The blob stores cluster arrays only up to the largest cluster count of any unit.
+ * Loading needs a handle created with the same B, H, Hkv, d, t, s, window, dtype, delta and seed (the Philox
+ * draws of later tokens depend on the seed and on the token index, which the blob carries); m_max may differ as
+ * long as it holds the stored clusters, which is also the way to continue a stream with a larger capacity.
+ * Everything the handle held before is discarded. After a load the handle continues the stream exactly as the
+ * saved one would have: the integer state stays identical token for token. All three calls are synchronous.
+ * host: ordinary host memory (pinned memory makes the copies faster). */
+int subgen_checkpoint_bytes(subgen_t* h, size_t* bytes);
+int subgen_checkpoint_save(subgen_t* h, void* host, size_t bytes, size_t* written);
+int subgen_checkpoint_load(subgen_t* h, const void* host, size_t bytes);
+
 /* Text of the calling thread's most recent error. */
 const char* subgen_last_error(void);
 

@@ -23,7 +23,7 @@ EXPORTS = [
     "subgen_workspace_bytes", "subgen_create", "subgen_create_ex", "subgen_destroy", "subgen_prefill",
     "subgen_prefill_varlen", "subgen_step", "subgen_step_host", "subgen_status", "subgen_export_state",
     "subgen_export_rows", "subgen_cache_stats", "subgen_profile_enable", "subgen_profile_read", "subgen_profile_prefill_read",
-    "subgen_launch_count", "subgen_last_error", "subgen_exact_create", "subgen_exact_destroy",
+    "subgen_launch_count", "subgen_last_error", "subgen_checkpoint_bytes", "subgen_checkpoint_save", "subgen_checkpoint_load", "subgen_exact_create", "subgen_exact_destroy",
     "subgen_exact_append", "subgen_exact_append_varlen", "subgen_exact_step", "subgen_exact_bytes",
     "subgen_exact_launch_count", "subgen_exact_attention_noalloc",
     "subgen_exact_kcenter_compress", "subgen_exact_kcenter_counters", "subgen_exact_export_tokens",
@@ -82,6 +82,9 @@ def load():
     L.subgen_profile_read.argtypes = [vp, C.POINTER(C.c_double), ip]
     L.subgen_profile_prefill_read.argtypes = [vp, C.POINTER(C.c_double)]
     L.subgen_launch_count.argtypes = [vp]
+    L.subgen_checkpoint_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
+    L.subgen_checkpoint_save.argtypes = [vp, vp, C.c_size_t, C.POINTER(C.c_size_t)]
+    L.subgen_checkpoint_load.argtypes = [vp, vp, C.c_size_t]
     L.subgen_launch_count.restype = C.c_uint64
     L.subgen_last_error.restype = C.c_char_p
     L.subgen_exact_create.restype = vp
@@ -240,6 +243,21 @@ class SubGen:
     @property
     def launch_count(self) -> int:
         return int(self._L.subgen_launch_count(self._h))
+
+    def checkpoint_save(self) -> torch.Tensor:
+        """The state between two calls as one pinned uint8 host tensor (see subgen_checkpoint_save)."""
+        n = C.c_size_t()
+        _check(self._L.subgen_checkpoint_bytes(self._h, C.byref(n)))
+        blob = torch.empty(n.value, dtype=torch.uint8, pin_memory=True)
+        w = C.c_size_t()
+        _check(self._L.subgen_checkpoint_save(self._h, blob.data_ptr(), n.value, C.byref(w)))
+        return blob[: w.value]
+
+    def checkpoint_load(self, blob: torch.Tensor):
+        """Replace this handle's state by a saved one; the configuration must match, m_max may be larger."""
+        if blob.dtype != torch.uint8 or blob.device.type != "cpu" or not blob.is_contiguous():
+            raise ValueError("blob must be a contiguous uint8 host tensor")
+        _check(self._L.subgen_checkpoint_load(self._h, blob.data_ptr(), blob.numel()))
 
 
 class ExactAttention:

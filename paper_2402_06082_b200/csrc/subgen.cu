@@ -655,6 +655,128 @@ uint64_t subgen_launch_count(const subgen_t* h) { return h ? h->launches : 0; }
 
 }  // extern "C"
 
+
+// ---- checkpoint: a handle's state as one host blob --------------------------------------------------------
+
+namespace {
+
+constexpr uint64_t kCkptMagic = 0x315450434e474253ull;   // "SBGNCPT1"
+
+struct CkptHeader {
+    uint64_t magic;
+    uint32_t version, dtype;
+    int32_t B, H, Hkv, d, t, s, window, m_rows;
+    float delta;
+    uint32_t pad;
+    uint64_t seed, payload_bytes;
+};
+
+struct CkptArray {
+    size_t off;        // offset in the workspace
+    size_t unit_cap;   // bytes per unit in the workspace
+    size_t unit_live;  // bytes per unit stored in the blob
+};
+
+// The arrays that make up the state between two calls, in blob order. Cluster arrays are stored up to m_rows
+// clusters per unit; partials, tickets and work queues are scratch of a single call and are not part of it.
+std::vector<CkptArray> ckpt_arrays(const subgen* h, int m_rows) {
+    const Dims& d = h->d;
+    const Layout& L = h->L;
+    const size_t row = (size_t)d.D * d.E, mm = (size_t)d.m_max, mr = (size_t)m_rows, s = (size_t)d.s, w = (size_t)d.w, t = (size_t)d.t;
+    return {
+        {L.X, mm * row, mr * row}, {L.S, mm * t * row, mr * t * row}, {L.xn, mm * 4, mr * 4}, {L.cnt, mm * 4, mr * 4},
+        {L.ctok, mm * 4, mr * 4}, {L.stok, mm * t * 4, mr * t * 4},
+        {L.Mk, s * row, s * row}, {L.Mv, s * row, s * row}, {L.MW, s * 8, s * 8}, {L.Mtok, s * 4, s * 4}, {L.MinvW, s * 4, s * 4},
+        {L.ringK, w * row, w * row}, {L.ringV, w * row, w * row},
+        {L.n_unit, 4, 4}, {L.m_unit, 4, 4}, {L.mu, 8, 8}, {L.status, 4, 4}, {L.last_cid, 4, 4}, {L.last_open, 4, 4},
+        {L.last_d2, 8, 8}, {L.pairs, 8, 8},
+    };
+}
+
+size_t ckpt_payload(const subgen* h, int m_rows) {
+    size_t n = 0;
+    for (const CkptArray& a : ckpt_arrays(h, m_rows)) n += a.unit_live * (size_t)h->d.U;
+    return n;
+}
+
+// Largest cluster count over the units. Synchronous.
+int ckpt_m_rows(subgen* h, int* out) {
+    std::vector<int> m(h->d.U);
+    CUDA_TRY(cudaStreamSynchronize(h->st));
+    CUDA_TRY(cudaMemcpy(m.data(), h->ws + h->L.m_unit, (size_t)h->d.U * 4, cudaMemcpyDeviceToHost));
+    int r = 0;
+    for (int x : m) r = x > r ? x : r;
+    *out = r;
+    return SUBGEN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int subgen_checkpoint_bytes(subgen_t* h, size_t* bytes) {
+    if (!h || !bytes) return fail(SUBGEN_EINVAL, "subgen_checkpoint_bytes: NULL argument");
+    int m_rows = 0;
+    if (int rc = ckpt_m_rows(h, &m_rows)) return rc;
+    *bytes = sizeof(CkptHeader) + ckpt_payload(h, m_rows);
+    return SUBGEN_OK;
+}
+
+int subgen_checkpoint_save(subgen_t* h, void* host, size_t bytes, size_t* written) {
+    if (!h || !host) return fail(SUBGEN_EINVAL, "subgen_checkpoint_save: NULL argument");
+    int m_rows = 0;
+    if (int rc = ckpt_m_rows(h, &m_rows)) return rc;
+    const size_t payload = ckpt_payload(h, m_rows), need = sizeof(CkptHeader) + payload;
+    if (bytes < need) return fail(SUBGEN_EINVAL, "subgen_checkpoint_save: buffer needs %zu bytes", need);
+    CkptHeader hd;
+    memset(&hd, 0, sizeof hd);
+    hd.magic = kCkptMagic; hd.version = 1; hd.dtype = (uint32_t)h->cfg.dtype;
+    hd.B = h->d.B; hd.H = h->d.H; hd.Hkv = h->d.Hkv; hd.d = h->d.D; hd.t = h->d.t; hd.s = h->d.s; hd.window = h->d.w;
+    hd.m_rows = m_rows; hd.delta = h->cfg.delta; hd.seed = h->cfg.seed; hd.payload_bytes = payload;
+    memcpy(host, &hd, sizeof hd);
+    char* dst = (char*)host + sizeof hd;
+    for (const CkptArray& a : ckpt_arrays(h, m_rows)) {
+        if (a.unit_live)
+            CUDA_TRY(cudaMemcpy2D(dst, a.unit_live, h->ws + a.off, a.unit_cap, a.unit_live, (size_t)h->d.U, cudaMemcpyDeviceToHost));
+        dst += a.unit_live * (size_t)h->d.U;
+    }
+    if (written) *written = need;
+    return SUBGEN_OK;
+}
+
+int subgen_checkpoint_load(subgen_t* h, const void* host, size_t bytes) {
+    if (!h || !host) return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: NULL argument");
+    if (bytes < sizeof(CkptHeader)) return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: blob shorter than its header");
+    CkptHeader hd;
+    memcpy(&hd, host, sizeof hd);
+    if (hd.magic != kCkptMagic || hd.version != 1) return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: not a checkpoint of this library version");
+    const Dims& d = h->d;
+    if (hd.B != d.B || hd.H != d.H || hd.Hkv != d.Hkv || hd.d != d.D || hd.t != d.t || hd.s != d.s || hd.window != d.w ||
+        (int)hd.dtype != h->cfg.dtype || hd.seed != h->cfg.seed || memcmp(&hd.delta, &h->cfg.delta, sizeof(float)) != 0)
+        return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: the checkpoint was written with another configuration "
+                    "(B, H, Hkv, d, t, s, window, dtype, delta and seed must match; only m_max may differ)");
+    if (hd.m_rows < 0 || hd.m_rows > d.m_max)
+        return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: the checkpoint holds %d clusters per unit, this handle's m_max is %d", hd.m_rows, d.m_max);
+    const size_t payload = ckpt_payload(h, hd.m_rows);
+    if (hd.payload_bytes != payload || bytes < sizeof hd + payload) return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: truncated or damaged blob");
+    CUDA_TRY(cudaStreamSynchronize(h->st));
+    // back to the state of a new handle, then the stored arrays on top
+    CUDA_TRY(cudaMemset(h->ws + h->L.book_begin, 0, h->L.book_end - h->L.book_begin));
+    CUDA_TRY(cudaMemset(h->ws + h->L.book_end, 0xFF, h->L.total - h->L.book_end));
+    const char* src = (const char*)host + sizeof hd;
+    for (const CkptArray& a : ckpt_arrays(h, hd.m_rows)) {
+        if (a.unit_live)
+            CUDA_TRY(cudaMemcpy2D(h->ws + a.off, a.unit_cap, src, a.unit_live, a.unit_live, (size_t)d.U, cudaMemcpyHostToDevice));
+        src += a.unit_live * (size_t)d.U;
+    }
+    std::vector<int> n(d.U);
+    CUDA_TRY(cudaMemcpy(n.data(), h->ws + h->L.n_unit, (size_t)d.U * 4, cudaMemcpyDeviceToHost));
+    for (int b = 0; b < d.B; ++b) h->n_host[b] = n[(size_t)b * d.Hkv];
+    return SUBGEN_OK;
+}
+
+}  // extern "C"
+
 // ------------------------------------------------------------------------------------------------
 // Exact comparison path.
 
