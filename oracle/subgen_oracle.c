@@ -121,6 +121,11 @@ typedef struct oracle_unit {
     int *m_tok;                  /* [s], -1 = null */
     uint64_t mu;
     int overflow_at;             /* token whose insertion found D full, or -1 */
+
+    /* bounded-m variant (see doubling_sweep): the threshold in force and how often it has doubled */
+    int bounded;
+    uint64_t thr2_fx;            /* starts as delta2_fx */
+    int level;
 } oracle_unit;
 
 oracle_unit *oracle_create(int d, float delta, int t, int s, int window, uint64_t seed,
@@ -131,6 +136,7 @@ oracle_unit *oracle_create(int d, float delta, int t, int s, int window, uint64_
     u->d = d; u->t = t; u->s = s; u->window = window; u->m_max = m_max;
     u->delta = delta;
     u->delta2_fx = (uint64_t)floor((double)delta * (double)delta * 4294967296.0);
+    u->thr2_fx = u->delta2_fx;
     u->key[0] = (uint32_t)seed; u->key[1] = (uint32_t)(seed >> 32);
     u->unit_id = unit_id;
     u->centre_tok = (int *)malloc(sizeof(int) * (size_t)m_max);
@@ -177,33 +183,97 @@ static uint32_t coin_word(const oracle_unit *u, int token, int slot, uint32_t do
     return out[slot % 4];
 }
 
+/*
+ * Bounded-m variant. The paper bounds the number of clusters only through the clusterability assumption and cites
+ * the incremental clustering of Charikar, Chekuri, Feder and Motwani as the inspiration of its online clustering;
+ * it does not say what to do when a budget of m_max clusters is exhausted. This is the reading taken, in the
+ * spirit of that doubling algorithm:
+ *   when token e has no representative within the threshold and m = m_max, the threshold doubles
+ *   (thr2 <- max(4 thr2, 1) in fixed point, capped at 2^62) and the clusters are swept in index order: cluster i
+ *   is kept if no already kept representative lies within the new threshold of x_i, otherwise it is merged into
+ *   the nearest kept one (ties: lowest kept index). Kept clusters are renumbered in order. Token e is then placed
+ *   against the kept representatives with the new threshold; if it still has to open a cluster and there is still
+ *   no room, the threshold doubles again.
+ * Merging cluster i (n_i members) into kept cluster j (n_j members): the count becomes n_j + n_i and every sample
+ * slot q of j independently takes slot q of i with probability n_i / (n_j + n_i), which keeps each slot uniform
+ * over the union, exactly as property (5) of Lemma 2 needs. The coin is
+ *   u * (n_j + n_i) < n_i * 2^32,  u = word q % 4 of Philox(counter = (e, unit, q / 4 + 256 * i, 2 + 4 * level)),
+ * i the index the merged cluster had before this sweep, level the number of doublings including this one.
+ */
+static uint32_t merge_coin_word(const oracle_unit *u, int token, int slot, int old_index) {
+    uint32_t ctr[4] = {(uint32_t)token, u->unit_id, (uint32_t)(slot / 4) + 256u * (uint32_t)old_index,
+                       2u + 4u * (uint32_t)u->level};
+    uint32_t out[4];
+    oracle_philox4x32_10(ctr, u->key, out);
+    return out[slot % 4];
+}
+
+static void doubling_sweep(oracle_unit *u, int e) {
+    u->level++;
+    if (u->thr2_fx >= ((uint64_t)1 << 60)) u->thr2_fx = (uint64_t)1 << 62;
+    else u->thr2_fx = u->thr2_fx ? 4 * u->thr2_fx : 1;
+    int *remap = (int *)malloc(sizeof(int) * (size_t)u->m);
+    int kept = 0;
+    for (int i = 0; i < u->m; ++i) {
+        const float *xi = u->K + (size_t)u->centre_tok[i] * u->d;
+        int best = -1;
+        uint64_t best_d2 = UINT64_MAX;
+        for (int j = 0; j < kept; ++j) {
+            uint64_t d2 = dist2_fx(u->K + (size_t)u->centre_tok[j] * u->d, xi, u->d);
+            if (d2 < best_d2) { best_d2 = d2; best = j; }
+        }
+        if (best >= 0 && best_d2 <= u->thr2_fx) {
+            uint64_t n_i = (uint64_t)u->count[i], n_new = (uint64_t)u->count[best] + n_i;
+            for (int q = 0; q < u->t; ++q) {
+                uint32_t w = merge_coin_word(u, e, q, i);
+                if ((uint64_t)w * n_new < (n_i << 32)) u->slot_tok[(size_t)best * u->t + q] = u->slot_tok[(size_t)i * u->t + q];
+            }
+            u->count[best] = (int)n_new;
+            remap[i] = best;
+        } else {
+            u->centre_tok[kept] = u->centre_tok[i];
+            u->count[kept] = u->count[i];
+            for (int q = 0; q < u->t; ++q) u->slot_tok[(size_t)kept * u->t + q] = u->slot_tok[(size_t)i * u->t + q];
+            remap[i] = kept++;
+        }
+    }
+    for (int tok = 0; tok < u->inserted; ++tok) u->assign[tok] = remap[u->assign[tok]];
+    u->m = kept;
+    free(remap);
+}
+
 /* Procedure UpdateSoftmaxNormalizer for token e. Returns 0, or -1 if D is full. */
 static int update_softmax_normalizer(oracle_unit *u, int e) {
     const float *k = u->K + (size_t)e * u->d;
-    int best = -1;
-    uint64_t best_d2 = UINT64_MAX;
-    for (int i = 0; i < u->m; ++i) {                    /* argmin over representatives */
-        uint64_t d2 = dist2_fx(u->K + (size_t)u->centre_tok[i] * u->d, k, u->d);
-        if (d2 < best_d2) { best_d2 = d2; best = i; }  /* strict: ties keep the lowest index */
-    }
-    u->ins_d2[e] = best_d2;
-    u->ins_near[e] = best;
-    if (best >= 0 && best_d2 <= u->delta2_fx) {
-        int n_new = ++u->count[best];
-        for (int j = 0; j < u->t; ++j) {               /* t independent size-1 reservoirs */
-            uint32_t w = coin_word(u, e, j, 0u);
-            if ((uint64_t)w * (uint64_t)n_new < 4294967296ull) u->slot_tok[(size_t)best * u->t + j] = e;
+    for (int round = 0;; ++round) {
+        int best = -1;
+        uint64_t best_d2 = UINT64_MAX;
+        for (int i = 0; i < u->m; ++i) {                    /* argmin over representatives */
+            uint64_t d2 = dist2_fx(u->K + (size_t)u->centre_tok[i] * u->d, k, u->d);
+            if (d2 < best_d2) { best_d2 = d2; best = i; }  /* strict: ties keep the lowest index */
         }
-        u->assign[e] = best;
-    } else {
-        if (u->m >= u->m_max) { if (u->overflow_at < 0) u->overflow_at = e; return -1; }
-        int c = u->m++;
-        u->centre_tok[c] = e;                           /* representative = first key of the cluster */
-        u->count[c] = 1;
-        for (int j = 0; j < u->t; ++j) u->slot_tok[(size_t)c * u->t + j] = e;   /* t copies */
-        u->assign[e] = c;
+        u->ins_d2[e] = best_d2;
+        u->ins_near[e] = best;
+        if (best >= 0 && best_d2 <= u->thr2_fx) {
+            int n_new = ++u->count[best];
+            for (int j = 0; j < u->t; ++j) {               /* t independent size-1 reservoirs */
+                uint32_t w = coin_word(u, e, j, 0u);
+                if ((uint64_t)w * (uint64_t)n_new < 4294967296ull) u->slot_tok[(size_t)best * u->t + j] = e;
+            }
+            u->assign[e] = best;
+            return 0;
+        }
+        if (u->m < u->m_max) {
+            int c = u->m++;
+            u->centre_tok[c] = e;                           /* representative = first key of the cluster */
+            u->count[c] = 1;
+            for (int j = 0; j < u->t; ++j) u->slot_tok[(size_t)c * u->t + j] = e;   /* t copies */
+            u->assign[e] = c;
+            return 0;
+        }
+        if (!u->bounded || round >= 40) { if (u->overflow_at < 0) u->overflow_at = e; return -1; }
+        doubling_sweep(u, e);
     }
-    return 0;
 }
 
 /* Procedure UpdateMatrixProduct for token e, with the mu of before this token. */
@@ -355,6 +425,10 @@ int oracle_inserted(const oracle_unit *u) { return u->inserted; }
 int oracle_m(const oracle_unit *u) { return u->m; }
 uint64_t oracle_mu(const oracle_unit *u) { return u->mu; }
 uint64_t oracle_delta2_fx(const oracle_unit *u) { return u->delta2_fx; }
+/* Switch on the bounded-m variant; valid only before the first token. */
+int oracle_set_bounded(oracle_unit *u, int on) { if (u->n) return -1; u->bounded = on != 0; return 0; }
+uint64_t oracle_thr2_fx(const oracle_unit *u) { return u->thr2_fx; }
+int oracle_level(const oracle_unit *u) { return u->level; }
 int oracle_overflow_at(const oracle_unit *u) { return u->overflow_at; }
 const int *oracle_counts(const oracle_unit *u) { return u->count; }
 const int *oracle_centre_tok(const oracle_unit *u) { return u->centre_tok; }

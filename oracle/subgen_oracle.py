@@ -63,7 +63,10 @@ def lib():
                 for name in ("oracle_n", "oracle_inserted", "oracle_m", "oracle_overflow_at"):
                     getattr(L, name).argtypes = [vp]
                     getattr(L, name).restype = C.c_int
-                for name in ("oracle_mu", "oracle_delta2_fx"):
+                L.oracle_set_bounded.argtypes = [vp, C.c_int]
+                L.oracle_level.argtypes = [vp]
+                L.oracle_level.restype = C.c_int
+                for name in ("oracle_mu", "oracle_delta2_fx", "oracle_thr2_fx"):
                     getattr(L, name).argtypes = [vp]
                     getattr(L, name).restype = C.c_uint64
                 for name in ("oracle_counts", "oracle_centre_tok", "oracle_slot_tok", "oracle_m_tok",
@@ -144,13 +147,17 @@ def kcenter_window_attention(K, V, q, k, r):
 class OracleUnit:
     """One stream = one (sequence, KV head) unit of the SubGen data structure."""
 
-    def __init__(self, d, delta, t, s, window, seed=0, unit_id=0, m_max=1 << 16):
+    def __init__(self, d, delta, t, s, window, seed=0, unit_id=0, m_max=1 << 16, bounded=False):
+        """bounded=True: m_max is a budget; when it is exhausted the threshold doubles and clusters merge
+        (the doubling_sweep of the C file) instead of the stream failing."""
         self.d, self.t, self.s, self.window, self.m_max = int(d), int(t), int(s), int(window), int(m_max)
         self._L = lib()
         self._h = self._L.oracle_create(self.d, float(np.float32(delta)), self.t, self.s, self.window,
                                         int(seed) & (2 ** 64 - 1), int(unit_id), self.m_max)
         if not self._h:
             raise ValueError("oracle_create rejected its arguments")
+        if bounded:
+            self._L.oracle_set_bounded(self._h, 1)
 
     def close(self):
         if getattr(self, "_h", None):
@@ -216,6 +223,10 @@ class OracleUnit:
     def mu(self): return int(self._L.oracle_mu(self._h))
     @property
     def delta2_fx(self): return int(self._L.oracle_delta2_fx(self._h))
+    @property
+    def thr2_fx(self): return int(self._L.oracle_thr2_fx(self._h))
+    @property
+    def level(self): return self._L.oracle_level(self._h)
     @property
     def overflow_at(self): return self._L.oracle_overflow_at(self._h)
     @property
