@@ -194,7 +194,7 @@ def workload_config(w):
                             w.name, w.B, w.H, w.Hkv, w.d, w.dtype, w.n_prompt, w.ncomp, w.sigma, w.outlier_frac, w.drift,
                             w.delta, w.t, w.s, w.window, w.philox_seed),
             "l2": "per-step working set (compressed cache) larger than the 126 MB L2; no explicit flush",
-            "accumulate": "fp32", "units": w.units}
+            "accumulate": "fp32", "units": w.units, "m_max": w.m_max}
 
 
 def run_subgen(args, w):
@@ -250,7 +250,7 @@ def run_subgen(args, w):
     torch.cuda.synchronize()
 
     sg = binding.SubGen(wr.B, wr.H, wr.d, wr.delta, wr.t, wr.s, wr.window, wr.philox_seed, Hkv=wr.Hkv, dtype=dt,
-                        m_max=wr.m_max, splits=args.splits)
+                        m_max=wr.m_max, splits=args.splits, bounded=args.bounded)
     out = torch.empty(wr.B, wr.H, wr.d, dtype=dt, device=dev)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
@@ -358,6 +358,9 @@ def run_subgen(args, w):
              "prefill_phases_ms": {"values": pf_values_ms, "score": pf_score_ms, "resolve": pf_resolve_ms},
              "prefill_score": tensor_roofline(pf_pairs, wr.d, pf_score_ms),
              "cache": {k: stats1[k] for k in ("clusters", "singleton_clusters", "m_filled", "window_rows", "tokens")}}
+    if args.bounded:
+        st0 = sg.export_state(0, 0)
+        extra["bounded"] = {"m_max": wr.m_max, "doublings_unit0": st0["doublings"], "clusters_unit0": st0["m"], "status": sg.status()}
 
     # ---- exact dense decode over full caches on the same inputs (comparison point) ----
     if args.exact and rank == 0:
@@ -490,6 +493,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--prompt", type=int, default=0, help="override the prompt length (smaller cases for profiling)")
     ap.add_argument("--batch", type=int, default=0, help="override the number of sequences")
+    ap.add_argument("--bounded", action="store_true",
+                    help="bounded-m variant: m_max is a budget (threshold doubling and merging), prompts inserted token by token")
+    ap.add_argument("--m-max", type=int, default=0, help="override the cluster capacity / budget per unit")
     ap.add_argument("--kcenter", default="", help="k,r: also time the one-shot k-center compression of the exact caches")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "subgen":
@@ -499,6 +505,8 @@ def main():
         w = w.scaled(n_prompt=args.prompt)
     if args.batch:
         w = w.scaled(B=args.batch)
+    if args.m_max:
+        w = w.scaled(m_max=args.m_max)
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -78,7 +78,24 @@ typedef struct subgen_config {
     void* workspace;        /* device, >= subgen_workspace_bytes(), 256-byte aligned, or NULL: the library allocates */
     size_t workspace_bytes;
     void* stream;           /* cudaStream_t, or NULL for the default stream */
+    int bounded;            /* 0: Algorithm 1 as printed, m_max is a capacity (exceeding it is an error);
+                             * 1: m_max is a budget, see "Bounded-m variant" below */
 } subgen_config;
+
+/* Bounded-m variant (subgen_config.bounded = 1). Algorithm 1 keeps as many clusters as the keys need; the
+ * paper bounds their number only through its clusterability assumption and names the incremental clustering of
+ * Charikar et al. as the inspiration of its online clustering (Section 1.1). With bounded = 1 a key that would
+ * need cluster number m_max + 1 makes the unit double its threshold instead (thr^2 <- max(4 thr^2, 1) in fixed
+ * point, capped at 2^62) and sweep its clusters in index order: cluster i is kept if no kept representative lies
+ * within the new threshold of x_i, else it is merged into the nearest kept one (ties: lowest kept index); kept
+ * clusters are renumbered in order. A merge adds the counts and lets each sample slot q of the surviving cluster
+ * take slot q of the merged one with probability n_i / (n_j + n_i), so that slots stay uniform over the union
+ * (property 5 of Lemma 2): coin u * (n_j + n_i) < n_i * 2^32 with u = word q % 4 of Philox(counter = (token,
+ * unit, q / 4 + 256 * i, 2 + 4 * doublings)), i the merged cluster's index before the sweep. The key is then
+ * placed under the new threshold; if it still needs a new cluster and none is free, the threshold doubles again.
+ * M, mu and the window are untouched. Such handles insert prompts token by token (the chunked prefill assumes
+ * stable cluster indices within a chunk), and a sweep is done by one thread block, so the step that triggers
+ * one takes milliseconds; thresholds double, so a unit sees few of them. */
 
 /* Bytes of device memory a handle of this configuration needs (0 on invalid configuration). */
 size_t subgen_workspace_bytes(const subgen_config* cfg);
@@ -131,6 +148,9 @@ typedef struct subgen_state_view {
     int* slot_tok;     /* [m_max * t]  token index held by S_i(j) */
     int* m_tok;        /* [s]          token index held by M(j), -1 = null */
     uint64_t* m_w;     /* [s]          W of that token, 0 = null */
+    /* outputs again */
+    uint64_t threshold2; /* squared threshold in force, fixed point: floor(delta^2 2^32) * 4^doublings */
+    int doublings;       /* threshold doublings so far (always 0 unless the handle is bounded) */
 } subgen_state_view;
 
 /* Synchronous copy of one unit's bookkeeping to the host (waits for the stream). */

@@ -34,14 +34,14 @@ class SubgenConfig(C.Structure):
     _fields_ = [("B", C.c_int), ("H", C.c_int), ("Hkv", C.c_int), ("d", C.c_int), ("delta", C.c_float),
                 ("t", C.c_int), ("s", C.c_int), ("window", C.c_int), ("seed", C.c_uint64), ("dtype", C.c_int),
                 ("m_max", C.c_int), ("splits", C.c_int), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-                ("stream", C.c_void_p)]
+                ("stream", C.c_void_p), ("bounded", C.c_int)]
 
 
 class StateView(C.Structure):
     _fields_ = [("n", C.c_int), ("inserted", C.c_int), ("m", C.c_int), ("status", C.c_int), ("mu", C.c_uint64),
                 ("last_cluster", C.c_int), ("last_opened", C.c_int), ("last_d2", C.c_uint64),
                 ("counts", C.c_void_p), ("centre_tok", C.c_void_p), ("slot_tok", C.c_void_p),
-                ("m_tok", C.c_void_p), ("m_w", C.c_void_p)]
+                ("m_tok", C.c_void_p), ("m_w", C.c_void_p), ("threshold2", C.c_uint64), ("doublings", C.c_int)]
 
 
 class Stats(C.Structure):
@@ -134,16 +134,17 @@ class SubGen:
     """One library handle: the SubGen caches of B sequences x Hkv KV heads on the current CUDA device."""
 
     def __init__(self, B, H, d, delta, t, s, window, seed=0, *, Hkv=None, dtype=torch.bfloat16, m_max=0, splits=0,
-                 stream: Optional[torch.cuda.Stream] = None):
+                 stream: Optional[torch.cuda.Stream] = None, bounded: bool = False):
         self._L = load()
         self._h = None
         if not torch.cuda.is_available():
             raise SubgenError("no CUDA device: this library has no CPU path")
+        self.bounded = bool(bounded)
         self.B, self.H, self.Hkv, self.d = int(B), int(H), int(Hkv or H), int(d)
         self.t, self.s, self.window, self.dtype = int(t), int(s), int(window), dtype
         self.stream = stream or torch.cuda.current_stream()
         cfg = SubgenConfig(self.B, self.H, self.Hkv, self.d, float(delta), self.t, self.s, self.window, int(seed),
-                           _dtype_code(dtype), int(m_max), int(splits), None, 0, self.stream.cuda_stream)
+                           _dtype_code(dtype), int(m_max), int(splits), None, 0, self.stream.cuda_stream, int(bool(bounded)))
         nbytes = self._L.subgen_workspace_bytes(C.byref(cfg))
         if nbytes == 0:
             raise SubgenError(self._L.subgen_last_error().decode())
@@ -212,7 +213,7 @@ class SubGen:
         return dict(n=v.n, inserted=v.inserted, m=m, status=v.status, mu=int(v.mu), last_cluster=v.last_cluster,
                     last_opened=v.last_opened, last_d2=int(v.last_d2), counts=counts[:m].copy(),
                     centre_tok=ctok[:m].copy(), slot_tok=stok.reshape(self.m_max, self.t)[:m].copy(),
-                    m_tok=mtok, m_w=mw)
+                    m_tok=mtok, m_w=mw, threshold2=int(v.threshold2), doublings=v.doublings)
 
     def export_rows(self, seq: int, kvhead: int, which: int) -> torch.Tensor:
         rows = {0: self.m_max, 1: self.m_max * self.t, 2: self.s, 3: self.s, 4: self.window, 5: self.window}[which]

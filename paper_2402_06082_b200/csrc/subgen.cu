@@ -47,6 +47,7 @@ size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
     size_t X, S, xn, cnt, ctok, stok, Mk, Mv, MW, Mtok, ringK, ringV;
     size_t n_unit, m_unit, mu, status, last_cid, last_open, last_d2, part1, part2, ticket1, ticket2, qnext, qnext2, part_tau, MinvW, pairs;
+    size_t thr2, level;
     size_t stage_q, stage_k, stage_v, stage_out, cu, stats;
     size_t book_begin, book_end;   // bookkeeping region cleared at creation
     size_t total;
@@ -139,6 +140,8 @@ Layout make_layout(const Dims& d) {
     L.qnext = take(U * sizeof(unsigned));
     L.qnext2 = take(U * sizeof(unsigned));
     L.pairs = take(U * sizeof(uint64_t));
+    L.thr2 = take(U * sizeof(uint64_t));
+    L.level = take(U * sizeof(int));
     L.MinvW = take(U * d.s * sizeof(float));
     L.MW = take(U * d.s * sizeof(uint64_t));
     L.stats = take(8 * sizeof(uint64_t));
@@ -177,6 +180,15 @@ struct subgen {
 
 namespace {
 
+// Every unit's threshold back to delta^2 (bounded handles). Synchronous.
+cudaError_t reset_thresholds(subgen* h) {
+    const unsigned long long d2 = (unsigned long long)floor((double)h->cfg.delta * (double)h->cfg.delta * 4294967296.0);
+    std::vector<unsigned long long> v((size_t)h->d.U, d2);
+    cudaError_t e = cudaStreamSynchronize(h->st);
+    if (e == cudaSuccess) e = cudaMemcpy(h->ws + h->L.thr2, v.data(), v.size() * 8, cudaMemcpyHostToDevice);
+    return e;
+}
+
 template <typename T> Cache<T> make_cache(const subgen* h) {
     const Dims& d = h->d;
     const Layout& L = h->L;
@@ -199,6 +211,8 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
     C.qnext = (unsigned*)(w + L.qnext); C.qnext2 = (unsigned*)(w + L.qnext2);
     C.part_tau = (float*)(w + L.part_tau); C.MinvW = (float*)(w + L.MinvW);
     C.pairs = (unsigned long long*)(w + L.pairs);
+    C.bounded = h->cfg.bounded ? 1 : 0;
+    C.thr2 = (unsigned long long*)(w + L.thr2); C.level = (int*)(w + L.level);
     return C;
 }
 
@@ -248,10 +262,13 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
         h->ev_used += 4;
         CUDA_TRY(cudaEventRecord(e[0], h->st));
     }
-    if constexpr (std::is_same<T, __nv_bfloat16>::value)
-        insert_mma_kernel<D><<<grid_i, kInsertMmaThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
-    else
-        insert_kernel<T, D><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        if (C.bounded) insert_mma_kernel<D, true><<<grid_i, kInsertMmaThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
+        else insert_mma_kernel<D, false><<<grid_i, kInsertMmaThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
+    } else {
+        if (C.bounded) insert_kernel<T, D, true><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
+        else insert_kernel<T, D, false><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
+    }
     if (e) CUDA_TRY(cudaEventRecord(e[1], h->st));
     launch_query<T, D>(C, h->d.G, grid_t, grid_z, h->st, q, out, e ? e[2] : nullptr);
     if (e) CUDA_TRY(cudaEventRecord(e[3], h->st));
@@ -269,7 +286,8 @@ int launch_step(subgen* h, const void* q, const void* k, const void* v, void* ou
 template <typename T, int D>
 int launch_prefill_td(subgen* h, const void* K, const void* V, int n, const int* cu_dev, int total) {
     Cache<T> C = make_cache<T>(h);
-    prefill_seq_kernel<T, D><<<h->d.U, kPrefillThreads, 0, h->st>>>(C, (const T*)K, (const T*)V, n, cu_dev, total);
+    if (C.bounded) prefill_seq_kernel<T, D, true><<<h->d.U, kPrefillThreads, 0, h->st>>>(C, (const T*)K, (const T*)V, n, cu_dev, total);
+    else prefill_seq_kernel<T, D, false><<<h->d.U, kPrefillThreads, 0, h->st>>>(C, (const T*)K, (const T*)V, n, cu_dev, total);
     CUDA_TRY(cudaGetLastError());
     h->launches += 1;
     return SUBGEN_OK;
@@ -440,6 +458,17 @@ subgen_t* subgen_create_ex(const subgen_config* cfg) {
     }
     h->n_host.assign(d.B, 0);
     if (const char* env = getenv("SUBGEN_PREFILL")) { h->seq_prefill = strcmp(env, "seq") == 0; h->mma_score = strcmp(env, "mma") == 0; }
+    if (h->cfg.bounded) {
+        // merges renumber the clusters in the middle of a chunk, which the chunked prefill does not handle:
+        // bounded handles insert their prompts token by token
+        h->seq_prefill = true;
+        if (reset_thresholds(h) != cudaSuccess) {
+            fail(SUBGEN_ECUDA, "subgen_create: threshold initialisation failed");
+            if (h->owns) cudaFree(h->ws);
+            delete h;
+            return nullptr;
+        }
+    }
     return h;
 }
 
@@ -555,6 +584,13 @@ int subgen_export_state(subgen_t* h, int seq, int kvhead, subgen_state_view* v) 
     CUDA_TRY(get(&v->last_opened, h->L.last_open + u * 4, 4));
     CUDA_TRY(get(&v->last_d2, h->L.last_d2 + u * 8, 8));
     v->inserted = v->n > d.w ? v->n - d.w : 0;
+    if (h->cfg.bounded) {
+        CUDA_TRY(get(&v->threshold2, h->L.thr2 + u * 8, 8));
+        CUDA_TRY(get(&v->doublings, h->L.level + u * 4, 4));
+    } else {
+        v->threshold2 = (uint64_t)floor((double)h->cfg.delta * (double)h->cfg.delta * 4294967296.0);
+        v->doublings = 0;
+    }
     if (v->counts) CUDA_TRY(get(v->counts, h->L.cnt + u * d.m_max * 4, (size_t)d.m_max * 4));
     if (v->centre_tok) CUDA_TRY(get(v->centre_tok, h->L.ctok + u * d.m_max * 4, (size_t)d.m_max * 4));
     if (v->slot_tok) CUDA_TRY(get(v->slot_tok, h->L.stok + u * d.m_max * d.t * 4, (size_t)d.m_max * d.t * 4));
@@ -689,7 +725,7 @@ std::vector<CkptArray> ckpt_arrays(const subgen* h, int m_rows) {
         {L.Mk, s * row, s * row}, {L.Mv, s * row, s * row}, {L.MW, s * 8, s * 8}, {L.Mtok, s * 4, s * 4}, {L.MinvW, s * 4, s * 4},
         {L.ringK, w * row, w * row}, {L.ringV, w * row, w * row},
         {L.n_unit, 4, 4}, {L.m_unit, 4, 4}, {L.mu, 8, 8}, {L.status, 4, 4}, {L.last_cid, 4, 4}, {L.last_open, 4, 4},
-        {L.last_d2, 8, 8}, {L.pairs, 8, 8},
+        {L.last_d2, 8, 8}, {L.pairs, 8, 8}, {L.thr2, 8, 8}, {L.level, 4, 4},
     };
 }
 
@@ -733,6 +769,7 @@ int subgen_checkpoint_save(subgen_t* h, void* host, size_t bytes, size_t* writte
     hd.magic = kCkptMagic; hd.version = 1; hd.dtype = (uint32_t)h->cfg.dtype;
     hd.B = h->d.B; hd.H = h->d.H; hd.Hkv = h->d.Hkv; hd.d = h->d.D; hd.t = h->d.t; hd.s = h->d.s; hd.window = h->d.w;
     hd.m_rows = m_rows; hd.delta = h->cfg.delta; hd.seed = h->cfg.seed; hd.payload_bytes = payload;
+    hd.pad = h->cfg.bounded ? 1u : 0u;
     memcpy(host, &hd, sizeof hd);
     char* dst = (char*)host + sizeof hd;
     for (const CkptArray& a : ckpt_arrays(h, m_rows)) {
@@ -752,9 +789,10 @@ int subgen_checkpoint_load(subgen_t* h, const void* host, size_t bytes) {
     if (hd.magic != kCkptMagic || hd.version != 1) return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: not a checkpoint of this library version");
     const Dims& d = h->d;
     if (hd.B != d.B || hd.H != d.H || hd.Hkv != d.Hkv || hd.d != d.D || hd.t != d.t || hd.s != d.s || hd.window != d.w ||
-        (int)hd.dtype != h->cfg.dtype || hd.seed != h->cfg.seed || memcmp(&hd.delta, &h->cfg.delta, sizeof(float)) != 0)
+        (int)hd.dtype != h->cfg.dtype || hd.seed != h->cfg.seed || memcmp(&hd.delta, &h->cfg.delta, sizeof(float)) != 0 ||
+        hd.pad != (h->cfg.bounded ? 1u : 0u))
         return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: the checkpoint was written with another configuration "
-                    "(B, H, Hkv, d, t, s, window, dtype, delta and seed must match; only m_max may differ)");
+                    "(B, H, Hkv, d, t, s, window, dtype, delta, seed and the bounded flag must match; only m_max may differ)");
     if (hd.m_rows < 0 || hd.m_rows > d.m_max)
         return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: the checkpoint holds %d clusters per unit, this handle's m_max is %d", hd.m_rows, d.m_max);
     const size_t payload = ckpt_payload(h, hd.m_rows);

@@ -112,7 +112,18 @@ template <typename T> struct Cache {
     unsigned* qnext;     // [U] next work item of the cluster scan's per-unit queue
     unsigned* qnext2;    // [U] same for the scan of M and the window
     unsigned long long* pairs;   // [U] (key, representative) pairs scored by the chunked prefill so far
+    // bounded-m variant: m_max is a budget, the threshold doubles and clusters merge when it is exhausted
+    int bounded;
+    unsigned long long* thr2;    // [U] threshold in force (fixed point), starts as delta2_fx
+    int* level;                  // [U] doublings so far
 };
+
+// The squared threshold a key of unit u is tested against. BND: the handle runs the bounded-m variant; it is a
+// template parameter of the insertion kernels so that the plain path carries none of the variant's code.
+template <bool BND, typename T>
+__device__ __forceinline__ unsigned long long threshold2(const Cache<T>& C, int u) {
+    return BND ? C.thr2[u] : C.delta2_fx;
+}
 
 // ---------------------------------------------------------------------------------------------
 // Nearest representative: scan rows [c0, c1) of X_u with `ngroups` row groups, every group keeps its
@@ -163,12 +174,97 @@ __device__ __forceinline__ Best block_best(Best b, Best* sm) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// Bounded-m variant: token e has no representative within the threshold and all m_max clusters are in use.
+// The paper fixes no rule for this; the one taken here follows the doubling idea of the incremental clustering
+// it cites: double the threshold (thr2 <- max(4 thr2, 1), capped at 2^62), sweep the clusters in index order,
+// keep cluster i if no kept representative lies within the new threshold of x_i, otherwise merge it into the
+// nearest kept one (ties: lowest kept index); kept clusters move to the front in order. Merging i (n_i members)
+// into j (n_j): count n_j + n_i, and slot q of j takes slot q of i with probability n_i / (n_j + n_i), coin
+//   u * (n_j + n_i) < n_i * 2^32,  u = word q % 4 of Philox(counter = (e, unit, q / 4 + 256 * i, 2 + 4 * level)),
+// which keeps every slot uniform over the union (property 5 of Lemma 2). Then e is placed against the kept
+// representatives; if it still must open a cluster and there is still no room, the threshold doubles again.
+// Executed by a whole block; on return best and m describe the placement of e under the new threshold.
+template <typename T, int D>
+__device__ void make_room(const Cache<T>& C, int u, int e, const uint4* krow, Best& best, int& m) {
+    constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, RPW = 32 / LPR;
+    __shared__ Best smb[32];
+    __shared__ uint4 xrow[LPR];
+    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, lr = lane % LPR, sub = lane / LPR;
+    const int group = warp * RPW + sub, ngroups = (nt >> 5) * RPW, t = C.t;
+    T* Xu = C.X + (size_t)u * C.m_max * D;
+    T* Su = C.S + (size_t)u * C.m_max * t * D;
+    int* cntu = C.cnt + (size_t)u * C.m_max;
+    int* ctoku = C.ctok + (size_t)u * C.m_max;
+    int* stoku = C.stok + (size_t)u * C.m_max * t;
+    float* xnu = C.xn + (size_t)u * C.m_max;
+    unsigned long long thr = C.thr2[u];
+    int level = C.level[u];
+    for (int round = 0; round < 40; ++round) {
+        ++level;
+        thr = thr >= (1ull << 60) ? (1ull << 62) : (thr ? 4ull * thr : 1ull);
+        int kept = 0;
+        for (int i = 0; i < m; ++i) {
+            __syncthreads();                       // rows and counts written for cluster i-1 are visible
+            if (tid < LPR) xrow[tid] = reinterpret_cast<const uint4*>(Xu + (size_t)i * D)[tid];
+            __syncthreads();
+            float xf[EPL];
+            Elem<T>::unpack(xrow[lr], xf);
+            Best b;
+            b.d2 = ~0ull; b.idx = INT_MAX; b.pad = 0;
+            scan_centres<T, D>(Xu, 0, kept, xf, group, ngroups, lr, b);
+            b = block_best(b, smb);
+            const int n_i = cntu[i];
+            if (kept > 0 && b.d2 <= thr) {
+                const int j = b.idx, n_j = cntu[j];
+                const unsigned long long n_new = (unsigned long long)n_i + (unsigned long long)n_j;
+                for (int p = tid; p < t * LPR; p += nt) {
+                    const int q = p / LPR, part = p % LPR;
+                    const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)(q >> 2) + 256u * (uint32_t)i,
+                                                             2u + 4u * (uint32_t)level), C.key0, C.key1);
+                    const uint32_t word = (q & 3) == 0 ? r.x : (q & 3) == 1 ? r.y : (q & 3) == 2 ? r.z : r.w;
+                    uint4* dst = reinterpret_cast<uint4*>(Su + ((size_t)j * t + q) * D) + part;
+                    if ((unsigned long long)word * n_new < ((unsigned long long)n_i << 32)) {
+                        *dst = n_i == 1 ? xrow[part] : reinterpret_cast<const uint4*>(Su + ((size_t)i * t + q) * D)[part];
+                        if (part == 0) stoku[(size_t)j * t + q] = stoku[(size_t)i * t + q];
+                    } else if (n_j == 1) {
+                        *dst = reinterpret_cast<const uint4*>(Xu + (size_t)j * D)[part];   // write out the implied copy
+                    }
+                }
+                __syncthreads();                   // n_j was read by everyone before it changes
+                if (tid == 0) cntu[j] = (int)n_new;
+            } else {
+                if (kept != i) {
+                    if (tid < LPR) reinterpret_cast<uint4*>(Xu + (size_t)kept * D)[tid] = xrow[tid];
+                    if (n_i >= 2)
+                        for (int p = tid; p < t * LPR; p += nt)
+                            reinterpret_cast<uint4*>(Su + (size_t)kept * t * D)[p] = reinterpret_cast<const uint4*>(Su + (size_t)i * t * D)[p];
+                    for (int q = tid; q < t; q += nt) stoku[(size_t)kept * t + q] = stoku[(size_t)i * t + q];
+                    if (tid == 0) { cntu[kept] = n_i; ctoku[kept] = ctoku[i]; xnu[kept] = xnu[i]; }
+                }
+                ++kept;
+            }
+        }
+        __syncthreads();
+        m = kept;
+        float kf[EPL];
+        Elem<T>::unpack(krow[lr], kf);
+        Best b;
+        b.d2 = ~0ull; b.idx = INT_MAX; b.pad = 0;
+        scan_centres<T, D>(Xu, 0, m, kf, group, ngroups, lr, b);
+        best = block_best(b, smb);
+        if ((m > 0 && best.d2 <= thr) || m < C.m_max) break;
+    }
+    if (tid == 0) { C.thr2[u] = thr; C.level[u] = level; }
+    __syncthreads();
+}
+
+// ---------------------------------------------------------------------------------------------
 // Insert token e (key/value rows already in shared memory) into D and M of unit u, given the nearest
 // representative. Executed by a whole block; ends with a __syncthreads(). Returns the new m.
 //   UpdateSoftmaxNormalizer: join (count, t coins) or open (representative, count 1; the t copies are
 //   implied while n_i = 1 and written out when the second member arrives);
 //   UpdateMatrixProduct: s coins with the OLD mu; then mu += W.
-template <typename T, int D>
+template <typename T, int D, bool BND = false>
 __device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, const uint4* krow, const uint4* vrow,
                             unsigned long long* sm_w /* shared, 2 elements */) {
     constexpr int EPL = Elem<T>::EPL, LPR = D / EPL;
@@ -207,7 +303,10 @@ __device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, c
     const unsigned long long W = sm_w[0];
     const unsigned long long mu_old = C.mu[u];
 
-    const bool join = (m > 0) && (best.d2 <= C.delta2_fx);
+    if constexpr (BND) {
+        if (!((m > 0) && (best.d2 <= C.thr2[u])) && m >= C.m_max) make_room<T, D>(C, u, e, krow, best, m);
+    }
+    const bool join = (m > 0) && (best.d2 <= threshold2<BND>(C, u));
     const bool full = !join && (m >= C.m_max);
     T* Xu = C.X + (size_t)u * C.m_max * D;
     T* Su = C.S + (size_t)u * C.m_max * t * D;

@@ -18,7 +18,7 @@ namespace sgk {
 
 constexpr int kInsertMmaThreads = 128;
 
-template <int D>
+template <int D, bool BND>
 __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ k_new,
                                                                     const __nv_bfloat16* __restrict__ v_new) {
     typedef __nv_bfloat16 T;
@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
     }
     kn += __shfl_xor_sync(0xffffffffu, kn, 1);
     kn += __shfl_xor_sync(0xffffffffu, kn, 2);
-    const float d2f = (float)((double)C.delta2_fx * (1.0 / 4294967296.0));
+    const float d2f = (float)((double)threshold2<BND>(C, u) * (1.0 / 4294967296.0));
 
     const int per = (((m + splits - 1) / splits) + 15) & ~15;       // slices are whole tiles
     const int c0 = blockIdx.x * per, c1 = min(m, c0 + per);
@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
     }
     if (tid < LPR) vrow[tid] = w ? ringv[tid] : vnew_u[tid];
     __syncthreads();
-    apply_insert<T, D>(C, u, e, b, m, krow, vrow, sm_w);
+    apply_insert<T, D, BND>(C, u, e, b, m, krow, vrow, sm_w);
     if (w) {
         if (tid < LPR) ringk[tid] = knew_u[tid];
         else if (tid < 2 * LPR) ringv[tid - LPR] = vnew_u[tid - LPR];

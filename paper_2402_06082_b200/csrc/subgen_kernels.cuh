@@ -16,7 +16,7 @@ constexpr int kPrefillThreads = 512;
 // (procedure UpdateSoftmaxNormalizer, argmin), the block that finishes last merges the slices and
 // applies the update (join/open, coins, UpdateMatrixProduct, mu) and then stores the new token in
 // the window row the old one occupied. Nothing waits on another block.
-template <typename T, int D>
+template <typename T, int D, bool BND>
 __global__ void __launch_bounds__(kInsertThreads) insert_kernel(Cache<T> C, const T* __restrict__ k_new,
                                                                 const T* __restrict__ v_new) {
     constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, RPW = 32 / LPR;
@@ -72,7 +72,7 @@ __global__ void __launch_bounds__(kInsertThreads) insert_kernel(Cache<T> C, cons
     }
     if (tid < LPR) vrow[tid] = w ? ringv[tid] : vnew_u[tid];
     __syncthreads();
-    apply_insert<T, D>(C, u, e, b, m, krow, vrow, sm_w);
+    apply_insert<T, D, BND>(C, u, e, b, m, krow, vrow, sm_w);
     if (w) {
         if (tid < LPR) ringk[tid] = knew_u[tid];
         else if (tid < 2 * LPR) ringv[tid - LPR] = vnew_u[tid - LPR];
@@ -221,7 +221,7 @@ __global__ void __launch_bounds__(kQueryThreads) query_kernel(Cache<T> C, const 
 // equals that of the same number of stream steps.
 // Rows of unit (b, h): K + (row0 + i) * D, row0 = (b*Hkv + h) * n_add (dense [B,Hkv,n,D]) or
 // h * total + cu[b] (packed [Hkv,total,D]).
-template <typename T, int D>
+template <typename T, int D, bool BND>
 __global__ void __launch_bounds__(kPrefillThreads) prefill_seq_kernel(Cache<T> C, const T* __restrict__ K,
                                                                       const T* __restrict__ V, int n_uniform,
                                                                       const int* __restrict__ cu, int total) {
@@ -250,7 +250,7 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_seq_kernel(Cache<T> C
         bst.d2 = ~0ull; bst.idx = INT_MAX; bst.pad = 0;
         scan_centres<T, D>(Xu, 0, m, kf, warp * RPW + sub, (nt >> 5) * RPW, lr, bst);
         bst = block_best(bst, smb);
-        m = apply_insert<T, D>(C, u, e, bst, m, krow, vrow, sm_w);
+        m = apply_insert<T, D, BND>(C, u, e, bst, m, krow, vrow, sm_w);
     }
     if (w) {
         const int lo = max(n_prev, n_tot - w);
