@@ -250,7 +250,7 @@ def run_subgen(args, w):
     torch.cuda.synchronize()
 
     sg = binding.SubGen(wr.B, wr.H, wr.d, wr.delta, wr.t, wr.s, wr.window, wr.philox_seed, Hkv=wr.Hkv, dtype=dt,
-                        m_max=wr.m_max, splits=args.splits, bounded=args.bounded)
+                        m_max=wr.m_max, splits=args.splits, bounded=args.bounded, nq_max=max(1, args.multi_query))
     out = torch.empty(wr.B, wr.H, wr.d, dtype=dt, device=dev)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
@@ -358,6 +358,27 @@ def run_subgen(args, w):
              "prefill_phases_ms": {"values": pf_values_ms, "score": pf_score_ms, "resolve": pf_resolve_ms},
              "prefill_score": tensor_roofline(pf_pairs, wr.d, pf_score_ms),
              "cache": {k: stats1[k] for k in ("clusters", "singleton_clusters", "m_filled", "window_rows", "tokens")}}
+    if args.multi_query > 1:
+        # read-only multi-query calls against the final state: same cache bytes as a step's query, nq answers each
+        nq = args.multi_query
+        probes = torch.randn(wr.B, wr.H, nq, wr.d, device=dev).to(dt)
+        pout = torch.empty_like(probes)
+        single = probes[:, :, :1].contiguous()
+        sout = torch.empty_like(single)
+        res = {}
+        for name, qq, oo in (("nq1", single, sout), ("nq%d" % nq, probes, pout)):
+            for _ in range(5):
+                sg.query(qq, oo)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(200):
+                sg.query(qq, oo)
+            e1.record()
+            torch.cuda.synchronize()
+            ms_q = e0.elapsed_time(e1) / 200
+            res[name] = {"ms_per_call": ms_q, "answers_per_s": wr.B * wr.H * qq.shape[2] / (ms_q * 1e-3),
+                         "achieved_GBps": stats1["query_bytes"] / (ms_q * 1e-3) / 1e9}
+        extra["multi_query"] = res
     if args.bounded:
         st0 = sg.export_state(0, 0)
         extra["bounded"] = {"m_max": wr.m_max, "doublings_unit0": st0["doublings"], "clusters_unit0": st0["m"], "status": sg.status()}
@@ -493,6 +514,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--prompt", type=int, default=0, help="override the prompt length (smaller cases for profiling)")
     ap.add_argument("--batch", type=int, default=0, help="override the number of sequences")
+    ap.add_argument("--multi-query", type=int, default=0,
+                    help="also time read-only subgen_query calls with this many queries per head (power of two, G*nq <= 8)")
     ap.add_argument("--bounded", action="store_true",
                     help="bounded-m variant: m_max is a budget (threshold doubling and merging), prompts inserted token by token")
     ap.add_argument("--m-max", type=int, default=0, help="override the cluster capacity / budget per unit")

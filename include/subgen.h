@@ -78,6 +78,7 @@ typedef struct subgen_config {
     void* workspace;        /* device, >= subgen_workspace_bytes(), 256-byte aligned, or NULL: the library allocates */
     size_t workspace_bytes;
     void* stream;           /* cudaStream_t, or NULL for the default stream */
+    int nq_max;             /* most queries per head one subgen_query call may carry; 0 = 1; (H / Hkv) * nq_max <= 8 */
     int bounded;            /* 0: Algorithm 1 as printed, m_max is a capacity (exceeding it is an error);
                              * 1: m_max is a budget, see "Bounded-m variant" below */
 } subgen_config;
@@ -125,6 +126,14 @@ int subgen_prefill_varlen(subgen_t* h, const void* K, const void* V, const int* 
  *   out = z / tau                       (no 1/sqrt(d): Eq. 1 has none)
  * q, out: device [B, H, d]; k, v: device [B, Hkv, d]. Query head h uses KV head h / (H/Hkv). */
 int subgen_step(subgen_t* h, const void* q, const void* k, const void* v, void* out);
+
+/* Procedure QueryStreamAttn alone, for nq queries per head at once, against the state as it stands (all tokens
+ * appended so far; nothing is inserted, nothing changes): out[b, h, j] = z / tau for query q[b, h, j]. The cache
+ * is read once for all nq queries: they ride in the spare columns of the tensor-core tiles that otherwise carry
+ * the H / Hkv heads of a KV head, so a call costs about what a step's query costs. Use: scoring several draft
+ * continuations, or several heads' worth of probes, against one context. q, out: device [B, H, nq, d]; nq a
+ * power of two, (H / Hkv) * nq <= 8 and nq <= the nq_max given at creation. Every sequence must hold a token. */
+int subgen_query(subgen_t* h, const void* q, int nq, void* out);
 
 /* subgen_step with HOST buffers: copies q, k, v to the device, runs the step, copies out back and
  * waits for it. Pinned host memory makes the copies asynchronous to the host until the final wait. */

@@ -55,6 +55,7 @@ struct Layout {
 
 struct Dims {
     int B, H, Hkv, G, D, t, s, w, m_max, splits, U;
+    int Gs;                        // columns the query scratch is sized for: G * max(1, nq_max)
     int sp_insert, sp_tau, sp_z;   // blocks per unit of the three step kernels (splits = their maximum)
     size_t E;   // bytes per element
 };
@@ -68,6 +69,8 @@ bool resolve(const subgen_config* c, Dims* o, const char** why) {
     if (d.H % d.Hkv) { *why = "H must be a multiple of Hkv"; return false; }
     d.G = d.H / d.Hkv;
     if (d.G != 1 && d.G != 2 && d.G != 4 && d.G != 8) { *why = "H / Hkv must be 1, 2, 4 or 8"; return false; }
+    if (c->nq_max < 0 || d.G * (c->nq_max ? c->nq_max : 1) > 8) { *why = "(H / Hkv) * nq_max must be <= 8"; return false; }
+    d.Gs = d.G * (c->nq_max ? c->nq_max : 1);
     if (d.D != 64 && d.D != 128) { *why = "d must be 64 or 128"; return false; }
     if (d.t < 1 || d.t > 64) { *why = "t must be in 1..64"; return false; }
     if (d.s < 1 || d.s > 65536) { *why = "s must be in 1..65536"; return false; }
@@ -125,8 +128,8 @@ Layout make_layout(const Dims& d) {
     L.stage_out = take((size_t)d.B * d.H * row);
     L.cu = take(((size_t)d.B + 1) * sizeof(int));
     L.part1 = take(U * d.splits * sizeof(Best));
-    L.part2 = take(U * d.splits * d.G * (size_t)(d.D + 2) * sizeof(float));
-    L.part_tau = take(U * d.splits * d.G * 2 * sizeof(float));
+    L.part2 = take(U * d.splits * d.Gs * (size_t)(d.D + 2) * sizeof(float));
+    L.part_tau = take(U * d.splits * d.Gs * 2 * sizeof(float));
     L.book_begin = off;
     L.cnt = take(U * d.m_max * sizeof(int));
     L.xn = take(U * d.m_max * sizeof(float));
@@ -218,28 +221,28 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
 
 // fp32 caches: CUDA-core dot products (full fp32 products). bf16 caches: tensor-core kernel.
 template <typename T, int D>
-void launch_query(const Cache<T>& C, int G, dim3 grid, dim3 grid_z, cudaStream_t st, const void* q, void* out, cudaEvent_t mid) {
+void launch_query(const Cache<T>& C, int G, dim3 grid, dim3 grid_z, cudaStream_t st, const void* q, void* out, cudaEvent_t mid, int advance = 1) {
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
         switch (G) {
             case 1: query_tau_kernel<D, 1><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                    query_z_kernel<D, 1><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
+                    query_z_kernel<D, 1><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x, advance); break;
             case 2: query_tau_kernel<D, 2><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                    query_z_kernel<D, 2><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
+                    query_z_kernel<D, 2><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x, advance); break;
             case 4: query_tau_kernel<D, 4><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                    query_z_kernel<D, 4><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
+                    query_z_kernel<D, 4><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x, advance); break;
             default: query_tau_kernel<D, 8><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                     query_z_kernel<D, 8><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x); break;
+                     query_z_kernel<D, 8><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x, advance); break;
         }
     } else {
         switch (G) {
-            case 1: query_kernel<T, D, 1><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
-            case 2: query_kernel<T, D, 2><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
-            case 4: query_kernel<T, D, 4><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
-            default: query_kernel<T, D, 8><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out); break;
+            case 1: query_kernel<T, D, 1><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out, advance); break;
+            case 2: query_kernel<T, D, 2><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out, advance); break;
+            case 4: query_kernel<T, D, 4><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out, advance); break;
+            default: query_kernel<T, D, 8><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out, advance); break;
         }
         if (mid) cudaEventRecord(mid, st);
     }
@@ -274,6 +277,19 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
     if (e) CUDA_TRY(cudaEventRecord(e[3], h->st));
     CUDA_TRY(cudaGetLastError());
     h->launches += std::is_same<T, __nv_bfloat16>::value ? 3 : 2;
+    return SUBGEN_OK;
+}
+
+// Read-only query with nq queries per head: the nq queries of the G heads of a KV head become G * nq columns.
+template <typename T, int D>
+int launch_query_only_td(subgen* h, const void* q, int nq, void* out) {
+    Cache<T> C = make_cache<T>(h);
+    C.H = h->d.H * nq;
+    C.G = h->d.G * nq;
+    const dim3 grid_t(h->d.sp_tau, h->d.U), grid_z(h->d.sp_z, h->d.U);
+    launch_query<T, D>(C, C.G, grid_t, grid_z, h->st, q, out, nullptr, 0);
+    CUDA_TRY(cudaGetLastError());
+    h->launches += std::is_same<T, __nv_bfloat16>::value ? 2 : 1;
     return SUBGEN_OK;
 }
 
@@ -539,6 +555,20 @@ int subgen_step(subgen_t* h, const void* q, const void* k, const void* v, void* 
     if (rc) return rc;
     for (int b = 0; b < h->d.B; ++b) h->n_host[b] += 1;
     return SUBGEN_OK;
+}
+
+int subgen_query(subgen_t* h, const void* q, int nq, void* out) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_query: handle is NULL");
+    if (!q || !out) return fail(SUBGEN_EINVAL, "subgen_query: q and out must not be NULL");
+    if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(SUBGEN_EINVAL, "subgen_query: pointers must be 16-byte aligned");
+    const int cols = h->d.G * nq;
+    if (nq < 1 || (nq & (nq - 1)) || cols > h->d.Gs)
+        return fail(SUBGEN_EINVAL, "subgen_query: nq must be a power of two with (H / Hkv) * nq <= %d (set nq_max at creation)", h->d.Gs);
+    for (int b = 0; b < h->d.B; ++b)
+        if (h->n_host[b] == 0) return fail(SUBGEN_ESTATE, "subgen_query: sequence %d has no tokens yet", b);
+    const bool f32 = h->cfg.dtype == SUBGEN_DTYPE_FP32;
+    if (h->d.D == 64) return f32 ? launch_query_only_td<float, 64>(h, q, nq, out) : launch_query_only_td<__nv_bfloat16, 64>(h, q, nq, out);
+    return f32 ? launch_query_only_td<float, 128>(h, q, nq, out) : launch_query_only_td<__nv_bfloat16, 128>(h, q, nq, out);
 }
 
 int subgen_step_host(subgen_t* h, const void* q, const void* k, const void* v, void* out) {

@@ -87,14 +87,15 @@ __global__ void __launch_bounds__(kInsertThreads) insert_kernel(Cache<T> C, cons
 // load. Blocks write (max, tau, z) partials; the block that finishes last merges them, divides,
 // writes out and advances the unit's token count.
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kQueryThreads) query_kernel(Cache<T> C, const T* __restrict__ q, T* __restrict__ out) {
+__global__ void __launch_bounds__(kQueryThreads) query_kernel(Cache<T> C, const T* __restrict__ q, T* __restrict__ out, int advance) {
     constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, RPW = 32 / LPR, STR = D + 2;
     __shared__ float sm[(kQueryThreads / 32) * G * STR];
     __shared__ int sm_last;
     const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5, lr = lane % LPR, sub = lane / LPR;
     const int b = u / C.Hkv, kvh = u % C.Hkv;
-    const int n = C.n_unit[u], w = C.w, t = C.t, s = C.s;
+    // advance = 1: the query of a stream step (its token is in the ring, not counted yet); 0: read-only query
+    const int n = C.n_unit[u] - (advance ? 0 : 1), w = C.w, t = C.t, s = C.s;
     const int wn = min(n + 1, w), m = C.m_unit[u];
     const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;
 
@@ -210,7 +211,7 @@ __global__ void __launch_bounds__(kQueryThreads) query_kernel(Cache<T> C, const 
     }
     final_merge<T, D, G>(part_u, splits, out + qrow0 * D, C.status[u] != 0);
     if (tid == 0) {
-        C.n_unit[u] = n + 1;
+        if (advance) C.n_unit[u] = n + 1;
         C.ticket2[u] = 0;
     }
 }

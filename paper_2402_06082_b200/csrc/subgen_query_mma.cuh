@@ -249,7 +249,7 @@ __global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfl
 // out = z / tau and advances the unit's token count.
 template <int D, int G>
 __global__ void __launch_bounds__(kQmThreads, 4) query_z_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ q,
-                                                                __nv_bfloat16* __restrict__ out, int splits_tau) {
+                                                                __nv_bfloat16* __restrict__ out, int splits_tau, int advance) {
     typedef __nv_bfloat16 T;
     constexpr int NC = D / 32, STR = D + 2, NW = kQmThreads / 32;
     __shared__ float sm[NW * G * STR];
@@ -257,7 +257,9 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_kernel(Cache<__nv_bfloa
     const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5, g = lane >> 2, tq = lane & 3;
     const int b = u / C.Hkv, kvh = u % C.Hkv;
-    const int n = C.n_unit[u], w = C.w, s = C.s;
+    // advance = 1: the query of a stream step, the step's token is in the ring but not counted yet;
+    // advance = 0: a read-only query of the state as it stands
+    const int n = C.n_unit[u] - (advance ? 0 : 1), w = C.w, s = C.s;
     const int wn = min(n + 1, w);
     const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;
 
@@ -361,7 +363,7 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_kernel(Cache<__nv_bfloa
     merge_partials<T, D, G>(part_u, splits, C.part_tau + (size_t)u * splits_tau * G * 2, splits_tau, out + qrow0 * D,
                             C.status[u] != 0, sred);
     if (tid == 0) {
-        C.n_unit[u] = n + 1;
+        if (advance) C.n_unit[u] = n + 1;
         C.ticket2[u] = 0;
         C.qnext[u] = 0;
         C.qnext2[u] = 0;
