@@ -179,7 +179,9 @@ typedef struct subgen_stats {
     uint64_t window_rows;        /* tokens currently in the windows */
     uint64_t tokens;             /* sum of n */
     uint64_t prefill_pairs;      /* (key, representative) pairs the chunked prefill has scored: 2*d flops each */
-    uint64_t insert_bytes;       /* bytes one step must read to place a key: the representatives */
+    uint64_t insert_bytes;       /* bytes one step must read to place a key: bf16, the first 32 coordinates of every
+                                  * representative and their norms (full rows follow only for those not ruled out
+                                  * by that lower bound); fp32, the representatives */
     uint64_t query_bytes;        /* bytes one step must read to answer the queries: cluster_bytes + value_bytes */
     uint64_t cluster_bytes;      /* cluster samples (t rows, or the representative alone while n_i = 1) and counts */
     uint64_t value_bytes;        /* M keys and values with their weights, window keys and values */

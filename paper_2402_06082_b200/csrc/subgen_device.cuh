@@ -28,6 +28,8 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1
     return c;
 }
 
+constexpr int kHeadDims = 32;   // coordinates of a representative kept in the packed head array
+
 template <typename T> struct Elem;
 template <> struct Elem<float> {
     static constexpr int EPL = 4;
@@ -86,6 +88,9 @@ template <typename T> struct Cache {
     T* X;            // [U, m_max, D]     representatives x_i
     T* S;            // [U, m_max, t, D]  cluster samples S_i (materialised once n_i >= 2)
     float* xn;       // [U, m_max]        ||x_i||^2 in fp32, used only to pre-filter distance candidates
+    T* Xh;           // [U, m_max, kHeadDims]  the first kHeadDims coordinates of x_i, packed: the step's insertion
+                     //                   reads these instead of the full rows to rule out far representatives
+    float* xhn;      // [U, m_max]        squared norm of that head in fp32
     int* cnt;        // [U, m_max]        n_i
     int* ctok;       // [U, m_max]        token index of x_i
     int* stok;       // [U, m_max, t]     token index in S_i(j)
@@ -235,11 +240,15 @@ __device__ void make_room(const Cache<T>& C, int u, int e, const uint4* krow, Be
             } else {
                 if (kept != i) {
                     if (tid < LPR) reinterpret_cast<uint4*>(Xu + (size_t)kept * D)[tid] = xrow[tid];
+                    if (tid < kHeadDims / EPL) reinterpret_cast<uint4*>(C.Xh + ((size_t)u * C.m_max + kept) * kHeadDims)[tid] = xrow[tid];
                     if (n_i >= 2)
                         for (int p = tid; p < t * LPR; p += nt)
                             reinterpret_cast<uint4*>(Su + (size_t)kept * t * D)[p] = reinterpret_cast<const uint4*>(Su + (size_t)i * t * D)[p];
                     for (int q = tid; q < t; q += nt) stoku[(size_t)kept * t + q] = stoku[(size_t)i * t + q];
-                    if (tid == 0) { cntu[kept] = n_i; ctoku[kept] = ctoku[i]; xnu[kept] = xnu[i]; }
+                    if (tid == 0) {
+                        cntu[kept] = n_i; ctoku[kept] = ctoku[i]; xnu[kept] = xnu[i];
+                        C.xhn[(size_t)u * C.m_max + kept] = C.xhn[(size_t)u * C.m_max + i];
+                    }
                 }
                 ++kept;
             }
@@ -274,28 +283,32 @@ __device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, c
     // W(v_e) and the input range check, by warp 0
     if (warp == 0) {
         unsigned long long acc = 0;
-        float kk = 0.f;
+        float kk = 0.f, kh = 0.f;
         bool bad = false;
         for (int p = lane; p < LPR; p += 32) {
             float vf[EPL], kf[EPL];
             Elem<T>::unpack(vrow[p], vf);
             Elem<T>::unpack(krow[p], kf);
+            float part = 0.f;
 #pragma unroll
             for (int j = 0; j < EPL; ++j) {
                 acc += fx_sq(vf[j]);
-                kk = fmaf(kf[j], kf[j], kk);
+                part = fmaf(kf[j], kf[j], part);
                 bad |= !(fabsf(vf[j]) <= kMaxAbsInput) || !(fabsf(kf[j]) <= kMaxAbsInput);
             }
+            kk += part;
+            if (p < kHeadDims / EPL) kh += part;
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
             acc += __shfl_xor_sync(0xffffffffu, acc, off);
             kk += __shfl_xor_sync(0xffffffffu, kk, off);
+            kh += __shfl_xor_sync(0xffffffffu, kh, off);
         }
         bad = __any_sync(0xffffffffu, bad);
         if (lane == 0) {
             sm_w[0] = acc;
-            sm_w[1] = (unsigned long long)__float_as_uint(kk);
+            sm_w[1] = (unsigned long long)__float_as_uint(kk) | ((unsigned long long)__float_as_uint(kh) << 32);
             if (bad) atomicOr(&C.status[u], 2);
         }
     }
@@ -335,11 +348,13 @@ __device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, c
     } else if (!full) {
         const int c = m;
         if (tid < LPR) reinterpret_cast<uint4*>(Xu + (size_t)c * D)[tid] = krow[tid];
+        if (tid < kHeadDims / EPL) reinterpret_cast<uint4*>(C.Xh + ((size_t)u * C.m_max + c) * kHeadDims)[tid] = krow[tid];
         for (int j = tid; j < t; j += nt) stoku[(size_t)c * t + j] = e;
         if (tid == 0) {
             cntu[c] = 1;
             C.ctok[(size_t)u * C.m_max + c] = e;
             C.xn[(size_t)u * C.m_max + c] = __uint_as_float((unsigned)sm_w[1]);
+            C.xhn[(size_t)u * C.m_max + c] = __uint_as_float((unsigned)(sm_w[1] >> 32));
         }
         m_new = m + 1;
     } else if (tid == 0) {

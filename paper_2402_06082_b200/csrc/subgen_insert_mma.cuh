@@ -1,16 +1,20 @@
-// Insert kernel for bf16 caches: the nearest-representative search with a tensor-core pre-filter.
+// Insert kernel for bf16 caches: the nearest-representative search with a tensor-core pre-filter over packed
+// heads of the representatives.
 //
-// Which cluster a key joins is decided by the exact fixed-point distance D2. Computing D2 for every
-// representative costs far more instructions per byte than HBM needs time to deliver the row, so the scan
-// first forms an approximate squared distance ||x||^2 + ||k||^2 - 2<x,k> with the inner products on the
-// tensor cores (m16n8k16, the key in column 0 of the B operand) and evaluates D2 exactly only for rows
-// whose approximation is within a proven guard band of delta^2:
-//     |approx - D2/2^32| < 2^-15 (||x||^2 + ||k||^2)      (fp32 accumulation of <= 128 exact products,
-//                                                           fp32 norms; see the design notes)
-//     flagged  <=>  approx <= delta^2 + 2^-13 (||x||^2 + ||k||^2)
-// Every row with D2 <= floor(delta^2 2^32) is flagged, so "no flagged row has D2 <= threshold" is
-// exactly the paper's "farther than delta from every representative" and the lexicographic minimum of
-// (D2, index) over the flagged rows is the argmin whenever the key joins.
+// Which cluster a key joins is decided by the exact fixed-point distance D2. D2 is a sum of non-negative terms,
+// so the distance over the first kHeadDims coordinates is a lower bound of it. The scan therefore reads only the
+// packed heads (kHeadDims coordinates per representative, a quarter of a d = 128 row) and their squared norms,
+// forms the approximate head distance ||xh||^2 + ||kh||^2 - 2<xh,kh> with the inner products on the tensor cores
+// (m16n8k16, the key's head in column 0 of the B operand) and evaluates D2 exactly, from the full row, only for
+// representatives whose head distance is within a proven guard band of the threshold:
+//     |approx - exact head distance| < 2^-15 (||xh||^2 + ||kh||^2)   (fp32 accumulation of <= 32 exact products,
+//                                                                     fp32 norms)
+//     flagged  <=>  approx <= delta^2 + 2^-13 (||xh||^2 + ||kh||^2)
+// Every row with D2 <= floor(delta^2 2^32) is flagged, so "no flagged row has D2 <= threshold" is exactly the
+// paper's "farther than delta from every representative" and the lexicographic minimum of (D2, index) over the
+// flagged rows is the argmin whenever the key joins. On keys that cluster, the flagged rows are the few
+// representatives near the key; on keys whose first coordinates carry no information every row is flagged and
+// the scan costs what a scan of the full rows costs.
 #pragma once
 #include "subgen_query_mma.cuh"
 
@@ -22,7 +26,7 @@ template <int D, bool BND>
 __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ k_new,
                                                                     const __nv_bfloat16* __restrict__ v_new) {
     typedef __nv_bfloat16 T;
-    constexpr int EPL = 8, LPR = D / EPL, NC = D / 32;
+    constexpr int EPL = 8, LPR = D / EPL;
     __shared__ uint4 krow[LPR], vrow[LPR];
     __shared__ Best smb[32];
     __shared__ unsigned long long sm_w[2];
@@ -47,20 +51,23 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
     __syncthreads();
     const int m = C.m_unit[u];
     const T* Xu = C.X + (size_t)u * C.m_max * D;
-    const float* xnu = C.xn + (size_t)u * C.m_max;
+    const T* Xhu = C.Xh + (size_t)u * C.m_max * kHeadDims;
+    const float* xhnu = C.xhn + (size_t)u * C.m_max;
 
-    // B operand (key in column 0) and ||k||^2
-    uint32_t kb[NC][4];
+    // B operand (head of the key in column 0) and the squared norm of that head. D2 is a sum of non-negative
+    // terms, so the distance over the first kHeadDims coordinates bounds it from below: a representative whose
+    // head distance is already beyond the threshold (plus the guard for the approximate arithmetic) cannot be
+    // joined, and only the others need their full row.
+    uint32_t kb[4];
     float kn = 0.f;
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
-        const uint4 r = krow[c * 4 + tq];
+    {
+        const uint4 r = krow[tq];
         float f[8];
         Elem<T>::unpack(r, f);
 #pragma unroll
         for (int j = 0; j < 8; ++j) kn = fmaf(f[j], f[j], kn);
-        kb[c][0] = g == 0 ? r.x : 0u; kb[c][1] = g == 0 ? r.y : 0u;
-        kb[c][2] = g == 0 ? r.z : 0u; kb[c][3] = g == 0 ? r.w : 0u;
+        kb[0] = g == 0 ? r.x : 0u; kb[1] = g == 0 ? r.y : 0u;
+        kb[2] = g == 0 ? r.z : 0u; kb[3] = g == 0 ? r.w : 0u;
     }
     kn += __shfl_xor_sync(0xffffffffu, kn, 1);
     kn += __shfl_xor_sync(0xffffffffu, kn, 2);
@@ -84,28 +91,34 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
         for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
         if (better(acc, row, b)) { b.d2 = acc; b.idx = row; }
     };
-    // approximate distances of one 16-row tile and the exact follow-up of its flagged rows
-    auto filter_tile = [&](int base, const uint4 (&ka)[NC], const uint4 (&kc)[NC], bool va, bool vb) {
-        const float xa = va ? xnu[base + g] : 0.f, xb = vb ? xnu[base + g + 8] : 0.f;
-        float sc[4] = {0.f, 0.f, 0.f, 0.f};
+    // kTiles tiles of 16 heads per warp and turn: all loads first, then the approximate head distances by MMA
+    // (lanes with tq == 0 hold <x, k> of rows g and g + 8) and the exact follow-up of the flagged rows
+    constexpr int kTiles = 4;
+    for (int base = c0 + warp * 16 * kTiles; base < c1; base += nw * 16 * kTiles) {
+        uint4 ka[kTiles], kc[kTiles];
+        float xa[kTiles], xb[kTiles];
 #pragma unroll
-        for (int c = 0; c < NC; ++c) {
-            mma_bf16_16816(sc, ka[c].x, kc[c].x, ka[c].y, kc[c].y, kb[c][0], kb[c][1]);
-            mma_bf16_16816(sc, ka[c].z, kc[c].z, ka[c].w, kc[c].w, kb[c][2], kb[c][3]);
+        for (int i = 0; i < kTiles; ++i) {
+            const int ra = base + i * 16 + g, rb = ra + 8;
+            const bool va = ra < c1, vb = rb < c1;
+            ka[i] = ldg16(Xhu + (size_t)(va ? ra : c1 - 1) * kHeadDims + tq * 8);
+            kc[i] = ldg16(Xhu + (size_t)(vb ? rb : c1 - 1) * kHeadDims + tq * 8);
+            xa[i] = va ? xhnu[ra] : 0.f;
+            xb[i] = vb ? xhnu[rb] : 0.f;
         }
-        // lanes with tq == 0 hold <x, k> of rows g (sc[0]) and g+8 (sc[2])
-        const float na = xa + kn, nb = xb + kn;
-        const bool fa = va && tq == 0 && (na - 2.f * sc[0]) <= d2f + 1.220703125e-4f * na;
-        const bool fb = vb && tq == 0 && (nb - 2.f * sc[2]) <= d2f + 1.220703125e-4f * nb;
-        unsigned ma = __ballot_sync(0xffffffffu, fa), mb = __ballot_sync(0xffffffffu, fb);
-        while (ma) { exact_row(base + ((__ffs(ma) - 1) >> 2)); ma &= ma - 1; }      // rare
-        while (mb) { exact_row(base + 8 + ((__ffs(mb) - 1) >> 2)); mb &= mb - 1; }
-    };
-    for (int base = c0 + warp * 16; base < c1; base += nw * 16) {
-        const bool va = base + g < c1, vb = base + g + 8 < c1;
-        uint4 ka[NC], kc[NC];
-        load_keys<D>(Xu + (size_t)(va ? base + g : c1 - 1) * D, Xu + (size_t)(vb ? base + g + 8 : c1 - 1) * D, tq, ka, kc);
-        filter_tile(base, ka, kc, va, vb);
+#pragma unroll
+        for (int i = 0; i < kTiles; ++i) {
+            const int ra = base + i * 16 + g, rb = ra + 8;
+            float sc[4] = {0.f, 0.f, 0.f, 0.f};
+            mma_bf16_16816(sc, ka[i].x, kc[i].x, ka[i].y, kc[i].y, kb[0], kb[1]);
+            mma_bf16_16816(sc, ka[i].z, kc[i].z, ka[i].w, kc[i].w, kb[2], kb[3]);
+            const float na = xa[i] + kn, nb = xb[i] + kn;
+            const bool fa = ra < c1 && tq == 0 && (na - 2.f * sc[0]) <= d2f + 1.220703125e-4f * na;
+            const bool fb = rb < c1 && tq == 0 && (nb - 2.f * sc[2]) <= d2f + 1.220703125e-4f * nb;
+            unsigned ma = __ballot_sync(0xffffffffu, fa), mb = __ballot_sync(0xffffffffu, fb);
+            while (ma) { exact_row(base + i * 16 + ((__ffs(ma) - 1) >> 2)); ma &= ma - 1; }
+            while (mb) { exact_row(base + i * 16 + 8 + ((__ffs(mb) - 1) >> 2)); mb &= mb - 1; }
+        }
     }
     b = block_best(b, smb);
     if (splits > 1) {

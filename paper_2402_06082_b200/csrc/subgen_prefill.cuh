@@ -452,6 +452,20 @@ __global__ void __launch_bounds__(kResolveThreads) prefill_resolve_kernel(Cache<
         const bool opened = is_open[j];
         if (opened) {
             if (lane < LPR) reinterpret_cast<uint4*>(Xu + (size_t)c * D)[lane] = src[lane];
+            {   // packed head of the representative and its squared norm
+                float hn = 0.f;
+                if (lane < kHeadDims / 8) {
+                    const uint4 r = src[lane];
+                    reinterpret_cast<uint4*>(C.Xh + ((size_t)u * C.m_max + c) * kHeadDims)[lane] = r;
+                    float f[8];
+                    Elem<T>::unpack(r, f);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) hn = fmaf(f[q], f[q], hn);
+                }
+                hn += __shfl_xor_sync(0xffffffffu, hn, 1);
+                hn += __shfl_xor_sync(0xffffffffu, hn, 2);
+                if (lane == 0) C.xhn[(size_t)u * C.m_max + c] = hn;
+            }
             if (!has_later[j])                                      // otherwise every slot gets its id from the key that wins it
                 for (int q = lane; q < t; q += 32) stoku[(size_t)c * t + q] = e;
             if (lane == 0) { C.ctok[(size_t)u * C.m_max + c] = e; C.xn[(size_t)u * C.m_max + c] = kn[j]; }

@@ -263,7 +263,7 @@ def test_cache_stats_and_profile():
     assert st["singleton_clusters"] == sum(int((o.counts == 1).sum()) for o in orcs.values())
     assert st["m_filled"] == sum(int((o.m_tok >= 0).sum()) for o in orcs.values())
     row = w.d * 2
-    assert st["insert_bytes"] == st["clusters"] * row
+    assert st["insert_bytes"] == st["clusters"] * (32 * 2 + 4)      # bf16: packed heads and their norms
     rows = st["singleton_clusters"] + (st["clusters"] - st["singleton_clusters"]) * w.t + 2 * st["m_filled"] + 2 * 64
     crow = st["singleton_clusters"] + (st["clusters"] - st["singleton_clusters"]) * w.t
     assert st["cluster_bytes"] == crow * row + st["clusters"] * 4
