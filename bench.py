@@ -356,7 +356,9 @@ def run_subgen(args, w):
     extra = {"prefill_ms": prefill_ms, "prefill_tokens_per_s": sum(lens) / (prefill_ms * 1e-3),
              "prefill_launches": prefill_launches,
              "prefill_phases_ms": {"values": pf_values_ms, "score": pf_score_ms, "resolve": pf_resolve_ms},
-             "prefill_score": tensor_roofline(pf_pairs, wr.d, pf_score_ms),
+             # the tcgen05 scoring kernel (d = 128, default) contracts the first 64 coordinates only
+             "prefill_score": tensor_roofline(pf_pairs, 64 if wr.d == 128 and os.environ.get("SUBGEN_PREFILL") is None else wr.d,
+                                              pf_score_ms),
              "cache": {k: stats1[k] for k in ("clusters", "singleton_clusters", "m_filled", "window_rows", "tokens")}}
     if args.multi_query > 1:
         # read-only multi-query calls against the final state: same cache bytes as a step's query, nq answers each

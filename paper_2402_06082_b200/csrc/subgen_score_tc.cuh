@@ -1,16 +1,19 @@
 // Prefill score kernel on the 5th-generation tensor cores (tcgen05), d = 128.
 //
 // One chunk of 128 keys (A, M = 128) against tiles of 128 representatives (B, N = 128): D[token][centre] =
-// <k, x> by tcgen05.mma.cta_group::1.kind::f16 (bf16 x bf16 -> fp32), K = 128 in eight K = 16 steps, the
-// accumulator in tensor memory (two buffers of 128 columns, so the MMAs of tile j+1 run while tile j is
-// read back). Operands sit in shared memory in the K-major 128-byte-swizzle layout the MMA descriptors
-// describe: 8-row groups of 128-byte rows (1024 bytes per group, 16-byte pieces XOR-ed with the row index
-// inside the group), one 16 KB block per 64-element half of d. The tiles are gathered with ordinary 16-byte
-// loads and stored straight into that layout (the rows of a unit are contiguous but the chunk may come from
-// the window ring, so no tensor map is involved), followed by a proxy fence before the MMA reads them.
+// <kh, xh> over the first 64 coordinates (the "head") by tcgen05.mma.cta_group::1.kind::f16 (bf16 x bf16 ->
+// fp32), K = 64 in four K = 16 steps, the accumulator in tensor memory (two buffers of 128 columns, so the MMAs
+// of tile j+1 run while tile j is read back). Operands sit in shared memory in the K-major 128-byte-swizzle
+// layout the MMA descriptors describe: 8-row groups of 128-byte rows (1024 bytes per group, 16-byte pieces
+// XOR-ed with the row index inside the group), one 16 KB block per 64-element half of d (the chunk keeps both
+// halves, for the exact distances; of the representatives only the head is staged). The tiles are gathered with
+// ordinary 16-byte loads and stored straight into that layout (the rows of a unit are contiguous but the chunk
+// may come from the window ring, so no tensor map is involved), followed by a proxy fence before the MMA reads
+// them.
 //
-// The MMA result is only a filter: a pair is flagged when <k,x> >= 1/2[(1-g)(||x||^2+||k||^2) - delta^2]
-// (the guard band of the insert kernel rearranged), and every flagged pair gets its exact fixed-point D2.
+// The MMA result is only a filter. D2 is a sum of non-negative terms, so the head distance bounds it from
+// below: a pair is flagged when <kh,xh> >= 1/2[(1-g)(||xh||^2+||kh||^2) - delta^2] (the guard band of the insert
+// kernel rearranged), and every flagged pair gets its exact fixed-point D2 over all coordinates.
 // Each thread owns one token row of the accumulator (tensor-memory lane = row) and scans its 128 columns.
 //
 // Waits: the only wait is on the mbarrier that the MMA commit arrives on; it is bounded, and when the bound is
@@ -22,13 +25,14 @@ namespace sgk {
 
 constexpr int kTcThreads = 128;
 constexpr int kTcTileN = 128;
+constexpr int kTcHeadPieces = 8;                 // 16-byte pieces of a row that make up the 64-coordinate head
 constexpr int kTcCand = 1024;                    // flagged pairs kept per tile before the exhaustive fallback
 constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((kTcTileN >> 3) << 17) | ((128u >> 4) << 24);
 constexpr unsigned kTcSpinLimit = 1u << 22;
 
 struct TcSmem {                                  // after a 1024-byte aligned base
     unsigned char A[2 * 128 * 128];              // chunk keys: [half of d][row][128 B swizzled]
-    unsigned char B[2][2 * kTcTileN * 128];      // two buffers of representatives, same layout
+    unsigned char B[2][kTcTileN * 128];          // two buffers of representative heads (64 coordinates), same layout
     float kn[kChunk];                            // 1/2 ((1-g) ||k||^2 - delta^2) per token
     float xa[2][kTcTileN];                       // 1/2 (1-g) ||x||^2 per representative of the tile (+inf: no row)
     unsigned long long wb_d2[4][kChunk];         // per warp: best exact (D2, index) per token
@@ -65,7 +69,6 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
         return;
     }
     const T* Xu = C.X + (size_t)u * C.m_max * D;
-    const float* xnu = C.xn + (size_t)u * C.m_max;
     const float d2f = (float)((double)C.delta2_fx * (1.0 / 4294967296.0));
     constexpr float kOneMinusG = 1.f - 1.220703125e-4f;
     const uint32_t sA = (uint32_t)__cvta_generic_to_shared(sm.A);
@@ -95,7 +98,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
     {
         const int j = tid;                                             // one token per thread
         float acc = 0.f;
-        for (int q = 0; q < LPR; ++q) {
+        for (int q = 0; q < kTcHeadPieces; ++q) {
             float f[8];
             Elem<T>::unpack(*reinterpret_cast<const uint4*>(sm.A + sw128_offset(j, q)), f);
 #pragma unroll
@@ -111,34 +114,42 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
     const int ntiles = (c1 - c0 + kTcTileN - 1) / kTcTileN;
 
     // representatives of tile j: global -> registers (tile_fetch), registers -> B[buf], xa[buf] (tile_store)
-    uint4 R[kTcTileN * LPR / kTcThreads];
-    float xr = INFINITY;
+    constexpr int kPer = kTcTileN * kTcHeadPieces / kTcThreads;      // pieces per thread and tile
+    uint4 R[kPer];
     auto tile_fetch = [&](int j) {
         const int row0 = c0 + j * kTcTileN;
 #pragma unroll
-        for (int i = 0; i < kTcTileN * LPR / kTcThreads; ++i) {
-            const int p = i * kTcThreads + tid, rr = p / LPR, q = p % LPR;
+        for (int i = 0; i < kPer; ++i) {
+            const int p = i * kTcThreads + tid, rr = p / kTcHeadPieces, q = p % kTcHeadPieces;
             R[i] = make_uint4(0, 0, 0, 0);
             if (row0 + rr < c1) R[i] = ldg16(Xu + (size_t)(row0 + rr) * D + q * 8);
         }
-        xr = row0 + tid < c1 ? 0.5f * kOneMinusG * xnu[row0 + tid] : INFINITY;
     };
-    auto tile_store = [&](int buf) {
+    auto tile_store = [&](int buf, int j) {
         unsigned char* dst = sm.B[buf];
+        const int row0 = c0 + j * kTcTileN;
 #pragma unroll
-        for (int i = 0; i < kTcTileN * LPR / kTcThreads; ++i) {
-            const int p = i * kTcThreads + tid;
-            *reinterpret_cast<uint4*>(dst + sw128_offset(p / LPR, p % LPR)) = R[i];
+        for (int i = 0; i < kPer; ++i) {
+            const int p = i * kTcThreads + tid, rr = p / kTcHeadPieces, q = p % kTcHeadPieces;
+            *reinterpret_cast<uint4*>(dst + sw128_offset(rr, q)) = R[i];
+            // squared norm of the head: the eight lanes that hold the row's pieces add up
+            float f[8], hn = 0.f;
+            Elem<T>::unpack(R[i], f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) hn = fmaf(f[e], f[e], hn);
+            hn += __shfl_xor_sync(0xffffffffu, hn, 1);
+            hn += __shfl_xor_sync(0xffffffffu, hn, 2);
+            hn += __shfl_xor_sync(0xffffffffu, hn, 4);
+            if (q == 0) sm.xa[buf][rr] = row0 + rr < c1 ? 0.5f * kOneMinusG * hn : INFINITY;
         }
-        sm.xa[buf][tid] = xr;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy stores -> visible to the MMA
     };
-    auto issue_mma = [&](int buf) {                                    // one thread: 8 MMAs of K = 16, then commit
+    auto issue_mma = [&](int buf) {                                    // one thread: 4 MMAs of K = 16, then commit
         const uint32_t sBb = buf ? sB1 : sB0;
         const uint32_t dcol = tmem + (uint32_t)(buf * kTcTileN);
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t off = (uint32_t)((ks >> 2) * (128 * 128) + (ks & 3) * 32);
+        for (int ks = 0; ks < 4; ++ks) {
+            const uint32_t off = (uint32_t)(ks * 32);
             const uint64_t da = umma_desc_sw128(sA + off), db = umma_desc_sw128(sBb + off);
             const uint32_t accum = ks ? 1u : 0u;
             asm volatile(
@@ -170,8 +181,8 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
     // Pipeline: the MMAs of tile j+1 run while tile j is read back, and the global loads of tile j+2 are in
     // flight (in registers) during both; they are stored once the MMAs of tile j have released their buffer.
     tile_fetch(0);
-    tile_store(0);
-    if (ntiles > 1) { tile_fetch(1); tile_store(1); }
+    tile_store(0, 0);
+    if (ntiles > 1) { tile_fetch(1); tile_store(1, 1); }
     __syncthreads();
     if (tid == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -239,7 +250,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
         __syncthreads();
         if (tid == 0) sm.ncand = 0;
         if (has2) {                                                       // buffer and accumulator `buf` are free now
-            tile_store(buf);
+            tile_store(buf, j + 2);
             __syncthreads();
             if (tid == 0) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
