@@ -326,7 +326,7 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         Lmax = hi - lo > Lmax ? hi - lo : Lmax;
     }
     const bool tc = D == 128 && !h->mma_score;           // tcgen05 scoring (d = 128), else warp-level MMAs
-    int slices = tc ? (148 * 2) / d.U : (148 * 4 + d.U - 1) / d.U;
+    int slices = tc ? (148 * 4) / d.U : (148 * 4 + d.U - 1) / d.U;
     slices = slices < 1 ? 1 : (slices > 32 ? 32 : slices);
     PrefillArgs a;
     a.K = (const T*)K; a.V = (const T*)V; a.n_uniform = n; a.cu = cu_dev; a.total = total; a.Lmax = Lmax; a.slices = slices;

@@ -2,11 +2,13 @@
 //
 // One chunk of 128 keys (A, M = 128) against tiles of 128 representatives (B, N = 128): D[token][centre] =
 // <kh, xh> over the first 64 coordinates (the "head") by tcgen05.mma.cta_group::1.kind::f16 (bf16 x bf16 ->
-// fp32), K = 64 in four K = 16 steps, the accumulator in tensor memory (two buffers of 128 columns, so the MMAs
-// of tile j+1 run while tile j is read back). Operands sit in shared memory in the K-major 128-byte-swizzle
+// fp32), K = 64 in four K = 16 steps, the accumulator in 128 columns of tensor memory. Four blocks share an SM
+// (54 KB of shared memory and a quarter of the tensor memory each), so one block's MMAs, read-back and exact
+// follow-up overlap the others'; within a block the MMAs of tile j+1 are issued as soon as tile j has been
+// read back and run during its exact follow-up. Operands sit in shared memory in the K-major 128-byte-swizzle
 // layout the MMA descriptors describe: 8-row groups of 128-byte rows (1024 bytes per group, 16-byte pieces
-// XOR-ed with the row index inside the group), one 16 KB block per 64-element half of d (the chunk keeps both
-// halves, for the exact distances; of the representatives only the head is staged). The tiles are gathered with
+// XOR-ed with the row index inside the group); only the heads are staged, the exact distances read full rows
+// from global memory. The tiles are gathered with
 // ordinary 16-byte loads and stored straight into that layout (the rows of a unit are contiguous but the chunk
 // may come from the window ring, so no tensor map is involved), followed by a proxy fence before the MMA reads
 // them.
@@ -26,32 +28,32 @@ namespace sgk {
 constexpr int kTcThreads = 128;
 constexpr int kTcTileN = 128;
 constexpr int kTcHeadPieces = 8;                 // 16-byte pieces of a row that make up the 64-coordinate head
-constexpr int kTcCand = 1024;                    // flagged pairs kept per tile before the exhaustive fallback
+constexpr int kTcCand = 512;                     // flagged pairs kept per tile before the exhaustive fallback
 constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((kTcTileN >> 3) << 17) | ((128u >> 4) << 24);
 constexpr unsigned kTcSpinLimit = 1u << 22;
 
 struct TcSmem {                                  // after a 1024-byte aligned base
-    unsigned char A[2 * 128 * 128];              // chunk keys: [half of d][row][128 B swizzled]
-    unsigned char B[2][kTcTileN * 128];          // two buffers of representative heads (64 coordinates), same layout
-    float kn[kChunk];                            // 1/2 ((1-g) ||k||^2 - delta^2) per token
-    float xa[2][kTcTileN];                       // 1/2 (1-g) ||x||^2 per representative of the tile (+inf: no row)
-    unsigned long long wb_d2[4][kChunk];         // per warp: best exact (D2, index) per token
-    int wb_idx[4][kChunk];
+    unsigned char A[128 * 128];                  // heads of the chunk keys: [row][128 B swizzled]
+    unsigned char B[2][kTcTileN * 128];          // two buffers of representative heads, same layout
+    float kn[kChunk];                            // 1/2 ((1-g) ||kh||^2 - delta^2) per token
+    float xa[2][kTcTileN];                       // 1/2 (1-g) ||xh||^2 per representative of the tile (+inf: no row)
+    unsigned long long wb_d2[kChunk];            // best exact (D2, index) per token; token j belongs to warp j % 4
+    int wb_idx[kChunk];
     unsigned cand[kTcCand];                      // token | row_in_tile << 8
-    unsigned long long mbar[2];
+    unsigned long long mbar;
     unsigned tmem_base, ncand, failed;
 };
 constexpr size_t kTcSmemBytes = sizeof(TcSmem) + 1024;
 
-__device__ __forceinline__ uint32_t sw128_offset(int row, int piece16) {      // piece16: 0..15 over the 256-byte row
-    return (uint32_t)((piece16 >> 3) * (128 * 128) + row * 128 + (((piece16 & 7) ^ (row & 7)) << 4));
+__device__ __forceinline__ uint32_t sw128_offset(int row, int piece16) {      // piece16: 0..7 over the 128-byte head
+    return (uint32_t)(row * 128 + (((piece16 & 7) ^ (row & 7)) << 4));
 }
 __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
     // start address >> 4 | LBO = 1 (16 B) << 16 | SBO = 1024 B >> 4 << 32 | version 1 << 46 | layout SWIZZLE_128B (2) << 61
     return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
 
-__global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<__nv_bfloat16> C, PrefillArgs a, int chunk) {
+__global__ void __launch_bounds__(kTcThreads, 4) prefill_score_tc_kernel(Cache<__nv_bfloat16> C, PrefillArgs a, int chunk) {
     typedef __nv_bfloat16 T;
     constexpr int D = 128, LPR = 16;
     extern __shared__ unsigned char dyn_raw[];
@@ -73,27 +75,26 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
     constexpr float kOneMinusG = 1.f - 1.220703125e-4f;
     const uint32_t sA = (uint32_t)__cvta_generic_to_shared(sm.A);
     const uint32_t sB0 = (uint32_t)__cvta_generic_to_shared(sm.B[0]), sB1 = (uint32_t)__cvta_generic_to_shared(sm.B[1]);
-    const uint32_t sBar0 = (uint32_t)__cvta_generic_to_shared(&sm.mbar[0]), sBar1 = (uint32_t)__cvta_generic_to_shared(&sm.mbar[1]);
+    const uint32_t sBar = (uint32_t)__cvta_generic_to_shared(&sm.mbar);
 
-    // ---- set-up: tensor memory (256 columns), barriers, the chunk ----
+    // ---- set-up: tensor memory (128 columns), the barrier, the chunk ----
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(&sm.tmem_base)), "r"(256u) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(&sm.tmem_base)), "r"(128u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sBar0) : "memory");
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sBar1) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sBar) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         sm.ncand = 0;
         sm.failed = 0;
     }
-    for (int p = tid; p < kChunk * LPR; p += kTcThreads) {            // chunk keys -> A (rows beyond cl are zero)
-        const int j = p / LPR, q = p % LPR;
+    for (int p = tid; p < kChunk * kTcHeadPieces; p += kTcThreads) {   // heads of the chunk keys -> A (rows beyond cl are zero)
+        const int j = p / kTcHeadPieces, q = p % kTcHeadPieces;
         uint4 v = make_uint4(0, 0, 0, 0);
         if (j < cl) v = reinterpret_cast<const uint4*>(key_row<D>(C, a, r, u, e0 + j))[q];
         *reinterpret_cast<uint4*>(sm.A + sw128_offset(j, q)) = v;
     }
-    for (int j = tid; j < 4 * kChunk; j += kTcThreads) { sm.wb_d2[j / kChunk][j % kChunk] = ~0ull; sm.wb_idx[j / kChunk][j % kChunk] = INT_MAX; }
+    for (int j = tid; j < kChunk; j += kTcThreads) { sm.wb_d2[j] = ~0ull; sm.wb_idx[j] = INT_MAX; }
     __syncthreads();
     {
         const int j = tid;                                             // one token per thread
@@ -106,6 +107,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
         }
         sm.kn[j] = 0.5f * (kOneMinusG * acc - d2f);
     }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the stores of A -> visible to the MMA
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -113,7 +115,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
     const float my_kn = sm.kn[tid];
     const int ntiles = (c1 - c0 + kTcTileN - 1) / kTcTileN;
 
-    // representatives of tile j: global -> registers (tile_fetch), registers -> B[buf], xa[buf] (tile_store)
+    // representative heads of tile j: global -> registers (tile_fetch), registers -> B[buf], xa[buf] (tile_store)
     constexpr int kPer = kTcTileN * kTcHeadPieces / kTcThreads;      // pieces per thread and tile
     uint4 R[kPer];
     auto tile_fetch = [&](int j) {
@@ -146,7 +148,6 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
     };
     auto issue_mma = [&](int buf) {                                    // one thread: 4 MMAs of K = 16, then commit
         const uint32_t sBb = buf ? sB1 : sB0;
-        const uint32_t dcol = tmem + (uint32_t)(buf * kTcTileN);
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks) {
             const uint32_t off = (uint32_t)(ks * 32);
@@ -155,17 +156,17 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
             asm volatile(
                 "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
-                ::"r"(dcol), "l"(da), "l"(db), "r"(kTcIdesc), "r"(accum), "r"(0u) : "memory");
+                ::"r"(tmem), "l"(da), "l"(db), "r"(kTcIdesc), "r"(accum), "r"(0u) : "memory");
         }
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(buf ? sBar1 : sBar0) : "memory");
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(sBar) : "memory");
     };
-    // exact D2 of (token tokj, representative row), by one warp; keeps the warp's best per token
+    // exact D2 of (token tokj, representative row), by one warp; only warp tokj % 4 ever handles token tokj
     auto exact_pair = [&](int tokj, int row) {
         unsigned long long acc = 0;
         if (lane < LPR) {
             float xf[8], kf[8];
             Elem<T>::unpack(*reinterpret_cast<const uint4*>(Xu + (size_t)row * D + lane * 8), xf);
-            Elem<T>::unpack(*reinterpret_cast<const uint4*>(sm.A + sw128_offset(tokj, lane)), kf);
+            Elem<T>::unpack(reinterpret_cast<const uint4*>(key_row<D>(C, a, r, u, e0 + tokj))[lane], kf);
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc += fx_sqdiff(xf[e], kf[e]);
         }
@@ -173,34 +174,32 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
         for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
         if (lane == 0) {
             Best cur;
-            cur.d2 = sm.wb_d2[warp][tokj]; cur.idx = sm.wb_idx[warp][tokj];
-            if (better(acc, row, cur)) { sm.wb_d2[warp][tokj] = acc; sm.wb_idx[warp][tokj] = row; }
+            cur.d2 = sm.wb_d2[tokj]; cur.idx = sm.wb_idx[tokj];
+            if (better(acc, row, cur)) { sm.wb_d2[tokj] = acc; sm.wb_idx[tokj] = row; }
         }
     };
 
-    // Pipeline: the MMAs of tile j+1 run while tile j is read back, and the global loads of tile j+2 are in
-    // flight (in registers) during both; they are stored once the MMAs of tile j have released their buffer.
+    // Pipeline: two tiles of heads are staged ahead in shared memory and a third is in flight in registers;
+    // the MMAs of tile j+1 are issued right after tile j has been read back from tensor memory.
     tile_fetch(0);
     tile_store(0, 0);
     if (ntiles > 1) { tile_fetch(1); tile_store(1, 1); }
+    if (ntiles > 2) tile_fetch(2);
     __syncthreads();
     if (tid == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         issue_mma(0);
-        if (ntiles > 1) issue_mma(1);
     }
     bool ok = true;
     for (int j = 0; j < ntiles; ++j) {
         const int buf = j & 1;
-        const bool has2 = j + 2 < ntiles;
-        if (has2) tile_fetch(j + 2);
         // wait for the MMAs of tile j (bounded)
         {
-            const uint32_t bar = buf ? sBar1 : sBar0, parity = (uint32_t)((j >> 1) & 1);
+            const uint32_t parity = (uint32_t)(j & 1);
             unsigned done = 0, spins = 0;
             while (!done && spins < kTcSpinLimit) {
                 asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
-                             : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+                             : "=r"(done) : "r"(sBar), "r"(parity) : "memory");
                 ++spins;
             }
             if (!done) sm.failed = 1;
@@ -208,12 +207,12 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
         __syncthreads();
         if (sm.failed) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        // epilogue: this thread's token row, 128 columns in four pieces of 32
+        // read-back: this thread's token row, 128 columns in four pieces of 32
         const float* xat = sm.xa[buf];
 #pragma unroll 1
         for (int cc = 0; cc < kTcTileN; cc += 32) {
             uint32_t v[32];
-            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * kTcTileN + cc);
+            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)cc;
             asm volatile(
                 "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
@@ -235,36 +234,36 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
-        // exact distances of the flagged pairs of this tile
+        // the accumulator is free: start tile j+1 (its heads were staged at least one barrier ago)
+        if (j + 1 < ntiles && tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            issue_mma(buf ^ 1);
+        }
+        // exact distances of the flagged pairs of this tile; warp w owns the tokens with index % 4 == w
         const unsigned nc = sm.ncand;
         const int row0 = c0 + j * kTcTileN;
         if (nc <= (unsigned)kTcCand) {
-            for (unsigned i = warp; i < nc; i += kTcThreads / 32) {
+            for (unsigned i = 0; i < nc; ++i) {
                 const unsigned cd = sm.cand[i];
-                exact_pair((int)(cd & 255u), row0 + (int)(cd >> 8));
+                if ((cd & 3u) == (unsigned)warp) exact_pair((int)(cd & 255u), row0 + (int)(cd >> 8));
             }
         } else {                                                          // too many to list: every pair of the tile
             const int nrow = min(kTcTileN, c1 - row0);
-            for (int i = warp; i < cl * nrow; i += kTcThreads / 32) exact_pair(i / nrow, row0 + i % nrow);
+            for (int tokj = warp; tokj < cl; tokj += kTcThreads / 32)
+                for (int rr = 0; rr < nrow; ++rr) exact_pair(tokj, row0 + rr);
         }
         __syncthreads();
         if (tid == 0) sm.ncand = 0;
-        if (has2) {                                                       // buffer and accumulator `buf` are free now
+        if (j + 2 < ntiles) {                                             // buffer `buf` is free since the MMAs of tile j ended
             tile_store(buf, j + 2);
-            __syncthreads();
-            if (tid == 0) {
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                issue_mma(buf);
-            }
+            if (j + 3 < ntiles) tile_fetch(j + 3);
         }
     }
     __syncthreads();
     if (ok) {
         for (int j = tid; j < kChunk; j += kTcThreads) {
             Best bb;
-            bb.d2 = sm.wb_d2[0][j]; bb.idx = sm.wb_idx[0][j]; bb.pad = 0;
-            for (int wv = 1; wv < 4; ++wv)
-                if (better(sm.wb_d2[wv][j], sm.wb_idx[wv][j], bb)) { bb.d2 = sm.wb_d2[wv][j]; bb.idx = sm.wb_idx[wv][j]; }
+            bb.d2 = sm.wb_d2[j]; bb.idx = sm.wb_idx[j]; bb.pad = 0;
             outp[j] = bb;
         }
     } else {
@@ -273,7 +272,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_score_tc_kernel(Cache<_
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(128u) : "memory");
 }
 
 }  // namespace sgk
