@@ -222,23 +222,39 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
     return C;
 }
 
+// Launch with the programmatic stream serialization attribute: the kernel may be scheduled while its predecessor
+// in the stream still runs and orders itself with pdl_wait(). SUBGEN_PDL=0 falls back to ordinary launches.
+template <typename... KArgs, typename... Args>
+void launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+    static const bool off = [] { const char* e = getenv("SUBGEN_PDL"); return e && e[0] == '0'; }();
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = off ? 0 : 1;
+    cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 // fp32 caches: CUDA-core dot products (full fp32 products). bf16 caches: tensor-core kernel.
 template <typename T, int D>
 void launch_query(const Cache<T>& C, int G, dim3 grid, dim3 grid_z, cudaStream_t st, const void* q, void* out, cudaEvent_t mid, int advance = 1) {
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
         switch (G) {
-            case 1: query_tau_kernel<D, 1><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
+            case 1: launch_pdl(query_tau_kernel<D, 1>, grid, dim3(kQmThreads), st, C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                    query_z_kernel<D, 1><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x, advance); break;
-            case 2: query_tau_kernel<D, 2><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
+                    launch_pdl(query_z_kernel<D, 1>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
+            case 2: launch_pdl(query_tau_kernel<D, 2>, grid, dim3(kQmThreads), st, C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                    query_z_kernel<D, 2><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x, advance); break;
-            case 4: query_tau_kernel<D, 4><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
+                    launch_pdl(query_z_kernel<D, 2>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
+            case 4: launch_pdl(query_tau_kernel<D, 4>, grid, dim3(kQmThreads), st, C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                    query_z_kernel<D, 4><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x, advance); break;
-            default: query_tau_kernel<D, 8><<<grid, kQmThreads, 0, st>>>(C, (const T*)q);
+                    launch_pdl(query_z_kernel<D, 4>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
+            default: launch_pdl(query_tau_kernel<D, 8>, grid, dim3(kQmThreads), st, C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                     query_z_kernel<D, 8><<<grid_z, kQmThreads, 0, st>>>(C, (const T*)q, (T*)out, (int)grid.x, advance); break;
+                     launch_pdl(query_z_kernel<D, 8>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
         }
     } else {
         switch (G) {
@@ -269,8 +285,8 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
         CUDA_TRY(cudaEventRecord(e[0], h->st));
     }
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
-        if (C.bounded) insert_mma_kernel<D, true><<<grid_i, kInsertMmaThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
-        else insert_mma_kernel<D, false><<<grid_i, kInsertMmaThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
+        if (C.bounded) launch_pdl(insert_mma_kernel<D, true>, grid_i, dim3(kInsertMmaThreads), h->st, C, (const T*)k, (const T*)v);
+        else launch_pdl(insert_mma_kernel<D, false>, grid_i, dim3(kInsertMmaThreads), h->st, C, (const T*)k, (const T*)v);
     } else {
         if (C.bounded) insert_kernel<T, D, true><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
         else insert_kernel<T, D, false><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);

@@ -28,6 +28,13 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1
     return c;
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start while
+// its predecessor in the stream is still running; pdl_wait() returns once that predecessor has completed and
+// its writes are visible (at once when the kernel was launched the ordinary way), pdl_trigger() lets the
+// successor start being scheduled. Everything a kernel reads that an earlier kernel wrote comes after pdl_wait().
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 constexpr int kHeadDims = 32;   // coordinates of a representative kept in the packed head array
 
 template <typename T> struct Elem;

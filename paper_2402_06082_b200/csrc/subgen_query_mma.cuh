@@ -157,16 +157,18 @@ __global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfl
     const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5, g = lane >> 2, tq = lane & 3;
     const int b = u / C.Hkv, kvh = u % C.Hkv;
-    const int t = C.t, m = C.m_unit[u];
     const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;
+    pdl_trigger();
 
-    uint32_t qb[NC][4];
+    uint32_t qb[NC][4];                   // the queries are an input of the call, not a predecessor's output
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
         uint4 r = make_uint4(0, 0, 0, 0);
         if (g < G) r = ldg16(q + (qrow0 + g) * D + c * 32 + tq * 8);
         qb[c][0] = r.x; qb[c][1] = r.y; qb[c][2] = r.z; qb[c][3] = r.w;
     }
+    pdl_wait();
+    const int t = C.t, m = C.m_unit[u];
     MmaState<16> S;                       // the accumulators stay untouched here and cost no registers
     S.m0 = S.m1 = -INFINITY;
     S.tau0 = S.tau1 = 0.f;
@@ -257,11 +259,8 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_kernel(Cache<__nv_bfloa
     const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5, g = lane >> 2, tq = lane & 3;
     const int b = u / C.Hkv, kvh = u % C.Hkv;
-    // advance = 1: the query of a stream step, the step's token is in the ring but not counted yet;
-    // advance = 0: a read-only query of the state as it stands
-    const int n = C.n_unit[u] - (advance ? 0 : 1), w = C.w, s = C.s;
-    const int wn = min(n + 1, w);
     const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;
+    pdl_trigger();
 
     uint32_t qb[NC][4];
 #pragma unroll
@@ -270,6 +269,11 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_kernel(Cache<__nv_bfloa
         if (g < G) r = ldg16(q + (qrow0 + g) * D + c * 32 + tq * 8);
         qb[c][0] = r.x; qb[c][1] = r.y; qb[c][2] = r.z; qb[c][3] = r.w;
     }
+    pdl_wait();
+    // advance = 1: the query of a stream step, the step's token is in the ring but not counted yet;
+    // advance = 0: a read-only query of the state as it stands
+    const int n = C.n_unit[u] - (advance ? 0 : 1), w = C.w, s = C.s;
+    const int wn = min(n + 1, w);
     MmaState<D> S;
     S.m0 = S.m1 = -INFINITY;
     S.tau0 = S.tau1 = 0.f;
