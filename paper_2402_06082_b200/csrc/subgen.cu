@@ -129,7 +129,7 @@ Layout make_layout(const Dims& d) {
     L.stage_out = take((size_t)d.B * d.H * row);
     L.cu = take(((size_t)d.B + 1) * sizeof(int));
     L.part1 = take(U * d.splits * sizeof(Best));
-    L.part2 = take(U * d.splits * d.Gs * (size_t)(d.D + 2) * sizeof(float));
+    L.part2 = take(U * (d.splits + 2) * d.Gs * (size_t)(d.D + 2) * sizeof(float));   // + 2: the evenly cut value scan
     L.part_tau = take(U * d.splits * d.Gs * 2 * sizeof(float));
     L.book_begin = off;
     L.cnt = take(U * d.m_max * sizeof(int));
@@ -240,21 +240,26 @@ void launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, 
 
 // fp32 caches: CUDA-core dot products (full fp32 products). bf16 caches: tensor-core kernel.
 template <typename T, int D>
-void launch_query(const Cache<T>& C, int G, dim3 grid, dim3 grid_z, cudaStream_t st, const void* q, void* out, cudaEvent_t mid, int advance = 1) {
+void launch_query(const Cache<T>& C, int G, dim3 grid, dim3 grid_z, cudaStream_t st, const void* q, void* out, cudaEvent_t mid, int advance = 1,
+                  int flat_ipu = 0, int flat_slots = 0) {
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
         switch (G) {
             case 1: launch_pdl(query_tau_kernel<D, 1>, grid, dim3(kQmThreads), st, C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                    launch_pdl(query_z_kernel<D, 1>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
+                    if (flat_ipu) launch_pdl(query_z_flat_kernel<D, 1>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance, flat_ipu, flat_slots);
+                    else launch_pdl(query_z_kernel<D, 1>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
             case 2: launch_pdl(query_tau_kernel<D, 2>, grid, dim3(kQmThreads), st, C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                    launch_pdl(query_z_kernel<D, 2>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
+                    if (flat_ipu) launch_pdl(query_z_flat_kernel<D, 2>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance, flat_ipu, flat_slots);
+                    else launch_pdl(query_z_kernel<D, 2>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
             case 4: launch_pdl(query_tau_kernel<D, 4>, grid, dim3(kQmThreads), st, C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                    launch_pdl(query_z_kernel<D, 4>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
+                    if (flat_ipu) launch_pdl(query_z_flat_kernel<D, 4>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance, flat_ipu, flat_slots);
+                    else launch_pdl(query_z_kernel<D, 4>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
             default: launch_pdl(query_tau_kernel<D, 8>, grid, dim3(kQmThreads), st, C, (const T*)q);
                     if (mid) cudaEventRecord(mid, st);
-                     launch_pdl(query_z_kernel<D, 8>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
+                     if (flat_ipu) launch_pdl(query_z_flat_kernel<D, 8>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance, flat_ipu, flat_slots);
+                    else launch_pdl(query_z_kernel<D, 8>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
         }
     } else {
         switch (G) {
@@ -265,6 +270,33 @@ void launch_query(const Cache<T>& C, int G, dim3 grid, dim3 grid_z, cudaStream_t
         }
         if (mid) cudaEventRecord(mid, st);
     }
+}
+
+// The value scan can be cut evenly over the grid when every unit has the same number of 16-row items, i.e. the same
+// window fill. That pays when the per-unit split needs more than one wave of blocks (many units: measured +2 % on
+// the step at 2048 units); with one wave or less the per-unit split with its work queue is faster (fewer units
+// per block, no second partial). Returns items per unit (0: use the per-unit split) and the grid size.
+// n_shift: 1 for a stream step (the step's token is already in the ring), 0 for a read-only query.
+int flat_value_scan(const subgen* h, int n_shift, int* grid) {
+    static const bool off = [] { const char* e = getenv("SUBGEN_FLAT"); return e && e[0] == '0'; }();
+    if (off || h->cfg.dtype != SUBGEN_DTYPE_BF16) return 0;
+    const Dims& d = h->d;
+    if ((long long)d.U * d.sp_z <= 148 * 4) return 0;
+    int wn0 = -1;
+    for (int b = 0; b < d.B; ++b) {
+        const long long n = (long long)h->n_host[b] + n_shift;
+        const int wn = n < d.w ? (int)n : d.w;
+        if (wn0 < 0) wn0 = wn;
+        else if (wn != wn0) return 0;
+    }
+    const int ipu = ((d.s + 15) >> 4) + ((wn0 + 15) >> 4);
+    const long long total = (long long)d.U * ipu;
+    const long long nb = total < 148 * 4 ? total : 148 * 4;
+    // a unit's partials must fit the room part2 has for it
+    const long long per_unit = (nb + d.U - 1) / d.U + 1;
+    if (per_unit > d.splits + 2) return 0;
+    *grid = (int)nb;
+    return ipu;
 }
 
 template <typename T, int D>
@@ -292,7 +324,9 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
         else insert_kernel<T, D, false><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
     }
     if (e) CUDA_TRY(cudaEventRecord(e[1], h->st));
-    launch_query<T, D>(C, h->d.G, grid_t, grid_z, h->st, q, out, e ? e[2] : nullptr);
+    int flat_grid = 0;
+    const int flat_ipu = flat_value_scan(h, 1, &flat_grid);
+    launch_query<T, D>(C, h->d.G, grid_t, flat_ipu ? dim3(flat_grid) : grid_z, h->st, q, out, e ? e[2] : nullptr, 1, flat_ipu, h->d.splits + 2);
     if (e) CUDA_TRY(cudaEventRecord(e[3], h->st));
     CUDA_TRY(cudaGetLastError());
     h->launches += std::is_same<T, __nv_bfloat16>::value ? 3 : 2;
@@ -306,7 +340,9 @@ int launch_query_only_td(subgen* h, const void* q, int nq, void* out) {
     C.H = h->d.H * nq;
     C.G = h->d.G * nq;
     const dim3 grid_t(h->d.sp_tau, h->d.U), grid_z(h->d.sp_z, h->d.U);
-    launch_query<T, D>(C, C.G, grid_t, grid_z, h->st, q, out, nullptr, 0);
+    int flat_grid = 0;
+    const int flat_ipu = flat_value_scan(h, 0, &flat_grid);
+    launch_query<T, D>(C, C.G, grid_t, flat_ipu ? dim3(flat_grid) : grid_z, h->st, q, out, nullptr, 0, flat_ipu, h->d.splits + 2);
     CUDA_TRY(cudaGetLastError());
     h->launches += std::is_same<T, __nv_bfloat16>::value ? 2 : 1;
     return SUBGEN_OK;

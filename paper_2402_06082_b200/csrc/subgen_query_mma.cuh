@@ -374,4 +374,137 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_kernel(Cache<__nv_bfloa
     }
 }
 
+// The same scan with the work cut evenly over the whole grid instead of per unit: all units have the same number
+// of 16-row items (ipu), block b takes the global items [b T / NB, (b+1) T / NB), T = U * ipu, which belong to one
+// unit or to a few consecutive ones. With NB equal to the number of resident blocks every block slot of the GPU
+// has the same share, whatever the ratio of slots to units. A unit's partials come from the blocks whose ranges
+// meet it; the block that delivers the last one merges. slots: partials a unit has room for in part2.
+template <int D, int G>
+__global__ void __launch_bounds__(kQmThreads, 4) query_z_flat_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ q,
+                                                                     __nv_bfloat16* __restrict__ out, int splits_tau, int advance,
+                                                                     int ipu, int slots) {
+    typedef __nv_bfloat16 T;
+    constexpr int NC = D / 32, STR = D + 2, NW = kQmThreads / 32;
+    __shared__ float sm[NW * G * STR];
+    __shared__ int sm_last;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, tq = lane & 3;
+    const long long NB = gridDim.x, Ttot = (long long)C.B * C.Hkv * ipu;
+    const long long i0 = (long long)blockIdx.x * Ttot / NB, i1 = ((long long)blockIdx.x + 1) * Ttot / NB;
+    pdl_trigger();
+    pdl_wait();
+    if (i0 >= i1) return;
+    const int w = C.w, s = C.s;
+    const int u_first = (int)(i0 / ipu), u_last = (int)((i1 - 1) / ipu);
+    for (int u = u_first; u <= u_last; ++u) {
+        const long long ulo = (long long)u * ipu;
+        const int lo = (int)(max(i0, ulo) - ulo), hi = (int)(min(i1, ulo + ipu) - ulo);
+        const int b = u / C.Hkv, kvh = u % C.Hkv;
+        const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;
+        uint32_t qb[NC][4];
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            uint4 r = make_uint4(0, 0, 0, 0);
+            if (g < G) r = ldg16(q + (qrow0 + g) * D + c * 32 + tq * 8);
+            qb[c][0] = r.x; qb[c][1] = r.y; qb[c][2] = r.z; qb[c][3] = r.w;
+        }
+        const int n = C.n_unit[u] - (advance ? 0 : 1);
+        const int wn = min(n + 1, w);
+        MmaState<D> S;
+        S.m0 = S.m1 = -INFINITY;
+        S.tau0 = S.tau1 = 0.f;
+#pragma unroll
+        for (int j = 0; j < D / 16; ++j) S.acc[j][0] = S.acc[j][1] = S.acc[j][2] = S.acc[j][3] = 0.f;
+        const T* Mku = C.Mk + (size_t)u * s * D;
+        const T* Mvu = C.Mv + (size_t)u * s * D;
+        const float* MiWu = C.MinvW + (size_t)u * s;
+        const T* Rk = C.ringK + (size_t)u * w * D;
+        const T* Rv = C.ringV + (size_t)u * w * D;
+        const float mu_over_s = (float)C.mu[u] / (float)s;
+        const int n_b = (s + 15) >> 4;
+        for (int item = lo + warp; item < hi; item += NW) {
+            // 16 value samples (weight mu/(s W), numerator only) or 16 window rows (weight 1, both sums)
+            const bool isM = item < n_b;
+            const int base = (isM ? item : item - n_b) * 16;
+            const int lim = isM ? s : wn;
+            const T* Kb = isM ? Mku : Rk;
+            const T* Vb = isM ? Mvu : Rv;
+            const int ia = min(base + g, lim - 1), ib = min(base + g + 8, lim - 1);
+            bool va = base + g < lim, vb = base + g + 8 < lim;
+            float wza = 1.f, wzb = 1.f;
+            if (isM) {
+                const float ia_w = MiWu[ia], ib_w = MiWu[ib];          // 1/W, 0 for a null slot
+                va = va && ia_w != 0.f;
+                vb = vb && ib_w != 0.f;
+                wza = va ? mu_over_s * ia_w : 0.f;
+                wzb = vb ? mu_over_s * ib_w : 0.f;
+            }
+            const T* pv[4];
+            pv[0] = Vb + (size_t)min(base + 2 * tq, lim - 1) * D;
+            pv[1] = Vb + (size_t)min(base + 2 * tq + 1, lim - 1) * D;
+            pv[2] = Vb + (size_t)min(base + 2 * tq + 8, lim - 1) * D;
+            pv[3] = Vb + (size_t)min(base + 2 * tq + 9, lim - 1) * D;
+            uint4 ka[NC], kb[NC], v[4][D / 64];
+            load_keys<D>(Kb + (size_t)ia * D, Kb + (size_t)ib * D, tq, ka, kb);      // keys and values in flight together
+            load_values<D>(pv, g, v);
+            float p[4];
+            tile_scores<D, D>(S, ka, kb, va, vb, qb, p);
+            if (!isM) {
+                S.tau0 += p[0] + p[2];
+                S.tau1 += p[1] + p[3];
+            }
+            const float pz[4] = {wza * p[0], wza * p[1], wzb * p[2], wzb * p[3]};
+            tile_values<D>(S, pz, v, g, tq);
+        }
+        // warp partial -> shared [warp][G][D+2]
+#pragma unroll
+        for (int off = 4; off < 32; off <<= 1) {
+            S.tau0 += __shfl_xor_sync(0xffffffffu, S.tau0, off);
+            S.tau1 += __shfl_xor_sync(0xffffffffu, S.tau1, off);
+        }
+        {
+            const int h0 = 2 * tq, h1 = 2 * tq + 1;
+            float* w0 = sm + ((size_t)warp * G + (h0 < G ? h0 : 0)) * STR;
+            float* w1 = sm + ((size_t)warp * G + (h1 < G ? h1 : 0)) * STR;
+            if (g == 0) {
+                if (h0 < G) { w0[0] = S.m0; w0[1] = S.tau0; }
+                if (h1 < G) { w1[0] = S.m1; w1[1] = S.tau1; }
+            }
+#pragma unroll
+            for (int j = 0; j < D / 16; ++j) {
+                const int col = (j >> 2) * 64 + g * 8 + 2 * (j & 3);
+                if (h0 < G) { w0[2 + col] = S.acc[j][0]; w0[2 + col + 1] = S.acc[j][2]; }
+                if (h1 < G) { w1[2 + col] = S.acc[j][1]; w1[2 + col + 1] = S.acc[j][3]; }
+            }
+        }
+        // which blocks meet this unit: the largest b with b T / NB <= x is ((x + 1) NB - 1) / T
+        const int b_first = (int)(((ulo + 1) * NB - 1) / Ttot), b_last = (int)(((ulo + ipu) * NB - 1) / Ttot);
+        const int np = b_last - b_first + 1;
+        float* part_u = C.part2 + (size_t)u * slots * G * STR;
+        block_combine<D, G>(sm, part_u + (size_t)((int)blockIdx.x - b_first) * G * STR);
+        __threadfence();
+        __syncthreads();
+        bool last = true;
+        if (np > 1) {
+            if (tid == 0) {
+                __threadfence();
+                sm_last = (atomicAdd(&C.ticket2[u], 1u) == (unsigned)np - 1u);
+            }
+            __syncthreads();
+            last = sm_last != 0;
+            if (last) __threadfence();
+        }
+        if (last) {
+            __shared__ float sred[16];
+            merge_partials<T, D, G>(part_u, np, C.part_tau + (size_t)u * splits_tau * G * 2, splits_tau, out + qrow0 * D,
+                                    C.status[u] != 0, sred);
+            if (tid == 0) {
+                if (advance) C.n_unit[u] = n + 1;
+                C.ticket2[u] = 0;
+                C.qnext[u] = 0;
+            }
+        }
+        __syncthreads();            // sm and sm_last are reused by the next unit
+    }
+}
+
 }  // namespace sgk
