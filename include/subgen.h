@@ -135,8 +135,9 @@ int subgen_step(subgen_t* h, const void* q, const void* k, const void* v, void* 
  * power of two, (H / Hkv) * nq <= 8 and nq <= the nq_max given at creation. Every sequence must hold a token. */
 int subgen_query(subgen_t* h, const void* q, int nq, void* out);
 
-/* subgen_step with HOST buffers: copies q, k, v to the device, runs the step, copies out back and
- * waits for it. Pinned host memory makes the copies asynchronous to the host until the final wait. */
+/* subgen_step with HOST buffers, returning when out is filled. With page-locked (pinned, mapped) buffers the
+ * step's kernels read q, k, v and write out across the bus themselves: no staging copies, one wait. With pageable
+ * buffers q, k, v are copied to the device first and out is copied back. */
 int subgen_step_host(subgen_t* h, const void* q, const void* k, const void* v, void* out);
 
 /* Waits for the stream, returns the OR of all units' status bits (>= 0) or a negative error. */

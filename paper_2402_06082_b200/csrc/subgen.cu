@@ -626,11 +626,31 @@ int subgen_query(subgen_t* h, const void* q, int nq, void* out) {
     return f32 ? launch_query_only_td<float, 128>(h, q, nq, out) : launch_query_only_td<__nv_bfloat16, 128>(h, q, nq, out);
 }
 
+// Device-side alias of a page-locked, mapped host buffer (what cudaHostAlloc / cudaHostRegister hand out under unified
+// addressing); false for pageable memory.
+static bool pinned_alias(const void* host, void** dev) {
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, host) != cudaSuccess) { cudaGetLastError(); return false; }
+    if (a.type != cudaMemoryTypeHost || !a.devicePointer) return false;
+    *dev = a.devicePointer;
+    return true;
+}
+
 int subgen_step_host(subgen_t* h, const void* q, const void* k, const void* v, void* out) {
     if (!h) return fail(SUBGEN_EINVAL, "subgen_step_host: handle is NULL");
     if (!q || !k || !v || !out) return fail(SUBGEN_EINVAL, "subgen_step_host: q, k, v, out must not be NULL");
     const size_t row = (size_t)h->d.D * h->d.E;
     const size_t qb = (size_t)h->d.B * h->d.H * row, kb = (size_t)h->d.U * row;
+    void *dq, *dk, *dv, *dout;
+    if (pinned_alias(q, &dq) && pinned_alias(k, &dk) && pinned_alias(v, &dv) && pinned_alias(out, &dout) &&
+        !(((uintptr_t)dq | (uintptr_t)dk | (uintptr_t)dv | (uintptr_t)dout) & 15)) {
+        // pinned buffers: the step's kernels read the inputs and write the result across the bus themselves
+        // (each input row is read by the few blocks of its unit, the result is written once)
+        int rc = subgen_step(h, dq, dk, dv, dout);
+        if (rc) return rc;
+        CUDA_TRY(cudaStreamSynchronize(h->st));
+        return SUBGEN_OK;
+    }
     char* w = h->ws;
     CUDA_TRY(cudaMemcpyAsync(w + h->L.stage_q, q, qb, cudaMemcpyHostToDevice, h->st));
     CUDA_TRY(cudaMemcpyAsync(w + h->L.stage_k, k, kb, cudaMemcpyHostToDevice, h->st));
