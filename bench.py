@@ -266,20 +266,29 @@ def run_subgen(args, w):
     torch.cuda.synchronize()
     warm.close()
     del warm, wk
-    sg.profile_enable(True)
+    def run_prefill(handle):
+        if varlen:
+            handle.prefill_varlen(Kp, Vp, np.concatenate([[0], np.cumsum(lens)]).astype(np.int64))
+        else:
+            handle.prefill(Kp, Vp)
+
+    # phases: the same prefill on a handle of its own with CUDA events between the kernels (they keep a kernel from
+    # starting while its predecessor drains, so the timed prefill below runs without them)
+    prof = binding.SubGen(wr.B, wr.H, wr.d, wr.delta, wr.t, wr.s, wr.window, wr.philox_seed, Hkv=wr.Hkv, dtype=dt,
+                          m_max=wr.m_max, splits=args.splits, bounded=args.bounded)
+    prof.profile_enable(True)
+    run_prefill(prof)
+    torch.cuda.synchronize()
+    pf_values_ms, pf_score_ms, pf_resolve_ms = prof.profile_prefill_read()
+    prof.close()
+    del prof
     l0 = sg.launch_count
     e0.record()
-    if varlen:
-        cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
-        sg.prefill_varlen(Kp, Vp, cu)
-    else:
-        sg.prefill(Kp, Vp)
+    run_prefill(sg)
     e1.record()
     torch.cuda.synchronize()
     prefill_ms = e0.elapsed_time(e1)
     prefill_launches = sg.launch_count - l0
-    pf_values_ms, pf_score_ms, pf_resolve_ms = sg.profile_prefill_read()
-    sg.profile_enable(False)
     pf_pairs = sg.cache_stats()["prefill_pairs"]
     st = sg.status()
     if st:

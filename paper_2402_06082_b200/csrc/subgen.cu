@@ -225,17 +225,21 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
 // Launch with the programmatic stream serialization attribute: the kernel may be scheduled while its predecessor
 // in the stream still runs and orders itself with pdl_wait(). SUBGEN_PDL=0 falls back to ordinary launches.
 template <typename... KArgs, typename... Args>
-void launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+void launch_pdl_smem(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
     static const bool off = [] { const char* e = getenv("SUBGEN_PDL"); return e && e[0] == '0'; }();
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = off ? 0 : 1;
     cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+template <typename... KArgs, typename... Args>
+void launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+    launch_pdl_smem(kern, grid, block, 0, st, args...);
 }
 
 // fp32 caches: CUDA-core dot products (full fp32 products). bf16 caches: tensor-core kernel.
@@ -436,10 +440,11 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
             configured = true;
         }
         for (int c = 0; c < nchunks; ++c) {
-            if (tc) prefill_score_tc_kernel<<<dim3(slices, d.U), kTcThreads, kTcSmemBytes, h->st>>>(C, a, c);
+            // both kernels stage their chunk keys before they wait for their predecessor in the stream
+            if (tc) launch_pdl_smem(prefill_score_tc_kernel, dim3(slices, d.U), dim3(kTcThreads), kTcSmemBytes, h->st, C, a, c);
             else prefill_score_kernel<D><<<dim3(slices, d.U), kScoreThreads, 0, h->st>>>(C, a, c);
             if (int rc = mark()) return rc;
-            prefill_resolve_kernel<D><<<d.U, kResolveThreads, 0, h->st>>>(C, a, c);
+            launch_pdl(prefill_resolve_kernel<D>, dim3(d.U), dim3(kResolveThreads), h->st, C, a, c);
             if (int rc = mark()) return rc;
         }
         launches += 2 * nchunks;

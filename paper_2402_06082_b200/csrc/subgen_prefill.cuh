@@ -333,17 +333,34 @@ __global__ void __launch_bounds__(kResolveThreads) prefill_resolve_kernel(Cache<
     const Range r = unit_range(C, a, u);
     const int e0 = r.ins_lo + chunk * kChunk, cl = min(kChunk, r.ins_hi - e0);
     if (cl <= 0) return;
-    const int m_old = C.m_unit[u], t = C.t;
+    const int t = C.t;
     const unsigned long long thr = C.delta2_fx;
     T* Xu = C.X + (size_t)u * C.m_max * D;
     T* Su = C.S + (size_t)u * C.m_max * t * D;
     int* cntu = C.cnt + (size_t)u * C.m_max;
     int* stoku = C.stok + (size_t)u * C.m_max * t;
 
+    // the chunk's keys and their norms depend on no earlier kernel of this call ...
     for (int p = tid; p < cl * LPR; p += kResolveThreads) {
         const int j = p / LPR, part = p % LPR;
         reinterpret_cast<uint4*>(keys + (size_t)j * D)[part] = reinterpret_cast<const uint4*>(key_row<D>(C, a, r, u, e0 + j))[part];
     }
+    __syncthreads();
+    for (int j = tid; j < cl; j += kResolveThreads) {                // ||k||^2 of a key that may become a representative
+        float acc = 0.f;
+        for (int p = 0; p < LPR; ++p) {
+            float f[8];
+            Elem<T>::unpack(reinterpret_cast<const uint4*>(keys + (size_t)j * D)[p], f);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc = fmaf(f[q], f[q], acc);
+        }
+        kn[j] = acc;
+    }
+    // ... the score kernel's results and the state the previous chunk left do: wait for them, then let the next
+    // kernel in the stream start staging its keys
+    pdl_wait();
+    pdl_trigger();
+    const int m_old = C.m_unit[u];
     for (int j = tid; j < cl; j += kResolveThreads) {
         Best bb; bb.d2 = ~0ull; bb.idx = INT_MAX; bb.pad = 0;
         if (m_old > 0)
@@ -357,16 +374,6 @@ __global__ void __launch_bounds__(kResolveThreads) prefill_resolve_kernel(Cache<
     }
     if (tid == 0) { sm_opened = 0; sm_full = 0; }
     __syncthreads();
-    for (int j = tid; j < cl; j += kResolveThreads) {                // ||k||^2 of a key that may become a representative
-        float acc = 0.f;
-        for (int p = 0; p < LPR; ++p) {
-            float f[8];
-            Elem<T>::unpack(reinterpret_cast<const uint4*>(keys + (size_t)j * D)[p], f);
-#pragma unroll
-            for (int q = 0; q < 8; ++q) acc = fmaf(f[q], f[q], acc);
-        }
-        kn[j] = acc;
-    }
 
     // Openings in stream order. Key j opens a representative iff its nearest representative so far (old ones
     // from the score kernel, new ones from this loop) is farther than delta.

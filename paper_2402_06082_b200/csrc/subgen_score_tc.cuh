@@ -62,14 +62,6 @@ __global__ void __launch_bounds__(kTcThreads, 4) prefill_score_tc_kernel(Cache<_
     const Range r = unit_range(C, a, u);
     const int e0 = r.ins_lo + chunk * kChunk, cl = min(kChunk, r.ins_hi - e0);
     if (cl <= 0) return;
-    const int m = C.m_unit[u];
-    Best* outp = a.pbest + ((size_t)u * slices + blockIdx.x) * kChunk;
-    const int per = (((m + slices - 1) / slices) + kTcTileN - 1) / kTcTileN * kTcTileN;
-    const int c0 = blockIdx.x * per, c1 = min(m, c0 + per);
-    if (c0 >= c1) {
-        for (int j = tid; j < kChunk; j += kTcThreads) { Best bb; bb.d2 = ~0ull; bb.idx = INT_MAX; bb.pad = 0; outp[j] = bb; }
-        return;
-    }
     const T* Xu = C.X + (size_t)u * C.m_max * D;
     const float d2f = (float)((double)C.delta2_fx * (1.0 / 4294967296.0));
     constexpr float kOneMinusG = 1.f - 1.220703125e-4f;
@@ -113,7 +105,15 @@ __global__ void __launch_bounds__(kTcThreads, 4) prefill_score_tc_kernel(Cache<_
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = sm.tmem_base;
     const float my_kn = sm.kn[tid];
-    const int ntiles = (c1 - c0 + kTcTileN - 1) / kTcTileN;
+    // Everything above touches only the chunk's keys. The representatives and their count come from the resolve
+    // kernel of the previous chunk, which may still be running: wait for it here, then let the next kernel in.
+    pdl_wait();
+    pdl_trigger();
+    const int m = C.m_unit[u];
+    Best* outp = a.pbest + ((size_t)u * slices + blockIdx.x) * kChunk;
+    const int per = (((m + slices - 1) / slices) + kTcTileN - 1) / kTcTileN * kTcTileN;
+    const int c0 = blockIdx.x * per, c1 = min(m, c0 + per);
+    const int ntiles = c0 < c1 ? (c1 - c0 + kTcTileN - 1) / kTcTileN : 0;      // 0: this slice holds no representative
 
     // representative heads of tile j: global -> registers (tile_fetch), registers -> B[buf], xa[buf] (tile_store)
     constexpr int kPer = kTcTileN * kTcHeadPieces / kTcThreads;      // pieces per thread and tile
@@ -181,12 +181,11 @@ __global__ void __launch_bounds__(kTcThreads, 4) prefill_score_tc_kernel(Cache<_
 
     // Pipeline: two tiles of heads are staged ahead in shared memory and a third is in flight in registers;
     // the MMAs of tile j+1 are issued right after tile j has been read back from tensor memory.
-    tile_fetch(0);
-    tile_store(0, 0);
+    if (ntiles > 0) { tile_fetch(0); tile_store(0, 0); }
     if (ntiles > 1) { tile_fetch(1); tile_store(1, 1); }
     if (ntiles > 2) tile_fetch(2);
     __syncthreads();
-    if (tid == 0) {
+    if (ntiles > 0 && tid == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         issue_mma(0);
     }
