@@ -184,8 +184,11 @@ typedef struct subgen_stats {
                                   * representative and their norms (full rows follow only for those not ruled out
                                   * by that lower bound); fp32, the representatives */
     uint64_t query_bytes;        /* bytes one step must read to answer the queries: cluster_bytes + value_bytes */
-    uint64_t cluster_bytes;      /* cluster samples (t rows, or the representative alone while n_i = 1) and counts */
+    uint64_t cluster_bytes;      /* cluster samples (bf16: each distinct sampled row once, as the t reservoirs of a
+                                  * cluster often hold the same token more than once; fp32: t rows; the
+                                  * representative alone while n_i = 1) with counts and slot aliases */
     uint64_t value_bytes;        /* M keys and values with their weights, window keys and values */
+    uint64_t distinct_sample_rows; /* over clusters with n_i > 1: slots that are the first to hold their token */
 } subgen_stats;
 
 /* Synchronous. Sums over all units, from the current state. */

@@ -46,7 +46,8 @@ class StateView(C.Structure):
 
 class Stats(C.Structure):
     _fields_ = [(k, C.c_uint64) for k in ("units", "clusters", "singleton_clusters", "m_filled", "window_rows",
-                                           "tokens", "prefill_pairs", "insert_bytes", "query_bytes", "cluster_bytes", "value_bytes")]
+                                           "tokens", "prefill_pairs", "insert_bytes", "query_bytes", "cluster_bytes", "value_bytes",
+                                           "distinct_sample_rows")]
 
 
 _lib = None

@@ -47,7 +47,7 @@ size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
     size_t X, S, xn, cnt, ctok, stok, Mk, Mv, MW, Mtok, ringK, ringV;
     size_t n_unit, m_unit, mu, status, last_cid, last_open, last_d2, part1, part2, ticket1, ticket2, qnext, qnext2, part_tau, MinvW, pairs;
-    size_t thr2, level, Xh, xhn;
+    size_t thr2, level, Xh, xhn, alias, ndist;
     size_t stage_q, stage_k, stage_v, stage_out, cu, stats;
     size_t book_begin, book_end;   // bookkeeping region cleared at creation
     size_t total;
@@ -135,6 +135,8 @@ Layout make_layout(const Dims& d) {
     L.cnt = take(U * d.m_max * sizeof(int));
     L.xn = take(U * d.m_max * sizeof(float));
     L.xhn = take(U * d.m_max * sizeof(float));
+    L.alias = take(U * d.m_max * (size_t)d.t + 16 * 64);   // + one item's worth: the cluster scan loads 16 rows at a time
+    L.ndist = take(U * d.m_max + 16);
     L.n_unit = take(U * sizeof(int));
     L.m_unit = take(U * sizeof(int));
     L.mu = take(U * sizeof(uint64_t));
@@ -203,7 +205,7 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
     C.delta2_fx = (unsigned long long)floor((double)h->cfg.delta * (double)h->cfg.delta * 4294967296.0);
     C.key0 = (uint32_t)h->cfg.seed; C.key1 = (uint32_t)(h->cfg.seed >> 32);
     C.X = (T*)(w + L.X); C.S = (T*)(w + L.S); C.xn = (float*)(w + L.xn);
-    C.Xh = (T*)(w + L.Xh); C.xhn = (float*)(w + L.xhn);
+    C.Xh = (T*)(w + L.Xh); C.xhn = (float*)(w + L.xhn); C.alias = (unsigned char*)(w + L.alias); C.ndist = (unsigned char*)(w + L.ndist);
     C.cnt = (int*)(w + L.cnt); C.ctok = (int*)(w + L.ctok); C.stok = (int*)(w + L.stok);
     C.Mk = (T*)(w + L.Mk); C.Mv = (T*)(w + L.Mv);
     C.MW = (unsigned long long*)(w + L.MW); C.Mtok = (int*)(w + L.Mtok);
@@ -453,6 +455,7 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
     for (int b = 0; b < d.B; ++b) longest = add[b] > longest ? add[b] : longest;
     int fx = (int)(((size_t)(longest < d.w ? longest : d.w) * (D / 8) + 255) / 256);
     fx = fx < 1 ? 1 : (fx > 16 ? 16 : fx);
+    if (Lmax > 0) { prefill_alias_kernel<<<dim3(8, d.U), 256, 0, h->st>>>(C); launches += 1; }
     prefill_finish_kernel<D><<<dim3(fx, d.U), 256, 0, h->st>>>(C, a);
     prefill_commit_kernel<<<(d.U + 255) / 256, 256, 0, h->st>>>(C, a, d.U);
     launches += 2;
@@ -749,7 +752,12 @@ int subgen_cache_stats(subgen_t* h, subgen_stats* out) {
     // bf16: packed heads and their norms (full rows only for the few representatives the heads do not rule out);
     // fp32: the exact scan reads the full rows
     out->insert_bytes = h->cfg.dtype == SUBGEN_DTYPE_BF16 ? r[0] * ((uint64_t)kHeadDims * h->d.E + 4) : r[0] * row;
-    out->cluster_bytes = (r[1] + (r[0] - r[1]) * (uint64_t)h->d.t) * row + r[0] * 4;
+    // bf16: the cluster scan fetches every distinct sampled row once (slots that repeat a token are read from their
+    // first copy) plus counts and alias rows; fp32: all t rows of every cluster with more than one member
+    out->distinct_sample_rows = r[6];
+    out->cluster_bytes = h->cfg.dtype == SUBGEN_DTYPE_BF16
+                             ? (r[1] + r[6]) * row + r[0] * (4 + (uint64_t)h->d.t)
+                             : (r[1] + (r[0] - r[1]) * (uint64_t)h->d.t) * row + r[0] * 4;
     out->value_bytes = (2 * r[2] + 2 * r[3]) * row + (uint64_t)h->d.U * h->d.s * 4;
     out->query_bytes = out->cluster_bytes + out->value_bytes;
     return SUBGEN_OK;
@@ -833,7 +841,7 @@ std::vector<CkptArray> ckpt_arrays(const subgen* h, int m_rows) {
     const size_t row = (size_t)d.D * d.E, mm = (size_t)d.m_max, mr = (size_t)m_rows, s = (size_t)d.s, w = (size_t)d.w, t = (size_t)d.t;
     return {
         {L.X, mm * row, mr * row}, {L.S, mm * t * row, mr * t * row}, {L.xn, mm * 4, mr * 4}, {L.cnt, mm * 4, mr * 4},
-        {L.Xh, mm * kHeadDims * d.E, mr * kHeadDims * d.E}, {L.xhn, mm * 4, mr * 4},
+        {L.Xh, mm * kHeadDims * d.E, mr * kHeadDims * d.E}, {L.xhn, mm * 4, mr * 4}, {L.alias, mm * t, mr * t}, {L.ndist, mm, mr},
         {L.ctok, mm * 4, mr * 4}, {L.stok, mm * t * 4, mr * t * 4},
         {L.Mk, s * row, s * row}, {L.Mv, s * row, s * row}, {L.MW, s * 8, s * 8}, {L.Mtok, s * 4, s * 4}, {L.MinvW, s * 4, s * 4},
         {L.ringK, w * row, w * row}, {L.ringV, w * row, w * row},

@@ -101,6 +101,12 @@ template <typename T> struct Cache {
     int* cnt;        // [U, m_max]        n_i
     int* ctok;       // [U, m_max]        token index of x_i
     int* stok;       // [U, m_max, t]     token index in S_i(j)
+    unsigned char* alias;   // [U, m_max, t]  the cluster's distinct sampled tokens. The t reservoirs sample with
+                     //                   replacement, so slots often repeat a token; entry k < ndist[c] names the
+                     //                   first slot holding the k-th distinct token and how many slots hold it:
+                     //                   slot | (copies - 1) << 4 for t <= 16, else the slot itself (no merging).
+                     //                   The query reads each distinct row once, weighted by its copies.
+    unsigned char* ndist;   // [U, m_max]     number of valid entries in the alias row (clusters with n_i > 1)
     T* Mk;           // [U, s, D]
     T* Mv;           // [U, s, D]
     unsigned long long* MW;    // [U, s]  W of the sampled token, 0 = null
@@ -185,6 +191,33 @@ __device__ __forceinline__ Best block_best(Best b, Best* sm) {
     return r;
 }
 
+// The distinct tokens among t slot tokens st[0..t), in slot order, in the encoding of Cache::alias. One thread.
+__device__ __forceinline__ int distinct_slots(const int* st, int t, unsigned char* al) {
+    if (t > 16) {
+        for (int j = 0; j < t; ++j) al[j] = (unsigned char)j;
+        return t;
+    }
+    int k = 0;
+    for (int j = 0; j < t; ++j) {
+        const int tok = st[j];
+        int hit = -1;
+        for (int i = 0; i < k; ++i) if (st[al[i] & 15] == tok) hit = i;
+        if (hit >= 0) al[hit] = (unsigned char)(al[hit] + 16);
+        else al[k++] = (unsigned char)j;
+    }
+    return k;
+}
+
+// Rebuild the alias row of cluster c of unit u from its slot tokens. Called by a whole block after the writes to
+// stok are visible (a __syncthreads() since them).
+template <typename T>
+__device__ __forceinline__ void rebuild_alias(const Cache<T>& C, int u, int c) {
+    if (threadIdx.x == 0) {
+        const size_t cc = (size_t)u * C.m_max + c;
+        C.ndist[cc] = (unsigned char)distinct_slots(C.stok + cc * C.t, C.t, C.alias + cc * C.t);
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Bounded-m variant: token e has no representative within the threshold and all m_max clusters are in use.
 // The paper fixes no rule for this; the one taken here follows the doubling idea of the incremental clustering
@@ -244,6 +277,7 @@ __device__ void make_room(const Cache<T>& C, int u, int e, const uint4* krow, Be
                 }
                 __syncthreads();                   // n_j was read by everyone before it changes
                 if (tid == 0) cntu[j] = (int)n_new;
+                rebuild_alias(C, u, j);
             } else {
                 if (kept != i) {
                     if (tid < LPR) reinterpret_cast<uint4*>(Xu + (size_t)kept * D)[tid] = xrow[tid];
@@ -251,7 +285,11 @@ __device__ void make_room(const Cache<T>& C, int u, int e, const uint4* krow, Be
                     if (n_i >= 2)
                         for (int p = tid; p < t * LPR; p += nt)
                             reinterpret_cast<uint4*>(Su + (size_t)kept * t * D)[p] = reinterpret_cast<const uint4*>(Su + (size_t)i * t * D)[p];
-                    for (int q = tid; q < t; q += nt) stoku[(size_t)kept * t + q] = stoku[(size_t)i * t + q];
+                    for (int q = tid; q < t; q += nt) {
+                        stoku[(size_t)kept * t + q] = stoku[(size_t)i * t + q];
+                        C.alias[((size_t)u * C.m_max + kept) * t + q] = C.alias[((size_t)u * C.m_max + i) * t + q];
+                    }
+                    if (tid == 0) C.ndist[(size_t)u * C.m_max + kept] = C.ndist[(size_t)u * C.m_max + i];
                     if (tid == 0) {
                         cntu[kept] = n_i; ctoku[kept] = ctoku[i]; xnu[kept] = xnu[i];
                         C.xhn[(size_t)u * C.m_max + kept] = C.xhn[(size_t)u * C.m_max + i];
@@ -352,6 +390,7 @@ __device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, c
         }
         __syncthreads();            // n_old was read by everyone before it changes
         if (tid == 0) cntu[c] = (int)n_new;
+        rebuild_alias(C, u, c);
     } else if (!full) {
         const int c = m;
         if (tid < LPR) reinterpret_cast<uint4*>(Xu + (size_t)c * D)[tid] = krow[tid];

@@ -267,15 +267,21 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_seq_kernel(Cache<T> C
 }
 
 // ---------------------------------------------------------------------------------------------
-// Sums for subgen_cache_stats: out[0..5] = clusters, singleton clusters, filled M slots, window rows,
-// tokens, 0.
+// Sums for subgen_cache_stats: out[0..6] = clusters, singleton clusters, filled M slots, window rows,
+// tokens, pairs scored by the prefill, distinct sample rows of the clusters with more than one member.
 template <typename T>
 __global__ void stats_kernel(Cache<T> C, int U, unsigned long long* out) {
     const int u = blockIdx.x;
     if (u >= U) return;
     const int m = C.m_unit[u], n = C.n_unit[u];
     unsigned long long single = 0, filled = 0;
-    for (int c = threadIdx.x; c < m; c += blockDim.x) single += C.cnt[(size_t)u * C.m_max + c] == 1;
+    unsigned long long distinct = 0;
+    for (int c = threadIdx.x; c < m; c += blockDim.x) {
+        const bool one = C.cnt[(size_t)u * C.m_max + c] == 1;
+        single += one;
+        if (!one) distinct += C.ndist[(size_t)u * C.m_max + c];
+    }
+    atomicAdd(&out[6], distinct);
     for (int i = threadIdx.x; i < C.s; i += blockDim.x) filled += C.MW[(size_t)u * C.s + i] != 0ull;
     atomicAdd(&out[1], single);
     atomicAdd(&out[2], filled);

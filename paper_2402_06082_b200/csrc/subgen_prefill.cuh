@@ -534,6 +534,15 @@ __global__ void prefill_finish_kernel(Cache<__nv_bfloat16> C, PrefillArgs a) {
 }
 
 // Last kernel of a prefill call: counters (after every block of every other kernel has read them).
+// Alias rows of every cluster (see Cache::alias) from the slot tokens the chunks left. grid (blocks, U).
+__global__ void prefill_alias_kernel(Cache<__nv_bfloat16> C) {
+    const int u = blockIdx.y, m = C.m_unit[u], t = C.t;
+    for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < m; c += gridDim.x * blockDim.x) {
+        const size_t cc = (size_t)u * C.m_max + c;
+        C.ndist[cc] = (unsigned char)distinct_slots(C.stok + cc * t, t, C.alias + cc * t);
+    }
+}
+
 __global__ void prefill_commit_kernel(Cache<__nv_bfloat16> C, PrefillArgs a, int U) {
     const int u = blockIdx.x * blockDim.x + threadIdx.x;
     if (u >= U) return;

@@ -142,6 +142,8 @@ __device__ __forceinline__ void tile_values(MmaState<D>& S, const float (&pz)[4]
     }
 }
 
+constexpr int kTauRows = 256 + 16;   // rows of one pass of the cluster scan: at most 256 sample rows and 16 singletons
+
 // floor(r / t) for small r by one multiply-high (t = 1 handled by the caller's magic = 0)
 __device__ __forceinline__ int div_small(int r, unsigned magic) { return magic ? (int)__umulhi((unsigned)r, magic) : r; }
 
@@ -153,7 +155,9 @@ __global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfl
     typedef __nv_bfloat16 T;
     constexpr int NC = D / 32, NW = kQmThreads / 32;
     __shared__ float sm[NW][G][2];
-    __shared__ int lst[NW][16], wcn[NW][16];
+    __shared__ unsigned als[NW][16 * 64 / 4];          // alias rows of the item's 16 clusters, t <= 64 bytes each
+    __shared__ int rix[NW][kTauRows];                  // row list of a pass: sample row index, or representative | 2^31
+    __shared__ float rwt[NW][kTauRows];
     const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5, g = lane >> 2, tq = lane & 3;
     const int b = u / C.Hkv, kvh = u % C.Hkv;
@@ -177,50 +181,76 @@ __global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfl
     const T* Xu = C.X + (size_t)u * C.m_max * D;
     const T* Su = C.S + (size_t)u * C.m_max * t * D;
     const int* cntu = C.cnt + (size_t)u * C.m_max;
+    const unsigned char* ndu = C.ndist + (size_t)u * C.m_max;
+    const unsigned* aliasu = reinterpret_cast<const unsigned*>(C.alias + (size_t)u * C.m_max * t);
     const float inv_t = 1.f / (float)t;
-    const unsigned magic = t > 1 ? (unsigned)(4294967296ull / (unsigned)t) + 1u : 0u;
     const int total = (m + 15) >> 4;
+    const int gsz = t <= 16 ? 16 : 256 / t;          // clusters whose rows fit one list of kTauRows entries (t <= 64)
     int item = 0;
     if (lane == 0) item = (int)atomicAdd(&C.qnext[u], 1u);
     item = __shfl_sync(0xffffffffu, item, 0);
     while (item < total) {
         int next = 0;
         if (lane == 0) next = (int)atomicAdd(&C.qnext[u], 1u);     // asked for early, needed late
-        // 16 clusters -> one list of rows: first the t samples of every cluster with n' > 1, then the
-        // representatives of the singletons
+        // 16 clusters -> one list of rows: first the distinct samples of every cluster with n' > 1, each weighted
+        // n'/t times the number of slots that hold it, then the representatives of the singletons
         const int c = item * 16 + lane;
         const int cn = (lane < 16 && c < m) ? cntu[c] : 0;
-        const unsigned ms = __ballot_sync(0xffffffffu, cn == 1), mm = __ballot_sync(0xffffffffu, cn > 1);
-        const unsigned lt = (1u << lane) - 1u;
-        const int nm = __popc(mm), ns = __popc(ms);
-        __syncwarp();
-        if (cn > 1) { const int r = __popc(mm & lt); lst[warp][r] = c; wcn[warp][r] = cn; }
-        if (cn == 1) lst[warp][nm + __popc(ms & lt)] = c;
-        __syncwarp();
-        const int rows_m = nm * t, rows = rows_m + ns;
-        // row r of the list -> pointer, weight, validity
-        auto resolve = [&](int r, const T*& ptr, float& wgt) -> bool {
-            ptr = Xu;
-            wgt = 1.f;
-            if (r < rows_m) {
-                const int ci = div_small(r, magic);
-                ptr = Su + ((size_t)lst[warp][ci] * t + (r - ci * t)) * D;
-                wgt = (float)wcn[warp][ci] * inv_t;
-            } else if (r < rows) {
-                ptr = Xu + (size_t)lst[warp][nm + r - rows_m] * D;
+        const int nd = (lane < 16 && c < m) ? (int)ndu[c] : 0;
+        // the 16 alias rows are contiguous (16 t bytes, 4-byte aligned; the array is padded by one item)
+        for (int i = lane; i < 4 * t; i += 32) als[warp][i] = aliasu[(size_t)item * 4 * t + i];
+        for (int p0 = 0; p0 < 16; p0 += gsz) {
+            const bool act = lane >= p0 && lane < p0 + gsz;
+            const int ndl = (act && cn > 1) ? nd : 0;
+            int incl = ndl;
+#pragma unroll
+            for (int off = 1; off < 16; off <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += v;
             }
-            return r < rows;
-        };
-        for (int r0 = 0; r0 < rows; r0 += 16) {
-            const T *pa, *pb;
-            float wa, wb;
-            const bool va = resolve(r0 + g, pa, wa), vb = resolve(r0 + g + 8, pb, wb);
-            uint4 ka[NC], kb[NC];
-            load_keys<D>(pa, pb, tq, ka, kb);
-            float p[4];
-            tile_scores<D, 16>(S, ka, kb, va, vb, qb, p);
-            S.tau0 += wa * p[0] + wb * p[2];
-            S.tau1 += wa * p[1] + wb * p[3];
+            const int rows_m = __shfl_sync(0xffffffffu, incl, 15);
+            const unsigned ms = __ballot_sync(0xffffffffu, act && cn == 1);
+            const int rows = rows_m + __popc(ms);
+            __syncwarp();
+            if (ndl) {
+                const unsigned char* al = reinterpret_cast<const unsigned char*>(als[warp]) + lane * t;
+                const float wc = (float)cn * inv_t;
+                for (int k = 0; k < ndl; ++k) {
+                    const int e = al[k];
+                    const int slot = t <= 16 ? (e & 15) : e, copies = t <= 16 ? (e >> 4) + 1 : 1;
+                    rix[warp][incl - ndl + k] = c * t + slot;
+                    rwt[warp][incl - ndl + k] = wc * (float)copies;
+                }
+            }
+            if (act && cn == 1) {
+                const int r = rows_m + __popc(ms & ((1u << lane) - 1u));
+                rix[warp][r] = c | (int)0x80000000;
+                rwt[warp][r] = 1.f;
+            }
+            __syncwarp();
+            // row r of the list -> pointer, weight, validity
+            auto resolve = [&](int r, const T*& ptr, float& wgt) -> bool {
+                ptr = Xu;
+                wgt = 1.f;
+                if (r < rows) {
+                    const int ix = rix[warp][r];
+                    ptr = ix < 0 ? Xu + (size_t)(ix & 0x7fffffff) * D : Su + (size_t)ix * D;
+                    wgt = rwt[warp][r];
+                }
+                return r < rows;
+            };
+            for (int r0 = 0; r0 < rows; r0 += 16) {
+                const T *pa, *pb;
+                float wa, wb;
+                const bool va = resolve(r0 + g, pa, wa), vb = resolve(r0 + g + 8, pb, wb);
+                uint4 ka[NC], kb[NC];
+                load_keys<D>(pa, pb, tq, ka, kb);
+                float p[4];
+                tile_scores<D, 16>(S, ka, kb, va, vb, qb, p);
+                S.tau0 += wa * p[0] + wb * p[2];
+                S.tau1 += wa * p[1] + wb * p[3];
+            }
+            __syncwarp();
         }
         item = __shfl_sync(0xffffffffu, next, 0);
     }

@@ -72,6 +72,9 @@ def test_budgeted_stream_matches_oracle(dtype, d, G, m_max):
     steps(n0 + n1 + n2, n)
     assert sg.status() == 0
     assert min(lv0) >= 1                                           # the budget was hit during the prompt already
+    if dtype == "bf16":                                            # the slot aliases survived the merges and moves
+        want = sum(len(set(r.tolist())) for o in orcs.values() for r in o.slot_tok[o.counts > 1])
+        assert sg.cache_stats()["distinct_sample_rows"] == want
     for (b, h), o in orcs.items():
         assert o.m <= m_max
         st = _same(sg, o, b, h, "end, unit %s" % ((b, h),))

@@ -60,6 +60,8 @@ def test_resume_continues_the_stream(dtype, d):
                 want = o.query(Qn[bb, h * G + g, i])
                 assert hp.rel_err(ob[bb, h * G + g], want) <= hp.TOL[w.torch_dtype]
                 assert hp.rel_err(oa[bb, h * G + g], want) <= hp.TOL[w.torch_dtype]
+    want = sum(len(set(r.tolist())) for o in orcs.values() for r in o.slot_tok[o.counts > 1])
+    assert a.cache_stats()["distinct_sample_rows"] == b.cache_stats()["distinct_sample_rows"] == want
     for (bb, h), o in orcs.items():
         sa, sb = a.export_state(bb, h), b.export_state(bb, h)
         hp.assert_state_equal(sb, o, "resumed handle, unit %s" % ((bb, h),))

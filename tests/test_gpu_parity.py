@@ -267,10 +267,12 @@ def test_cache_stats_and_profile():
     assert st["m_filled"] == sum(int((o.m_tok >= 0).sum()) for o in orcs.values())
     row = w.d * 2
     assert st["insert_bytes"] == st["clusters"] * (32 * 2 + 4)      # bf16: packed heads and their norms
-    rows = st["singleton_clusters"] + (st["clusters"] - st["singleton_clusters"]) * w.t + 2 * st["m_filled"] + 2 * 64
-    crow = st["singleton_clusters"] + (st["clusters"] - st["singleton_clusters"]) * w.t
-    assert st["cluster_bytes"] == crow * row + st["clusters"] * 4
-    assert st["value_bytes"] == (rows - crow) * row + 2 * w.s * 4
+    distinct = sum(len(set(r.tolist())) for o in orcs.values() for r in o.slot_tok[o.counts > 1])
+    assert st["distinct_sample_rows"] == distinct
+    assert distinct < (st["clusters"] - st["singleton_clusters"]) * w.t          # reservoirs do repeat tokens
+    crow = st["singleton_clusters"] + distinct
+    assert st["cluster_bytes"] == crow * row + st["clusters"] * (4 + w.t)
+    assert st["value_bytes"] == (2 * st["m_filled"] + 2 * 64) * row + 2 * w.s * 4
     assert st["query_bytes"] == st["cluster_bytes"] + st["value_bytes"]
     sg.profile_enable(True)
     K, V, Q = synth.batch_stream(w, 3, "cuda")
