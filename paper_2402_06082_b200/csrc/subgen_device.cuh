@@ -209,13 +209,29 @@ __device__ __forceinline__ int distinct_slots(const int* st, int t, unsigned cha
 }
 
 // Rebuild the alias row of cluster c of unit u from its slot tokens. Called by a whole block after the writes to
-// stok are visible (a __syncthreads() since them).
+// stok are visible (a __syncthreads() since them); the first warp does the work, one slot per lane.
 template <typename T>
 __device__ __forceinline__ void rebuild_alias(const Cache<T>& C, int u, int c) {
-    if (threadIdx.x == 0) {
-        const size_t cc = (size_t)u * C.m_max + c;
-        C.ndist[cc] = (unsigned char)distinct_slots(C.stok + cc * C.t, C.t, C.alias + cc * C.t);
+    if (threadIdx.x >= 32) return;
+    const int lane = threadIdx.x, t = C.t;
+    const size_t cc = (size_t)u * C.m_max + c;
+    const int* st = C.stok + cc * t;
+    unsigned char* al = C.alias + cc * t;
+    if (t > 16) {                                   // no merging: every slot stands for itself
+        for (int j = lane; j < t; j += 32) al[j] = (unsigned char)j;
+        if (lane == 0) C.ndist[cc] = (unsigned char)t;
+        return;
     }
+    const int tok = lane < t ? st[lane] : -2 - lane;          // lanes beyond t hold tokens nobody shares
+    bool first = lane < t;
+    int copies = 0;
+    for (int i = 0; i < t; ++i) {
+        const int other = __shfl_sync(0xffffffffu, tok, i);
+        if (other == tok) { copies += 1; if (i < lane) first = false; }
+    }
+    const unsigned firsts = __ballot_sync(0xffffffffu, first);
+    if (first) al[__popc(firsts & ((1u << lane) - 1u))] = (unsigned char)(lane | ((copies - 1) << 4));
+    if (lane == 0) C.ndist[cc] = (unsigned char)__popc(firsts);
 }
 
 // ---------------------------------------------------------------------------------------------
