@@ -182,7 +182,8 @@ __global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfl
     const T* Su = C.S + (size_t)u * C.m_max * t * D;
     const int* cntu = C.cnt + (size_t)u * C.m_max;
     const unsigned char* ndu = C.ndist + (size_t)u * C.m_max;
-    const unsigned* aliasu = reinterpret_cast<const unsigned*>(C.alias + (size_t)u * C.m_max * t);
+    const unsigned char* alias_bytes = C.alias + (size_t)u * C.m_max * t;
+    const unsigned* alias_words = (reinterpret_cast<uintptr_t>(alias_bytes) & 3) ? nullptr : reinterpret_cast<const unsigned*>(alias_bytes);
     const float inv_t = 1.f / (float)t;
     const int total = (m + 15) >> 4;
     const int gsz = t <= 16 ? 16 : 256 / t;          // clusters whose rows fit one list of kTauRows entries (t <= 64)
@@ -197,8 +198,14 @@ __global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfl
         const int c = item * 16 + lane;
         const int cn = (lane < 16 && c < m) ? cntu[c] : 0;
         const int nd = (lane < 16 && c < m) ? (int)ndu[c] : 0;
-        // the 16 alias rows are contiguous (16 t bytes, 4-byte aligned; the array is padded by one item)
-        for (int i = lane; i < 4 * t; i += 32) als[warp][i] = aliasu[(size_t)item * 4 * t + i];
+        // the 16 alias rows are contiguous (16 t bytes; the array is padded by one item): word loads when the
+        // unit's rows start on a 4-byte boundary (m_max t a multiple of 4, or unit 0), else byte by byte
+        if (alias_words) {
+            for (int i = lane; i < 4 * t; i += 32) als[warp][i] = alias_words[(size_t)item * 4 * t + i];
+        } else {
+            unsigned char* dst = reinterpret_cast<unsigned char*>(als[warp]);
+            for (int i = lane; i < 16 * t; i += 32) dst[i] = alias_bytes[(size_t)item * 16 * t + i];
+        }
         for (int p0 = 0; p0 < 16; p0 += gsz) {
             const bool act = lane >= p0 && lane < p0 + gsz;
             const int ndl = (act && cn > 1) ? nd : 0;

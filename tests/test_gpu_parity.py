@@ -423,3 +423,29 @@ def test_benchmark_workload_full_size_sampled_units():
     for bh in sample:
         hp.assert_state_equal(sg.export_state(*bh), orcs[bh], "full-size steps unit %s" % (bh,))
     assert sg.status() == 0
+
+
+@pytest.mark.parametrize("t,m_max,bounded", [(3, 512, False), (3, 6, True), (17, 512, False), (33, 7, True), (64, 512, False), (1, 512, False)])
+def test_odd_sample_counts_and_unaligned_units(t, m_max, bounded):
+    """t that is not a multiple of 4 (the per-unit alias rows then start at odd byte offsets) and t > 16 (alias
+    lists keep every slot; the cluster scan goes through its rows in several passes)."""
+    from paper_2402_06082_b200.binding import SubGen
+    from oracle import subgen_oracle as orc
+    w = synth.CFG3.scaled(B=1, H=5, Hkv=5, d=128, n_prompt=150, ncomp=10, s=7, window=1, m_max=m_max, t=t, delta=0.5)
+    n0, nd = 150, 9
+    K, V, Q = synth.batch_stream(w, n0 + nd, "cuda")
+    sg = SubGen(1, 5, 128, w.delta, t, w.s, w.window, w.philox_seed, Hkv=5, dtype=torch.bfloat16, m_max=m_max, bounded=bounded)
+    orcs = {h: orc.OracleUnit(128, w.delta, t, w.s, w.window, seed=w.philox_seed, unit_id=h, m_max=m_max, bounded=bounded) for h in range(5)}
+    sg.prefill(K[:, :, :n0].contiguous(), V[:, :, :n0].contiguous())
+    for h, o in orcs.items():
+        o.push_many(f32(K[0, h, :n0]), f32(V[0, h, :n0]))
+    for i in range(n0, n0 + nd):
+        out = f32(sg.step(Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous()))
+        for h, o in orcs.items():
+            o.push(f32(K[0, h, i]), f32(V[0, h, i]))
+            assert hp.rel_err(out[0, h], o.query(f32(Q[0, h, i]))) <= hp.TOL[torch.bfloat16]
+    want = 0
+    for h, o in orcs.items():
+        hp.assert_state_equal(sg.export_state(0, h), o, "unit %d" % h)
+        want += sum(len(set(r.tolist())) if t <= 16 else t for r in o.slot_tok[o.counts > 1])
+    assert sg.cache_stats()["distinct_sample_rows"] == want
