@@ -19,8 +19,7 @@
  *   mu = sum of ||v||^2         -> mu (fixed point, see below)
  *   window                      -> the last `window` token indices
  *
- * Readings of points the paper leaves open (each one is also listed in the
- * design notes of the repository):
+ * Readings of points the paper leaves open:
  *  - Window (Section 3.2 keeps "the most recent r tokens" next to the
  *    clustered rest and gives no estimator for the combination): a token
  *    enters D and M when it LEAVES the window; window tokens enter numerator
