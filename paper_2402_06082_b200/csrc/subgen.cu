@@ -1163,7 +1163,8 @@ int kcenter_compress_td(subgen_exact* h, int k, int r, int k_iter, int keep_max,
     gi = gi > 32 ? 32 : gi;
     kcenter_init_kernel<T, D><<<dim3(gi, h->U), 256, 0, h->st>>>(E, r, head, dist);
     for (int t = 0; t < k_iter; ++t)
-        kcenter_iter_kernel<T, D><<<dim3(S, h->U), kKcThreads, smem, h->st>>>(E, t, k, r, head, dist, centres, part[(t + 1) & 1], part[t & 1], counters);
+        launch_pdl_smem(kcenter_iter_kernel<T, D>, dim3(S, h->U), dim3(kKcThreads), smem, h->st, E, t, k, r, (const uint4*)head, dist, centres,
+                        (const Best*)part[(t + 1) & 1], part[t & 1], counters);
     int gx = (int)(((size_t)keep_max * (D / Elem<T>::EPL) + 255) / 256);
     gx = gx < 1 ? 1 : (gx > 32 ? 32 : gx);
     kcenter_gather_kernel<T, D><<<dim3(gx, h->U), 256, 0, h->st>>>(E, k, r, centres, Kt, Vt, tokt, keep_max);

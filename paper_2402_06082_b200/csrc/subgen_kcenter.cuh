@@ -66,6 +66,8 @@ __global__ void __launch_bounds__(kKcThreads) kcenter_iter_kernel(ExactCache<T> 
     __shared__ int nsurv;
     const int u = blockIdx.y, S = gridDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = kKcThreads >> 5;
     const int lr = lane % LPR, sub = lane / LPR;
+    pdl_trigger();                       // the next pass may be scheduled; it waits for this one right here
+    pdl_wait();
     const int n = E.n_unit[u], n_old = max(0, n - r);
     if (t >= min(k, n_old)) return;
     // the newest centre
