@@ -388,12 +388,13 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
     slices = slices < 1 ? 1 : (slices > 32 ? 32 : slices);
     PrefillArgs a;
     a.K = (const T*)K; a.V = (const T*)V; a.n_uniform = n; a.cu = cu_dev; a.total = total; a.Lmax = Lmax; a.slices = slices;
-    a.Wbuf = nullptr; a.Tot = nullptr; a.Thr = nullptr; a.Mwin = nullptr; a.pbest = nullptr;
+    a.Wbuf = nullptr; a.Tot = nullptr; a.Thr = nullptr; a.Mwin = nullptr; a.pbest = nullptr; a.mhist = nullptr;
     int launches = 0;
     if (Lmax > 0) {
         const size_t b_w = align_up((size_t)d.U * Lmax * 8), b_m = align_up((size_t)d.U * d.s * 4);
         const size_t b_p = align_up((size_t)d.U * slices * kChunk * sizeof(Best));
-        const size_t need = 3 * b_w + b_m + b_p;
+        const size_t b_h = align_up((size_t)d.U * 2 * sizeof(int));
+        const size_t need = 3 * b_w + b_m + b_p + b_h;
         if (need > h->scratch_bytes) {
             if (h->scratch) { CUDA_TRY(cudaStreamSynchronize(h->st)); CUDA_TRY(cudaFree(h->scratch)); h->scratch = nullptr; h->scratch_bytes = 0; }
             cudaError_t e = cudaMalloc((void**)&h->scratch, need);
@@ -405,6 +406,7 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         a.Thr = (unsigned long long*)(h->scratch + 2 * b_w);
         a.Mwin = (int*)(h->scratch + 3 * b_w);
         a.pbest = (Best*)(h->scratch + 3 * b_w + b_m);
+        a.mhist = (int*)(h->scratch + 3 * b_w + b_m + b_p);
         auto mark = [&]() -> int {                       // profiling: one event on the stream
             if (!h->prof) return SUBGEN_OK;
             if (h->pev_used == h->pev.size()) {
@@ -436,6 +438,8 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         launches += 4;
         if (int rc = mark()) return rc;
         const int nchunks = (Lmax + kChunk - 1) / kChunk;
+        prefill_mhist_kernel<<<(d.U + 255) / 256, 256, 0, h->st>>>(C, a, d.U);
+        launches += 1;
         static bool configured = false;
         if (tc && !configured) {
             CUDA_TRY(cudaFuncSetAttribute(prefill_score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes));

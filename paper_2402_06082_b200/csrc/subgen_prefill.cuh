@@ -40,6 +40,8 @@ struct PrefillArgs {
     unsigned long long* Thr;           // [U, Lmax] coin threshold ceil(W 2^32 / tot): the coin succeeds iff u < Thr
     int* Mwin;                         // [U, s] winning token per M slot, -1 none
     Best* pbest;                       // [U, slices, kChunk] partial nearest old representative per chunk token
+    int* mhist;                        // [U, 2] cluster count after chunk c in slot c & 1 (both slots: the count before
+                                       //        the call, until chunks 0 and 1 have been resolved)
     int slices;
 };
 
@@ -504,6 +506,7 @@ __global__ void __launch_bounds__(kResolveThreads) prefill_resolve_kernel(Cache<
     if (tid == 0) {
         C.pairs[u] += (unsigned long long)cl * (unsigned long long)m_old;
         C.m_unit[u] = m_old + sm_opened;
+        a.mhist[2 * u + (chunk & 1)] = m_old + sm_opened;
         if (sm_full) atomicOr(&C.status[u], 1);
         const int j = cl - 1;
         if (e0 + j == r.ins_hi - 1) {                               // the most recent insertion of this unit
@@ -534,6 +537,12 @@ __global__ void prefill_finish_kernel(Cache<__nv_bfloat16> C, PrefillArgs a) {
 }
 
 // Last kernel of a prefill call: counters (after every block of every other kernel has read them).
+// Both slots of mhist start as the cluster count before the call. One thread per unit.
+__global__ void prefill_mhist_kernel(Cache<__nv_bfloat16> C, PrefillArgs a, int U) {
+    const int u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u < U) { a.mhist[2 * u] = C.m_unit[u]; a.mhist[2 * u + 1] = C.m_unit[u]; }
+}
+
 // Alias rows of every cluster (see Cache::alias) from the slot tokens the chunks left. grid (blocks, U).
 __global__ void prefill_alias_kernel(Cache<__nv_bfloat16> C) {
     const int u = blockIdx.y, m = C.m_unit[u], t = C.t;

@@ -105,31 +105,30 @@ __global__ void __launch_bounds__(kTcThreads, 4) prefill_score_tc_kernel(Cache<_
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = sm.tmem_base;
     const float my_kn = sm.kn[tid];
-    // Everything above touches only the chunk's keys. The representatives and their count come from the resolve
-    // kernel of the previous chunk, which may still be running: wait for it here, then let the next kernel in.
-    pdl_wait();
-    pdl_trigger();
-    const int m = C.m_unit[u];
+    // Everything above touches only the chunk's keys. Tiles of 128 representatives are dealt to the blocks of the
+    // unit round-robin. The resolve kernel of the previous chunk may still be running: it appends representatives
+    // and never touches those that exist, so the tiles that lay entirely below the count the chunk before it left
+    // (ms_safe, written two kernels ago, read from L2) are scored at once; then the kernel waits for its
+    // predecessor and scores the rest with the final count.
     Best* outp = a.pbest + ((size_t)u * slices + blockIdx.x) * kChunk;
-    const int per = (((m + slices - 1) / slices) + kTcTileN - 1) / kTcTileN * kTcTileN;
-    const int c0 = blockIdx.x * per, c1 = min(m, c0 + per);
-    const int ntiles = c0 < c1 ? (c1 - c0 + kTcTileN - 1) / kTcTileN : 0;      // 0: this slice holds no representative
+    const int m_safe = __ldcg(a.mhist + 2 * u + (chunk & 1));        // count after chunk - 2
+    const int JA = m_safe / kTcTileN;                                  // tiles [0, JA) are final
 
     // representative heads of tile j: global -> registers (tile_fetch), registers -> B[buf], xa[buf] (tile_store)
     constexpr int kPer = kTcTileN * kTcHeadPieces / kTcThreads;      // pieces per thread and tile
     uint4 R[kPer];
-    auto tile_fetch = [&](int j) {
-        const int row0 = c0 + j * kTcTileN;
+    auto tile_fetch = [&](int j, int limit) {
+        const int row0 = j * kTcTileN;
 #pragma unroll
         for (int i = 0; i < kPer; ++i) {
             const int p = i * kTcThreads + tid, rr = p / kTcHeadPieces, q = p % kTcHeadPieces;
             R[i] = make_uint4(0, 0, 0, 0);
-            if (row0 + rr < c1) R[i] = ldg16(Xu + (size_t)(row0 + rr) * D + q * 8);
+            if (row0 + rr < limit) R[i] = ldg16(Xu + (size_t)(row0 + rr) * D + q * 8);
         }
     };
-    auto tile_store = [&](int buf, int j) {
+    auto tile_store = [&](int buf, int j, int limit) {
         unsigned char* dst = sm.B[buf];
-        const int row0 = c0 + j * kTcTileN;
+        const int row0 = j * kTcTileN;
 #pragma unroll
         for (int i = 0; i < kPer; ++i) {
             const int p = i * kTcThreads + tid, rr = p / kTcHeadPieces, q = p % kTcHeadPieces;
@@ -142,7 +141,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) prefill_score_tc_kernel(Cache<_
             hn += __shfl_xor_sync(0xffffffffu, hn, 1);
             hn += __shfl_xor_sync(0xffffffffu, hn, 2);
             hn += __shfl_xor_sync(0xffffffffu, hn, 4);
-            if (q == 0) sm.xa[buf][rr] = row0 + rr < c1 ? 0.5f * kOneMinusG * hn : INFINITY;
+            if (q == 0) sm.xa[buf][rr] = row0 + rr < limit ? 0.5f * kOneMinusG * hn : INFINITY;
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy stores -> visible to the MMA
     };
@@ -179,85 +178,102 @@ __global__ void __launch_bounds__(kTcThreads, 4) prefill_score_tc_kernel(Cache<_
         }
     };
 
-    // Pipeline: two tiles of heads are staged ahead in shared memory and a third is in flight in registers;
-    // the MMAs of tile j+1 are issued right after tile j has been read back from tensor memory.
-    if (ntiles > 0) { tile_fetch(0); tile_store(0, 0); }
-    if (ntiles > 1) { tile_fetch(1); tile_store(1, 1); }
-    if (ntiles > 2) tile_fetch(2);
-    __syncthreads();
-    if (ntiles > 0 && tid == 0) {
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        issue_mma(0);
-    }
+    // A run of cnt tiles j0, j0 + slices, ...: two tiles of heads are staged ahead in shared memory and a third is
+    // in flight in registers; the MMAs of a tile are issued right after its predecessor has been read back from
+    // tensor memory. done: MMA commits of this block so far (barrier phase and buffer of the next tile).
+    int done = 0;
     bool ok = true;
-    for (int j = 0; j < ntiles; ++j) {
-        const int buf = j & 1;
-        // wait for the MMAs of tile j (bounded)
-        {
-            const uint32_t parity = (uint32_t)(j & 1);
-            unsigned done = 0, spins = 0;
-            while (!done && spins < kTcSpinLimit) {
-                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
-                             : "=r"(done) : "r"(sBar), "r"(parity) : "memory");
-                ++spins;
-            }
-            if (!done) sm.failed = 1;
-        }
+    auto run = [&](int j0, int cnt, int limit) {
+        if (cnt <= 0 || !ok) return;
+        tile_fetch(j0, limit);
+        tile_store(done & 1, j0, limit);
+        if (cnt > 1) { tile_fetch(j0 + slices, limit); tile_store((done + 1) & 1, j0 + slices, limit); }
+        if (cnt > 2) tile_fetch(j0 + 2 * slices, limit);
         __syncthreads();
-        if (sm.failed) { ok = false; break; }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        // read-back: this thread's token row, 128 columns in four pieces of 32
-        const float* xat = sm.xa[buf];
+        if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            issue_mma(done & 1);
+        }
+        for (int i = 0; i < cnt; ++i) {
+            const int buf = (done + i) & 1;
+            // wait for the MMAs of this tile (bounded)
+            {
+                const uint32_t parity = (uint32_t)((done + i) & 1);
+                unsigned fin = 0, spins = 0;
+                while (!fin && spins < kTcSpinLimit) {
+                    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                                 : "=r"(fin) : "r"(sBar), "r"(parity) : "memory");
+                    ++spins;
+                }
+                if (!fin) sm.failed = 1;
+            }
+            __syncthreads();
+            if (sm.failed) { ok = false; return; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            // read-back: this thread's token row, 128 columns in four pieces of 32
+            const float* xat = sm.xa[buf];
 #pragma unroll 1
-        for (int cc = 0; cc < kTcTileN; cc += 32) {
-            uint32_t v[32];
-            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)cc;
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
-                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-                  "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-                  "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-                  "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                : "r"(taddr) : "memory");
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            if (tid < cl) {
+            for (int cc = 0; cc < kTcTileN; cc += 32) {
+                uint32_t v[32];
+                const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)cc;
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                      "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+                      "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+                      "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                    : "r"(taddr) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (tid < cl) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    if (__uint_as_float(v[i]) >= xat[cc + i] + my_kn) {          // rare
-                        const unsigned slot = atomicAdd(&sm.ncand, 1u);
-                        if (slot < (unsigned)kTcCand) sm.cand[slot] = (unsigned)tid | ((unsigned)(cc + i) << 8);
+                    for (int q = 0; q < 32; ++q) {
+                        if (__uint_as_float(v[q]) >= xat[cc + q] + my_kn) {          // rare
+                            const unsigned slot = atomicAdd(&sm.ncand, 1u);
+                            if (slot < (unsigned)kTcCand) sm.cand[slot] = (unsigned)tid | ((unsigned)(cc + q) << 8);
+                        }
                     }
                 }
             }
-        }
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
-        // the accumulator is free: start tile j+1 (its heads were staged at least one barrier ago)
-        if (j + 1 < ntiles && tid == 0) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            issue_mma(buf ^ 1);
-        }
-        // exact distances of the flagged pairs of this tile; warp w owns the tokens with index % 4 == w
-        const unsigned nc = sm.ncand;
-        const int row0 = c0 + j * kTcTileN;
-        if (nc <= (unsigned)kTcCand) {
-            for (unsigned i = 0; i < nc; ++i) {
-                const unsigned cd = sm.cand[i];
-                if ((cd & 3u) == (unsigned)warp) exact_pair((int)(cd & 255u), row0 + (int)(cd >> 8));
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncthreads();
+            // the accumulator is free: start the next tile (its heads were staged at least one barrier ago)
+            if (i + 1 < cnt && tid == 0) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                issue_mma(buf ^ 1);
             }
-        } else {                                                          // too many to list: every pair of the tile
-            const int nrow = min(kTcTileN, c1 - row0);
-            for (int tokj = warp; tokj < cl; tokj += kTcThreads / 32)
-                for (int rr = 0; rr < nrow; ++rr) exact_pair(tokj, row0 + rr);
+            // exact distances of the flagged pairs of this tile; warp w owns the tokens with index % 4 == w
+            const unsigned nc = sm.ncand;
+            const int row0 = (j0 + i * slices) * kTcTileN;
+            if (nc <= (unsigned)kTcCand) {
+                for (unsigned q = 0; q < nc; ++q) {
+                    const unsigned cd = sm.cand[q];
+                    if ((cd & 3u) == (unsigned)warp) exact_pair((int)(cd & 255u), row0 + (int)(cd >> 8));
+                }
+            } else {                                                          // too many to list: every pair of the tile
+                const int nrow = min(kTcTileN, limit - row0);
+                for (int tokj = warp; tokj < cl; tokj += kTcThreads / 32)
+                    for (int rr = 0; rr < nrow; ++rr) exact_pair(tokj, row0 + rr);
+            }
+            __syncthreads();
+            if (tid == 0) sm.ncand = 0;
+            if (i + 2 < cnt) {                                                // this tile's buffer is free since its MMAs ended
+                tile_store(buf, j0 + (i + 2) * slices, limit);
+                if (i + 3 < cnt) tile_fetch(j0 + (i + 3) * slices, limit);
+            }
         }
-        __syncthreads();
-        if (tid == 0) sm.ncand = 0;
-        if (j + 2 < ntiles) {                                             // buffer `buf` is free since the MMAs of tile j ended
-            tile_store(buf, j + 2);
-            if (j + 3 < ntiles) tile_fetch(j + 3);
-        }
-    }
+        done += cnt;
+    };
+    const int bx = (int)blockIdx.x;
+    const int nA = JA > bx ? (JA - bx + slices - 1) / slices : 0;      // this block's tiles below JA
+    run(bx, nA, JA * kTcTileN);
+    pdl_wait();
+    pdl_trigger();
+    const int m = C.m_unit[u];
+    const int JT = (m + kTcTileN - 1) / kTcTileN;
+    const int jB = bx + nA * slices;                                   // this block's first tile at or above JA
+    const int nB = JT > jB ? (JT - jB + slices - 1) / slices : 0;
+    run(jB, nB, m);
     __syncthreads();
     if (ok) {
         for (int j = tid; j < kChunk; j += kTcThreads) {
