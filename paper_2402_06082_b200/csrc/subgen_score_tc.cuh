@@ -246,9 +246,61 @@ __global__ void __launch_bounds__(kTcThreads, 4) prefill_score_tc_kernel(Cache<_
             const unsigned nc = sm.ncand;
             const int row0 = (j0 + i * slices) * kTcTileN;
             if (nc <= (unsigned)kTcCand) {
-                for (unsigned q = 0; q < nc; ++q) {
-                    const unsigned cd = sm.cand[q];
-                    if ((cd & 3u) == (unsigned)warp) exact_pair((int)(cd & 255u), row0 + (int)(cd >> 8));
+                // four pairs per turn, two per half-warp with both rows of each pair requested before any is used:
+                // a pair's exact distance is a chain of two global loads and a reduction, so the pairs of a tile
+                // are evaluated side by side instead of one after the other
+                for (unsigned base = 0; base < nc; base += 32) {
+                    const bool have = base + lane < nc;
+                    const unsigned cd = have ? sm.cand[base + lane] : 0u;
+                    unsigned mine = __ballot_sync(0xffffffffu, have && (cd & 3u) == (unsigned)warp);
+                    while (mine) {
+                        int sel[4];
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) {
+                            sel[x] = mine ? __ffs(mine) - 1 : -1;
+                            if (mine) mine &= mine - 1;
+                        }
+                        const int half = lane >> 4, l16 = lane & 15;
+                        unsigned long long acc[2];
+                        unsigned cdv[2];
+                        uint4 xr[2], kr[2];
+#pragma unroll
+                        for (int y = 0; y < 2; ++y) {
+                            const int sidx = sel[2 * y + half];
+                            cdv[y] = __shfl_sync(0xffffffffu, cd, sidx < 0 ? 0 : sidx);
+                            if (sidx >= 0) {
+                                xr[y] = *reinterpret_cast<const uint4*>(Xu + (size_t)(row0 + (int)(cdv[y] >> 8)) * D + l16 * 8);
+                                kr[y] = reinterpret_cast<const uint4*>(key_row<D>(C, a, r, u, e0 + (int)(cdv[y] & 255u)))[l16];
+                            } else {
+                                xr[y] = make_uint4(0, 0, 0, 0);
+                                kr[y] = make_uint4(0, 0, 0, 0);
+                            }
+                        }
+#pragma unroll
+                        for (int y = 0; y < 2; ++y) {
+                            float xf[8], kf[8];
+                            Elem<T>::unpack(xr[y], xf);
+                            Elem<T>::unpack(kr[y], kf);
+                            acc[y] = 0;
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) acc[y] += fx_sqdiff(xf[e], kf[e]);
+#pragma unroll
+                            for (int off = 8; off > 0; off >>= 1) acc[y] += __shfl_xor_sync(0xffffffffu, acc[y], off);
+                        }
+                        // lane 0 applies the (up to) four results one after the other: they may concern one token
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) {
+                            const int y = x >> 1, hsrc = (x & 1) * 16;
+                            const unsigned long long d2 = __shfl_sync(0xffffffffu, acc[y], hsrc);
+                            const unsigned cdx = __shfl_sync(0xffffffffu, cdv[y], hsrc);
+                            if (lane == 0 && sel[x] >= 0) {
+                                const int tokj = (int)(cdx & 255u), row = row0 + (int)(cdx >> 8);
+                                Best cur;
+                                cur.d2 = sm.wb_d2[tokj]; cur.idx = sm.wb_idx[tokj];
+                                if (better(d2, row, cur)) { sm.wb_d2[tokj] = d2; sm.wb_idx[tokj] = row; }
+                            }
+                        }
+                    }
                 }
             } else {                                                          // too many to list: every pair of the tile
                 const int nrow = min(kTcTileN, limit - row0);
