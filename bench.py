@@ -371,6 +371,9 @@ def run_subgen(args, w):
     else:
         dom = ("query_kernel", cbytes + vbytes, c_ms)
     achieved = gbs(dom[1], dom[2])
+    row_b = wr.d * (2 if dt == torch.bfloat16 else 4)
+    nominal_c = 0.5 * sum((st_["singleton_clusters"] + (st_["clusters"] - st_["singleton_clusters"]) * wr.t) * row_b + st_["clusters"] * 4
+                          for st_ in (stats1, stats2))
     step_bytes = avg_main("cluster_bytes") + avg_main("value_bytes") + avg_main("insert_bytes")
     traffic = None
     if NCU_TRAFFIC.get(dom[0]) and NCU_TRAFFIC[dom[0]]["workload"] == wr.name and not args.prompt:          # DRAM bytes of one launch from the ncu capture, scaled by the units processed
@@ -380,7 +383,9 @@ def run_subgen(args, w):
                 "unit": "GB/s", "frac": achieved / peak if achieved else None, "traffic": traffic,
                 "algorithmic_bytes_per_launch": dom[1], "ms_per_launch": dom[2],
                 "kernels": {"insert": {"algorithmic_bytes_per_launch": ibytes, "ms_per_launch": i_ms, "achieved": gbs(ibytes, i_ms)},
-                            "cluster_scan": {"algorithmic_bytes_per_launch": cbytes, "ms_per_launch": c_ms, "achieved": gbs(cbytes, c_ms)},
+                            "cluster_scan": {"algorithmic_bytes_per_launch": cbytes, "ms_per_launch": c_ms, "achieved": gbs(cbytes, c_ms),
+                                             # for comparison: all t sample slots of every cluster, repeats included
+                                             "bytes_with_repeated_slots": nominal_c, "achieved_with_repeated_slots": gbs(nominal_c, c_ms)},
                             "value_scan": {"algorithmic_bytes_per_launch": vbytes, "ms_per_launch": v_ms, "achieved": gbs(vbytes, v_ms)}},
                 "timing": "per-kernel durations from a second pass of %d steps with CUDA events around every kernel; "
                           "the step figure from the timed region (no events between kernels)" % P_steps,
