@@ -49,7 +49,10 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
         return;
     }
     const int e = n - w;
+    // key and value of the token that leaves the window: both fetched now, so that the block that ends up applying
+    // the insertion does not wait for the value row after the scan
     if (tid < LPR) krow[tid] = w ? ringk[tid] : knew_u[tid];
+    else if (tid < 2 * LPR) vrow[tid - LPR] = w ? ringv[tid - LPR] : vnew_u[tid - LPR];
     __syncthreads();
     const int m = C.m_unit[u];
     const T* Xu = C.X + (size_t)u * C.m_max * D;
@@ -142,8 +145,6 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
         b = block_best(bb, smb);
         if (tid == 0) C.ticket1[u] = 0;
     }
-    if (tid < LPR) vrow[tid] = w ? ringv[tid] : vnew_u[tid];
-    __syncthreads();
     apply_insert<T, D, BND>(C, u, e, b, m, krow, vrow, sm_w);
     if (w) {
         if (tid < LPR) ringk[tid] = knew_u[tid];
