@@ -31,11 +31,6 @@ from paper_2402_06082_b200 import sharding, synth  # noqa: E402
 
 METRIC = "SubGen decode steps/s (B x H heads) at 32K ctx"
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised in
-# profiles/step_kernels_cfg3.md (cfg3 state at 32K tokens, 64 units). Valid for cfg3 only; set an entry to
-# None when its kernel changes.
-NCU_TRAFFIC = {"query_tau_kernel": {"dram_bytes": 132.43e6, "units": 64, "workload": "cfg3"}}
-
 
 # ------------------------------------------------------------------------------------------ helpers
 def measured_peaks():
@@ -61,7 +56,7 @@ def tensor_roofline(pairs, d, ms):
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU every 50 ms through NVML while running."""
+    """Samples SM clock and throttle reasons of one GPU every 20 ms through NVML while running."""
 
     def __init__(self, device_index: int):
         self.samples, self.reasons, self.max_mhz = [], set(), None
@@ -96,7 +91,7 @@ class ClockSampler:
                         self.reasons.add(k)
             except Exception:
                 pass
-            self._stop.wait(0.05)
+            self._stop.wait(0.02)
 
     def __enter__(self):
         if self._h is not None:
@@ -197,31 +192,31 @@ def workload_config(w):
             "accumulate": "fp32", "units": w.units, "m_max": w.m_max}
 
 
-def run_subgen(args, w):
-    from paper_2402_06082_b200 import binding, build
-    build.build()
-    N = args.gpus
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
-    torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    # weak scaling: every rank serves its own batch of B sequences (units are independent, no data-path collective)
-    wr = sharding.rank_workload(w, rank)
-    K_steps = args.steps
-    W_steps = args.warmup
-    n_e2e = args.e2e_steps
-    P_steps = min(K_steps, 256)          # second, shorter pass with CUDA events between the kernels
-    n_dec = W_steps + K_steps + P_steps + n_e2e + 4
+def plan_repeats(K_steps, est_ms_per_step):
+    """How often the K-step timed region is repeated: enough for about 0.6 s of GPU time, at most 4096 steps in all
+    (every step lengthens the context by one token, so the workload must not drift far), at least 3 regions when K
+    allows it."""
+    want = int(min(4096, max(K_steps, 600.0 / max(est_ms_per_step, 1e-3))))
+    R = (want + K_steps - 1) // K_steps
+    if R < 3 and 3 * K_steps <= 4096:
+        R = 3
+    return max(1, min(R, 256))
+
+
+def measure(wr, args, K_steps, W_steps, world, rank, local, dist, headline):
+    """Prefill + decode of one workload on this rank's GPU. headline = True adds the prefill phase profile, the exact
+    comparison, the per-kernel roofline block; False gives the compact entry of the per-config table."""
+    from paper_2402_06082_b200 import binding
+    n_e2e = args.e2e_steps if headline else min(args.e2e_steps, 16)
+    P_steps = min(K_steps, 256 if headline else 64)          # second, shorter pass with CUDA events between the kernels
     lens = wr.prompt_lens()
     varlen = wr.varlen is not None
     dev = "cuda"
     dt = wr.torch_dtype
+    R_max = 256 if K_steps * 256 <= 4096 else max(3, 4096 // K_steps)
+    # a workload streamed from empty (cfg1) first runs half of its stated stream length untimed
+    lead = wr.n_decode // 2 if not max(lens) else 0
+    n_dec = lead + W_steps + 64 + K_steps * R_max + P_steps + n_e2e + 4
 
     # ---- inputs, resident in HBM ----
     qs = torch.empty(n_dec, wr.B, wr.H, wr.d, dtype=dt, device=dev)
@@ -267,23 +262,26 @@ def run_subgen(args, w):
     warm.close()
     del warm, wk
     torch.cuda.empty_cache()
+
     def run_prefill(handle):
         if varlen:
             handle.prefill_varlen(Kp, Vp, np.concatenate([[0], np.cumsum(lens)]).astype(np.int64))
-        else:
+        elif max(lens):
             handle.prefill(Kp, Vp)
 
     # phases: the same prefill on a handle of its own with CUDA events between the kernels (they keep a kernel from
     # starting while its predecessor drains, so the timed prefill below runs without them)
-    prof = binding.SubGen(wr.B, wr.H, wr.d, wr.delta, wr.t, wr.s, wr.window, wr.philox_seed, Hkv=wr.Hkv, dtype=dt,
-                          m_max=wr.m_max, splits=args.splits, bounded=args.bounded)
-    prof.profile_enable(True)
-    run_prefill(prof)
-    torch.cuda.synchronize()
-    pf_values_ms, pf_score_ms, pf_resolve_ms = prof.profile_prefill_read()
-    prof.close()
-    del prof
-    torch.cuda.empty_cache()          # the exact comparison allocates with cudaMalloc, outside torch's cache
+    pf_values_ms = pf_score_ms = pf_resolve_ms = None
+    if headline:
+        prof = binding.SubGen(wr.B, wr.H, wr.d, wr.delta, wr.t, wr.s, wr.window, wr.philox_seed, Hkv=wr.Hkv, dtype=dt,
+                              m_max=wr.m_max, splits=args.splits, bounded=args.bounded)
+        prof.profile_enable(True)
+        run_prefill(prof)
+        torch.cuda.synchronize()
+        pf_values_ms, pf_score_ms, pf_resolve_ms = prof.profile_prefill_read()
+        prof.close()
+        del prof
+        torch.cuda.empty_cache()          # the exact comparison allocates with cudaMalloc, outside torch's cache
     l0 = sg.launch_count
     e0.record()
     run_prefill(sg)
@@ -294,71 +292,93 @@ def run_subgen(args, w):
     pf_pairs = sg.cache_stats()["prefill_pairs"]
     st = sg.status()
     if st:
-        raise SystemExit("device status %d after prefill (1 = cluster capacity, 2 = input range)" % st)
+        raise SystemExit("%s: device status %d after prefill (1 = cluster capacity, 2 = input range)" % (wr.name, st))
     del Kp, Vp
-
-    # ---- decode: warm-up, then the timed region ----
-    for i in range(W_steps):
+    for i in range(lead):
         sg.step(qs[i], ks[i], vs[i], out)
+    pos = lead
+
+    # ---- decode: warm-up, an estimate of the step time, then R timed regions of exactly K steps each ----
+    for i in range(W_steps):
+        sg.step(qs[pos + i], ks[pos + i], vs[pos + i], out)
+    pos += W_steps
     torch.cuda.synchronize()
+    e0.record()
+    for i in range(64):
+        sg.step(qs[pos + i], ks[pos + i], vs[pos + i], out)
+    e1.record()
+    torch.cuda.synchronize()
+    pos += 64
+    R = min(plan_repeats(K_steps, e0.elapsed_time(e1) / 64), R_max)
+    if dist:                              # every rank must run the same number of regions
+        t = torch.tensor([R], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MIN)
+        R = int(t.item())
     stats0 = sg.cache_stats()
-    if dist:
-        dist.barrier()
-    torch.cuda.synchronize()
     launches0 = sg.launch_count
+    region_ms = []
     with ClockSampler(local) as clk:
-        e0.record()
-        for i in range(W_steps, W_steps + K_steps):
-            sg.step(qs[i], ks[i], vs[i], out)
-        e1.record()
-        torch.cuda.synchronize()
-    if dist:
-        dist.barrier()
-    ms = e0.elapsed_time(e1)
-    launches = sg.launch_count - launches0
+        for r in range(R):
+            if dist:
+                dist.barrier()
+            torch.cuda.synchronize()
+            e0.record()
+            for i in range(pos, pos + K_steps):
+                sg.step(qs[i], ks[i], vs[i], out)
+            e1.record()
+            torch.cuda.synchronize()
+            if dist:
+                dist.barrier()
+            region_ms.append(sharding.max_over_ranks(e0.elapsed_time(e1), dist, dev))
+            pos += K_steps
+    launches = (sg.launch_count - launches0) // R
     stats1 = sg.cache_stats()
+    ms = float(np.median(region_ms))
     # per-kernel durations: the same loop again, shorter, with CUDA events recorded on the handle's stream around
     # every kernel (events between kernels cost time and keep a kernel from being scheduled while its predecessor
     # drains, so the headline above is taken without them)
     sg.profile_enable(True)
-    for i in range(W_steps + K_steps, W_steps + K_steps + P_steps):
+    for i in range(pos, pos + P_steps):
         sg.step(qs[i], ks[i], vs[i], out)
     torch.cuda.synchronize()
+    pos += P_steps
     ins_ms, tau_ms, z_ms, nprof = sg.profile_read()
     sg.profile_enable(False)
     stats2 = sg.cache_stats()
-    ms = sharding.max_over_ranks(ms, dist, dev)
     ms_per_step = ms / K_steps
     value = sharding.job_steps_per_s(world, K_steps, ms)
 
     # ---- end to end through the host-buffer entry point ----
-    base = W_steps + K_steps + P_steps
-    hq = qs[base:base + n_e2e].cpu().pin_memory()
-    hk = ks[base:base + n_e2e].cpu().pin_memory()
-    hv = vs[base:base + n_e2e].cpu().pin_memory()
+    hq = qs[pos:pos + n_e2e].cpu().pin_memory()
+    hk = ks[pos:pos + n_e2e].cpu().pin_memory()
+    hv = vs[pos:pos + n_e2e].cpu().pin_memory()
     hout = torch.empty(wr.B, wr.H, wr.d, dtype=dt).pin_memory()
+    for i in range(min(2, n_e2e)):        # the first host-buffer call resolves the pinned mappings
+        sg.step_host(hq[i], hk[i], hv[i], hout)
     if dist:
         dist.barrier()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
-    for i in range(n_e2e):
+    for i in range(min(2, n_e2e), n_e2e):
         sg.step_host(hq[i], hk[i], hv[i], hout)
     t_e2e = time.perf_counter() - t0
     t_e2e = sharding.max_over_ranks(t_e2e, dist, dev)
+    n_timed_e2e = max(1, n_e2e - min(2, n_e2e))
     esz = 2 if dt == torch.bfloat16 else 4
     h2d = (wr.B * wr.H + 2 * wr.B * wr.Hkv) * wr.d * esz
     d2h = wr.B * wr.H * wr.d * esz
-    e2e = {"value": world * n_e2e / t_e2e, "unit": "steps/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-           "steps": n_e2e}
+    e2e = {"value": world * n_timed_e2e / t_e2e, "unit": "steps/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+           "steps": n_timed_e2e}
     if sg.status():
-        raise SystemExit("device status %d after decode" % sg.status())
+        raise SystemExit("%s: device status %d after decode" % (wr.name, sg.status()))
 
-    # ---- roofline of the dominant kernel (query_kernel) ----
+    # ---- roofline of the dominant kernel ----
     peak, which = measured_peaks()
+
     def avg(key):                       # bytes of the profiled pass (per-kernel figures)
         return 0.5 * (stats1[key] + stats2[key])
 
-    def avg_main(key):                  # bytes of the timed region (whole-step figure)
+    def avg_main(key):                  # bytes of the timed regions (whole-step figure)
         return 0.5 * (stats0[key] + stats1[key])
 
     def gbs(nbytes, ms_):
@@ -375,10 +395,18 @@ def run_subgen(args, w):
     nominal_c = 0.5 * sum((st_["singleton_clusters"] + (st_["clusters"] - st_["singleton_clusters"]) * wr.t) * row_b + st_["clusters"] * 4
                           for st_ in (stats1, stats2))
     step_bytes = avg_main("cluster_bytes") + avg_main("value_bytes") + avg_main("insert_bytes")
-    traffic = None
-    if NCU_TRAFFIC.get(dom[0]) and NCU_TRAFFIC[dom[0]]["workload"] == wr.name and not args.prompt:          # DRAM bytes of one launch from the ncu capture, scaled by the units processed
-        t = NCU_TRAFFIC[dom[0]]
-        traffic = t["dram_bytes"] * wr.units / t["units"]
+    step_gbs = gbs(step_bytes, ms_per_step)
+    clocks = clk.summary()
+    if not headline:
+        sg.close()
+        return {"units": wr.units, "steps_per_s": value, "ms_per_step": ms_per_step, "repeats": R,
+                "ms_per_step_min": min(region_ms) / K_steps, "ms_per_step_max": max(region_ms) / K_steps,
+                "step_bytes": step_bytes, "step_GBps": step_gbs, "frac_of_hbm_peak": step_gbs / peak if step_gbs else None,
+                "kernel_ms": {"insert": i_ms, "cluster_scan": c_ms, "value_scan": v_ms},
+                "prefill_ms": prefill_ms, "prefill_tokens_per_s": sum(lens) / (prefill_ms * 1e-3) if sum(lens) else None,
+                "e2e_steps_per_s": e2e["value"], "gpu_launches_per_region": int(launches), "clocks": clocks,
+                "clusters_per_unit": stats1["clusters"] / wr.units}
+    traffic = ncu_traffic(dom[0], wr) if not args.prompt else None
     roofline = {"bound": "hbm", "kernel": dom[0], "achieved": achieved, "peak": peak, "peak_source": which,
                 "unit": "GB/s", "frac": achieved / peak if achieved else None, "traffic": traffic,
                 "algorithmic_bytes_per_launch": dom[1], "ms_per_launch": dom[2],
@@ -388,12 +416,10 @@ def run_subgen(args, w):
                                              "bytes_with_repeated_slots": nominal_c, "achieved_with_repeated_slots": gbs(nominal_c, c_ms)},
                             "value_scan": {"algorithmic_bytes_per_launch": vbytes, "ms_per_launch": v_ms, "achieved": gbs(vbytes, v_ms)}},
                 "timing": "per-kernel durations from a second pass of %d steps with CUDA events around every kernel; "
-                          "the step figure from the timed region (no events between kernels)" % P_steps,
-                "step": {"algorithmic_bytes": step_bytes,
-                         "achieved": gbs(step_bytes, ms_per_step),
-                         "frac": gbs(step_bytes, ms_per_step) / peak}}
+                          "the step figure from the timed regions (no events between kernels)" % P_steps,
+                "step": {"algorithmic_bytes": step_bytes, "achieved": step_gbs, "frac": step_gbs / peak}}
 
-    extra = {"prefill_ms": prefill_ms, "prefill_tokens_per_s": sum(lens) / (prefill_ms * 1e-3),
+    extra = {"prefill_ms": prefill_ms, "prefill_tokens_per_s": sum(lens) / (prefill_ms * 1e-3) if sum(lens) else None,
              "prefill_launches": prefill_launches,
              "prefill_phases_ms": {"values": pf_values_ms, "score": pf_score_ms, "resolve": pf_resolve_ms},
              # the tcgen05 scoring kernel (d = 128, default) contracts the first 64 coordinates only
@@ -424,6 +450,9 @@ def run_subgen(args, w):
     if args.bounded:
         st0 = sg.export_state(0, 0)
         extra["bounded"] = {"m_max": wr.m_max, "doublings_unit0": st0["doublings"], "clusters_unit0": st0["m"], "status": sg.status()}
+    sg.close()
+    del sg
+    torch.cuda.empty_cache()
 
     # ---- exact dense decode over full caches on the same inputs (comparison point) ----
     if args.exact and rank == 0:
@@ -433,9 +462,68 @@ def run_subgen(args, w):
                 kc = tuple(int(x) for x in args.kcenter.split(","))
             elif wr.kc_k:
                 kc = (wr.kc_k, wr.kc_r)
-            extra["exact"] = run_exact(wr, lens, n_dec, K_steps, W_steps, qs, ks, vs, peak, kc)
+            extra["exact"] = run_exact(wr, lens, n_dec, min(K_steps, 200), W_steps, qs, ks, vs, peak, kc)
         except Exception as ex:  # report, do not hide
             extra["exact"] = {"error": str(ex)[:200]}
+    return {"value": value, "ms_per_step": ms_per_step, "repeats": R, "region_ms": region_ms, "clocks": clocks, "e2e": e2e,
+            "launches": int(launches), "roofline": roofline, "extra": extra, "lens": lens, "varlen": varlen}
+
+
+def ncu_traffic(kernel, wr):
+    """DRAM bytes of one launch of `kernel` from the tracked record of an ncu capture (profiles/ncu_traffic.json),
+    scaled by the units processed (units share nothing, so traffic grows in proportion). None when there is no
+    record for this kernel and workload, or when the kernel's source file has changed since the capture."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        rec = json.load(f).get(kernel)
+    if not rec or rec.get("workload") != wr.name:
+        return None
+    try:
+        with open(os.path.join(ROOT, rec["source"]), "rb") as f:
+            data = f.read()
+    except OSError:
+        return None
+    blob = hashlib.sha1(b"blob %d\0" % len(data) + data).hexdigest()      # what `git hash-object` prints
+    if blob != rec.get("source_blob"):
+        return None
+    return rec["dram_bytes"] * wr.units / rec["units"]
+
+
+def run_subgen(args, w):
+    from paper_2402_06082_b200 import build
+    build.build()
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    # weak scaling: every rank serves its own batch of B sequences (units are independent, no data-path collective)
+    wr = sharding.rank_workload(w, rank)
+    K_steps, W_steps = args.steps, args.warmup
+    res = measure(wr, args, K_steps, W_steps, world, rank, local, dist, True)
+    extra = res["extra"]
+    lens, varlen = res["lens"], res["varlen"]
+
+    # ---- the other workloads of the benchmark definition, one compact entry each (single GPU only) ----
+    if args.configs and world == 1 and not (args.prompt or args.batch or args.m_max or args.bounded):
+        table = {}
+        for name in ("cfg1", "cfg2", "cfg4b", "cfg4", "cfg5"):
+            if name == wr.name:
+                continue
+            try:
+                table[name] = measure(synth.CONFIGS[name], args, min(K_steps, 200), max(W_steps, 3), 1, 0, local, None, False)
+            except Exception as ex:  # report, do not hide
+                table[name] = {"error": str(ex)[:200]}
+            torch.cuda.empty_cache()
+        extra["configs"] = table
 
     cpu = None
     if rank == 0 and world == 1 and args.cpu_baseline:
@@ -448,10 +536,14 @@ def run_subgen(args, w):
                "prefill_tokens_per_s": r["prefill_tokens_per_s"]}
 
     if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world, "steps": K_steps, "warmup": W_steps,
-                "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        dt = wr.torch_dtype
+        reg = res["region_ms"]
+        line = {"metric": METRIC, "value": res["value"], "unit": "steps/s", "n_gpus": world, "steps": K_steps, "warmup": W_steps,
+                "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16" if dt == torch.bfloat16 else "f32", "data": "synthetic", "config": workload_config(wr),
-                "clocks": clk.summary(), "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+                "timed_regions": {"repeats": res["repeats"], "steps_each": K_steps, "statistic": "median",
+                                  "ms_per_step_min": min(reg) / K_steps, "ms_per_step_max": max(reg) / K_steps},
+                "clocks": res["clocks"], "e2e": res["e2e"], "gpu_launches": res["launches"], "roofline": res["roofline"],
                 "cpu_baseline": cpu, "extra": extra}
         print(json.dumps(line), flush=True)
     if dist:
@@ -554,6 +646,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=32)
     ap.add_argument("--no-exact", dest="exact", action="store_false")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--no-configs", dest="configs", action="store_false",
+                    help="skip the compact entries for the other workloads of the benchmark definition")
     ap.add_argument("--prompt", type=int, default=0, help="override the prompt length (smaller cases for profiling)")
     ap.add_argument("--batch", type=int, default=0, help="override the number of sequences")
     ap.add_argument("--multi-query", type=int, default=0,

@@ -226,8 +226,20 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
 
 // Launch with the programmatic stream serialization attribute: the kernel may be scheduled while its predecessor
 // in the stream still runs and orders itself with pdl_wait(). SUBGEN_PDL=0 falls back to ordinary launches.
+// plain = true launches the ordinary way (a full dependency on everything earlier in the stream): used for the
+// first kernel of a call when that kernel touches the caller's inputs before its dependency wait.
+// A failed launch is remembered in g_launch_err, which take_launch_error() returns and clears.
+thread_local cudaError_t g_launch_err = cudaSuccess;
+
+cudaError_t take_launch_error() {
+    cudaError_t e = g_launch_err;
+    g_launch_err = cudaSuccess;
+    const cudaError_t last = cudaGetLastError();
+    return e != cudaSuccess ? e : last;
+}
+
 template <typename... KArgs, typename... Args>
-void launch_pdl_smem(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+void launch_pdl_opt(bool plain, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
     static const bool off = [] { const char* e = getenv("SUBGEN_PDL"); return e && e[0] == '0'; }();
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
@@ -236,36 +248,42 @@ void launch_pdl_smem(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
-    cfg.numAttrs = off ? 0 : 1;
-    cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+    cfg.numAttrs = (off || plain) ? 0 : 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+    if (e != cudaSuccess && g_launch_err == cudaSuccess) g_launch_err = e;
+}
+template <typename... KArgs, typename... Args>
+void launch_pdl_smem(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    launch_pdl_opt(false, kern, grid, block, smem, st, args...);
 }
 template <typename... KArgs, typename... Args>
 void launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
-    launch_pdl_smem(kern, grid, block, 0, st, args...);
+    launch_pdl_opt(false, kern, grid, block, 0, st, args...);
 }
 
-// fp32 caches: CUDA-core dot products (full fp32 products). bf16 caches: tensor-core kernel.
+// The two query kernels of a bf16 handle for G columns. first_plain: the cluster scan is the first kernel of the
+// call (read-only queries) and loads the caller's q before its dependency wait, so it is launched the ordinary way.
+template <int D, int G>
+void launch_query_bf16(const Cache<__nv_bfloat16>& C, dim3 grid, dim3 grid_z, cudaStream_t st, const __nv_bfloat16* q,
+                       __nv_bfloat16* out, cudaEvent_t mid, int advance, int flat_ipu, int flat_slots, bool first_plain) {
+    launch_pdl_opt(first_plain, query_tau_kernel<D, G>, grid, dim3(kQmThreads), 0, st, C, q);
+    if (mid) cudaEventRecord(mid, st);
+    if (flat_ipu) launch_pdl(query_z_flat_kernel<D, G>, grid_z, dim3(kQmThreads), st, C, q, out, (int)grid.x, advance, flat_ipu, flat_slots);
+    else launch_pdl(query_z_kernel<D, G>, grid_z, dim3(kQmThreads), st, C, q, out, (int)grid.x, advance);
+}
+
+// fp32 caches: CUDA-core dot products (full fp32 products). bf16 caches: tensor-core kernels.
 template <typename T, int D>
 void launch_query(const Cache<T>& C, int G, dim3 grid, dim3 grid_z, cudaStream_t st, const void* q, void* out, cudaEvent_t mid, int advance = 1,
-                  int flat_ipu = 0, int flat_slots = 0) {
+                  int flat_ipu = 0, int flat_slots = 0, bool first_plain = false) {
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        const T* qq = (const T*)q;
+        T* oo = (T*)out;
         switch (G) {
-            case 1: launch_pdl(query_tau_kernel<D, 1>, grid, dim3(kQmThreads), st, C, (const T*)q);
-                    if (mid) cudaEventRecord(mid, st);
-                    if (flat_ipu) launch_pdl(query_z_flat_kernel<D, 1>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance, flat_ipu, flat_slots);
-                    else launch_pdl(query_z_kernel<D, 1>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
-            case 2: launch_pdl(query_tau_kernel<D, 2>, grid, dim3(kQmThreads), st, C, (const T*)q);
-                    if (mid) cudaEventRecord(mid, st);
-                    if (flat_ipu) launch_pdl(query_z_flat_kernel<D, 2>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance, flat_ipu, flat_slots);
-                    else launch_pdl(query_z_kernel<D, 2>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
-            case 4: launch_pdl(query_tau_kernel<D, 4>, grid, dim3(kQmThreads), st, C, (const T*)q);
-                    if (mid) cudaEventRecord(mid, st);
-                    if (flat_ipu) launch_pdl(query_z_flat_kernel<D, 4>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance, flat_ipu, flat_slots);
-                    else launch_pdl(query_z_kernel<D, 4>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
-            default: launch_pdl(query_tau_kernel<D, 8>, grid, dim3(kQmThreads), st, C, (const T*)q);
-                    if (mid) cudaEventRecord(mid, st);
-                     if (flat_ipu) launch_pdl(query_z_flat_kernel<D, 8>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance, flat_ipu, flat_slots);
-                    else launch_pdl(query_z_kernel<D, 8>, grid_z, dim3(kQmThreads), st, C, (const T*)q, (T*)out, (int)grid.x, advance); break;
+            case 1: launch_query_bf16<D, 1>(C, grid, grid_z, st, qq, oo, mid, advance, flat_ipu, flat_slots, first_plain); break;
+            case 2: launch_query_bf16<D, 2>(C, grid, grid_z, st, qq, oo, mid, advance, flat_ipu, flat_slots, first_plain); break;
+            case 4: launch_query_bf16<D, 4>(C, grid, grid_z, st, qq, oo, mid, advance, flat_ipu, flat_slots, first_plain); break;
+            default: launch_query_bf16<D, 8>(C, grid, grid_z, st, qq, oo, mid, advance, flat_ipu, flat_slots, first_plain); break;
         }
     } else {
         switch (G) {
@@ -334,7 +352,7 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
     const int flat_ipu = flat_value_scan(h, 1, &flat_grid);
     launch_query<T, D>(C, h->d.G, grid_t, flat_ipu ? dim3(flat_grid) : grid_z, h->st, q, out, e ? e[2] : nullptr, 1, flat_ipu, h->d.splits + 2);
     if (e) CUDA_TRY(cudaEventRecord(e[3], h->st));
-    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(take_launch_error());
     h->launches += std::is_same<T, __nv_bfloat16>::value ? 3 : 2;
     return SUBGEN_OK;
 }
@@ -348,8 +366,8 @@ int launch_query_only_td(subgen* h, const void* q, int nq, void* out) {
     const dim3 grid_t(h->d.sp_tau, h->d.U), grid_z(h->d.sp_z, h->d.U);
     int flat_grid = 0;
     const int flat_ipu = flat_value_scan(h, 0, &flat_grid);
-    launch_query<T, D>(C, C.G, grid_t, flat_ipu ? dim3(flat_grid) : grid_z, h->st, q, out, nullptr, 0, flat_ipu, h->d.splits + 2);
-    CUDA_TRY(cudaGetLastError());
+    launch_query<T, D>(C, C.G, grid_t, flat_ipu ? dim3(flat_grid) : grid_z, h->st, q, out, nullptr, 0, flat_ipu, h->d.splits + 2, true);
+    CUDA_TRY(take_launch_error());
     h->launches += std::is_same<T, __nv_bfloat16>::value ? 2 : 1;
     return SUBGEN_OK;
 }
@@ -365,7 +383,7 @@ int launch_prefill_td(subgen* h, const void* K, const void* V, int n, const int*
     Cache<T> C = make_cache<T>(h);
     if (C.bounded) prefill_seq_kernel<T, D, true><<<h->d.U, kPrefillThreads, 0, h->st>>>(C, (const T*)K, (const T*)V, n, cu_dev, total);
     else prefill_seq_kernel<T, D, false><<<h->d.U, kPrefillThreads, 0, h->st>>>(C, (const T*)K, (const T*)V, n, cu_dev, total);
-    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(take_launch_error());
     h->launches += 1;
     return SUBGEN_OK;
 }
@@ -440,14 +458,10 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         const int nchunks = (Lmax + kChunk - 1) / kChunk;
         prefill_mhist_kernel<<<(d.U + 255) / 256, 256, 0, h->st>>>(C, a, d.U);
         launches += 1;
-        static bool configured = false;
-        if (tc && !configured) {
-            CUDA_TRY(cudaFuncSetAttribute(prefill_score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes));
-            configured = true;
-        }
         for (int c = 0; c < nchunks; ++c) {
             // both kernels stage their chunk keys before they wait for their predecessor in the stream
-            if (tc) launch_pdl_smem(prefill_score_tc_kernel, dim3(slices, d.U), dim3(kTcThreads), kTcSmemBytes, h->st, C, a, c);
+            // chunk 0 reads the cluster-count history its immediate predecessor wrote before it waits: ordinary launch
+            if (tc) launch_pdl_opt(c == 0, prefill_score_tc_kernel, dim3(slices, d.U), dim3(kTcThreads), kTcSmemBytes, h->st, C, a, c);
             else prefill_score_kernel<D><<<dim3(slices, d.U), kScoreThreads, 0, h->st>>>(C, a, c);
             if (int rc = mark()) return rc;
             launch_pdl(prefill_resolve_kernel<D>, dim3(d.U), dim3(kResolveThreads), h->st, C, a, c);
@@ -463,7 +477,7 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
     prefill_finish_kernel<D><<<dim3(fx, d.U), 256, 0, h->st>>>(C, a);
     prefill_commit_kernel<<<(d.U + 255) / 256, 256, 0, h->st>>>(C, a, d.U);
     launches += 2;
-    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(take_launch_error());
     h->launches += launches;
     return SUBGEN_OK;
 }
@@ -540,6 +554,15 @@ subgen_t* subgen_create_ex(const subgen_config* cfg) {
         return nullptr;
     }
     h->n_host.assign(d.B, 0);
+    // the tcgen05 score kernel needs more dynamic shared memory than the default limit; the attribute is per device,
+    // so it is set for the device of every handle that can launch the kernel
+    if (cfg->dtype == SUBGEN_DTYPE_BF16 && d.D == 128 &&
+        cudaFuncSetAttribute(prefill_score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) != cudaSuccess) {
+        fail(SUBGEN_ECUDA, "subgen_create: cudaFuncSetAttribute failed: %s", cudaGetErrorString(cudaGetLastError()));
+        if (h->owns) cudaFree(h->ws);
+        delete h;
+        return nullptr;
+    }
     if (const char* env = getenv("SUBGEN_PREFILL")) { h->seq_prefill = strcmp(env, "seq") == 0; h->mma_score = strcmp(env, "mma") == 0; }
     if (h->cfg.bounded) {
         // merges renumber the clusters in the middle of a chunk, which the chunked prefill does not handle:
@@ -744,7 +767,7 @@ int subgen_cache_stats(subgen_t* h, subgen_stats* out) {
     CUDA_TRY(cudaMemsetAsync(dev, 0, 8 * sizeof(uint64_t), h->st));
     if (h->cfg.dtype == SUBGEN_DTYPE_FP32) stats_kernel<float><<<h->d.U, 256, 0, h->st>>>(make_cache<float>(h), h->d.U, dev);
     else stats_kernel<__nv_bfloat16><<<h->d.U, 256, 0, h->st>>>(make_cache<__nv_bfloat16>(h), h->d.U, dev);
-    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(take_launch_error());
     h->launches += 1;
     uint64_t r[8];
     CUDA_TRY(cudaMemcpyAsync(r, dev, sizeof r, cudaMemcpyDeviceToHost, h->st));
@@ -976,7 +999,7 @@ int exact_append_td(subgen_exact* h, const void* K, const void* V, int n, const 
     bx = bx < 1 ? 1 : (bx > 64 ? 64 : bx);
     exact_append_kernel<T, D><<<dim3(bx, h->U), 256, 0, h->st>>>(E, (const T*)K, (const T*)V, n, cu_dev, total);
     exact_advance_kernel<T><<<(h->U + 255) / 256, 256, 0, h->st>>>(E, h->U, n, cu_dev);
-    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(take_launch_error());
     h->launches += 2;
     return SUBGEN_OK;
 }
@@ -1000,7 +1023,7 @@ int exact_step_td(subgen_exact* h, const void* q, const void* k, const void* v, 
         case 4: exact_step_kernel<T, D, 4><<<grid, kQueryThreads, 0, h->st>>>(E, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
         default: exact_step_kernel<T, D, 8><<<grid, kQueryThreads, 0, h->st>>>(E, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
     }
-    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(take_launch_error());
     h->launches += 1;
     return SUBGEN_OK;
 }
@@ -1019,7 +1042,7 @@ int exact_step_mma(subgen_exact* h, const void* q, const void* k, const void* v,
         case 4: exact_mma_kernel<D, 4><<<grid, kQmThreads, 0, h->st>>>(E, (const T*)q, (T*)out); break;
         default: exact_mma_kernel<D, 8><<<grid, kQmThreads, 0, h->st>>>(E, (const T*)q, (T*)out); break;
     }
-    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(take_launch_error());
     h->launches += 1;
     return SUBGEN_OK;
 }
@@ -1174,7 +1197,7 @@ int kcenter_compress_td(subgen_exact* h, int k, int r, int k_iter, int keep_max,
     kcenter_gather_kernel<T, D><<<dim3(gx, h->U), 256, 0, h->st>>>(E, k, r, centres, Kt, Vt, tokt, keep_max);
     kcenter_scatter_kernel<T, D><<<dim3(gx, h->U), 256, 0, h->st>>>(E, k, r, Kt, Vt, tokt, keep_max);
     kcenter_commit_kernel<T><<<(h->U + 255) / 256, 256, 0, h->st>>>(E, h->U, k, r);
-    cudaError_t le = cudaGetLastError();
+    cudaError_t le = take_launch_error();
     cudaError_t se = cudaMemcpyAsync(h->kc_counters, counters, 16, cudaMemcpyDeviceToHost, h->st);
     if (se == cudaSuccess) se = cudaStreamSynchronize(h->st);
     cudaFree(scratch);
@@ -1374,6 +1397,6 @@ extern "C" int subgen_exact_attention_noalloc(const void* q, const void* K, cons
         if (f32) launch_attend_static<float, 128>(G, grid, st, q, K, V, out, n, H, Hkv, part, ticket);
         else launch_attend_static<__nv_bfloat16, 128>(G, grid, st, q, K, V, out, n, H, Hkv, part, ticket);
     }
-    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(take_launch_error());
     return SUBGEN_OK;
 }

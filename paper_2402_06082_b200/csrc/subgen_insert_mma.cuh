@@ -33,8 +33,10 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
     __shared__ int sm_last;
     const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, nw = nt >> 5, g = lane >> 2, tq = lane & 3;
-    pdl_trigger();
+    // The successor (the cluster scan) loads the call's queries before its own dependency wait, so it may only be
+    // scheduled once everything that precedes this call in the stream has completed: wait first, then trigger.
     pdl_wait();
+    pdl_trigger();
     const int n = C.n_unit[u], w = C.w;
     const uint4* knew_u = reinterpret_cast<const uint4*>(k_new + (size_t)u * D);
     const uint4* vnew_u = reinterpret_cast<const uint4*>(v_new + (size_t)u * D);

@@ -108,8 +108,13 @@ __global__ void __launch_bounds__(kTcThreads, 4) prefill_score_tc_kernel(Cache<_
     // Everything above touches only the chunk's keys. Tiles of 128 representatives are dealt to the blocks of the
     // unit round-robin. The resolve kernel of the previous chunk may still be running: it appends representatives
     // and never touches those that exist, so the tiles that lay entirely below the count the chunk before it left
-    // (ms_safe, written two kernels ago, read from L2) are scored at once; then the kernel waits for its
-    // predecessor and scores the rest with the final count.
+    // (m_safe, read from L2) are scored at once; then the kernel waits for its predecessor and scores the rest with
+    // the final count. Who wrote m_safe: for chunk c >= 2 the resolve kernel of chunk c - 2, which had completed
+    // before the score kernel of chunk c - 1 passed its own wait, and this kernel is scheduled only after every
+    // block of the resolve kernel of chunk c - 1 has passed its wait, which is later still. For chunk 1 the writer
+    // is the history-initialisation kernel, three launches back and complete for the same reason. For chunk 0 that
+    // kernel is the immediate predecessor, so chunk 0 is launched the ordinary way (the host does that), which makes
+    // everything earlier in the stream complete before this kernel starts.
     Best* outp = a.pbest + ((size_t)u * slices + blockIdx.x) * kChunk;
     const int m_safe = __ldcg(a.mhist + 2 * u + (chunk & 1));        // count after chunk - 2
     const int JA = m_safe / kTcTileN;                                  // tiles [0, JA) are final

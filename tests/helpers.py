@@ -47,6 +47,32 @@ def rel_err(got: np.ndarray, want: np.ndarray) -> float:
     return float(np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30))
 
 
+def out_ulp(want: np.ndarray, dtype) -> np.ndarray:
+    """One unit in the last place of the OUTPUT format at each wanted value (bf16: 8 significant bits; fp32: 24)."""
+    a = np.abs(np.asarray(want, np.float64))
+    bits = 8 if dtype == torch.bfloat16 else 24
+    e = np.floor(np.log2(np.maximum(a, 2.0 ** -126)))
+    return 2.0 ** (e - (bits - 1))
+
+
+def elem_err(got: np.ndarray, want: np.ndarray, dtype) -> float:
+    """Largest per-coordinate error in units of the tolerance: (|got_j - want_j| - ulp_j) / (tol * max_j |want_j|).
+    A norm can hide a wrong small coordinate under a few large ones; this cannot."""
+    got = np.asarray(got, np.float64); want = np.asarray(want, np.float64)
+    scale = TOL[dtype] * max(float(np.max(np.abs(want))), 1e-30)
+    return float(np.max((np.abs(got - want) - out_ulp(want, dtype)) / scale))
+
+
+def assert_output(got: np.ndarray, want: np.ndarray, dtype, where="") -> None:
+    """An output vector against the oracle's: relative L2 error within the tolerance of the dtype AND every
+    coordinate within tol * max|want| plus one unit in the last place of the output format."""
+    assert np.all(np.isfinite(np.asarray(got, np.float64))), "%s: non-finite output" % (where,)
+    r = rel_err(got, want)
+    assert r <= TOL[dtype], "%s: relative L2 error %.3g > %.3g" % (where, r, TOL[dtype])
+    e = elem_err(got, want, dtype)
+    assert e <= 1.0, "%s: a coordinate is off by %.3g x the per-element tolerance" % (where, e)
+
+
 def assert_rows_match_tokens(sg, seq, kvhead, gpu_state, K_unit: torch.Tensor, V_unit: torch.Tensor):
     """Stored vectors are bit copies of the input rows named by the token indices."""
     st = gpu_state

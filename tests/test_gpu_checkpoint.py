@@ -58,8 +58,8 @@ def test_resume_continues_the_stream(dtype, d):
             o.push(Kn[bb, h, i], Vn[bb, h, i])
             for g in range(G):
                 want = o.query(Qn[bb, h * G + g, i])
-                assert hp.rel_err(ob[bb, h * G + g], want) <= hp.TOL[w.torch_dtype]
-                assert hp.rel_err(oa[bb, h * G + g], want) <= hp.TOL[w.torch_dtype]
+                hp.assert_output(ob[bb, h * G + g], want, w.torch_dtype)
+                hp.assert_output(oa[bb, h * G + g], want, w.torch_dtype)
     want = sum(len(set(r.tolist())) for o in orcs.values() for r in o.slot_tok[o.counts > 1])
     assert a.cache_stats()["distinct_sample_rows"] == b.cache_stats()["distinct_sample_rows"] == want
     for (bb, h), o in orcs.items():

@@ -38,7 +38,7 @@ def test_evenly_cut_value_scan_matches_oracle(d, G, s, window, n0):
             o.push(f32(K[b, h, i]), f32(V[b, h, i]))
             for g in range(G):
                 err = hp.rel_err(out[b, h * G + g], o.query(f32(Q[b, h * G + g, i])))
-                assert err <= hp.TOL[torch.bfloat16], "step %d unit %s head %d: rel err %.3g" % (i, (b, h), g, err)
+                hp.assert_output(out[b, h * G + g], o.query(f32(Q[b, h * G + g, i])), torch.bfloat16, "step %d unit %s head %d: rel err %.3g" % (i, (b, h), g, err))
     # the read-only multi-query call takes the same path
     probes = Q[:, :, n0:n0 + 2].contiguous()
     got = f32(sg.query(probes))
@@ -46,5 +46,5 @@ def test_evenly_cut_value_scan_matches_oracle(d, G, s, window, n0):
         hp.assert_state_equal(sg.export_state(b, h), o, "unit %s" % ((b, h),))
         for g in range(G):
             for j in range(2):
-                assert hp.rel_err(got[b, h * G + g, j], o.query(f32(probes[b, h * G + g, j]))) <= hp.TOL[torch.bfloat16]
+                hp.assert_output(got[b, h * G + g, j], o.query(f32(probes[b, h * G + g, j])), torch.bfloat16)
     assert sg.status() == 0

@@ -184,7 +184,7 @@ def test_varlen_prefill_bf16():
         for (b, h), o in orcs.items():
             o.push(f32(k)[b, h], f32(v)[b, h])
             for g in range(G):
-                assert hp.rel_err(out[b, h * G + g], o.query(f32(q)[b, h * G + g])) <= hp.TOL[torch.bfloat16]
+                hp.assert_output(out[b, h * G + g], o.query(f32(q)[b, h * G + g]), torch.bfloat16)
     for (b, h), o in orcs.items():
         hp.assert_state_equal(sg.export_state(b, h), o, "varlen steps %s" % ((b, h),))
 
@@ -347,7 +347,7 @@ def test_exact_attention_matches_eq1(dtype, G):
         for b in range(w.B):
             for hq in range(w.H):
                 want = orc.exact_attention(Kn[b, hq // G, : i + 1], Vn[b, hq // G, : i + 1], Qn[b, hq, i])
-                assert hp.rel_err(out[b, hq], want) <= hp.TOL[w.torch_dtype]
+                hp.assert_output(out[b, hq], want, w.torch_dtype)
     assert ex.bytes_per_step() == 2 * w.B * w.Hkv * (n0 + nd) * w.d * (4 if dtype == "fp32" else 2)
     with pytest.raises(Exception):
         ex.step(Q[:, :, 0].contiguous(), K[:, :, 0].contiguous(), V[:, :, 0].contiguous())   # cache full
@@ -375,7 +375,8 @@ def test_exact_varlen_and_short_window_agreement():
             for hq in range(w.H):
                 want = orc.exact_attention(f32(streams[b][0])[hq // 2, : lens[b] + i + 1],
                                            f32(streams[b][1])[hq // 2, : lens[b] + i + 1], f32(q)[b, hq])
-                assert hp.rel_err(a[b, hq], want) <= 2e-2 and hp.rel_err(e[b, hq], want) <= 2e-2
+                hp.assert_output(a[b, hq], want, torch.bfloat16)
+                hp.assert_output(e[b, hq], want, torch.bfloat16)
 
 
 # ------------------------------------------------------------------------------------------- full size
@@ -419,7 +420,7 @@ def test_benchmark_workload_full_size_sampled_units():
             Kh, Vh, Qh = host[(b, h)]
             orcs[(b, h)].push(Kh[n0 + i], Vh[n0 + i])
             err = hp.rel_err(out[b, h], orcs[(b, h)].query(Qh[n0 + i]))
-            assert err <= hp.TOL[torch.bfloat16], "step %d unit %s: %.3g" % (i, (b, h), err)
+            hp.assert_output(out[b, h], orcs[(b, h)].query(Qh[n0 + i]), torch.bfloat16, "step %d unit %s: %.3g" % (i, (b, h), err))
     for bh in sample:
         hp.assert_state_equal(sg.export_state(*bh), orcs[bh], "full-size steps unit %s" % (bh,))
     assert sg.status() == 0
@@ -443,7 +444,7 @@ def test_odd_sample_counts_and_unaligned_units(t, m_max, bounded):
         out = f32(sg.step(Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous()))
         for h, o in orcs.items():
             o.push(f32(K[0, h, i]), f32(V[0, h, i]))
-            assert hp.rel_err(out[0, h], o.query(f32(Q[0, h, i]))) <= hp.TOL[torch.bfloat16]
+            hp.assert_output(out[0, h], o.query(f32(Q[0, h, i])), torch.bfloat16)
     want = 0
     for h, o in orcs.items():
         hp.assert_state_equal(sg.export_state(0, h), o, "unit %d" % h)

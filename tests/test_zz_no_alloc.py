@@ -6,7 +6,10 @@ synchronisation. For them the library offers one exact-attention call whose scra
 the library image. This test calls it through the C ABI twice in a row, with different shapes so that the
 second call finds the first call's leftovers in the shared array, and checks both results against the
 handle-based exact path (subgen_exact_append + subgen_exact_step), within the tolerances of the other
-GPU tests. It is collected last on purpose.
+GPU tests, and on a few (sequence, head) pairs also against the CPU oracle's statement of Eq. 1. The cases
+cover every branch of the kernel: several blocks per unit with the arrival counter, a single block per unit
+(fewer than 64 tokens), group sizes 1, 4 and 8, both element types and both head dimensions. It is collected
+last on purpose.
 """
 import ctypes
 import os
@@ -47,10 +50,23 @@ def _rel(a, b):
     return float(((a - b).norm(dim=-1) / b.norm(dim=-1).clamp_min(1e-30)).max())
 
 
+def _check_against_oracle(B, H, Hkv, d, n, dtype, q, K, V, out):
+    """Eq. 1 from the CPU oracle for the first and the last head of the first and the last sequence."""
+    import helpers as hp
+    from oracle import subgen_oracle as orc
+    G = H // Hkv
+    for b in sorted({0, B - 1}):
+        for hq in sorted({0, H - 1}):
+            want = orc.exact_attention(hp.f32(K[b, hq // G]), hp.f32(V[b, hq // G]), hp.f32(q[b, hq]))
+            hp.assert_output(hp.f32(out[b, hq]), want, dtype, "no-alloc entry point vs oracle, seq %d head %d" % (b, hq))
+
+
 def test_two_calls_in_a_row_match_the_handle_based_path():
     from paper_2402_06082_b200 import binding
     L = binding.load()
-    cases = [(2, 8, 2, 128, 3001, torch.bfloat16, 1), (3, 4, 4, 64, 517, torch.float32, 2)]
+    cases = [(2, 8, 2, 128, 3001, torch.bfloat16, 1), (3, 4, 4, 64, 517, torch.float32, 2),
+             (2, 2, 2, 128, 40, torch.bfloat16, 3),       # fewer than 64 tokens: one block per unit, no arrival counter
+             (1, 16, 2, 64, 700, torch.bfloat16, 4)]      # eight query heads per KV head
     for (B, H, Hkv, d, n, dtype, seed) in cases:
         q, K, V = _case(B, H, Hkv, d, n, dtype, seed)
         out = torch.full((B, H, d), float("nan"), dtype=dtype, device="cuda")
@@ -61,6 +77,7 @@ def test_two_calls_in_a_row_match_the_handle_based_path():
         want = _reference(B, H, Hkv, d, n, dtype, q, K, V)
         assert torch.isfinite(out).all()
         assert _rel(out, want) <= TOL[dtype]
+        _check_against_oracle(B, H, Hkv, d, n, dtype, q, K, V, out)
     # same call again on the first shape: the array now holds the second call's leftovers
     B, H, Hkv, d, n, dtype, seed = cases[0]
     q, K, V = _case(B, H, Hkv, d, n, dtype, seed)
