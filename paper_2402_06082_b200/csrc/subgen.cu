@@ -16,6 +16,7 @@
 #include "subgen_insert_mma.cuh"
 #include "subgen_prefill.cuh"
 #include "subgen_score_tc.cuh"
+#include "subgen_prefill_persist.cuh"
 #include "subgen_exact_mma.cuh"
 #include "subgen_kcenter.cuh"
 
@@ -183,6 +184,10 @@ struct subgen {
     size_t scratch_bytes = 0;
     bool seq_prefill = false;     // SUBGEN_PREFILL=seq: token-by-token prefill also for bf16
     bool mma_score = false;       // SUBGEN_PREFILL=mma: chunk scoring with warp-level MMAs instead of tcgen05 (d = 128)
+    int persist = -1;             // key phase as one persistent kernel (d = 128): -1 chosen from the unit count,
+                                  // 0 / 1 forced by SUBGEN_PREFILL=chunk / persist
+    bool pf_persist = false;      // the most recent profiled prefill used the persistent kernel
+    unsigned long long* pf_phase_dev = nullptr;   // its per-unit phase times (inside scratch)
 };
 
 namespace {
@@ -412,7 +417,8 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         const size_t b_w = align_up((size_t)d.U * Lmax * 8), b_m = align_up((size_t)d.U * d.s * 4);
         const size_t b_p = align_up((size_t)d.U * slices * kChunk * sizeof(Best));
         const size_t b_h = align_up((size_t)d.U * 2 * sizeof(int));
-        const size_t need = 3 * b_w + b_m + b_p + b_h;
+        const size_t b_ns = align_up((size_t)d.U * kPpPhases * sizeof(unsigned long long));
+        const size_t need = 3 * b_w + b_m + b_p + b_h + b_ns;
         if (need > h->scratch_bytes) {
             if (h->scratch) { CUDA_TRY(cudaStreamSynchronize(h->st)); CUDA_TRY(cudaFree(h->scratch)); h->scratch = nullptr; h->scratch_bytes = 0; }
             cudaError_t e = cudaMalloc((void**)&h->scratch, need);
@@ -425,6 +431,7 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         a.Mwin = (int*)(h->scratch + 3 * b_w);
         a.pbest = (Best*)(h->scratch + 3 * b_w + b_m);
         a.mhist = (int*)(h->scratch + 3 * b_w + b_m + b_p);
+        unsigned long long* phase_ns = (unsigned long long*)(h->scratch + 3 * b_w + b_m + b_p + b_h);
         auto mark = [&]() -> int {                       // profiling: one event on the stream
             if (!h->prof) return SUBGEN_OK;
             if (h->pev_used == h->pev.size()) {
@@ -455,19 +462,31 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         prefill_gather_kernel<D><<<dim3(gx, d.U), 256, 0, h->st>>>(C, a);
         launches += 4;
         if (int rc = mark()) return rc;
-        const int nchunks = (Lmax + kChunk - 1) / kChunk;
-        prefill_mhist_kernel<<<(d.U + 255) / 256, 256, 0, h->st>>>(C, a, d.U);
-        launches += 1;
-        for (int c = 0; c < nchunks; ++c) {
-            // both kernels stage their chunk keys before they wait for their predecessor in the stream
-            // chunk 0 reads the cluster-count history its immediate predecessor wrote before it waits: ordinary launch
-            if (tc) launch_pdl_opt(c == 0, prefill_score_tc_kernel, dim3(slices, d.U), dim3(kTcThreads), kTcSmemBytes, h->st, C, a, c);
-            else prefill_score_kernel<D><<<dim3(slices, d.U), kScoreThreads, 0, h->st>>>(C, a, c);
+        // Key phase. Many units with few representatives each: one persistent block per unit walks its chunks
+        // (subgen_prefill_persist.cuh). Few units: a score and a resolve kernel per chunk, the representatives of a
+        // unit spread over many blocks.
+        const bool persist = tc && (h->persist >= 0 ? h->persist == 1 : d.U >= 24);
+        h->pf_persist = persist && h->prof;
+        if (persist) {
+            h->pf_phase_dev = phase_ns;
+            prefill_keys_persist_kernel<<<d.U, kPpThreads, kPpSmemBytes, h->st>>>(C, a, h->prof ? phase_ns : nullptr);
+            launches += 1;
             if (int rc = mark()) return rc;
-            launch_pdl(prefill_resolve_kernel<D>, dim3(d.U), dim3(kResolveThreads), h->st, C, a, c);
-            if (int rc = mark()) return rc;
+        } else {
+            const int nchunks = (Lmax + kChunk - 1) / kChunk;
+            prefill_mhist_kernel<<<(d.U + 255) / 256, 256, 0, h->st>>>(C, a, d.U);
+            launches += 1;
+            for (int c = 0; c < nchunks; ++c) {
+                // both kernels stage their chunk keys before they wait for their predecessor in the stream;
+                // chunk 0 reads the cluster-count history its immediate predecessor wrote before it waits: ordinary launch
+                if (tc) launch_pdl_opt(c == 0, prefill_score_tc_kernel, dim3(slices, d.U), dim3(kTcThreads), kTcSmemBytes, h->st, C, a, c);
+                else prefill_score_kernel<D><<<dim3(slices, d.U), kScoreThreads, 0, h->st>>>(C, a, c);
+                if (int rc = mark()) return rc;
+                launch_pdl(prefill_resolve_kernel<D>, dim3(d.U), dim3(kResolveThreads), h->st, C, a, c);
+                if (int rc = mark()) return rc;
+            }
+            launches += 2 * nchunks;
         }
-        launches += 2 * nchunks;
     }
     int longest = 0;
     for (int b = 0; b < d.B; ++b) longest = add[b] > longest ? add[b] : longest;
@@ -557,13 +576,18 @@ subgen_t* subgen_create_ex(const subgen_config* cfg) {
     // the tcgen05 score kernel needs more dynamic shared memory than the default limit; the attribute is per device,
     // so it is set for the device of every handle that can launch the kernel
     if (cfg->dtype == SUBGEN_DTYPE_BF16 && d.D == 128 &&
-        cudaFuncSetAttribute(prefill_score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) != cudaSuccess) {
+        (cudaFuncSetAttribute(prefill_score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) != cudaSuccess ||
+         cudaFuncSetAttribute(prefill_keys_persist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPpSmemBytes) != cudaSuccess)) {
         fail(SUBGEN_ECUDA, "subgen_create: cudaFuncSetAttribute failed: %s", cudaGetErrorString(cudaGetLastError()));
         if (h->owns) cudaFree(h->ws);
         delete h;
         return nullptr;
     }
-    if (const char* env = getenv("SUBGEN_PREFILL")) { h->seq_prefill = strcmp(env, "seq") == 0; h->mma_score = strcmp(env, "mma") == 0; }
+    if (const char* env = getenv("SUBGEN_PREFILL")) {
+        h->seq_prefill = strcmp(env, "seq") == 0; h->mma_score = strcmp(env, "mma") == 0;
+        if (strcmp(env, "chunk") == 0) h->persist = 0;
+        if (strcmp(env, "persist") == 0) h->persist = 1;
+    }
     if (h->cfg.bounded) {
         // merges renumber the clusters in the middle of a chunk, which the chunked prefill does not handle:
         // bounded handles insert their prompts token by token
@@ -821,12 +845,31 @@ int subgen_profile_prefill_read(subgen_t* h, double* ms) {
         float x = 0;
         CUDA_TRY(cudaEventElapsedTime(&x, h->pev[0], h->pev[1]));
         acc[0] = x;
-        for (size_t i = 1; i + 2 < h->pev_used; i += 2) {       // chunk: events i -> i+1 (score) -> i+2 (resolve)
-            float sc = 0, rs = 0;
-            CUDA_TRY(cudaEventElapsedTime(&sc, h->pev[i], h->pev[i + 1]));
-            CUDA_TRY(cudaEventElapsedTime(&rs, h->pev[i + 1], h->pev[i + 2]));
-            acc[1] += sc;
-            acc[2] += rs;
+        if (h->pf_persist && h->pev_used >= 3) {
+            // one kernel for all chunks: its wall time, split in the proportion of the time the units' blocks spent
+            // scoring (staging included) and resolving
+            float wall = 0;
+            CUDA_TRY(cudaEventElapsedTime(&wall, h->pev[1], h->pev[2]));
+            std::vector<unsigned long long> ns((size_t)h->d.U * kPpPhases);
+            CUDA_TRY(cudaMemcpy(ns.data(), h->pf_phase_dev, ns.size() * 8, cudaMemcpyDeviceToHost));
+            double ph[kPpPhases] = {0};
+            for (int u = 0; u < h->d.U; ++u)
+                for (int i = 0; i < kPpPhases; ++i) ph[i] += (double)ns[(size_t)kPpPhases * u + i];
+            const double sc = ph[0] + ph[1] + ph[2] + ph[3] + ph[4], rs = ph[5] + ph[6] + ph[7];
+            if (getenv("SUBGEN_TRACE"))
+                fprintf(stderr, "subgen prefill phases (share of block time): stage %.3f wait %.3f readback %.3f store+issue %.3f "
+                        "follow-up %.3f | openings %.3f ranks+coins %.3f writes %.3f; mean block cycles %.0f\n",
+                        ph[0] / (sc + rs), ph[1] / (sc + rs), ph[2] / (sc + rs), ph[3] / (sc + rs), ph[4] / (sc + rs),
+                        ph[5] / (sc + rs), ph[6] / (sc + rs), ph[7] / (sc + rs), (sc + rs) / h->d.U);
+            if (sc + rs > 0) { acc[1] = wall * sc / (sc + rs); acc[2] = wall * rs / (sc + rs); }
+        } else {
+            for (size_t i = 1; i + 2 < h->pev_used; i += 2) {       // chunk: events i -> i+1 (score) -> i+2 (resolve)
+                float sc = 0, rs = 0;
+                CUDA_TRY(cudaEventElapsedTime(&sc, h->pev[i], h->pev[i + 1]));
+                CUDA_TRY(cudaEventElapsedTime(&rs, h->pev[i + 1], h->pev[i + 2]));
+                acc[1] += sc;
+                acc[2] += rs;
+            }
         }
     }
     if (ms) { ms[0] = acc[0]; ms[1] = acc[1]; ms[2] = acc[2]; }

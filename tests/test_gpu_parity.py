@@ -158,7 +158,9 @@ def test_empty_prefill_and_zero_values():
     hp.assert_state_equal(sg.export_state(0, 0), o, "after zero value")
 
 
-def test_varlen_prefill_bf16():
+@pytest.mark.parametrize("mode", ["chunk", "persist"])
+def test_varlen_prefill_bf16(mode, monkeypatch):
+    monkeypatch.setenv("SUBGEN_PREFILL", mode)
     w = synth.CFG5.scaled(B=3, H=4, Hkv=2, ncomp=16, s=64, window=32, m_max=256)
     lens = [5, 333, 90]
     n_dec = 6
@@ -293,27 +295,31 @@ def test_chunked_prefill_equals_token_by_token_prefill(monkeypatch):
     b = _sg(w)
     monkeypatch.setenv("SUBGEN_PREFILL", "mma")  # chunk scoring with warp-level MMAs
     c = _sg(w)
+    monkeypatch.setenv("SUBGEN_PREFILL", "persist")  # all chunks of a call in one persistent kernel (tcgen05)
+    p = _sg(w)
     monkeypatch.delenv("SUBGEN_PREFILL")
     for lo, hi in ((0, 7), (7, 300), (300, 301), (301, 1000)):
-        for sg in (a, b, c):
+        for sg in (a, b, c, p):
             sg.prefill(K[:, :, lo:hi].contiguous(), V[:, :, lo:hi].contiguous())
         for bb in range(w.B):
             for h in range(w.Hkv):
                 s2 = b.export_state(bb, h)
                 hp.assert_rows_match_tokens(b, bb, h, s2, K[bb, h], V[bb, h])
-                for sg in (a, c):
+                for sg in (a, c, p):
                     s1 = sg.export_state(bb, h)
                     for key in ("m", "mu", "n", "last_cluster", "last_opened", "status"):
                         assert s1[key] == s2[key], (key, lo, hi)
                     for key in ("counts", "centre_tok", "slot_tok", "m_tok", "m_w"):
                         np.testing.assert_array_equal(s1[key], s2[key], err_msg="%s after [%d,%d)" % (key, lo, hi))
                     hp.assert_rows_match_tokens(sg, bb, h, s1, K[bb, h], V[bb, h])
-    assert a.launch_count > b.launch_count
+    assert a.launch_count > p.launch_count > b.launch_count
 
 
-def test_tcgen05_scoring_many_tiles_and_dense_candidates():
+@pytest.mark.parametrize("mode", ["chunk", "persist"])
+def test_tcgen05_scoring_many_tiles_and_dense_candidates(mode, monkeypatch):
     """Several 128-representative tiles per chunk, and a radius so large that every pair is inside the guard band
-    (the exhaustive path of the score kernel): state must equal the oracle's."""
+    (the exhaustive path of the score kernel): state must equal the oracle's. Both tcgen05 prefill paths."""
+    monkeypatch.setenv("SUBGEN_PREFILL", mode)
     w = synth.CFG3.scaled(B=1, H=2, Hkv=2, n_prompt=2500, ncomp=400, s=64, t=4, window=16, m_max=1024)
     _run_stream(w, 2500, 4)
     w = synth.CFG2.scaled(B=1, H=1, Hkv=1, n_prompt=600, ncomp=4, sigma=0.5, delta=30.0, s=32, t=4, window=8, m_max=64)
@@ -321,8 +327,10 @@ def test_tcgen05_scoring_many_tiles_and_dense_candidates():
     assert orcs[(0, 0)].m == 1
 
 
-def test_prefill_capacity_overflow_is_reported():
+@pytest.mark.parametrize("mode", ["chunk", "persist"])
+def test_prefill_capacity_overflow_is_reported(mode, monkeypatch):
     from paper_2402_06082_b200 import binding
+    monkeypatch.setenv("SUBGEN_PREFILL", mode)
     w = synth.CFG3.scaled(B=1, H=2, Hkv=2, n_prompt=400, ncomp=64, s=32, window=8, m_max=16)
     K, V, _ = synth.batch_stream(w, 400, "cuda")
     sg = _sg(w)

@@ -38,9 +38,13 @@ def _draw(seed):
 
 
 @pytest.mark.parametrize("seed", list(range(40)))
-def test_random_configuration(seed):
+def test_random_configuration(seed, monkeypatch):
     from paper_2402_06082_b200.binding import SubGen
     c = _draw(seed)
+    # unbounded bf16 handles with d = 128 have two prefill paths (a score and a resolve kernel per chunk, or one
+    # persistent kernel per call); the default picks by unit count, so odd seeds force the persistent one
+    if seed % 2:
+        monkeypatch.setenv("SUBGEN_PREFILL", "persist")
     B, Hkv, G, d, t, s, window = c["B"], c["Hkv"], c["G"], c["d"], c["t"], c["s"], c["window"]
     w = synth.CFG3.scaled(B=B, H=Hkv * G, Hkv=Hkv, d=d, dtype=c["dtype"], n_prompt=c["n0"], ncomp=c["ncomp"], s=s, window=window,
                           m_max=c["m_max"], t=t, delta=c["delta"], philox_seed=c["philox"], data_seed=seed)
