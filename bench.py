@@ -386,7 +386,10 @@ def measure(wr, args, K_steps, W_steps, world, rank, local, dist, headline):
 
     cbytes, vbytes, ibytes = avg("cluster_bytes"), avg("value_bytes"), avg("insert_bytes")
     c_ms, v_ms, i_ms = tau_ms / max(nprof, 1), z_ms / max(nprof, 1), ins_ms / max(nprof, 1)
-    if v_ms > 0:
+    nk = sg.step_kernels
+    if nk == 1:                         # the whole step is one kernel
+        dom = ("step_fused_kernel", cbytes + vbytes + ibytes, c_ms)
+    elif v_ms > 0:
         dom = ("query_tau_kernel", cbytes, c_ms) if c_ms >= v_ms else ("query_z_kernel", vbytes, v_ms)
     else:
         dom = ("query_kernel", cbytes + vbytes, c_ms)
@@ -402,15 +405,16 @@ def measure(wr, args, K_steps, W_steps, world, rank, local, dist, headline):
         return {"units": wr.units, "steps_per_s": value, "ms_per_step": ms_per_step, "repeats": R,
                 "ms_per_step_min": min(region_ms) / K_steps, "ms_per_step_max": max(region_ms) / K_steps,
                 "step_bytes": step_bytes, "step_GBps": step_gbs, "frac_of_hbm_peak": step_gbs / peak if step_gbs else None,
-                "kernel_ms": {"insert": i_ms, "cluster_scan": c_ms, "value_scan": v_ms},
-                "prefill_ms": prefill_ms, "prefill_tokens_per_s": sum(lens) / (prefill_ms * 1e-3) if sum(lens) else None,
+                "kernel_ms": {"step_fused": c_ms} if nk == 1 else {"insert": i_ms, "cluster_scan": c_ms, "value_scan": v_ms},
+                "step_kernels": nk, "prefill_ms": prefill_ms, "prefill_tokens_per_s": sum(lens) / (prefill_ms * 1e-3) if sum(lens) else None,
                 "e2e_steps_per_s": e2e["value"], "gpu_launches_per_region": int(launches), "clocks": clocks,
                 "clusters_per_unit": stats1["clusters"] / wr.units}
     traffic = ncu_traffic(dom[0], wr) if not args.prompt else None
     roofline = {"bound": "hbm", "kernel": dom[0], "achieved": achieved, "peak": peak, "peak_source": which,
                 "unit": "GB/s", "frac": achieved / peak if achieved else None, "traffic": traffic,
                 "algorithmic_bytes_per_launch": dom[1], "ms_per_launch": dom[2],
-                "kernels": {"insert": {"algorithmic_bytes_per_launch": ibytes, "ms_per_launch": i_ms, "achieved": gbs(ibytes, i_ms)},
+                "kernels": {"step_fused": {"algorithmic_bytes_per_launch": dom[1], "ms_per_launch": c_ms, "achieved": gbs(dom[1], c_ms)}} if nk == 1 else
+                           {"insert": {"algorithmic_bytes_per_launch": ibytes, "ms_per_launch": i_ms, "achieved": gbs(ibytes, i_ms)},
                             "cluster_scan": {"algorithmic_bytes_per_launch": cbytes, "ms_per_launch": c_ms, "achieved": gbs(cbytes, c_ms),
                                              # for comparison: all t sample slots of every cluster, repeats included
                                              "bytes_with_repeated_slots": nominal_c, "achieved_with_repeated_slots": gbs(nominal_c, c_ms)},

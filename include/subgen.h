@@ -81,7 +81,14 @@ typedef struct subgen_config {
     int nq_max;             /* most queries per head one subgen_query call may carry; 0 = 1; (H / Hkv) * nq_max <= 8 */
     int bounded;            /* 0: Algorithm 1 as printed, m_max is a capacity (exceeding it is an error);
                              * 1: m_max is a budget, see "Bounded-m variant" below */
+    int step_mode;          /* how subgen_step runs on bf16 handles: SUBGEN_STEP_AUTO (0) picks by the number of
+                             * units, SUBGEN_STEP_FUSED one kernel per step, SUBGEN_STEP_SPLIT three kernels
+                             * (insertion, cluster scan, value scan). Same results either way. */
 } subgen_config;
+
+#define SUBGEN_STEP_AUTO 0
+#define SUBGEN_STEP_FUSED 1
+#define SUBGEN_STEP_SPLIT 2
 
 /* Bounded-m variant (subgen_config.bounded = 1). Algorithm 1 keeps as many clusters as the keys need; the
  * paper bounds their number only through its clusterability assumption and names the incremental clustering of
@@ -207,6 +214,9 @@ int subgen_profile_prefill_read(subgen_t* h, double ms[3]);
 
 /* Number of kernels this handle has launched so far. */
 uint64_t subgen_launch_count(const subgen_t* h);
+/* Kernels one subgen_step launches on this handle: 1 (fused step: its whole duration is reported in ms[1] of
+ * subgen_profile_read, ms[0] and ms[2] are 0), 2 (fp32) or 3. */
+int subgen_step_kernels(const subgen_t* h);
 
 /* Checkpoint and resume. The paper describes a stream that never stops; a serving process has to move a
  * conversation between GPUs or survive a restart, so the state between two calls (D with its samples and counts, M

@@ -18,12 +18,13 @@ LIB_PATH = os.path.join(_HERE, "libsubgen.so")
 
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 ST_CAPACITY, ST_RANGE = 1, 2
+STEP_MODES = {"auto": 0, "fused": 1, "split": 2}
 
 EXPORTS = [
     "subgen_workspace_bytes", "subgen_create", "subgen_create_ex", "subgen_destroy", "subgen_prefill",
     "subgen_prefill_varlen", "subgen_step", "subgen_step_host", "subgen_status", "subgen_export_state",
     "subgen_export_rows", "subgen_cache_stats", "subgen_profile_enable", "subgen_profile_read", "subgen_profile_prefill_read",
-    "subgen_query", "subgen_launch_count", "subgen_last_error", "subgen_checkpoint_bytes", "subgen_checkpoint_save", "subgen_checkpoint_load", "subgen_exact_create", "subgen_exact_destroy",
+    "subgen_query", "subgen_launch_count", "subgen_step_kernels", "subgen_last_error", "subgen_checkpoint_bytes", "subgen_checkpoint_save", "subgen_checkpoint_load", "subgen_exact_create", "subgen_exact_destroy",
     "subgen_exact_append", "subgen_exact_append_varlen", "subgen_exact_step", "subgen_exact_bytes",
     "subgen_exact_launch_count", "subgen_exact_attention_noalloc",
     "subgen_exact_kcenter_compress", "subgen_exact_kcenter_counters", "subgen_exact_export_tokens",
@@ -34,7 +35,7 @@ class SubgenConfig(C.Structure):
     _fields_ = [("B", C.c_int), ("H", C.c_int), ("Hkv", C.c_int), ("d", C.c_int), ("delta", C.c_float),
                 ("t", C.c_int), ("s", C.c_int), ("window", C.c_int), ("seed", C.c_uint64), ("dtype", C.c_int),
                 ("m_max", C.c_int), ("splits", C.c_int), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-                ("stream", C.c_void_p), ("nq_max", C.c_int), ("bounded", C.c_int)]
+                ("stream", C.c_void_p), ("nq_max", C.c_int), ("bounded", C.c_int), ("step_mode", C.c_int)]
 
 
 class StateView(C.Structure):
@@ -83,6 +84,7 @@ def load():
     L.subgen_profile_read.argtypes = [vp, C.POINTER(C.c_double), ip]
     L.subgen_profile_prefill_read.argtypes = [vp, C.POINTER(C.c_double)]
     L.subgen_launch_count.argtypes = [vp]
+    L.subgen_step_kernels.argtypes = [vp]
     L.subgen_query.argtypes = [vp, vp, C.c_int, vp]
     L.subgen_checkpoint_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
     L.subgen_checkpoint_save.argtypes = [vp, vp, C.c_size_t, C.POINTER(C.c_size_t)]
@@ -136,7 +138,8 @@ class SubGen:
     """One library handle: the SubGen caches of B sequences x Hkv KV heads on the current CUDA device."""
 
     def __init__(self, B, H, d, delta, t, s, window, seed=0, *, Hkv=None, dtype=torch.bfloat16, m_max=0, splits=0,
-                 stream: Optional[torch.cuda.Stream] = None, bounded: bool = False, nq_max: int = 1):
+                 stream: Optional[torch.cuda.Stream] = None, bounded: bool = False, nq_max: int = 1,
+                 step_mode: str = "auto"):
         self._L = load()
         self._h = None
         if not torch.cuda.is_available():
@@ -146,7 +149,8 @@ class SubGen:
         self.t, self.s, self.window, self.dtype = int(t), int(s), int(window), dtype
         self.stream = stream or torch.cuda.current_stream()
         cfg = SubgenConfig(self.B, self.H, self.Hkv, self.d, float(delta), self.t, self.s, self.window, int(seed),
-                           _dtype_code(dtype), int(m_max), int(splits), None, 0, self.stream.cuda_stream, int(nq_max), int(bool(bounded)))
+                           _dtype_code(dtype), int(m_max), int(splits), None, 0, self.stream.cuda_stream, int(nq_max), int(bool(bounded)),
+                           STEP_MODES[step_mode])
         nbytes = self._L.subgen_workspace_bytes(C.byref(cfg))
         if nbytes == 0:
             raise SubgenError(self._L.subgen_last_error().decode())
@@ -255,6 +259,11 @@ class SubGen:
     @property
     def launch_count(self) -> int:
         return int(self._L.subgen_launch_count(self._h))
+
+    @property
+    def step_kernels(self) -> int:
+        """Kernels one step launches: 1 (fused step), 2 (fp32) or 3."""
+        return _check(self._L.subgen_step_kernels(self._h))
 
     def checkpoint_save(self) -> torch.Tensor:
         """The state between two calls as one pinned uint8 host tensor (see subgen_checkpoint_save)."""

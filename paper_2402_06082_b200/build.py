@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsubgen.so")
 SOURCES = ["subgen.cu"]
-HEADERS = ["subgen_device.cuh", "subgen_kernels.cuh", "subgen_query_mma.cuh", "subgen_insert_mma.cuh", "subgen_prefill.cuh", "subgen_score_tc.cuh", "subgen_prefill_persist.cuh", "subgen_exact_mma.cuh", "subgen_kcenter.cuh", os.path.join("..", "..", "include", "subgen.h")]
+HEADERS = ["subgen_device.cuh", "subgen_kernels.cuh", "subgen_query_mma.cuh", "subgen_insert_mma.cuh", "subgen_step_fused.cuh", "subgen_prefill.cuh", "subgen_score_tc.cuh", "subgen_prefill_persist.cuh", "subgen_exact_mma.cuh", "subgen_kcenter.cuh", os.path.join("..", "..", "include", "subgen.h")]
 
 
 def _stale() -> bool:

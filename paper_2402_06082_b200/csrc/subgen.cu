@@ -14,6 +14,7 @@
 #include "subgen_kernels.cuh"
 #include "subgen_query_mma.cuh"
 #include "subgen_insert_mma.cuh"
+#include "subgen_step_fused.cuh"
 #include "subgen_prefill.cuh"
 #include "subgen_score_tc.cuh"
 #include "subgen_prefill_persist.cuh"
@@ -58,6 +59,7 @@ struct Dims {
     int B, H, Hkv, G, D, t, s, w, m_max, splits, U;
     int Gs;                        // columns the query scratch is sized for: G * max(1, nq_max)
     int sp_insert, sp_tau, sp_z;   // blocks per unit of the three step kernels (splits = their maximum)
+    int sp_fused;                  // blocks per unit of the one-kernel step
     size_t E;   // bytes per element
 };
 
@@ -79,6 +81,7 @@ bool resolve(const subgen_config* c, Dims* o, const char** why) {
     if (d.m_max < 1) { *why = "m_max must be positive"; return false; }
     if (!(c->delta >= 0.f) || !isfinite(c->delta) || c->delta > 32768.f) { *why = "delta must be finite, in [0, 32768]"; return false; }
     if (c->dtype != SUBGEN_DTYPE_FP32 && c->dtype != SUBGEN_DTYPE_BF16) { *why = "unknown dtype"; return false; }
+    if (c->step_mode < SUBGEN_STEP_AUTO || c->step_mode > SUBGEN_STEP_SPLIT) { *why = "unknown step_mode"; return false; }
     if ((long long)d.B * d.Hkv > 65535) { *why = "B * Hkv must be <= 65535"; return false; }
     d.E = c->dtype == SUBGEN_DTYPE_FP32 ? 4 : 2;
     d.U = d.B * d.Hkv;
@@ -108,6 +111,14 @@ bool resolve(const subgen_config* c, Dims* o, const char** why) {
     }
     d.splits = d.sp_insert > d.sp_tau ? d.sp_insert : d.sp_tau;
     if (d.sp_z > d.splits) d.splits = d.sp_z;
+    // one-kernel step: 256-thread blocks, two per SM, one resident wave
+    d.sp_fused = c->splits ? c->splits : (148 * 2) / d.U;
+    d.sp_fused = d.sp_fused < 1 ? 1 : (d.sp_fused > 64 ? 64 : d.sp_fused);
+    if (const char* env = getenv("SUBGEN_FUSED_SPLITS")) {
+        const int a = atoi(env);
+        if (a > 0 && a <= 128) d.sp_fused = a;
+    }
+    if (d.sp_fused > d.splits) d.splits = d.sp_fused;
     *o = d;
     return true;
 }
@@ -187,6 +198,7 @@ struct subgen {
     int persist = -1;             // key phase as one persistent kernel (d = 128): -1 chosen from the unit count,
                                   // 0 / 1 forced by SUBGEN_PREFILL=chunk / persist
     bool pf_persist = false;      // the most recent profiled prefill used the persistent kernel
+    bool fused = false;           // stream steps run as one kernel (bf16, not bounded): few units, or SUBGEN_STEP=fused
     unsigned long long* pf_phase_dev = nullptr;   // its per-unit phase times (inside scratch)
 };
 
@@ -346,6 +358,20 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
         CUDA_TRY(cudaEventRecord(e[0], h->st));
     }
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        if (h->fused) {
+            const dim3 grid_f(h->d.sp_fused, h->d.U);
+            if (e) CUDA_TRY(cudaEventRecord(e[1], h->st));          // the whole step is reported as the middle interval
+            switch (h->d.G) {
+                case 1: launch_pdl(step_fused_kernel<D, 1>, grid_f, dim3(kFsThreads), h->st, C, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
+                case 2: launch_pdl(step_fused_kernel<D, 2>, grid_f, dim3(kFsThreads), h->st, C, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
+                case 4: launch_pdl(step_fused_kernel<D, 4>, grid_f, dim3(kFsThreads), h->st, C, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
+                default: launch_pdl(step_fused_kernel<D, 8>, grid_f, dim3(kFsThreads), h->st, C, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
+            }
+            if (e) { CUDA_TRY(cudaEventRecord(e[2], h->st)); CUDA_TRY(cudaEventRecord(e[3], h->st)); }
+            CUDA_TRY(take_launch_error());
+            h->launches += 1;
+            return SUBGEN_OK;
+        }
         if (C.bounded) launch_pdl(insert_mma_kernel<D, true>, grid_i, dim3(kInsertMmaThreads), h->st, C, (const T*)k, (const T*)v);
         else launch_pdl(insert_mma_kernel<D, false>, grid_i, dim3(kInsertMmaThreads), h->st, C, (const T*)k, (const T*)v);
     } else {
@@ -587,6 +613,16 @@ subgen_t* subgen_create_ex(const subgen_config* cfg) {
         h->seq_prefill = strcmp(env, "seq") == 0; h->mma_score = strcmp(env, "mma") == 0;
         if (strcmp(env, "chunk") == 0) h->persist = 0;
         if (strcmp(env, "persist") == 0) h->persist = 1;
+    }
+    // Stream steps as one kernel when the units are too few for the three-kernel chain to hide its own latency
+    // (SUBGEN_STEP=fused / split forces either way). Bounded handles and fp32 handles keep their kernels.
+    const bool can_fuse = cfg->dtype == SUBGEN_DTYPE_BF16 && !cfg->bounded;
+    h->fused = can_fuse && d.U <= 148;
+    if (cfg->step_mode == SUBGEN_STEP_FUSED) h->fused = can_fuse;
+    if (cfg->step_mode == SUBGEN_STEP_SPLIT) h->fused = false;
+    if (const char* env = getenv("SUBGEN_STEP")) {
+        if (strcmp(env, "fused") == 0) h->fused = can_fuse;
+        if (strcmp(env, "split") == 0) h->fused = false;
     }
     if (h->cfg.bounded) {
         // merges renumber the clusters in the middle of a chunk, which the chunked prefill does not handle:
@@ -878,6 +914,11 @@ int subgen_profile_prefill_read(subgen_t* h, double* ms) {
 }
 
 uint64_t subgen_launch_count(const subgen_t* h) { return h ? h->launches : 0; }
+
+int subgen_step_kernels(const subgen_t* h) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_step_kernels: handle is NULL");
+    return h->cfg.dtype == SUBGEN_DTYPE_FP32 ? 2 : (h->fused ? 1 : 3);
+}
 
 }  // extern "C"
 

@@ -329,59 +329,64 @@ __device__ void make_room(const Cache<T>& C, int u, int e, const uint4* krow, Be
 }
 
 // ---------------------------------------------------------------------------------------------
-// Insert token e (key/value rows already in shared memory) into D and M of unit u, given the nearest
-// representative. Executed by a whole block; ends with a __syncthreads(). Returns the new m.
-//   UpdateSoftmaxNormalizer: join (count, t coins) or open (representative, count 1; the t copies are
-//   implied while n_i = 1 and written out when the second member arrives);
-//   UpdateMatrixProduct: s coins with the OLD mu; then mu += W.
-template <typename T, int D, bool BND = false>
-__device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, const uint4* krow, const uint4* vrow,
-                            unsigned long long* sm_w /* shared, 2 elements */) {
+// Insertion of token e (key/value rows already in shared memory) into D and M of unit u, in three parts that the
+// step's insertion kernel runs one after the other in one block (apply_insert) and that the fused step kernel
+// spreads over its blocks.
+
+// W(v_e), ||k_e||^2 (whole row and packed head, fp32) and the input range check. Called by ONE warp; leaves
+// sm_w[0] = W and sm_w[1] = {||k||^2, ||k head||^2} in shared memory (visible to the block after a barrier).
+template <typename T, int D>
+__device__ __forceinline__ void token_weights(const Cache<T>& C, int u, const uint4* krow, const uint4* vrow,
+                                              unsigned long long* sm_w) {
     constexpr int EPL = Elem<T>::EPL, LPR = D / EPL;
-    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5;
-    const int t = C.t, s = C.s;
-
-    // W(v_e) and the input range check, by warp 0
-    if (warp == 0) {
-        unsigned long long acc = 0;
-        float kk = 0.f, kh = 0.f;
-        bool bad = false;
-        for (int p = lane; p < LPR; p += 32) {
-            float vf[EPL], kf[EPL];
-            Elem<T>::unpack(vrow[p], vf);
-            Elem<T>::unpack(krow[p], kf);
-            float part = 0.f;
+    const int lane = threadIdx.x & 31;
+    unsigned long long acc = 0;
+    float kk = 0.f, kh = 0.f;
+    bool bad = false;
+    for (int p = lane; p < LPR; p += 32) {
+        float vf[EPL], kf[EPL];
+        Elem<T>::unpack(vrow[p], vf);
+        Elem<T>::unpack(krow[p], kf);
+        float part = 0.f;
 #pragma unroll
-            for (int j = 0; j < EPL; ++j) {
-                acc += fx_sq(vf[j]);
-                part = fmaf(kf[j], kf[j], part);
-                bad |= !(fabsf(vf[j]) <= kMaxAbsInput) || !(fabsf(kf[j]) <= kMaxAbsInput);
-            }
-            kk += part;
-            if (p < kHeadDims / EPL) kh += part;
+        for (int j = 0; j < EPL; ++j) {
+            acc += fx_sq(vf[j]);
+            part = fmaf(kf[j], kf[j], part);
+            bad |= !(fabsf(vf[j]) <= kMaxAbsInput) || !(fabsf(kf[j]) <= kMaxAbsInput);
         }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            acc += __shfl_xor_sync(0xffffffffu, acc, off);
-            kk += __shfl_xor_sync(0xffffffffu, kk, off);
-            kh += __shfl_xor_sync(0xffffffffu, kh, off);
-        }
-        bad = __any_sync(0xffffffffu, bad);
-        if (lane == 0) {
-            sm_w[0] = acc;
-            sm_w[1] = (unsigned long long)__float_as_uint(kk) | ((unsigned long long)__float_as_uint(kh) << 32);
-            if (bad) atomicOr(&C.status[u], 2);
-        }
+        kk += part;
+        if (p < kHeadDims / EPL) kh += part;
     }
-    __syncthreads();
-    const unsigned long long W = sm_w[0];
-    const unsigned long long mu_old = C.mu[u];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        kk += __shfl_xor_sync(0xffffffffu, kk, off);
+        kh += __shfl_xor_sync(0xffffffffu, kh, off);
+    }
+    bad = __any_sync(0xffffffffu, bad);
+    if (lane == 0) {
+        sm_w[0] = acc;
+        sm_w[1] = (unsigned long long)__float_as_uint(kk) | ((unsigned long long)__float_as_uint(kh) << 32);
+        if (bad) atomicOr(&C.status[u], 2);
+    }
+}
 
+// UpdateSoftmaxNormalizer for token e given its nearest representative: join (count, t coins) or open
+// (representative, count 1; the t copies are implied while n_i = 1 and written out when the second member
+// arrives). Executed by a whole block after token_weights and a barrier. Returns the new m; join / full report
+// what happened (full: the key needed a new cluster and none was free). On bounded handles best and m are
+// replaced by the placement under the threshold in force after make_room.
+template <typename T, int D, bool BND = false>
+__device__ int apply_cluster(const Cache<T>& C, int u, int e, Best& best, int& m, const uint4* krow,
+                             const unsigned long long* sm_w, bool& join, bool& full) {
+    constexpr int EPL = Elem<T>::EPL, LPR = D / EPL;
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int t = C.t;
     if constexpr (BND) {
         if (!((m > 0) && (best.d2 <= C.thr2[u])) && m >= C.m_max) make_room<T, D>(C, u, e, krow, best, m);
     }
-    const bool join = (m > 0) && (best.d2 <= threshold2<BND>(C, u));
-    const bool full = !join && (m >= C.m_max);
+    join = (m > 0) && (best.d2 <= threshold2<BND>(C, u));
+    full = !join && (m >= C.m_max);
     T* Xu = C.X + (size_t)u * C.m_max * D;
     T* Su = C.S + (size_t)u * C.m_max * t * D;
     int* cntu = C.cnt + (size_t)u * C.m_max;
@@ -422,26 +427,48 @@ __device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, c
     } else if (tid == 0) {
         atomicOr(&C.status[u], 1);
     }
+    return m_new;
+}
+
+// M slot i takes (k_e, v_e) with weight W. One thread.
+template <typename T, int D>
+__device__ __forceinline__ void store_value_sample(const Cache<T>& C, int u, int i, int e, unsigned long long W,
+                                                   const uint4* krow, const uint4* vrow) {
+    constexpr int LPR = D / Elem<T>::EPL;
+    uint4* dk = reinterpret_cast<uint4*>(C.Mk + ((size_t)u * C.s + i) * D);
+    uint4* dv = reinterpret_cast<uint4*>(C.Mv + ((size_t)u * C.s + i) * D);
+    for (int p = 0; p < LPR; ++p) { dk[p] = krow[p]; dv[p] = vrow[p]; }
+    C.MW[(size_t)u * C.s + i] = W;
+    C.MinvW[(size_t)u * C.s + i] = 1.f / (float)W;
+    C.Mtok[(size_t)u * C.s + i] = e;
+}
+
+// Insert token e into D and M of unit u, given the nearest representative. Executed by a whole block; ends with
+// a __syncthreads(). Returns the new m.
+//   UpdateSoftmaxNormalizer: apply_cluster;
+//   UpdateMatrixProduct: s coins with the OLD mu; then mu += W.
+template <typename T, int D, bool BND = false>
+__device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, const uint4* krow, const uint4* vrow,
+                            unsigned long long* sm_w /* shared, 2 elements */) {
+    const int tid = threadIdx.x, nt = blockDim.x, warp = tid >> 5;
+    const int s = C.s;
+    if (warp == 0) token_weights<T, D>(C, u, krow, vrow, sm_w);
+    __syncthreads();
+    const unsigned long long W = sm_w[0];
+    const unsigned long long mu_old = C.mu[u];
+    bool join, full;
+    const int m_new = apply_cluster<T, D, BND>(C, u, e, best, m, krow, sm_w, join, full);
 
     // UpdateMatrixProduct: slot i flips its own coin; winners copy (k_e, v_e)
     if (W > 0) {
         const unsigned long long tot = mu_old + W;
-        T* Mku = C.Mk + (size_t)u * s * D;
-        T* Mvu = C.Mv + (size_t)u * s * D;
         for (int blk = tid; blk * 4 < s; blk += nt) {
             const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)blk, 1u), C.key0, C.key1);
             const uint32_t words[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const int i = blk * 4 + q;
-                if (i < s && coin_value(words[q], tot, W)) {
-                    uint4* dk = reinterpret_cast<uint4*>(Mku + (size_t)i * D);
-                    uint4* dv = reinterpret_cast<uint4*>(Mvu + (size_t)i * D);
-                    for (int p = 0; p < LPR; ++p) { dk[p] = krow[p]; dv[p] = vrow[p]; }
-                    C.MW[(size_t)u * s + i] = W;
-                    C.MinvW[(size_t)u * s + i] = 1.f / (float)W;
-                    C.Mtok[(size_t)u * s + i] = e;
-                }
+                if (i < s && coin_value(words[q], tot, W)) store_value_sample<T, D>(C, u, i, e, W, krow, vrow);
             }
         }
     }

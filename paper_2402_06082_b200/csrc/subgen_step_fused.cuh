@@ -1,0 +1,499 @@
+// One-kernel stream step for bf16 caches (main loop of Algorithm 1: UpdateSoftmaxNormalizer, UpdateMatrixProduct,
+// mu update, QueryStreamAttn; window of Section 3.2).
+//
+// The three-kernel step (insertion, cluster scan, value scan) is a chain of dependent launches: the query must see
+// the state after the insertion. With few (sequence, KV head) units each of those kernels is short and the chain
+// itself is the cost. Here one grid does the whole step in one pass over the state as it was BEFORE the insertion,
+// and nobody waits for anybody:
+//
+//   every block   loads the queries, the token e that leaves the window and W(v_e); scans its slice of the packed
+//                 representative heads for the nearest representative of k_e (as insert_mma_kernel does); then takes
+//                 items from the unit's queue: 16 clusters (partition function), 16 slots of M, 16 window rows
+//   M             which slots of M the token e replaces depends only on (seed, unit, e, slot, mu, W): the warp that
+//                 scans a tile of M flips the tile's 16 coins itself, scores (k_e, v_e) with weight mu/(s W_e) in place
+//                 of a replaced slot and writes the slot. No other warp touches that slot in this step.
+//   window        the row the new token (k, v) will take is scored from the call's input instead of from the ring
+//   last block    (arrival ticket) merges the slices' nearest representatives, decides join / open, and corrects the
+//                 partition function for the one cluster that changes: it scores that cluster's t sample rows (or its
+//                 representative) and k_e, and adds  new contribution - old contribution  as one more partial;
+//                 then it applies the cluster update, stores the new token in the window, merges all partials and
+//                 writes out = z / tau.
+//
+// mu after the insertion (mu + W_e) is known from the start, so the scan weights M with the final mu.
+#pragma once
+#include "subgen_insert_mma.cuh"
+
+namespace sgk {
+
+constexpr int kFsThreads = 256;
+constexpr int kFsWarps = kFsThreads / 32;
+
+// Scores of one 16-row tile against q without the softmax bookkeeping: sc = (row g, head 2tq), (g, 2tq+1),
+// (g+8, 2tq), (g+8, 2tq+1).
+template <int D>
+__device__ __forceinline__ void tile_raw_scores(const uint4 (&ka)[D / 32], const uint4 (&kb)[D / 32], const uint32_t (&qb)[D / 32][4],
+                                                float (&sc)[4]) {
+    sc[0] = sc[1] = sc[2] = sc[3] = 0.f;
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+        mma_bf16_16816(sc, ka[c].x, kb[c].x, ka[c].y, kb[c].y, qb[c][0], qb[c][1]);
+        mma_bf16_16816(sc, ka[c].z, kb[c].z, ka[c].w, kb[c].w, qb[c][2], qb[c][3]);
+    }
+}
+
+template <int D, int G>
+__global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ q,
+                                                                  const __nv_bfloat16* __restrict__ k_new,
+                                                                  const __nv_bfloat16* __restrict__ v_new,
+                                                                  __nv_bfloat16* __restrict__ out) {
+    typedef __nv_bfloat16 T;
+    constexpr int NC = D / 32, LPR = D / 8, STR = D + 2, NW = kFsWarps;
+    // During the scan every warp keeps the row list of its item here; afterwards the same bytes hold the warps'
+    // partials [warp][G][D+2].
+    constexpr int kListBytes = NW * (16 * 64 + 2 * kTauRows * 4);
+    constexpr int kPartBytes = NW * G * STR * 4;
+    constexpr int kScratchBytes = kListBytes > kPartBytes ? kListBytes : kPartBytes;
+    __shared__ __align__(16) unsigned char scratch[kScratchBytes];
+    __shared__ uint4 krow[LPR], vrow[LPR];
+    __shared__ Best smb[32];
+    __shared__ unsigned long long sm_w[2];
+    __shared__ float psc[65][8];          // last block: raw scores of the changing cluster's rows and of k_e
+    __shared__ float sred[16];
+    __shared__ int sm_last;
+    const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5, g = lane >> 2, tq = lane & 3;
+    const int b = u / C.Hkv, kvh = u % C.Hkv;
+    const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;
+    // The call's inputs may come from the kernel that precedes this one in the stream: everything waits for it.
+    pdl_wait();
+    pdl_trigger();
+
+    uint32_t qb[NC][4];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        uint4 r = make_uint4(0, 0, 0, 0);
+        if (g < G) r = ldg16(q + (qrow0 + g) * D + c * 32 + tq * 8);
+        qb[c][0] = r.x; qb[c][1] = r.y; qb[c][2] = r.z; qb[c][3] = r.w;
+    }
+    const int n = C.n_unit[u], m = C.m_unit[u];
+    const unsigned long long mu_old = C.mu[u];
+    const int w = C.w, s = C.s, t = C.t;
+    const bool has_ins = n >= w;                     // a token leaves the window (w = 0: the new token itself)
+    const int e = n - w;
+    const int slot = w ? n % w : 0;
+    const T* knew_u = k_new + (size_t)u * D;
+    const T* vnew_u = v_new + (size_t)u * D;
+    const T* kE = w ? C.ringK + ((size_t)u * w + slot) * D : knew_u;      // rows of the token that leaves
+    const T* vE = w ? C.ringV + ((size_t)u * w + slot) * D : vnew_u;
+    if (has_ins) {
+        if (tid < LPR) krow[tid] = reinterpret_cast<const uint4*>(kE)[tid];
+        else if (tid < 2 * LPR) vrow[tid - LPR] = reinterpret_cast<const uint4*>(vE)[tid - LPR];
+    }
+    __syncthreads();
+    if (has_ins && warp == 0) token_weights<T, D>(C, u, krow, vrow, sm_w);
+    __syncthreads();
+    const unsigned long long W = has_ins ? sm_w[0] : 0ull;
+    const unsigned long long tot = mu_old + W;       // mu after this step's insertion
+
+    const T* Xu = C.X + (size_t)u * C.m_max * D;
+    const T* Su = C.S + (size_t)u * C.m_max * t * D;
+    const int* cntu = C.cnt + (size_t)u * C.m_max;
+
+    // ---- nearest representative of k_e over this block's slice of the packed heads ----
+    Best bst;
+    bst.d2 = ~0ull; bst.idx = INT_MAX; bst.pad = 0;
+    if (has_ins) {
+        if (m > 0) {
+            const T* Xhu = C.Xh + (size_t)u * C.m_max * kHeadDims;
+            const float* xhnu = C.xhn + (size_t)u * C.m_max;
+            uint32_t kb0[4];
+            float kn = 0.f;
+            {
+                const uint4 r = krow[tq];
+                float f[8];
+                Elem<T>::unpack(r, f);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) kn = fmaf(f[j], f[j], kn);
+                kb0[0] = g == 0 ? r.x : 0u; kb0[1] = g == 0 ? r.y : 0u;
+                kb0[2] = g == 0 ? r.z : 0u; kb0[3] = g == 0 ? r.w : 0u;
+            }
+            kn += __shfl_xor_sync(0xffffffffu, kn, 1);
+            kn += __shfl_xor_sync(0xffffffffu, kn, 2);
+            const float d2f = (float)((double)C.delta2_fx * (1.0 / 4294967296.0));
+            const int per = (((m + splits - 1) / splits) + 15) & ~15;       // slices are whole tiles
+            const int c0 = blockIdx.x * per, c1 = min(m, c0 + per);
+            auto exact_row = [&](int row) {                                  // exact D2 of one flagged row, by the warp
+                unsigned long long acc = 0;
+                if (lane < LPR) {
+                    float xf[8], kf[8];
+                    Elem<T>::unpack(*reinterpret_cast<const uint4*>(Xu + (size_t)row * D + lane * 8), xf);
+                    Elem<T>::unpack(krow[lane], kf);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc += fx_sqdiff(xf[j], kf[j]);
+                }
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+                if (better(acc, row, bst)) { bst.d2 = acc; bst.idx = row; }
+            };
+            constexpr int kTiles = 2;
+            for (int base = c0 + warp * 16 * kTiles; base < c1; base += NW * 16 * kTiles) {
+                uint4 ha[kTiles], hc[kTiles];
+                float xa[kTiles], xb[kTiles];
+#pragma unroll
+                for (int i = 0; i < kTiles; ++i) {
+                    const int ra = base + i * 16 + g, rb = ra + 8;
+                    const bool va = ra < c1, vb = rb < c1;
+                    ha[i] = ldg16(Xhu + (size_t)(va ? ra : c1 - 1) * kHeadDims + tq * 8);
+                    hc[i] = ldg16(Xhu + (size_t)(vb ? rb : c1 - 1) * kHeadDims + tq * 8);
+                    xa[i] = va ? xhnu[ra] : 0.f;
+                    xb[i] = vb ? xhnu[rb] : 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < kTiles; ++i) {
+                    const int ra = base + i * 16 + g, rb = ra + 8;
+                    float sc[4] = {0.f, 0.f, 0.f, 0.f};
+                    mma_bf16_16816(sc, ha[i].x, hc[i].x, ha[i].y, hc[i].y, kb0[0], kb0[1]);
+                    mma_bf16_16816(sc, ha[i].z, hc[i].z, ha[i].w, hc[i].w, kb0[2], kb0[3]);
+                    const float na = xa[i] + kn, nb = xb[i] + kn;
+                    const bool fa = ra < c1 && tq == 0 && (na - 2.f * sc[0]) <= d2f + 1.220703125e-4f * na;
+                    const bool fb = rb < c1 && tq == 0 && (nb - 2.f * sc[2]) <= d2f + 1.220703125e-4f * nb;
+                    unsigned ma = __ballot_sync(0xffffffffu, fa), mb = __ballot_sync(0xffffffffu, fb);
+                    while (ma) { exact_row(base + i * 16 + ((__ffs(ma) - 1) >> 2)); ma &= ma - 1; }
+                    while (mb) { exact_row(base + i * 16 + 8 + ((__ffs(mb) - 1) >> 2)); mb &= mb - 1; }
+                }
+            }
+        }
+        bst = block_best(bst, smb);
+        if (tid == 0) C.part1[(size_t)u * splits + blockIdx.x] = bst;
+    }
+
+    // ---- scan of the state as it stands before the insertion ----
+    MmaState<D> S;
+    S.m0 = S.m1 = -INFINITY;
+    S.tau0 = S.tau1 = 0.f;
+#pragma unroll
+    for (int j = 0; j < D / 16; ++j) S.acc[j][0] = S.acc[j][1] = S.acc[j][2] = S.acc[j][3] = 0.f;
+    {
+        unsigned* als = reinterpret_cast<unsigned*>(scratch) + warp * (16 * 64 / 4);
+        int* rix = reinterpret_cast<int*>(scratch + NW * 16 * 64) + warp * kTauRows;
+        float* rwt = reinterpret_cast<float*>(scratch + NW * (16 * 64 + kTauRows * 4)) + warp * kTauRows;
+        const unsigned char* ndu = C.ndist + (size_t)u * C.m_max;
+        const unsigned char* alias_bytes = C.alias + (size_t)u * C.m_max * t;
+        const unsigned* alias_words = (reinterpret_cast<uintptr_t>(alias_bytes) & 3) ? nullptr : reinterpret_cast<const unsigned*>(alias_bytes);
+        const float inv_t = 1.f / (float)t;
+        const int gsz = t <= 16 ? 16 : 256 / t;
+        const T* Mku = C.Mk + (size_t)u * s * D;
+        const T* Mvu = C.Mv + (size_t)u * s * D;
+        const float* MiWu = C.MinvW + (size_t)u * s;
+        const T* Rk = C.ringK + (size_t)u * w * D;
+        const T* Rv = C.ringV + (size_t)u * w * D;
+        const float mu_over_s = (float)tot / (float)s;
+        const float inv_we = W ? 1.f / (float)W : 0.f;
+        const int wn = min(n + 1, w);
+        const int n_a = (m + 15) >> 4, n_b = (s + 15) >> 4, n_c = (wn + 15) >> 4, total = n_a + n_b + n_c;
+        int item = 0;
+        if (lane == 0) item = (int)atomicAdd(&C.qnext[u], 1u);
+        item = __shfl_sync(0xffffffffu, item, 0);
+        while (item < total) {
+            int next = 0;
+            if (lane == 0) next = (int)atomicAdd(&C.qnext[u], 1u);     // asked for early, needed late
+            if (item < n_a) {
+                // 16 clusters -> one list of rows: the distinct samples of every cluster with n' > 1, each weighted
+                // n'/t times the number of slots that hold it, then the representatives of the singletons
+                const int c = item * 16 + lane;
+                const int cn = (lane < 16 && c < m) ? cntu[c] : 0;
+                const int nd = (lane < 16 && c < m) ? (int)ndu[c] : 0;
+                if (alias_words) {
+                    for (int i = lane; i < 4 * t; i += 32) als[i] = alias_words[(size_t)item * 4 * t + i];
+                } else {
+                    unsigned char* dst = reinterpret_cast<unsigned char*>(als);
+                    for (int i = lane; i < 16 * t; i += 32) dst[i] = alias_bytes[(size_t)item * 16 * t + i];
+                }
+                for (int p0 = 0; p0 < 16; p0 += gsz) {
+                    const bool act = lane >= p0 && lane < p0 + gsz;
+                    const int ndl = (act && cn > 1) ? nd : 0;
+                    int incl = ndl;
+#pragma unroll
+                    for (int off = 1; off < 16; off <<= 1) {
+                        const int v = __shfl_up_sync(0xffffffffu, incl, off);
+                        if (lane >= off) incl += v;
+                    }
+                    const int rows_m = __shfl_sync(0xffffffffu, incl, 15);
+                    const unsigned ms = __ballot_sync(0xffffffffu, act && cn == 1);
+                    const int rows = rows_m + __popc(ms);
+                    __syncwarp();
+                    if (ndl) {
+                        const unsigned char* al = reinterpret_cast<const unsigned char*>(als) + lane * t;
+                        const float wc = (float)cn * inv_t;
+                        for (int k = 0; k < ndl; ++k) {
+                            const int ee = al[k];
+                            const int sl = t <= 16 ? (ee & 15) : ee, copies = t <= 16 ? (ee >> 4) + 1 : 1;
+                            rix[incl - ndl + k] = c * t + sl;
+                            rwt[incl - ndl + k] = wc * (float)copies;
+                        }
+                    }
+                    if (act && cn == 1) {
+                        const int r = rows_m + __popc(ms & ((1u << lane) - 1u));
+                        rix[r] = c | (int)0x80000000;
+                        rwt[r] = 1.f;
+                    }
+                    __syncwarp();
+                    auto resolve = [&](int r, const T*& ptr, float& wgt) -> bool {
+                        ptr = Xu;
+                        wgt = 1.f;
+                        if (r < rows) {
+                            const int ix = rix[r];
+                            ptr = ix < 0 ? Xu + (size_t)(ix & 0x7fffffff) * D : Su + (size_t)ix * D;
+                            wgt = rwt[r];
+                        }
+                        return r < rows;
+                    };
+                    for (int r0 = 0; r0 < rows; r0 += 16) {
+                        const T *pa, *pb;
+                        float wa, wb;
+                        const bool va = resolve(r0 + g, pa, wa), vb = resolve(r0 + g + 8, pb, wb);
+                        uint4 ka[NC], kb[NC];
+                        load_keys<D>(pa, pb, tq, ka, kb);
+                        float p[4];
+                        tile_scores<D, D>(S, ka, kb, va, vb, qb, p);
+                        S.tau0 += wa * p[0] + wb * p[2];
+                        S.tau1 += wa * p[1] + wb * p[3];
+                    }
+                    __syncwarp();
+                }
+            } else {
+                // 16 value samples (weight mu/(s W), numerator only) or 16 window rows (weight 1, both sums)
+                const bool isM = item < n_a + n_b;
+                const int base = (isM ? item - n_a : item - n_a - n_b) * 16;
+                const int lim = isM ? s : wn;
+                const T* Kb = isM ? Mku : Rk;
+                const T* Vb = isM ? Mvu : Rv;
+                const int ia = min(base + g, lim - 1), ib = min(base + g + 8, lim - 1);
+                bool va = base + g < lim, vb = base + g + 8 < lim;
+                const int iv[4] = {min(base + 2 * tq, lim - 1), min(base + 2 * tq + 1, lim - 1), min(base + 2 * tq + 8, lim - 1),
+                                   min(base + 2 * tq + 9, lim - 1)};
+                const T* pka = Kb + (size_t)ia * D;
+                const T* pkb = Kb + (size_t)ib * D;
+                const T* pv[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) pv[i] = Vb + (size_t)iv[i] * D;
+                float wa_in = 1.f, wb_in = 1.f;
+                unsigned sub = 0;                     // rows of this tile that are scored from another place
+                if (isM) {
+                    wa_in = MiWu[ia];                 // 1/W, 0 for a null slot
+                    wb_in = MiWu[ib];
+                } else if (w && slot >= base && slot < base + 16) {
+                    // the new token's row: not in the ring yet, read from the call's input
+                    sub = 1u << (slot - base);
+                    if (ia == slot) pka = knew_u;
+                    if (ib == slot) pkb = knew_u;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) if (iv[i] == slot) pv[i] = vnew_u;
+                }
+                uint4 ka[NC], kb[NC], v[4][D / 64];
+                load_keys<D>(pka, pkb, tq, ka, kb);                  // keys and values in flight together
+                load_values<D>(pv, g, v);
+                if (isM && W > 0) {
+                    // UpdateMatrixProduct for the 16 slots of this tile: four Philox blocks, flipped while the rows
+                    // are on their way; a slot that takes the leaving token is scored from that token's rows
+                    unsigned nib = 0;
+                    if (lane < 4) {
+                        const int blk = (base >> 2) + lane;
+                        if (blk * 4 < s) {
+                            const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)blk, 1u), C.key0, C.key1);
+                            const uint32_t words[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                            for (int qq = 0; qq < 4; ++qq)
+                                if (blk * 4 + qq < s && coin_value(words[qq], tot, W)) nib |= 1u << qq;
+                        }
+                    }
+                    sub = __shfl_sync(0xffffffffu, nib, 0) | (__shfl_sync(0xffffffffu, nib, 1) << 4) |
+                          (__shfl_sync(0xffffffffu, nib, 2) << 8) | (__shfl_sync(0xffffffffu, nib, 3) << 12);
+                    if (sub) {                        // rare: about s / (tokens inserted) slots per step
+                        if ((sub >> g) & 1u) { wa_in = inv_we; for (int c = 0; c < NC; ++c) ka[c] = ldg16(kE + c * 32 + tq * 8); }
+                        if ((sub >> (g + 8)) & 1u) { wb_in = inv_we; for (int c = 0; c < NC; ++c) kb[c] = ldg16(kE + c * 32 + tq * 8); }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int r = 2 * tq + (i & 1) + (i >> 1) * 8;
+                            if ((sub >> r) & 1u)
+                                for (int cc = 0; cc < D / 64; ++cc) v[i][cc] = ldg16(vE + cc * 64 + g * 8);
+                        }
+                    }
+                }
+                float wza = 1.f, wzb = 1.f;
+                if (isM) {
+                    va = va && wa_in != 0.f;
+                    vb = vb && wb_in != 0.f;
+                    wza = va ? mu_over_s * wa_in : 0.f;
+                    wzb = vb ? mu_over_s * wb_in : 0.f;
+                }
+                float p[4];
+                tile_scores<D, D>(S, ka, kb, va, vb, qb, p);
+                if (!isM) {
+                    S.tau0 += p[0] + p[2];
+                    S.tau1 += p[1] + p[3];
+                }
+                const float pz[4] = {wza * p[0], wza * p[1], wzb * p[2], wzb * p[3]};
+                tile_values<D>(S, pz, v, g, tq);
+                if (isM && sub) {                     // the replaced slots take (k_e, v_e): half a warp per row
+                    unsigned todo = sub;
+                    while (todo) {
+                        const int i = base + __ffs(todo) - 1;
+                        todo &= todo - 1;
+                        if (lane < LPR) reinterpret_cast<uint4*>(C.Mk + ((size_t)u * s + i) * D)[lane] = krow[lane];
+                        else if (lane < 2 * LPR) reinterpret_cast<uint4*>(C.Mv + ((size_t)u * s + i) * D)[lane - LPR] = vrow[lane - LPR];
+                        if (lane == 31) {
+                            C.MW[(size_t)u * s + i] = W;
+                            C.MinvW[(size_t)u * s + i] = inv_we;
+                            C.Mtok[(size_t)u * s + i] = e;
+                        }
+                    }
+                }
+            }
+            item = __shfl_sync(0xffffffffu, next, 0);
+        }
+    }
+    __syncthreads();                                  // the row lists are dead: their bytes take the partials
+
+    // ---- warp partial -> shared [warp][G][D+2] -> block partial in global memory ----
+    float* smp = reinterpret_cast<float*>(scratch);
+#pragma unroll
+    for (int off = 4; off < 32; off <<= 1) {
+        S.tau0 += __shfl_xor_sync(0xffffffffu, S.tau0, off);
+        S.tau1 += __shfl_xor_sync(0xffffffffu, S.tau1, off);
+    }
+    {
+        const int h0 = 2 * tq, h1 = 2 * tq + 1;
+        float* w0 = smp + ((size_t)warp * G + (h0 < G ? h0 : 0)) * STR;
+        float* w1 = smp + ((size_t)warp * G + (h1 < G ? h1 : 0)) * STR;
+        if (g == 0) {
+            if (h0 < G) { w0[0] = S.m0; w0[1] = S.tau0; }
+            if (h1 < G) { w1[0] = S.m1; w1[1] = S.tau1; }
+        }
+#pragma unroll
+        for (int j = 0; j < D / 16; ++j) {
+            const int col = (j >> 2) * 64 + g * 8 + 2 * (j & 3);
+            if (h0 < G) { w0[2 + col] = S.acc[j][0]; w0[2 + col + 1] = S.acc[j][2]; }
+            if (h1 < G) { w1[2 + col] = S.acc[j][1]; w1[2 + col + 1] = S.acc[j][3]; }
+        }
+    }
+    float* part_u = C.part2 + (size_t)u * splits * G * STR;
+    block_combine<D, G>(smp, part_u + (size_t)blockIdx.x * G * STR);
+    __threadfence();
+    __syncthreads();
+    if (splits > 1) {
+        if (tid == 0) {
+            __threadfence();
+            sm_last = (atomicAdd(&C.ticket2[u], 1u) == (unsigned)splits - 1u);
+        }
+        __syncthreads();
+        if (!sm_last) return;
+        __threadfence();
+    }
+
+    // ---- last block of the unit: the insertion's cluster half, the correction of tau, the window, the output ----
+    float* patch = C.part_tau + (size_t)u * splits * G * 2;       // one more {max, tau} partial per head
+    int np_t = 0;
+    if (has_ins) {
+        Best bb;
+        bb.d2 = ~0ull; bb.idx = INT_MAX; bb.pad = 0;
+        for (int i = tid; i < splits; i += kFsThreads) {
+            const ulonglong2 raw = __ldcg(reinterpret_cast<const ulonglong2*>(C.part1 + (size_t)u * splits + i));
+            const int idx = (int)(raw.y & 0xffffffffull);
+            if (better(raw.x, idx, bb)) { bb.d2 = raw.x; bb.idx = idx; }
+        }
+        bb = block_best(bb, smb);
+        const bool joins = (m > 0) && (bb.d2 <= C.delta2_fx);
+        const bool is_full = !joins && (m >= C.m_max);
+        if (!is_full) {
+            np_t = 1;
+            if (warp == 0) {
+                // rows whose scores the correction needs: the cluster's sample rows (its representative while it is
+                // a singleton), then k_e
+                const int c = joins ? bb.idx : 0;
+                const int n_old = joins ? cntu[c] : 0;
+                const int nrow_old = !joins ? 0 : (n_old >= 2 ? t : 1);
+                const int R = nrow_old + 1;
+                auto rowptr = [&](int r) -> const T* {
+                    if (r >= nrow_old) return kE;
+                    return n_old >= 2 ? Su + ((size_t)c * t + r) * D : Xu + (size_t)c * D;
+                };
+                for (int r0 = 0; r0 < R; r0 += 16) {
+                    const int ra = r0 + g, rb = r0 + g + 8;
+                    uint4 ka[NC], kb[NC];
+                    load_keys<D>(rowptr(min(ra, R - 1)), rowptr(min(rb, R - 1)), tq, ka, kb);
+                    float sc[4];
+                    tile_raw_scores<D>(ka, kb, qb, sc);
+                    if (ra < R) { psc[ra][2 * tq] = sc[0]; psc[ra][2 * tq + 1] = sc[1]; }
+                    if (rb < R) { psc[rb][2 * tq] = sc[2]; psc[rb][2 * tq + 1] = sc[3]; }
+                }
+                // the cluster coins of e (the same draws apply_cluster takes)
+                unsigned long long coins = 0;
+                if (joins) {
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        const int j = half * 32 + lane;
+                        bool hit = false;
+                        if (j < t) {
+                            const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)(j >> 2), 0u), C.key0, C.key1);
+                            const uint32_t word = (j & 3) == 0 ? r.x : (j & 3) == 1 ? r.y : (j & 3) == 2 ? r.z : r.w;
+                            hit = coin_cluster(word, (uint32_t)n_old + 1u);
+                        }
+                        coins |= (unsigned long long)__ballot_sync(0xffffffffu, hit) << (32 * half);
+                    }
+                }
+                __syncwarp();
+                if (lane < G) {
+                    const float se = psc[nrow_old][lane];
+                    float mx = se;
+                    for (int r = 0; r < nrow_old; ++r) mx = fmaxf(mx, psc[r][lane]);
+                    const float ee = __expf(se - mx);
+                    float delta;
+                    if (!joins) {
+                        delta = ee;                                   // a new singleton cluster: weight 1
+                    } else if (n_old >= 2) {
+                        float so = 0.f, sn = 0.f;
+                        for (int j = 0; j < t; ++j) {
+                            const float ej = __expf(psc[j][lane] - mx);
+                            so += ej;
+                            sn += ((coins >> j) & 1ull) ? ee : ej;
+                        }
+                        delta = ((float)(n_old + 1) * sn - (float)n_old * so) / (float)t;
+                    } else {
+                        const float ex = __expf(psc[0][lane] - mx);
+                        const int ne = __popcll(coins);
+                        delta = 2.f * ((float)ne * ee + (float)(t - ne) * ex) / (float)t - ex;
+                    }
+                    patch[lane * 2] = mx;
+                    patch[lane * 2 + 1] = delta;
+                }
+            }
+        }
+        __syncthreads();                              // the old sample rows have been read
+        bool join2, full2;
+        int m_ref = m;
+        const int m_new = apply_cluster<T, D, false>(C, u, e, bb, m_ref, krow, sm_w, join2, full2);
+        if (tid == 0) {
+            C.mu[u] = tot;
+            C.m_unit[u] = m_new;
+            C.last_cid[u] = join2 ? bb.idx : (full2 ? -1 : m);
+            C.last_open[u] = join2 ? 0 : 1;
+            C.last_d2[u] = bb.d2;
+        }
+    }
+    if (w) {                                          // the new token takes the window row the leaving one had
+        uint4* ringk = reinterpret_cast<uint4*>(C.ringK + ((size_t)u * w + slot) * D);
+        uint4* ringv = reinterpret_cast<uint4*>(C.ringV + ((size_t)u * w + slot) * D);
+        if (tid < LPR) ringk[tid] = reinterpret_cast<const uint4*>(knew_u)[tid];
+        else if (tid < 2 * LPR) ringv[tid - LPR] = reinterpret_cast<const uint4*>(vnew_u)[tid - LPR];
+    }
+    __syncthreads();                                  // the correction partial and the status bits are written
+    merge_partials<T, D, G>(part_u, splits, patch, np_t, out + qrow0 * D, C.status[u] != 0, sred);
+    if (tid == 0) {
+        C.n_unit[u] = n + 1;
+        C.ticket2[u] = 0;
+        C.qnext[u] = 0;
+    }
+}
+
+}  // namespace sgk

@@ -259,9 +259,10 @@ def test_step_host_matches_step(pinned):
                 np.testing.assert_array_equal(s1[key], s2[key])
 
 
-def test_cache_stats_and_profile():
+@pytest.mark.parametrize("mode", ["split", "fused"])
+def test_cache_stats_and_profile(mode):
     w = synth.CFG3.scaled(B=1, H=2, Hkv=2, n_prompt=600, ncomp=16, s=64, window=32, m_max=256)
-    sg, orcs, _ = _run_stream(w, 600, 4)
+    sg, orcs, _ = _run_stream(w, 600, 4, step_mode=mode)
     st = sg.cache_stats()
     assert st["units"] == 2 and st["tokens"] == 2 * 604 and st["window_rows"] == 64
     assert st["clusters"] == sum(o.m for o in orcs.values())
@@ -282,7 +283,9 @@ def test_cache_stats_and_profile():
     for i in range(3):
         sg.step(Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous())
     ins, tau, zz, steps = sg.profile_read()
-    assert steps == 3 and ins > 0 and tau > 0 and zz > 0 and sg.launch_count == before + 9
+    nk = sg.step_kernels
+    assert nk == (3 if mode == "split" else 1) and steps == 3 and sg.launch_count == before + 3 * nk
+    assert tau > 0 and ((ins > 0 and zz > 0) if nk == 3 else (ins < tau and zz < tau))     # one kernel: its time is in tau
 
 
 def test_chunked_prefill_equals_token_by_token_prefill(monkeypatch):

@@ -1,0 +1,151 @@
+"""The two ways a bf16 handle can run a stream step (one fused kernel, or insertion + cluster scan + value scan)
+against the CPU oracle and against each other.
+
+Both must leave the same integer state, bit for bit, and give outputs within the bf16 tolerance of the oracle
+(main loop of Algorithm 1 with the window of Section 3.2). The fused kernel scans the state as it was before the
+step's insertion and corrects for the insertion afterwards, so the cases below aim at that correction: a token that
+joins a singleton cluster, one that opens a cluster, value slots replaced during the scan, windows of 0 and 1 row,
+a window that is not yet full, grouped queries, many blocks per unit and a single one.
+"""
+import os
+import sys
+
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+
+import numpy as np
+import pytest
+import torch
+
+import helpers as hp
+from helpers import f32
+from paper_2402_06082_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+MODES = ["fused", "split"]
+
+
+def _sg(w, **kw):
+    from paper_2402_06082_b200.binding import SubGen
+    args = dict(Hkv=w.Hkv, dtype=w.torch_dtype, m_max=w.m_max)
+    args.update(kw)
+    return SubGen(w.B, w.H, w.d, w.delta, w.t, w.s, w.window, w.philox_seed, **args)
+
+
+def _stream(w, n_prefill, n_steps, mode, **kw):
+    """Prefill, then n_steps stream steps with every output checked per coordinate; final state bit for bit."""
+    n = n_prefill + n_steps
+    K, V, Q = synth.batch_stream(w, n, "cuda")
+    sg = _sg(w, step_mode=mode, **kw)
+    assert sg.step_kernels == (1 if mode == "fused" else 3)
+    units = [(b, h) for b in range(w.B) for h in range(w.Hkv)]
+    orcs = {bh: hp.oracle_unit(w, *bh) for bh in units}
+    Kn, Vn, Qn = f32(K), f32(V), f32(Q)
+    if n_prefill:
+        sg.prefill(K[:, :, :n_prefill].contiguous(), V[:, :, :n_prefill].contiguous())
+        for (b, h), o in orcs.items():
+            o.push_many(Kn[b, h, :n_prefill], Vn[b, h, :n_prefill])
+    outs = [f32(sg.step(Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous())) for i in range(n_prefill, n)]
+    G = w.H // w.Hkv
+    opened = joined_singleton = replaced = 0
+    for j, i in enumerate(range(n_prefill, n)):
+        for (b, h), o in orcs.items():
+            m0, cnt0, mt0 = o.m, o.counts.copy(), o.m_tok.copy()
+            o.push(Kn[b, h, i], Vn[b, h, i])
+            if o.inserted:
+                e = o.inserted - 1
+                c = int(o.assign[e])
+                opened += int(o.m > m0)
+                joined_singleton += int(o.m == m0 and c < len(cnt0) and cnt0[c] == 1)
+                replaced += int(np.sum(o.m_tok != mt0))
+            for g in range(G):
+                hp.assert_output(outs[j][b, h * G + g], o.query(Qn[b, h * G + g, i]), w.torch_dtype,
+                                 "%s step %d unit %s head %d" % (mode, i, (b, h), g))
+    for (b, h), o in orcs.items():
+        st = sg.export_state(b, h)
+        hp.assert_state_equal(st, o, "%s after steps unit %s" % (mode, (b, h)))
+        hp.assert_rows_match_tokens(sg, b, h, st, K[b, h], V[b, h])
+    assert sg.status() == 0
+    return dict(opened=opened, joined_singleton=joined_singleton, replaced=replaced), sg
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_outliers_gqa(mode):
+    """Outliers open clusters and leave singletons that later members join; G = 4 heads share a unit."""
+    w = synth.CFG3.scaled(B=2, H=8, Hkv=2, n_prompt=700, ncomp=24, s=256, window=32, m_max=512)
+    ev, _ = _stream(w, 700, 80, mode)
+    assert ev["opened"] > 0 and ev["replaced"] > 0
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_from_empty_through_window_fill(mode):
+    """A stream from nothing: steps before the window is full, the first insertion (M takes the token in every
+    slot), then ordinary steps; a small s / n ratio makes value slots change in most steps."""
+    w = synth.CFG2.scaled(B=1, H=2, Hkv=2, ncomp=6, s=48, t=4, window=9, m_max=128)
+    ev, _ = _stream(w, 0, 120, mode)
+    assert ev["replaced"] > 48 and ev["joined_singleton"] > 0
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("window", [0, 1])
+def test_tiny_windows(mode, window):
+    w = synth.CFG2.scaled(B=1, H=4, Hkv=2, ncomp=5, s=40, t=3, window=window, m_max=128, outlier_frac=0.1)
+    _stream(w, 50, 70, mode)
+    _stream(w, 0, 5, mode)
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("splits", [1, 2, 7, 23])
+def test_block_splits(mode, splits):
+    """One block per unit (no arrival ticket), a few, and more blocks than the unit has work items."""
+    w = synth.CFG3.scaled(B=1, H=2, Hkv=2, n_prompt=400, ncomp=12, s=96, window=24, m_max=256)
+    _stream(w, 400, 30, mode, splits=splits)
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("d,G,t", [(64, 1, 5), (64, 8, 8), (128, 2, 16), (128, 8, 33)])
+def test_geometries(mode, d, G, t):
+    """Both head dimensions, group sizes up to 8, t beyond 16 (no slot merging) and beyond 32 (two coin words)."""
+    w = synth.CFG2.scaled(B=1, H=2 * G, Hkv=2, d=d, n_prompt=300, ncomp=8, s=64, t=t, window=16, m_max=128)
+    _stream(w, 300, 40, mode)
+
+
+def test_modes_agree_and_many_units_fused():
+    """More units than the automatic choice would fuse (one block per unit, several waves): fused and split handles
+    fed the same stream end in the same state and give the same outputs up to rounding."""
+    w = synth.CFG3.scaled(B=5, H=32, Hkv=32, n_prompt=300, ncomp=8, s=64, window=16, m_max=128)
+    n0, nd = 300, 12
+    K, V, Q = synth.batch_stream(w, n0 + nd, "cuda")
+    a, b = _sg(w, step_mode="fused"), _sg(w, step_mode="split")
+    for sg in (a, b):
+        sg.prefill(K[:, :, :n0].contiguous(), V[:, :, :n0].contiguous())
+    for i in range(n0, n0 + nd):
+        q, k, v = Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous()
+        oa, ob = f32(a.step(q, k, v)), f32(b.step(q, k, v))
+        for bb in range(w.B):
+            for h in range(w.H):
+                hp.assert_output(oa[bb, h], ob[bb, h], w.torch_dtype, "step %d seq %d head %d" % (i, bb, h))
+    for bb in range(w.B):
+        for h in range(0, w.Hkv, 5):
+            sa, sb = a.export_state(bb, h), b.export_state(bb, h)
+            for key in ("n", "m", "mu", "last_cluster", "last_opened"):
+                assert sa[key] == sb[key], key
+            for key in ("counts", "centre_tok", "slot_tok", "m_tok", "m_w"):
+                np.testing.assert_array_equal(sa[key], sb[key], err_msg=key)
+    o = hp.oracle_unit(w, 4, 31)
+    Kn, Vn = f32(K[4, 31]), f32(V[4, 31])
+    o.push_many(Kn, Vn)
+    hp.assert_state_equal(a.export_state(4, 31), o, "fused, last unit")
+    assert a.status() == 0 and b.status() == 0
+
+
+def test_fused_capacity_overflow_sets_status():
+    """A key that needs a cluster when none is free: status bit, NaN outputs, no fault (fused path)."""
+    w = synth.CFG1.scaled(dtype="bf16", d=64, delta=0.0, window=2, s=16, m_max=8)
+    K, V, Q = synth.batch_stream(w, 40, "cuda")
+    sg = _sg(w, step_mode="fused")
+    out = None
+    for i in range(40):
+        out = sg.step(Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous())
+    assert sg.status() & 1
+    assert torch.isnan(out.float()).all()
