@@ -46,6 +46,19 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 __device__ __forceinline__ uint4 ldg16(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
 
+// 16-byte load of a row that is read once per step: not kept in L1 and first in line for eviction from L2. A step
+// streams hundreds of megabytes of sampled rows; loaded the ordinary way they push out of the L2 everything that
+// IS read again in the next step or by the next kernel (counts, alias rows, packed heads, partials, the kernels'
+// own instructions), which then comes from DRAM at the head of every dependent chain.
+__device__ __forceinline__ uint4 ldg16_stream(const void* p) {
+    uint64_t pol;
+    asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p), "l"(pol));
+    return r;
+}
+
 // Per-warp running state. Lane = 4*g + tq. The lane keeps the running maxima and partial partition
 // sums of heads 2tq and 2tq+1, and z^T accumulators acc[cc*4+j] = {z[2tq][c], z[2tq+1][c], z[2tq][c+1],
 // z[2tq+1][c+1]} with c = cc*64 + g*8 + 2j.
@@ -64,6 +77,16 @@ __device__ __forceinline__ void load_keys(const __nv_bfloat16* pa, const __nv_bf
     for (int c = 0; c < D / 32; ++c) {
         ka[c] = ldg16(pa + c * 32 + tq * 8);
         kb[c] = ldg16(pb + c * 32 + tq * 8);
+    }
+}
+// the same for rows that are read once per step (see ldg16_stream)
+template <int D>
+__device__ __forceinline__ void load_keys_stream(const __nv_bfloat16* pa, const __nv_bfloat16* pb, int tq, uint4 (&ka)[D / 32],
+                                                 uint4 (&kb)[D / 32]) {
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+        ka[c] = ldg16_stream(pa + c * 32 + tq * 8);
+        kb[c] = ldg16_stream(pb + c * 32 + tq * 8);
     }
 }
 
@@ -117,6 +140,13 @@ __device__ __forceinline__ void load_values(const __nv_bfloat16* const (&pv)[4],
 #pragma unroll
         for (int cc = 0; cc < D / 64; ++cc) v[i][cc] = ldg16(pv[i] + cc * 64 + g * 8);
 }
+template <int D>
+__device__ __forceinline__ void load_values_stream(const __nv_bfloat16* const (&pv)[4], int g, uint4 (&v)[4][D / 64]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int cc = 0; cc < D / 64; ++cc) v[i][cc] = ldg16_stream(pv[i] + cc * 64 + g * 8);
+}
 
 template <int D>
 __device__ __forceinline__ void tile_values(MmaState<D>& S, const float (&pz)[4], const uint4 (&v)[4][D / 64], int g, int tq) {
@@ -146,6 +176,137 @@ constexpr int kTauRows = 256 + 16;   // rows of one pass of the cluster scan: at
 
 // floor(r / t) for small r by one multiply-high (t = 1 handled by the caller's magic = 0)
 __device__ __forceinline__ int div_small(int r, unsigned magic) { return magic ? (int)__umulhi((unsigned)r, magic) : r; }
+
+// ---------------------------------------------------------------------------------------------
+// The cluster part of the partition function for one warp, as a software pipeline over items of 16 clusters:
+//   tau_D += sum over the item's clusters of n'/t sum over the t samples of exp<q,k>
+// (a cluster with n' = 1 is read as its representative with weight 1; slots that hold the same token are read once
+// and weighted by their number). While the rows of item i are scored, the counts and alias rows of item i+1 are
+// already on their way and the ticket for item i+2 has been asked for, so the only memory round trip a warp waits
+// for per item is that of the rows themselves. UN tiles of 16 rows are requested together.
+//   first, second  the warp's first two items (known without a memory access)
+//   counter, base  later items are base + atomicAdd(counter, 1)
+//   als, rix, rwt  this warp's shared-memory scratch: 16 * 64 bytes, kTauRows ints, kTauRows floats
+template <int D, int DA, int UN>
+__device__ __forceinline__ void cluster_scan(MmaState<DA>& S, const uint32_t (&qb)[D / 32][4], const Cache<__nv_bfloat16>& C, int u,
+                                             int m, int first, int second, unsigned* counter, int base, unsigned* als, int* rix,
+                                             float* rwt) {
+    typedef __nv_bfloat16 T;
+    constexpr int NC = D / 32;
+    const int lane = threadIdx.x & 31, g = lane >> 2, tq = lane & 3;
+    const int t = C.t;
+    const T* Xu = C.X + (size_t)u * C.m_max * D;
+    const T* Su = C.S + (size_t)u * C.m_max * t * D;
+    const int* cntu = C.cnt + (size_t)u * C.m_max;
+    const unsigned char* ndu = C.ndist + (size_t)u * C.m_max;
+    const unsigned char* alias_bytes = C.alias + (size_t)u * C.m_max * t;
+    // alias rows of an item are 16 t contiguous bytes (the array is padded by one item); they travel through two
+    // registers per lane when t <= 16 and the unit's rows start on a 4-byte boundary, else they are read in place
+    const bool fast = t <= 16 && !(reinterpret_cast<uintptr_t>(alias_bytes) & 3);
+    const unsigned* alias_words = reinterpret_cast<const unsigned*>(alias_bytes);
+    const float inv_t = 1.f / (float)t;
+    const int total = (m + 15) >> 4;
+    const int gsz = t <= 16 ? 16 : 256 / t;          // clusters whose rows fit one list of kTauRows entries (t <= 64)
+    const int nwords = 4 * t;                        // alias words per item (fast path: <= 64)
+    int item = first, next = second;
+    int cn = 0, nd = 0;
+    unsigned aw0 = 0, aw1 = 0;
+    auto fetch = [&](int it, int& cn_, int& nd_, unsigned& a0, unsigned& a1) {
+        cn_ = 0; nd_ = 0; a0 = 0; a1 = 0;
+        if (it < total) {
+            const int c = it * 16 + lane;
+            if (lane < 16 && c < m) { cn_ = cntu[c]; nd_ = (int)ndu[c]; }
+            if (fast) {
+                if (lane < nwords) a0 = alias_words[(size_t)it * nwords + lane];
+                if (lane + 32 < nwords) a1 = alias_words[(size_t)it * nwords + lane + 32];
+            }
+        }
+    };
+    fetch(item, cn, nd, aw0, aw1);
+    while (item < total) {
+        int next2 = 0;
+        if (lane == 0) next2 = base + (int)atomicAdd(counter, 1u);       // asked for now, needed two items later
+        int cn_n, nd_n;
+        unsigned aw0_n, aw1_n;
+        fetch(next, cn_n, nd_n, aw0_n, aw1_n);
+        const int c = item * 16 + lane;
+        if (fast) {
+            if (lane < nwords) als[lane] = aw0;
+            if (lane + 32 < nwords) als[lane + 32] = aw1;
+        } else {
+            unsigned char* dst = reinterpret_cast<unsigned char*>(als);
+            for (int i = lane; i < 16 * t; i += 32) dst[i] = alias_bytes[(size_t)item * 16 * t + i];
+        }
+        for (int p0 = 0; p0 < 16; p0 += gsz) {
+            const bool act = lane >= p0 && lane < p0 + gsz;
+            const int ndl = (act && cn > 1) ? nd : 0;
+            int incl = ndl;
+#pragma unroll
+            for (int off = 1; off < 16; off <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += v;
+            }
+            const int rows_m = __shfl_sync(0xffffffffu, incl, 15);
+            const unsigned ms = __ballot_sync(0xffffffffu, act && cn == 1);
+            const int rows = rows_m + __popc(ms);
+            __syncwarp();
+            if (ndl) {
+                const unsigned char* al = reinterpret_cast<const unsigned char*>(als) + lane * t;
+                const float wc = (float)cn * inv_t;
+                for (int k = 0; k < ndl; ++k) {
+                    const int e = al[k];
+                    const int slot = t <= 16 ? (e & 15) : e, copies = t <= 16 ? (e >> 4) + 1 : 1;
+                    rix[incl - ndl + k] = c * t + slot;
+                    rwt[incl - ndl + k] = wc * (float)copies;
+                }
+            }
+            if (act && cn == 1) {
+                const int r = rows_m + __popc(ms & ((1u << lane) - 1u));
+                rix[r] = c | (int)0x80000000;
+                rwt[r] = 1.f;
+            }
+            __syncwarp();
+            // row r of the list -> pointer, weight, validity
+            auto resolve = [&](int r, const T*& ptr, float& wgt) -> bool {
+                ptr = Xu;
+                wgt = 1.f;
+                if (r < rows) {
+                    const int ix = rix[r];
+                    ptr = ix < 0 ? Xu + (size_t)(ix & 0x7fffffff) * D : Su + (size_t)ix * D;
+                    wgt = rwt[r];
+                }
+                return r < rows;
+            };
+            for (int r0 = 0; r0 < rows; r0 += 16 * UN) {
+                const T *pa[UN], *pb[UN];
+                float wa[UN], wb[UN];
+                bool va[UN], vb[UN];
+                uint4 ka[UN][NC], kb[UN][NC];
+#pragma unroll
+                for (int i = 0; i < UN; ++i) {
+                    va[i] = resolve(r0 + 16 * i + g, pa[i], wa[i]);
+                    vb[i] = resolve(r0 + 16 * i + g + 8, pb[i], wb[i]);
+                }
+#pragma unroll
+                for (int i = 0; i < UN; ++i)
+                    if (i == 0 || r0 + 16 * i < rows) load_keys_stream<D>(pa[i], pb[i], tq, ka[i], kb[i]);
+#pragma unroll
+                for (int i = 0; i < UN; ++i) {
+                    if (i == 0 || r0 + 16 * i < rows) {
+                        float p[4];
+                        tile_scores<D, DA>(S, ka[i], kb[i], va[i], vb[i], qb, p);
+                        S.tau0 += wa[i] * p[0] + wb[i] * p[2];
+                        S.tau1 += wa[i] * p[1] + wb[i] * p[3];
+                    }
+                }
+            }
+            __syncwarp();
+        }
+        item = next;
+        next = __shfl_sync(0xffffffffu, next2, 0);
+        cn = cn_n; nd = nd_n; aw0 = aw0_n; aw1 = aw1_n;
+    }
+}
 
 // ---------------------------------------------------------------------------------------------
 // Clusters: tau_D = sum over clusters of n'/t sum over the t samples of exp<q,k>; a cluster with n' = 1
@@ -251,7 +412,7 @@ __global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfl
                 float wa, wb;
                 const bool va = resolve(r0 + g, pa, wa), vb = resolve(r0 + g + 8, pb, wb);
                 uint4 ka[NC], kb[NC];
-                load_keys<D>(pa, pb, tq, ka, kb);
+                load_keys_stream<D>(pa, pb, tq, ka, kb);
                 float p[4];
                 tile_scores<D, 16>(S, ka, kb, va, vb, qb, p);
                 S.tau0 += wa * p[0] + wb * p[2];
@@ -352,8 +513,8 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_kernel(Cache<__nv_bfloa
         pv[2] = Vb + (size_t)min(base + 2 * tq + 8, lim - 1) * D;
         pv[3] = Vb + (size_t)min(base + 2 * tq + 9, lim - 1) * D;
         uint4 ka[NC], kb[NC], v[4][D / 64];
-        load_keys<D>(Kb + (size_t)ia * D, Kb + (size_t)ib * D, tq, ka, kb);      // keys and values in flight together
-        load_values<D>(pv, g, v);
+        load_keys_stream<D>(Kb + (size_t)ia * D, Kb + (size_t)ib * D, tq, ka, kb);      // keys and values in flight together
+        load_values_stream<D>(pv, g, v);
         float p[4];
         tile_scores<D, D>(S, ka, kb, va, vb, qb, p);
         if (!isM) {
@@ -481,8 +642,8 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_flat_kernel(Cache<__nv_
             pv[2] = Vb + (size_t)min(base + 2 * tq + 8, lim - 1) * D;
             pv[3] = Vb + (size_t)min(base + 2 * tq + 9, lim - 1) * D;
             uint4 ka[NC], kb[NC], v[4][D / 64];
-            load_keys<D>(Kb + (size_t)ia * D, Kb + (size_t)ib * D, tq, ka, kb);      // keys and values in flight together
-            load_values<D>(pv, g, v);
+            load_keys_stream<D>(Kb + (size_t)ia * D, Kb + (size_t)ib * D, tq, ka, kb);      // keys and values in flight together
+            load_values_stream<D>(pv, g, v);
             float p[4];
             tile_scores<D, D>(S, ka, kb, va, vb, qb, p);
             if (!isM) {

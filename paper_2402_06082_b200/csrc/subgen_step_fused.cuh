@@ -7,8 +7,11 @@
 // and nobody waits for anybody:
 //
 //   every block   loads the queries, the token e that leaves the window and W(v_e); scans its slice of the packed
-//                 representative heads for the nearest representative of k_e (as insert_mma_kernel does); then takes
-//                 items from the unit's queue: 16 clusters (partition function), 16 slots of M, 16 window rows
+//                 representative heads for the nearest representative of k_e (as insert_mma_kernel does); then its
+//                 warps take items from the unit's two queues: 16 clusters (partition function), or 16 slots of M /
+//                 16 window rows (numerator). A warp starts in one role: cluster warps need no numerator
+//                 accumulators and spend those registers on a second tile of rows in flight (cluster_scan with two
+//                 tiles); when its queue is empty a warp helps with the other one.
 //   M             which slots of M the token e replaces depends only on (seed, unit, e, slot, mu, W): the warp that
 //                 scans a tile of M flips the tile's 16 coins itself, scores (k_e, v_e) with weight mu/(s W_e) in place
 //                 of a replaced slot and writes the slot. No other warp touches that slot in this step.
@@ -167,21 +170,50 @@ __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bf
         if (tid == 0) C.part1[(size_t)u * splits + blockIdx.x] = bst;
     }
 
+
     // ---- scan of the state as it stands before the insertion ----
+    unsigned* als = reinterpret_cast<unsigned*>(scratch) + warp * (16 * 64 / 4);
+    int* rix = reinterpret_cast<int*>(scratch + NW * 16 * 64) + warp * kTauRows;
+    float* rwt = reinterpret_cast<float*>(scratch + NW * (16 * 64 + kTauRows * 4)) + warp * kTauRows;
+    const int wn = min(n + 1, w);
+    const int n_a = (m + 15) >> 4, n_b = (s + 15) >> 4, n_c = (wn + 15) >> 4, n_v = n_b + n_c;
+    // Roles. The unit's TW warps are dealt to the two queues in proportion to the rows behind them (cluster rows
+    // are not counted anywhere: at most t per cluster and at most one per inserted token, at least one per cluster).
+    const int TW = splits * NW, gw = blockIdx.x * NW + warp;
+    int VW;
+    {
+        long long ec = min((long long)m * t, (long long)max(n - w, 0));
+        ec = max(ec, (long long)m);
+        const long long ev = 2ll * (s + wn);
+        VW = (int)(((long long)TW * ev + (ev + ec) / 2) / (ev + ec));
+        if (n_a == 0) VW = TW;
+        else VW = TW == 1 ? 0 : max(1, min(VW, TW - 1));
+    }
+    const int CW = TW - VW;
+    const int vi = (int)((long long)gw * VW / TW), ci = gw - vi;
+    const bool is_v = (int)((long long)(gw + 1) * VW / TW) > vi;
+    // the first ticket(s) of the queue this warp will help with later: asked for now, needed then
+    int t1 = 0, t2 = 0;
+    if (lane == 0) {
+        if (is_v) {
+            t1 = 2 * CW + (int)atomicAdd(&C.qnext[u], 1u);
+            t2 = 2 * CW + (int)atomicAdd(&C.qnext[u], 1u);
+        } else {
+            t1 = VW + (int)atomicAdd(&C.qnext2[u], 1u);
+        }
+    }
     MmaState<D> S;
-    S.m0 = S.m1 = -INFINITY;
-    S.tau0 = S.tau1 = 0.f;
+    {
+        MmaState<16> SA;                  // cluster warps: running maxima and partition sums only
+        SA.m0 = SA.m1 = -INFINITY;
+        SA.tau0 = SA.tau1 = 0.f;
+        SA.acc[0][0] = SA.acc[0][1] = SA.acc[0][2] = SA.acc[0][3] = 0.f;
+        if (!is_v) cluster_scan<D, 16, 2>(SA, qb, C, u, m, ci, CW + ci, &C.qnext[u], 2 * CW, als, rix, rwt);
+        S.m0 = SA.m0; S.m1 = SA.m1; S.tau0 = SA.tau0; S.tau1 = SA.tau1;
+    }
 #pragma unroll
     for (int j = 0; j < D / 16; ++j) S.acc[j][0] = S.acc[j][1] = S.acc[j][2] = S.acc[j][3] = 0.f;
     {
-        unsigned* als = reinterpret_cast<unsigned*>(scratch) + warp * (16 * 64 / 4);
-        int* rix = reinterpret_cast<int*>(scratch + NW * 16 * 64) + warp * kTauRows;
-        float* rwt = reinterpret_cast<float*>(scratch + NW * (16 * 64 + kTauRows * 4)) + warp * kTauRows;
-        const unsigned char* ndu = C.ndist + (size_t)u * C.m_max;
-        const unsigned char* alias_bytes = C.alias + (size_t)u * C.m_max * t;
-        const unsigned* alias_words = (reinterpret_cast<uintptr_t>(alias_bytes) & 3) ? nullptr : reinterpret_cast<const unsigned*>(alias_bytes);
-        const float inv_t = 1.f / (float)t;
-        const int gsz = t <= 16 ? 16 : 256 / t;
         const T* Mku = C.Mk + (size_t)u * s * D;
         const T* Mvu = C.Mv + (size_t)u * s * D;
         const float* MiWu = C.MinvW + (size_t)u * s;
@@ -189,170 +221,99 @@ __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bf
         const T* Rv = C.ringV + (size_t)u * w * D;
         const float mu_over_s = (float)tot / (float)s;
         const float inv_we = W ? 1.f / (float)W : 0.f;
-        const int wn = min(n + 1, w);
-        const int n_a = (m + 15) >> 4, n_b = (s + 15) >> 4, n_c = (wn + 15) >> 4, total = n_a + n_b + n_c;
-        int item = 0;
-        if (lane == 0) item = (int)atomicAdd(&C.qnext[u], 1u);
-        item = __shfl_sync(0xffffffffu, item, 0);
-        while (item < total) {
+        int item = is_v ? vi : __shfl_sync(0xffffffffu, t1, 0);
+        while (item < n_v) {
             int next = 0;
-            if (lane == 0) next = (int)atomicAdd(&C.qnext[u], 1u);     // asked for early, needed late
-            if (item < n_a) {
-                // 16 clusters -> one list of rows: the distinct samples of every cluster with n' > 1, each weighted
-                // n'/t times the number of slots that hold it, then the representatives of the singletons
-                const int c = item * 16 + lane;
-                const int cn = (lane < 16 && c < m) ? cntu[c] : 0;
-                const int nd = (lane < 16 && c < m) ? (int)ndu[c] : 0;
-                if (alias_words) {
-                    for (int i = lane; i < 4 * t; i += 32) als[i] = alias_words[(size_t)item * 4 * t + i];
-                } else {
-                    unsigned char* dst = reinterpret_cast<unsigned char*>(als);
-                    for (int i = lane; i < 16 * t; i += 32) dst[i] = alias_bytes[(size_t)item * 16 * t + i];
-                }
-                for (int p0 = 0; p0 < 16; p0 += gsz) {
-                    const bool act = lane >= p0 && lane < p0 + gsz;
-                    const int ndl = (act && cn > 1) ? nd : 0;
-                    int incl = ndl;
+            if (lane == 0) next = VW + (int)atomicAdd(&C.qnext2[u], 1u);     // asked for early, needed late
+            // 16 value samples (weight mu/(s W), numerator only) or 16 window rows (weight 1, both sums)
+            const bool isM = item < n_b;
+            const int base = (isM ? item : item - n_b) * 16;
+            const int lim = isM ? s : wn;
+            const T* Kb = isM ? Mku : Rk;
+            const T* Vb = isM ? Mvu : Rv;
+            const int ia = min(base + g, lim - 1), ib = min(base + g + 8, lim - 1);
+            bool va = base + g < lim, vb = base + g + 8 < lim;
+            const int iv[4] = {min(base + 2 * tq, lim - 1), min(base + 2 * tq + 1, lim - 1), min(base + 2 * tq + 8, lim - 1),
+                               min(base + 2 * tq + 9, lim - 1)};
+            const T* pka = Kb + (size_t)ia * D;
+            const T* pkb = Kb + (size_t)ib * D;
+            const T* pv[4];
 #pragma unroll
-                    for (int off = 1; off < 16; off <<= 1) {
-                        const int v = __shfl_up_sync(0xffffffffu, incl, off);
-                        if (lane >= off) incl += v;
-                    }
-                    const int rows_m = __shfl_sync(0xffffffffu, incl, 15);
-                    const unsigned ms = __ballot_sync(0xffffffffu, act && cn == 1);
-                    const int rows = rows_m + __popc(ms);
-                    __syncwarp();
-                    if (ndl) {
-                        const unsigned char* al = reinterpret_cast<const unsigned char*>(als) + lane * t;
-                        const float wc = (float)cn * inv_t;
-                        for (int k = 0; k < ndl; ++k) {
-                            const int ee = al[k];
-                            const int sl = t <= 16 ? (ee & 15) : ee, copies = t <= 16 ? (ee >> 4) + 1 : 1;
-                            rix[incl - ndl + k] = c * t + sl;
-                            rwt[incl - ndl + k] = wc * (float)copies;
-                        }
-                    }
-                    if (act && cn == 1) {
-                        const int r = rows_m + __popc(ms & ((1u << lane) - 1u));
-                        rix[r] = c | (int)0x80000000;
-                        rwt[r] = 1.f;
-                    }
-                    __syncwarp();
-                    auto resolve = [&](int r, const T*& ptr, float& wgt) -> bool {
-                        ptr = Xu;
-                        wgt = 1.f;
-                        if (r < rows) {
-                            const int ix = rix[r];
-                            ptr = ix < 0 ? Xu + (size_t)(ix & 0x7fffffff) * D : Su + (size_t)ix * D;
-                            wgt = rwt[r];
-                        }
-                        return r < rows;
-                    };
-                    for (int r0 = 0; r0 < rows; r0 += 16) {
-                        const T *pa, *pb;
-                        float wa, wb;
-                        const bool va = resolve(r0 + g, pa, wa), vb = resolve(r0 + g + 8, pb, wb);
-                        uint4 ka[NC], kb[NC];
-                        load_keys<D>(pa, pb, tq, ka, kb);
-                        float p[4];
-                        tile_scores<D, D>(S, ka, kb, va, vb, qb, p);
-                        S.tau0 += wa * p[0] + wb * p[2];
-                        S.tau1 += wa * p[1] + wb * p[3];
-                    }
-                    __syncwarp();
-                }
-            } else {
-                // 16 value samples (weight mu/(s W), numerator only) or 16 window rows (weight 1, both sums)
-                const bool isM = item < n_a + n_b;
-                const int base = (isM ? item - n_a : item - n_a - n_b) * 16;
-                const int lim = isM ? s : wn;
-                const T* Kb = isM ? Mku : Rk;
-                const T* Vb = isM ? Mvu : Rv;
-                const int ia = min(base + g, lim - 1), ib = min(base + g + 8, lim - 1);
-                bool va = base + g < lim, vb = base + g + 8 < lim;
-                const int iv[4] = {min(base + 2 * tq, lim - 1), min(base + 2 * tq + 1, lim - 1), min(base + 2 * tq + 8, lim - 1),
-                                   min(base + 2 * tq + 9, lim - 1)};
-                const T* pka = Kb + (size_t)ia * D;
-                const T* pkb = Kb + (size_t)ib * D;
-                const T* pv[4];
+            for (int i = 0; i < 4; ++i) pv[i] = Vb + (size_t)iv[i] * D;
+            float wa_in = 1.f, wb_in = 1.f;
+            unsigned sub = 0;                     // rows of this tile that are scored from another place
+            if (isM) {
+                wa_in = MiWu[ia];                 // 1/W, 0 for a null slot
+                wb_in = MiWu[ib];
+            } else if (w && slot >= base && slot < base + 16) {
+                // the new token's row: not in the ring yet, read from the call's input
+                if (ia == slot) pka = knew_u;
+                if (ib == slot) pkb = knew_u;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) pv[i] = Vb + (size_t)iv[i] * D;
-                float wa_in = 1.f, wb_in = 1.f;
-                unsigned sub = 0;                     // rows of this tile that are scored from another place
-                if (isM) {
-                    wa_in = MiWu[ia];                 // 1/W, 0 for a null slot
-                    wb_in = MiWu[ib];
-                } else if (w && slot >= base && slot < base + 16) {
-                    // the new token's row: not in the ring yet, read from the call's input
-                    sub = 1u << (slot - base);
-                    if (ia == slot) pka = knew_u;
-                    if (ib == slot) pkb = knew_u;
+                for (int i = 0; i < 4; ++i) if (iv[i] == slot) pv[i] = vnew_u;
+            }
+            uint4 ka[NC], kb[NC], v[4][D / 64];
+            load_keys_stream<D>(pka, pkb, tq, ka, kb);           // keys and values in flight together
+            load_values_stream<D>(pv, g, v);
+            if (isM && W > 0) {
+                // UpdateMatrixProduct for the 16 slots of this tile: four Philox blocks, flipped while the rows
+                // are on their way; a slot that takes the leaving token is scored from that token's rows
+                unsigned nib = 0;
+                if (lane < 4) {
+                    const int blk = (base >> 2) + lane;
+                    if (blk * 4 < s) {
+                        const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)blk, 1u), C.key0, C.key1);
+                        const uint32_t words[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) if (iv[i] == slot) pv[i] = vnew_u;
-                }
-                uint4 ka[NC], kb[NC], v[4][D / 64];
-                load_keys<D>(pka, pkb, tq, ka, kb);                  // keys and values in flight together
-                load_values<D>(pv, g, v);
-                if (isM && W > 0) {
-                    // UpdateMatrixProduct for the 16 slots of this tile: four Philox blocks, flipped while the rows
-                    // are on their way; a slot that takes the leaving token is scored from that token's rows
-                    unsigned nib = 0;
-                    if (lane < 4) {
-                        const int blk = (base >> 2) + lane;
-                        if (blk * 4 < s) {
-                            const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)blk, 1u), C.key0, C.key1);
-                            const uint32_t words[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-                            for (int qq = 0; qq < 4; ++qq)
-                                if (blk * 4 + qq < s && coin_value(words[qq], tot, W)) nib |= 1u << qq;
-                        }
-                    }
-                    sub = __shfl_sync(0xffffffffu, nib, 0) | (__shfl_sync(0xffffffffu, nib, 1) << 4) |
-                          (__shfl_sync(0xffffffffu, nib, 2) << 8) | (__shfl_sync(0xffffffffu, nib, 3) << 12);
-                    if (sub) {                        // rare: about s / (tokens inserted) slots per step
-                        if ((sub >> g) & 1u) { wa_in = inv_we; for (int c = 0; c < NC; ++c) ka[c] = ldg16(kE + c * 32 + tq * 8); }
-                        if ((sub >> (g + 8)) & 1u) { wb_in = inv_we; for (int c = 0; c < NC; ++c) kb[c] = ldg16(kE + c * 32 + tq * 8); }
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int r = 2 * tq + (i & 1) + (i >> 1) * 8;
-                            if ((sub >> r) & 1u)
-                                for (int cc = 0; cc < D / 64; ++cc) v[i][cc] = ldg16(vE + cc * 64 + g * 8);
-                        }
+                        for (int qq = 0; qq < 4; ++qq)
+                            if (blk * 4 + qq < s && coin_value(words[qq], tot, W)) nib |= 1u << qq;
                     }
                 }
-                float wza = 1.f, wzb = 1.f;
-                if (isM) {
-                    va = va && wa_in != 0.f;
-                    vb = vb && wb_in != 0.f;
-                    wza = va ? mu_over_s * wa_in : 0.f;
-                    wzb = vb ? mu_over_s * wb_in : 0.f;
-                }
-                float p[4];
-                tile_scores<D, D>(S, ka, kb, va, vb, qb, p);
-                if (!isM) {
-                    S.tau0 += p[0] + p[2];
-                    S.tau1 += p[1] + p[3];
-                }
-                const float pz[4] = {wza * p[0], wza * p[1], wzb * p[2], wzb * p[3]};
-                tile_values<D>(S, pz, v, g, tq);
-                if (isM && sub) {                     // the replaced slots take (k_e, v_e): half a warp per row
-                    unsigned todo = sub;
-                    while (todo) {
-                        const int i = base + __ffs(todo) - 1;
-                        todo &= todo - 1;
-                        if (lane < LPR) reinterpret_cast<uint4*>(C.Mk + ((size_t)u * s + i) * D)[lane] = krow[lane];
-                        else if (lane < 2 * LPR) reinterpret_cast<uint4*>(C.Mv + ((size_t)u * s + i) * D)[lane - LPR] = vrow[lane - LPR];
-                        if (lane == 31) {
-                            C.MW[(size_t)u * s + i] = W;
-                            C.MinvW[(size_t)u * s + i] = inv_we;
-                            C.Mtok[(size_t)u * s + i] = e;
-                        }
+                sub = __shfl_sync(0xffffffffu, nib, 0) | (__shfl_sync(0xffffffffu, nib, 1) << 4) |
+                      (__shfl_sync(0xffffffffu, nib, 2) << 8) | (__shfl_sync(0xffffffffu, nib, 3) << 12);
+                if (sub) {                        // rare: about s / (tokens inserted) slots per step
+                    if ((sub >> g) & 1u) { wa_in = inv_we; for (int c = 0; c < NC; ++c) ka[c] = ldg16(kE + c * 32 + tq * 8); }
+                    if ((sub >> (g + 8)) & 1u) { wb_in = inv_we; for (int c = 0; c < NC; ++c) kb[c] = ldg16(kE + c * 32 + tq * 8); }
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int r = 2 * tq + (i & 1) + (i >> 1) * 8;
+                        if ((sub >> r) & 1u)
+                            for (int cc = 0; cc < D / 64; ++cc) v[i][cc] = ldg16(vE + cc * 64 + g * 8);
                     }
+                }
+            }
+            float wza = 1.f, wzb = 1.f;
+            if (isM) {
+                va = va && wa_in != 0.f;
+                vb = vb && wb_in != 0.f;
+                wza = va ? mu_over_s * wa_in : 0.f;
+                wzb = vb ? mu_over_s * wb_in : 0.f;
+            }
+            float p[4];
+            tile_scores<D, D>(S, ka, kb, va, vb, qb, p);
+            if (!isM) {
+                S.tau0 += p[0] + p[2];
+                S.tau1 += p[1] + p[3];
+            }
+            const float pz[4] = {wza * p[0], wza * p[1], wzb * p[2], wzb * p[3]};
+            tile_values<D>(S, pz, v, g, tq);
+            while (sub) {                         // the replaced slots take (k_e, v_e): half a warp per row
+                const int i = base + __ffs(sub) - 1;
+                sub &= sub - 1;
+                if (lane < LPR) reinterpret_cast<uint4*>(C.Mk + ((size_t)u * s + i) * D)[lane] = krow[lane];
+                else if (lane < 2 * LPR) reinterpret_cast<uint4*>(C.Mv + ((size_t)u * s + i) * D)[lane - LPR] = vrow[lane - LPR];
+                if (lane == 31) {
+                    C.MW[(size_t)u * s + i] = W;
+                    C.MinvW[(size_t)u * s + i] = inv_we;
+                    C.Mtok[(size_t)u * s + i] = e;
                 }
             }
             item = __shfl_sync(0xffffffffu, next, 0);
         }
     }
+    // value warps that are done help with whatever clusters are left (one tile in flight: the accumulators are live)
+    if (is_v) cluster_scan<D, D, 1>(S, qb, C, u, m, __shfl_sync(0xffffffffu, t1, 0), __shfl_sync(0xffffffffu, t2, 0), &C.qnext[u],
+                                    2 * CW, als, rix, rwt);
     __syncthreads();                                  // the row lists are dead: their bytes take the partials
 
     // ---- warp partial -> shared [warp][G][D+2] -> block partial in global memory ----
@@ -379,97 +340,137 @@ __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bf
     }
     float* part_u = C.part2 + (size_t)u * splits * G * STR;
     block_combine<D, G>(smp, part_u + (size_t)blockIdx.x * G * STR);
-    __threadfence();
     __syncthreads();
     if (splits > 1) {
+        // arrival ticket: the release half of the atomic publishes this block's partials (ordered before it by the
+        // barrier), the acquire half lets the last block read everybody else's
         if (tid == 0) {
-            __threadfence();
-            sm_last = (atomicAdd(&C.ticket2[u], 1u) == (unsigned)splits - 1u);
+            unsigned old;
+            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(&C.ticket2[u]) : "memory");
+            sm_last = (old == (unsigned)splits - 1u);
         }
         __syncthreads();
         if (!sm_last) return;
-        __threadfence();
     }
 
-    // ---- last block of the unit: the insertion's cluster half, the correction of tau, the window, the output ----
-    float* patch = C.part_tau + (size_t)u * splits * G * 2;       // one more {max, tau} partial per head
-    int np_t = 0;
+    // ---- last block of the unit ----
+    // Nearest representative over all slices, then two things side by side: warp 0 scores the one cluster that
+    // changes (its sample rows, or its representative while it is a singleton, and k_e) and forms the correction
+    // new contribution - old contribution of the partition function; the other warps merge the blocks' partials.
+    Best bb;
+    bb.d2 = ~0ull; bb.idx = INT_MAX; bb.pad = 0;
+    bool joins = false, is_full = false;
     if (has_ins) {
-        Best bb;
-        bb.d2 = ~0ull; bb.idx = INT_MAX; bb.pad = 0;
         for (int i = tid; i < splits; i += kFsThreads) {
             const ulonglong2 raw = __ldcg(reinterpret_cast<const ulonglong2*>(C.part1 + (size_t)u * splits + i));
             const int idx = (int)(raw.y & 0xffffffffull);
             if (better(raw.x, idx, bb)) { bb.d2 = raw.x; bb.idx = idx; }
         }
         bb = block_best(bb, smb);
-        const bool joins = (m > 0) && (bb.d2 <= C.delta2_fx);
-        const bool is_full = !joins && (m >= C.m_max);
-        if (!is_full) {
-            np_t = 1;
-            if (warp == 0) {
-                // rows whose scores the correction needs: the cluster's sample rows (its representative while it is
-                // a singleton), then k_e
-                const int c = joins ? bb.idx : 0;
-                const int n_old = joins ? cntu[c] : 0;
-                const int nrow_old = !joins ? 0 : (n_old >= 2 ? t : 1);
-                const int R = nrow_old + 1;
-                auto rowptr = [&](int r) -> const T* {
-                    if (r >= nrow_old) return kE;
-                    return n_old >= 2 ? Su + ((size_t)c * t + r) * D : Xu + (size_t)c * D;
-                };
-                for (int r0 = 0; r0 < R; r0 += 16) {
-                    const int ra = r0 + g, rb = r0 + g + 8;
-                    uint4 ka[NC], kb[NC];
-                    load_keys<D>(rowptr(min(ra, R - 1)), rowptr(min(rb, R - 1)), tq, ka, kb);
-                    float sc[4];
-                    tile_raw_scores<D>(ka, kb, qb, sc);
-                    if (ra < R) { psc[ra][2 * tq] = sc[0]; psc[ra][2 * tq + 1] = sc[1]; }
-                    if (rb < R) { psc[rb][2 * tq] = sc[2]; psc[rb][2 * tq + 1] = sc[3]; }
-                }
-                // the cluster coins of e (the same draws apply_cluster takes)
-                unsigned long long coins = 0;
-                if (joins) {
+        joins = (m > 0) && (bb.d2 <= C.delta2_fx);
+        is_full = !joins && (m >= C.m_max);
+    }
+    const bool patched = has_ins && !is_full;
+    float* pmx = sred;                                // [G] maximum the correction is relative to
+    float* pdl = sred + 8;                            // [G] the correction
+    if (warp == 0) {
+        if (patched) {
+            const int c = joins ? bb.idx : 0;
+            const int n_old = joins ? cntu[c] : 0;
+            const int nrow_old = !joins ? 0 : (n_old >= 2 ? t : 1);
+            const int R = nrow_old + 1;
+            auto rowptr = [&](int r) -> const T* {
+                if (r >= nrow_old) return kE;
+                return n_old >= 2 ? Su + ((size_t)c * t + r) * D : Xu + (size_t)c * D;
+            };
+            for (int r0 = 0; r0 < R; r0 += 16) {
+                const int ra = r0 + g, rb = r0 + g + 8;
+                uint4 ka[NC], kb[NC];
+                load_keys<D>(rowptr(min(ra, R - 1)), rowptr(min(rb, R - 1)), tq, ka, kb);
+                float sc[4];
+                tile_raw_scores<D>(ka, kb, qb, sc);
+                if (ra < R) { psc[ra][2 * tq] = sc[0]; psc[ra][2 * tq + 1] = sc[1]; }
+                if (rb < R) { psc[rb][2 * tq] = sc[2]; psc[rb][2 * tq + 1] = sc[3]; }
+            }
+            // the cluster coins of e (the same draws apply_cluster takes)
+            unsigned long long coins = 0;
+            if (joins) {
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        const int j = half * 32 + lane;
-                        bool hit = false;
-                        if (j < t) {
-                            const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)(j >> 2), 0u), C.key0, C.key1);
-                            const uint32_t word = (j & 3) == 0 ? r.x : (j & 3) == 1 ? r.y : (j & 3) == 2 ? r.z : r.w;
-                            hit = coin_cluster(word, (uint32_t)n_old + 1u);
-                        }
-                        coins |= (unsigned long long)__ballot_sync(0xffffffffu, hit) << (32 * half);
+                for (int half = 0; half < 2; ++half) {
+                    const int j = half * 32 + lane;
+                    bool hit = false;
+                    if (j < t) {
+                        const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)(j >> 2), 0u), C.key0, C.key1);
+                        const uint32_t word = (j & 3) == 0 ? r.x : (j & 3) == 1 ? r.y : (j & 3) == 2 ? r.z : r.w;
+                        hit = coin_cluster(word, (uint32_t)n_old + 1u);
                     }
-                }
-                __syncwarp();
-                if (lane < G) {
-                    const float se = psc[nrow_old][lane];
-                    float mx = se;
-                    for (int r = 0; r < nrow_old; ++r) mx = fmaxf(mx, psc[r][lane]);
-                    const float ee = __expf(se - mx);
-                    float delta;
-                    if (!joins) {
-                        delta = ee;                                   // a new singleton cluster: weight 1
-                    } else if (n_old >= 2) {
-                        float so = 0.f, sn = 0.f;
-                        for (int j = 0; j < t; ++j) {
-                            const float ej = __expf(psc[j][lane] - mx);
-                            so += ej;
-                            sn += ((coins >> j) & 1ull) ? ee : ej;
-                        }
-                        delta = ((float)(n_old + 1) * sn - (float)n_old * so) / (float)t;
-                    } else {
-                        const float ex = __expf(psc[0][lane] - mx);
-                        const int ne = __popcll(coins);
-                        delta = 2.f * ((float)ne * ee + (float)(t - ne) * ex) / (float)t - ex;
-                    }
-                    patch[lane * 2] = mx;
-                    patch[lane * 2 + 1] = delta;
+                    coins |= (unsigned long long)__ballot_sync(0xffffffffu, hit) << (32 * half);
                 }
             }
+            __syncwarp();
+            if (lane < G) {
+                const float se = psc[nrow_old][lane];
+                float mx = se;
+                for (int r = 0; r < nrow_old; ++r) mx = fmaxf(mx, psc[r][lane]);
+                const float ee = __expf(se - mx);
+                float delta;
+                if (!joins) {
+                    delta = ee;                                   // a new singleton cluster: weight 1
+                } else if (n_old >= 2) {
+                    float so = 0.f, sn = 0.f;
+                    for (int j = 0; j < t; ++j) {
+                        const float ej = __expf(psc[j][lane] - mx);
+                        so += ej;
+                        sn += ((coins >> j) & 1ull) ? ee : ej;
+                    }
+                    delta = ((float)(n_old + 1) * sn - (float)n_old * so) / (float)t;
+                } else {
+                    const float ex = __expf(psc[0][lane] - mx);
+                    const int ne = __popcll(coins);
+                    delta = 2.f * ((float)ne * ee + (float)(t - ne) * ex) / (float)t - ex;
+                }
+                pmx[lane] = mx;
+                pdl[lane] = delta;
+            }
+        } else if (lane < G) {
+            pmx[lane] = -INFINITY;
+            pdl[lane] = 0.f;
         }
-        __syncthreads();                              // the old sample rows have been read
+    }
+    // Merge of the blocks' partials {max, tau, z[D]}, first half: per head the maximum over the partials, the
+    // partition sum under it and every partial's factor exp(max_i - max) (warps 1.. while warp 0 is busy above).
+    float* fac = smp;                                 // [splits][8]
+    float* hmx = smp + 128 * 8;                       // [G] maximum over the partials
+    float* htau = hmx + 8;                            // [G] partition sum relative to it
+    float4* zsum = reinterpret_cast<float4*>(smp + 128 * 8 + 16);    // [kFsThreads] column quads per group of partials
+    if (warp > 0) {
+        for (int hh = warp - 1; hh < G; hh += NW - 1) {
+            float mx = -INFINITY;
+            float2 ph[4];                             // splits <= 128: four partials per lane
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int i = lane + 32 * k;
+                ph[k] = make_float2(-INFINITY, 0.f);
+                if (i < splits) ph[k] = __ldcg(reinterpret_cast<const float2*>(part_u + ((size_t)i * G + hh) * STR));
+                mx = fmaxf(mx, ph[k].x);
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+            float tau = 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int i = lane + 32 * k;
+                const float f = ph[k].x == -INFINITY ? 0.f : __expf(ph[k].x - mx);
+                if (i < splits) fac[i * 8 + hh] = f;
+                tau = fmaf(ph[k].y, f, tau);
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) tau += __shfl_xor_sync(0xffffffffu, tau, off);
+            if (lane == 0) { hmx[hh] = mx; htau[hh] = tau; }
+        }
+    }
+    __syncthreads();                                  // the correction is in shared memory; the old sample rows were read
+    if (has_ins) {
         bool join2, full2;
         int m_ref = m;
         const int m_new = apply_cluster<T, D, false>(C, u, e, bb, m_ref, krow, sm_w, join2, full2);
@@ -487,12 +488,60 @@ __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bf
         if (tid < LPR) ringk[tid] = reinterpret_cast<const uint4*>(knew_u)[tid];
         else if (tid < 2 * LPR) ringv[tid - LPR] = reinterpret_cast<const uint4*>(vnew_u)[tid - LPR];
     }
-    __syncthreads();                                  // the correction partial and the status bits are written
-    merge_partials<T, D, G>(part_u, splits, patch, np_t, out + qrow0 * D, C.status[u] != 0, sred);
+    __syncthreads();                                  // status bits of this step are set
+    const bool poisoned = C.status[u] != 0;
+    // second half: the numerators. A thread takes one quad of neighbouring columns and every P-th partial, so that
+    // all its loads are independent; the P groups meet in shared memory.
+    constexpr int NQ = G * D / 4, P = kFsThreads / NQ;
+    {
+        const int qd = tid % NQ, pg = tid / NQ;
+        const int hh = (4 * qd) / D, cc = (4 * qd) % D;
+        float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i0 = pg; i0 < splits; i0 += 8 * P) {
+            float4 pz[8];
+            float f[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int i = i0 + k * P;
+                f[k] = i < splits ? fac[i * 8 + hh] : 0.f;
+                // rows of a partial start 8 bytes into a 16-byte slot pattern (D + 2 floats): two 8-byte loads
+                const float* pp = part_u + ((size_t)min(i, splits - 1) * G + hh) * STR + 2 + cc;
+                const float2 lo = __ldcg(reinterpret_cast<const float2*>(pp)), hi = __ldcg(reinterpret_cast<const float2*>(pp + 2));
+                pz[k] = make_float4(lo.x, lo.y, hi.x, hi.y);
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                acc4.x = fmaf(pz[k].x, f[k], acc4.x); acc4.y = fmaf(pz[k].y, f[k], acc4.y);
+                acc4.z = fmaf(pz[k].z, f[k], acc4.z); acc4.w = fmaf(pz[k].w, f[k], acc4.w);
+            }
+        }
+        zsum[tid] = acc4;
+    }
+    __syncthreads();
+    if (tid < NQ) {
+        const int hh = (4 * tid) / D, cc = (4 * tid) % D;
+        float4 z = zsum[tid];
+#pragma unroll
+        for (int pg = 1; pg < P; ++pg) {
+            const float4 o = zsum[pg * NQ + tid];
+            z.x += o.x; z.y += o.y; z.z += o.z; z.w += o.w;
+        }
+        const float mf = fmaxf(hmx[hh], pmx[hh]);
+        const float fa = hmx[hh] == -INFINITY ? 0.f : __expf(hmx[hh] - mf);
+        const float fb = pmx[hh] == -INFINITY ? 0.f : __expf(pmx[hh] - mf);
+        const float tau = htau[hh] * fa + pdl[hh] * fb;
+        const float sc = tau > 0.f ? fa / tau : 0.f;
+        float r0 = z.x * sc, r1 = z.y * sc, r2 = z.z * sc, r3 = z.w * sc;
+        if (poisoned) r0 = r1 = r2 = r3 = __int_as_float(0x7fc00000);
+        __nv_bfloat162* dst = reinterpret_cast<__nv_bfloat162*>(out + qrow0 * D + (size_t)hh * D + cc);
+        dst[0] = __floats2bfloat162_rn(r0, r1);
+        dst[1] = __floats2bfloat162_rn(r2, r3);
+    }
     if (tid == 0) {
         C.n_unit[u] = n + 1;
         C.ticket2[u] = 0;
         C.qnext[u] = 0;
+        C.qnext2[u] = 0;
     }
 }
 
