@@ -52,8 +52,8 @@ __global__ void __launch_bounds__(kQmThreads, 4) exact_mma_kernel(ExactCache<__n
         pv[2] = Vu + (size_t)min(base + 2 * tq + 8, n - 1) * D;
         pv[3] = Vu + (size_t)min(base + 2 * tq + 9, n - 1) * D;
         uint4 ka[NC], kb[NC], v[4][D / 64];
-        load_keys_stream<D>(Ku + (size_t)ia * D, Ku + (size_t)ib * D, tq, ka, kb);
-        load_values_stream<D>(pv, g, v);
+        load_keys<D>(Ku + (size_t)ia * D, Ku + (size_t)ib * D, tq, ka, kb);
+        load_values<D>(pv, g, v);
         float p[4];
         tile_scores<D, D>(S, ka, kb, va, vb, qb, p);
         S.tau0 += p[0] + p[2];

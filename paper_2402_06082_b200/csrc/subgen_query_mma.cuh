@@ -46,7 +46,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 __device__ __forceinline__ uint4 ldg16(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
 
-// 16-byte load of a row that is read once per step: not kept in L1 and first in line for eviction from L2. A step
+// 16-byte load of a row that is read once per step: first in line for eviction from L2. A step
 // streams hundreds of megabytes of sampled rows; loaded the ordinary way they push out of the L2 everything that
 // IS read again in the next step or by the next kernel (counts, alias rows, packed heads, partials, the kernels'
 // own instructions), which then comes from DRAM at the head of every dependent chain.
@@ -54,7 +54,7 @@ __device__ __forceinline__ uint4 ldg16_stream(const void* p) {
     uint64_t pol;
     asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
     uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+    asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
                  : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p), "l"(pol));
     return r;
 }
