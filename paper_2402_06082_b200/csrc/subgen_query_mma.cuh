@@ -308,6 +308,101 @@ __device__ __forceinline__ void cluster_scan(MmaState<DA>& S, const uint32_t (&q
     }
 }
 
+// The cluster part of the partition function for one warp, items of 16 clusters taken from the unit's counter one
+// at a time (the plain loop; cluster_scan above is the pipelined one). als, rix, rwt: this warp's shared-memory
+// scratch as for cluster_scan.
+template <int D>
+__device__ __forceinline__ void cluster_scan_queue(MmaState<16>& S, const uint32_t (&qb)[D / 32][4], const Cache<__nv_bfloat16>& C,
+                                                   int u, int m, unsigned* als, int* rix, float* rwt) {
+    typedef __nv_bfloat16 T;
+    constexpr int NC = D / 32;
+    const int lane = threadIdx.x & 31, g = lane >> 2, tq = lane & 3;
+    const int t = C.t;
+    const T* Xu = C.X + (size_t)u * C.m_max * D;
+    const T* Su = C.S + (size_t)u * C.m_max * t * D;
+    const int* cntu = C.cnt + (size_t)u * C.m_max;
+    const unsigned char* ndu = C.ndist + (size_t)u * C.m_max;
+    const unsigned char* alias_bytes = C.alias + (size_t)u * C.m_max * t;
+    const unsigned* alias_words = (reinterpret_cast<uintptr_t>(alias_bytes) & 3) ? nullptr : reinterpret_cast<const unsigned*>(alias_bytes);
+    const float inv_t = 1.f / (float)t;
+    const int total = (m + 15) >> 4;
+    const int gsz = t <= 16 ? 16 : 256 / t;          // clusters whose rows fit one list of kTauRows entries (t <= 64)
+    int item = 0;
+    if (lane == 0) item = (int)atomicAdd(&C.qnext[u], 1u);
+    item = __shfl_sync(0xffffffffu, item, 0);
+    while (item < total) {
+        int next = 0;
+        if (lane == 0) next = (int)atomicAdd(&C.qnext[u], 1u);     // asked for early, needed late
+        // 16 clusters -> one list of rows: first the distinct samples of every cluster with n' > 1, each weighted
+        // n'/t times the number of slots that hold it, then the representatives of the singletons
+        const int c = item * 16 + lane;
+        const int cn = (lane < 16 && c < m) ? cntu[c] : 0;
+        const int nd = (lane < 16 && c < m) ? (int)ndu[c] : 0;
+        // the 16 alias rows are contiguous (16 t bytes; the array is padded by one item): word loads when the
+        // unit's rows start on a 4-byte boundary (m_max t a multiple of 4, or unit 0), else byte by byte
+        if (alias_words) {
+            for (int i = lane; i < 4 * t; i += 32) als[i] = alias_words[(size_t)item * 4 * t + i];
+        } else {
+            unsigned char* dst = reinterpret_cast<unsigned char*>(als);
+            for (int i = lane; i < 16 * t; i += 32) dst[i] = alias_bytes[(size_t)item * 16 * t + i];
+        }
+        for (int p0 = 0; p0 < 16; p0 += gsz) {
+            const bool act = lane >= p0 && lane < p0 + gsz;
+            const int ndl = (act && cn > 1) ? nd : 0;
+            int incl = ndl;
+#pragma unroll
+            for (int off = 1; off < 16; off <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += v;
+            }
+            const int rows_m = __shfl_sync(0xffffffffu, incl, 15);
+            const unsigned ms = __ballot_sync(0xffffffffu, act && cn == 1);
+            const int rows = rows_m + __popc(ms);
+            __syncwarp();
+            if (ndl) {
+                const unsigned char* al = reinterpret_cast<const unsigned char*>(als) + lane * t;
+                const float wc = (float)cn * inv_t;
+                for (int k = 0; k < ndl; ++k) {
+                    const int e = al[k];
+                    const int slot = t <= 16 ? (e & 15) : e, copies = t <= 16 ? (e >> 4) + 1 : 1;
+                    rix[incl - ndl + k] = c * t + slot;
+                    rwt[incl - ndl + k] = wc * (float)copies;
+                }
+            }
+            if (act && cn == 1) {
+                const int r = rows_m + __popc(ms & ((1u << lane) - 1u));
+                rix[r] = c | (int)0x80000000;
+                rwt[r] = 1.f;
+            }
+            __syncwarp();
+            // row r of the list -> pointer, weight, validity
+            auto resolve = [&](int r, const T*& ptr, float& wgt) -> bool {
+                ptr = Xu;
+                wgt = 1.f;
+                if (r < rows) {
+                    const int ix = rix[r];
+                    ptr = ix < 0 ? Xu + (size_t)(ix & 0x7fffffff) * D : Su + (size_t)ix * D;
+                    wgt = rwt[r];
+                }
+                return r < rows;
+            };
+            for (int r0 = 0; r0 < rows; r0 += 16) {
+                const T *pa, *pb;
+                float wa, wb;
+                const bool va = resolve(r0 + g, pa, wa), vb = resolve(r0 + g + 8, pb, wb);
+                uint4 ka[NC], kb[NC];
+                load_keys_stream<D>(pa, pb, tq, ka, kb);
+                float p[4];
+                tile_scores<D, 16>(S, ka, kb, va, vb, qb, p);
+                S.tau0 += wa * p[0] + wb * p[2];
+                S.tau1 += wa * p[1] + wb * p[3];
+            }
+            __syncwarp();
+        }
+        item = __shfl_sync(0xffffffffu, next, 0);
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Clusters: tau_D = sum over clusters of n'/t sum over the t samples of exp<q,k>; a cluster with n' = 1
 // is read as its representative with weight 1. Writes per block {max, tau} per head to part_tau.
@@ -333,95 +428,13 @@ __global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfl
         qb[c][0] = r.x; qb[c][1] = r.y; qb[c][2] = r.z; qb[c][3] = r.w;
     }
     pdl_wait();
-    const int t = C.t, m = C.m_unit[u];
+    const int m = C.m_unit[u];
     MmaState<16> S;                       // the accumulators stay untouched here and cost no registers
     S.m0 = S.m1 = -INFINITY;
     S.tau0 = S.tau1 = 0.f;
     S.acc[0][0] = S.acc[0][1] = S.acc[0][2] = S.acc[0][3] = 0.f;
 
-    const T* Xu = C.X + (size_t)u * C.m_max * D;
-    const T* Su = C.S + (size_t)u * C.m_max * t * D;
-    const int* cntu = C.cnt + (size_t)u * C.m_max;
-    const unsigned char* ndu = C.ndist + (size_t)u * C.m_max;
-    const unsigned char* alias_bytes = C.alias + (size_t)u * C.m_max * t;
-    const unsigned* alias_words = (reinterpret_cast<uintptr_t>(alias_bytes) & 3) ? nullptr : reinterpret_cast<const unsigned*>(alias_bytes);
-    const float inv_t = 1.f / (float)t;
-    const int total = (m + 15) >> 4;
-    const int gsz = t <= 16 ? 16 : 256 / t;          // clusters whose rows fit one list of kTauRows entries (t <= 64)
-    int item = 0;
-    if (lane == 0) item = (int)atomicAdd(&C.qnext[u], 1u);
-    item = __shfl_sync(0xffffffffu, item, 0);
-    while (item < total) {
-        int next = 0;
-        if (lane == 0) next = (int)atomicAdd(&C.qnext[u], 1u);     // asked for early, needed late
-        // 16 clusters -> one list of rows: first the distinct samples of every cluster with n' > 1, each weighted
-        // n'/t times the number of slots that hold it, then the representatives of the singletons
-        const int c = item * 16 + lane;
-        const int cn = (lane < 16 && c < m) ? cntu[c] : 0;
-        const int nd = (lane < 16 && c < m) ? (int)ndu[c] : 0;
-        // the 16 alias rows are contiguous (16 t bytes; the array is padded by one item): word loads when the
-        // unit's rows start on a 4-byte boundary (m_max t a multiple of 4, or unit 0), else byte by byte
-        if (alias_words) {
-            for (int i = lane; i < 4 * t; i += 32) als[warp][i] = alias_words[(size_t)item * 4 * t + i];
-        } else {
-            unsigned char* dst = reinterpret_cast<unsigned char*>(als[warp]);
-            for (int i = lane; i < 16 * t; i += 32) dst[i] = alias_bytes[(size_t)item * 16 * t + i];
-        }
-        for (int p0 = 0; p0 < 16; p0 += gsz) {
-            const bool act = lane >= p0 && lane < p0 + gsz;
-            const int ndl = (act && cn > 1) ? nd : 0;
-            int incl = ndl;
-#pragma unroll
-            for (int off = 1; off < 16; off <<= 1) {
-                const int v = __shfl_up_sync(0xffffffffu, incl, off);
-                if (lane >= off) incl += v;
-            }
-            const int rows_m = __shfl_sync(0xffffffffu, incl, 15);
-            const unsigned ms = __ballot_sync(0xffffffffu, act && cn == 1);
-            const int rows = rows_m + __popc(ms);
-            __syncwarp();
-            if (ndl) {
-                const unsigned char* al = reinterpret_cast<const unsigned char*>(als[warp]) + lane * t;
-                const float wc = (float)cn * inv_t;
-                for (int k = 0; k < ndl; ++k) {
-                    const int e = al[k];
-                    const int slot = t <= 16 ? (e & 15) : e, copies = t <= 16 ? (e >> 4) + 1 : 1;
-                    rix[warp][incl - ndl + k] = c * t + slot;
-                    rwt[warp][incl - ndl + k] = wc * (float)copies;
-                }
-            }
-            if (act && cn == 1) {
-                const int r = rows_m + __popc(ms & ((1u << lane) - 1u));
-                rix[warp][r] = c | (int)0x80000000;
-                rwt[warp][r] = 1.f;
-            }
-            __syncwarp();
-            // row r of the list -> pointer, weight, validity
-            auto resolve = [&](int r, const T*& ptr, float& wgt) -> bool {
-                ptr = Xu;
-                wgt = 1.f;
-                if (r < rows) {
-                    const int ix = rix[warp][r];
-                    ptr = ix < 0 ? Xu + (size_t)(ix & 0x7fffffff) * D : Su + (size_t)ix * D;
-                    wgt = rwt[warp][r];
-                }
-                return r < rows;
-            };
-            for (int r0 = 0; r0 < rows; r0 += 16) {
-                const T *pa, *pb;
-                float wa, wb;
-                const bool va = resolve(r0 + g, pa, wa), vb = resolve(r0 + g + 8, pb, wb);
-                uint4 ka[NC], kb[NC];
-                load_keys_stream<D>(pa, pb, tq, ka, kb);
-                float p[4];
-                tile_scores<D, 16>(S, ka, kb, va, vb, qb, p);
-                S.tau0 += wa * p[0] + wb * p[2];
-                S.tau1 += wa * p[1] + wb * p[3];
-            }
-            __syncwarp();
-        }
-        item = __shfl_sync(0xffffffffu, next, 0);
-    }
+    cluster_scan_queue<D>(S, qb, C, u, m, als[warp], rix[warp], rwt[warp]);
 #pragma unroll
     for (int off = 4; off < 32; off <<= 1) {
         S.tau0 += __shfl_xor_sync(0xffffffffu, S.tau0, off);

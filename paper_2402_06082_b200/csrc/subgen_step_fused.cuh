@@ -44,6 +44,278 @@ __device__ __forceinline__ void tile_raw_scores(const uint4 (&ka)[D / 32], const
     }
 }
 
+// What a step knows about its two tokens once the unit's counters are read: the new token (k, v) of the call and the
+// token e that leaves the window and is inserted into D and M (the new token itself when there is no window).
+struct StepToken {
+    int n;                            // tokens seen before this step
+    int e;                            // index of the token that leaves the window (n - window)
+    int slot;                         // window row both tokens use: e leaves it, the new token takes it
+    bool has_ins;                     // a token leaves the window in this step
+    unsigned long long W;             // W(v_e), 0 without insertion
+    unsigned long long tot;           // mu after the insertion
+    const __nv_bfloat16 *kE, *vE;     // rows of token e (in the window ring, or the call's input when window = 0)
+    const __nv_bfloat16 *knew, *vnew; // rows of the new token (the call's input)
+};
+
+// Nearest representative of the key in krow over rows [c0, c1) of the unit's packed heads: the tensor-core filter
+// and exact follow-up of insert_mma_kernel. Warps take KT tiles of 16 heads per turn; every thread ends with the
+// best (D2, index) its warp has seen (bst is updated, not reset).
+template <int D, int KT>
+__device__ __forceinline__ void head_scan_slice(const Cache<__nv_bfloat16>& C, int u, int c0, int c1, const uint4* krow, int nwarps,
+                                                Best& bst) {
+    typedef __nv_bfloat16 T;
+    constexpr int LPR = D / 8;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, tq = lane & 3;
+    const T* Xu = C.X + (size_t)u * C.m_max * D;
+    const T* Xhu = C.Xh + (size_t)u * C.m_max * kHeadDims;
+    const float* xhnu = C.xhn + (size_t)u * C.m_max;
+    uint32_t kb0[4];
+    float kn = 0.f;
+    {
+        const uint4 r = krow[tq];
+        float f[8];
+        Elem<T>::unpack(r, f);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) kn = fmaf(f[j], f[j], kn);
+        kb0[0] = g == 0 ? r.x : 0u; kb0[1] = g == 0 ? r.y : 0u;
+        kb0[2] = g == 0 ? r.z : 0u; kb0[3] = g == 0 ? r.w : 0u;
+    }
+    kn += __shfl_xor_sync(0xffffffffu, kn, 1);
+    kn += __shfl_xor_sync(0xffffffffu, kn, 2);
+    const float d2f = (float)((double)C.delta2_fx * (1.0 / 4294967296.0));
+    auto exact_row = [&](int row) {                                  // exact D2 of one flagged row, by the warp
+        unsigned long long acc = 0;
+        if (lane < LPR) {
+            float xf[8], kf[8];
+            Elem<T>::unpack(*reinterpret_cast<const uint4*>(Xu + (size_t)row * D + lane * 8), xf);
+            Elem<T>::unpack(krow[lane], kf);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc += fx_sqdiff(xf[j], kf[j]);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        if (better(acc, row, bst)) { bst.d2 = acc; bst.idx = row; }
+    };
+    for (int base = c0 + warp * 16 * KT; base < c1; base += nwarps * 16 * KT) {
+        uint4 ha[KT], hc[KT];
+        float xa[KT], xb[KT];
+#pragma unroll
+        for (int i = 0; i < KT; ++i) {
+            const int ra = base + i * 16 + g, rb = ra + 8;
+            const bool va = ra < c1, vb = rb < c1;
+            ha[i] = ldg16(Xhu + (size_t)(va ? ra : c1 - 1) * kHeadDims + tq * 8);
+            hc[i] = ldg16(Xhu + (size_t)(vb ? rb : c1 - 1) * kHeadDims + tq * 8);
+            xa[i] = va ? xhnu[ra] : 0.f;
+            xb[i] = vb ? xhnu[rb] : 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < KT; ++i) {
+            const int ra = base + i * 16 + g, rb = ra + 8;
+            float sc[4] = {0.f, 0.f, 0.f, 0.f};
+            mma_bf16_16816(sc, ha[i].x, hc[i].x, ha[i].y, hc[i].y, kb0[0], kb0[1]);
+            mma_bf16_16816(sc, ha[i].z, hc[i].z, ha[i].w, hc[i].w, kb0[2], kb0[3]);
+            const float na = xa[i] + kn, nb = xb[i] + kn;
+            const bool fa = ra < c1 && tq == 0 && (na - 2.f * sc[0]) <= d2f + 1.220703125e-4f * na;
+            const bool fb = rb < c1 && tq == 0 && (nb - 2.f * sc[2]) <= d2f + 1.220703125e-4f * nb;
+            unsigned ma = __ballot_sync(0xffffffffu, fa), mb = __ballot_sync(0xffffffffu, fb);
+            while (ma) { exact_row(base + i * 16 + ((__ffs(ma) - 1) >> 2)); ma &= ma - 1; }
+            while (mb) { exact_row(base + i * 16 + 8 + ((__ffs(mb) - 1) >> 2)); mb &= mb - 1; }
+        }
+    }
+}
+
+// One warp's share of the numerator: items of 16 slots of M (weight mu/(s W), numerator only), then items of 16
+// window rows (weight 1, numerator and partition function), on the state as it stands BEFORE the step's insertion,
+// with the step's two changes made on the fly:
+//   UpdateMatrixProduct  the warp flips the 16 value coins of its tile of M (four Philox blocks, while the rows are on
+//                        their way), scores (k_e, v_e) with weight mu/(s W_e) in place of a slot that takes token e
+//                        and writes that slot; no other warp touches the slot in this step;
+//   window               the row the new token will take is scored from the call's input.
+// first: the warp's first item; later ones are base + atomicAdd(counter, 1). krow / vrow: token e in shared memory.
+template <int D>
+__device__ __forceinline__ void value_scan(MmaState<D>& S, const uint32_t (&qb)[D / 32][4], const Cache<__nv_bfloat16>& C, int u,
+                                           const StepToken& tk, const uint4* krow, const uint4* vrow, int first, unsigned* counter,
+                                           int base_ticket) {
+    typedef __nv_bfloat16 T;
+    constexpr int NC = D / 32, LPR = D / 8;
+    const int lane = threadIdx.x & 31, g = lane >> 2, tq = lane & 3;
+    const int w = C.w, s = C.s;
+    const T* Mku = C.Mk + (size_t)u * s * D;
+    const T* Mvu = C.Mv + (size_t)u * s * D;
+    const float* MiWu = C.MinvW + (size_t)u * s;
+    const T* Rk = C.ringK + (size_t)u * w * D;
+    const T* Rv = C.ringV + (size_t)u * w * D;
+    const unsigned long long W = tk.W, tot = tk.tot;
+    const float mu_over_s = (float)tot / (float)s;
+    const float inv_we = W ? 1.f / (float)W : 0.f;
+    const int wn = min(tk.n + 1, w), slot = tk.slot;
+    const int n_b = (s + 15) >> 4, n_v = n_b + ((wn + 15) >> 4);
+    int item = first;
+    while (item < n_v) {
+        int next = 0;
+        if (lane == 0) next = base_ticket + (int)atomicAdd(counter, 1u);     // asked for early, needed late
+        const bool isM = item < n_b;
+        const int base = (isM ? item : item - n_b) * 16;
+        const int lim = isM ? s : wn;
+        const T* Kb = isM ? Mku : Rk;
+        const T* Vb = isM ? Mvu : Rv;
+        const int ia = min(base + g, lim - 1), ib = min(base + g + 8, lim - 1);
+        bool va = base + g < lim, vb = base + g + 8 < lim;
+        const int iv[4] = {min(base + 2 * tq, lim - 1), min(base + 2 * tq + 1, lim - 1), min(base + 2 * tq + 8, lim - 1),
+                           min(base + 2 * tq + 9, lim - 1)};
+        const T* pka = Kb + (size_t)ia * D;
+        const T* pkb = Kb + (size_t)ib * D;
+        const T* pv[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) pv[i] = Vb + (size_t)iv[i] * D;
+        float wa_in = 1.f, wb_in = 1.f;
+        unsigned sub = 0;                     // slots of this tile that take token e
+        if (isM) {
+            wa_in = MiWu[ia];                 // 1/W, 0 for a null slot
+            wb_in = MiWu[ib];
+        } else if (w && slot >= base && slot < base + 16) {
+            // the new token's row: not in the ring yet, read from the call's input
+            if (ia == slot) pka = tk.knew;
+            if (ib == slot) pkb = tk.knew;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) if (iv[i] == slot) pv[i] = tk.vnew;
+        }
+        uint4 ka[NC], kb[NC], v[4][D / 64];
+        load_keys_stream<D>(pka, pkb, tq, ka, kb);           // keys and values in flight together
+        load_values_stream<D>(pv, g, v);
+        if (isM && W > 0) {
+            unsigned nib = 0;
+            if (lane < 4) {
+                const int blk = (base >> 2) + lane;
+                if (blk * 4 < s) {
+                    const uint4 r = philox4x32_10(make_uint4((uint32_t)tk.e, (uint32_t)u, (uint32_t)blk, 1u), C.key0, C.key1);
+                    const uint32_t words[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                    for (int qq = 0; qq < 4; ++qq)
+                        if (blk * 4 + qq < s && coin_value(words[qq], tot, W)) nib |= 1u << qq;
+                }
+            }
+            sub = __shfl_sync(0xffffffffu, nib, 0) | (__shfl_sync(0xffffffffu, nib, 1) << 4) |
+                  (__shfl_sync(0xffffffffu, nib, 2) << 8) | (__shfl_sync(0xffffffffu, nib, 3) << 12);
+            if (sub) {                        // rare: about s / (tokens inserted) slots per step
+                if ((sub >> g) & 1u) { wa_in = inv_we; for (int c = 0; c < NC; ++c) ka[c] = ldg16(tk.kE + c * 32 + tq * 8); }
+                if ((sub >> (g + 8)) & 1u) { wb_in = inv_we; for (int c = 0; c < NC; ++c) kb[c] = ldg16(tk.kE + c * 32 + tq * 8); }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int r = 2 * tq + (i & 1) + (i >> 1) * 8;
+                    if ((sub >> r) & 1u)
+                        for (int cc = 0; cc < D / 64; ++cc) v[i][cc] = ldg16(tk.vE + cc * 64 + g * 8);
+                }
+            }
+        }
+        float wza = 1.f, wzb = 1.f;
+        if (isM) {
+            va = va && wa_in != 0.f;
+            vb = vb && wb_in != 0.f;
+            wza = va ? mu_over_s * wa_in : 0.f;
+            wzb = vb ? mu_over_s * wb_in : 0.f;
+        }
+        float p[4];
+        tile_scores<D, D>(S, ka, kb, va, vb, qb, p);
+        if (!isM) {
+            S.tau0 += p[0] + p[2];
+            S.tau1 += p[1] + p[3];
+        }
+        const float pz[4] = {wza * p[0], wza * p[1], wzb * p[2], wzb * p[3]};
+        tile_values<D>(S, pz, v, g, tq);
+        while (sub) {                         // the replaced slots take (k_e, v_e): half a warp per row
+            const int i = base + __ffs(sub) - 1;
+            sub &= sub - 1;
+            if (lane < LPR) reinterpret_cast<uint4*>(C.Mk + ((size_t)u * s + i) * D)[lane] = krow[lane];
+            else if (lane < 2 * LPR) reinterpret_cast<uint4*>(C.Mv + ((size_t)u * s + i) * D)[lane - LPR] = vrow[lane - LPR];
+            if (lane == 31) {
+                C.MW[(size_t)u * s + i] = W;
+                C.MinvW[(size_t)u * s + i] = inv_we;
+                C.Mtok[(size_t)u * s + i] = tk.e;
+            }
+        }
+        item = __shfl_sync(0xffffffffu, next, 0);
+    }
+}
+
+// The partition function changes in one cluster per step: token e joins cluster c (count + 1, some of its t slots
+// take k_e) or opens a new one (weight 1). The scan saw the cluster as it was; this computes, per head,
+//   pdl = new contribution - old contribution,  relative to the maximum pmx of the scores involved,
+// from the scores of the cluster's sample rows (its representative while it is a singleton) and of k_e. The coins
+// are the draws apply_cluster takes. Called by ONE warp; psc: shared [65][8]; pmx, pdl: shared [G]. Must run before
+// apply_cluster overwrites the sample rows.
+template <int D, int G>
+__device__ __forceinline__ void tau_correction(const Cache<__nv_bfloat16>& C, int u, const StepToken& tk,
+                                               const uint32_t (&qb)[D / 32][4], bool patched, bool joins, int c_join,
+                                               float (*psc)[8], float* pmx, float* pdl) {
+    typedef __nv_bfloat16 T;
+    constexpr int NC = D / 32;
+    const int lane = threadIdx.x & 31, g = lane >> 2, tq = lane & 3;
+    const int t = C.t;
+    if (!patched) {
+        if (lane < G) { pmx[lane] = -INFINITY; pdl[lane] = 0.f; }
+        return;
+    }
+    const T* Xu = C.X + (size_t)u * C.m_max * D;
+    const T* Su = C.S + (size_t)u * C.m_max * t * D;
+    const int c = joins ? c_join : 0;
+    const int n_old = joins ? C.cnt[(size_t)u * C.m_max + c] : 0;
+    const int nrow_old = !joins ? 0 : (n_old >= 2 ? t : 1);
+    const int R = nrow_old + 1;
+    auto rowptr = [&](int r) -> const T* {
+        if (r >= nrow_old) return tk.kE;
+        return n_old >= 2 ? Su + ((size_t)c * t + r) * D : Xu + (size_t)c * D;
+    };
+    for (int r0 = 0; r0 < R; r0 += 16) {
+        const int ra = r0 + g, rb = r0 + g + 8;
+        uint4 ka[NC], kb[NC];
+        load_keys<D>(rowptr(min(ra, R - 1)), rowptr(min(rb, R - 1)), tq, ka, kb);
+        float sc[4];
+        tile_raw_scores<D>(ka, kb, qb, sc);
+        if (ra < R) { psc[ra][2 * tq] = sc[0]; psc[ra][2 * tq + 1] = sc[1]; }
+        if (rb < R) { psc[rb][2 * tq] = sc[2]; psc[rb][2 * tq + 1] = sc[3]; }
+    }
+    unsigned long long coins = 0;
+    if (joins) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int j = half * 32 + lane;
+            bool hit = false;
+            if (j < t) {
+                const uint4 r = philox4x32_10(make_uint4((uint32_t)tk.e, (uint32_t)u, (uint32_t)(j >> 2), 0u), C.key0, C.key1);
+                const uint32_t word = (j & 3) == 0 ? r.x : (j & 3) == 1 ? r.y : (j & 3) == 2 ? r.z : r.w;
+                hit = coin_cluster(word, (uint32_t)n_old + 1u);
+            }
+            coins |= (unsigned long long)__ballot_sync(0xffffffffu, hit) << (32 * half);
+        }
+    }
+    __syncwarp();
+    if (lane < G) {
+        const float se = psc[nrow_old][lane];
+        float mx = se;
+        for (int r = 0; r < nrow_old; ++r) mx = fmaxf(mx, psc[r][lane]);
+        const float ee = __expf(se - mx);
+        float delta;
+        if (!joins) {
+            delta = ee;                                   // a new singleton cluster: weight 1
+        } else if (n_old >= 2) {
+            float so = 0.f, sn = 0.f;
+            for (int j = 0; j < t; ++j) {
+                const float ej = __expf(psc[j][lane] - mx);
+                so += ej;
+                sn += ((coins >> j) & 1ull) ? ee : ej;
+            }
+            delta = ((float)(n_old + 1) * sn - (float)n_old * so) / (float)t;
+        } else {
+            const float ex = __expf(psc[0][lane] - mx);
+            const int ne = __popcll(coins);
+            delta = 2.f * ((float)ne * ee + (float)(t - ne) * ex) / (float)t - ex;
+        }
+        pmx[lane] = mx;
+        pdl[lane] = delta;
+    }
+}
+
 template <int D, int G>
 __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ q,
                                                                   const __nv_bfloat16* __restrict__ k_new,
@@ -97,74 +369,18 @@ __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bf
     __syncthreads();
     const unsigned long long W = has_ins ? sm_w[0] : 0ull;
     const unsigned long long tot = mu_old + W;       // mu after this step's insertion
-
-    const T* Xu = C.X + (size_t)u * C.m_max * D;
-    const T* Su = C.S + (size_t)u * C.m_max * t * D;
-    const int* cntu = C.cnt + (size_t)u * C.m_max;
+    StepToken tk;
+    tk.n = n; tk.e = e; tk.slot = slot; tk.has_ins = has_ins; tk.W = W; tk.tot = tot;
+    tk.kE = kE; tk.vE = vE; tk.knew = knew_u; tk.vnew = vnew_u;
 
     // ---- nearest representative of k_e over this block's slice of the packed heads ----
     Best bst;
     bst.d2 = ~0ull; bst.idx = INT_MAX; bst.pad = 0;
     if (has_ins) {
         if (m > 0) {
-            const T* Xhu = C.Xh + (size_t)u * C.m_max * kHeadDims;
-            const float* xhnu = C.xhn + (size_t)u * C.m_max;
-            uint32_t kb0[4];
-            float kn = 0.f;
-            {
-                const uint4 r = krow[tq];
-                float f[8];
-                Elem<T>::unpack(r, f);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) kn = fmaf(f[j], f[j], kn);
-                kb0[0] = g == 0 ? r.x : 0u; kb0[1] = g == 0 ? r.y : 0u;
-                kb0[2] = g == 0 ? r.z : 0u; kb0[3] = g == 0 ? r.w : 0u;
-            }
-            kn += __shfl_xor_sync(0xffffffffu, kn, 1);
-            kn += __shfl_xor_sync(0xffffffffu, kn, 2);
-            const float d2f = (float)((double)C.delta2_fx * (1.0 / 4294967296.0));
             const int per = (((m + splits - 1) / splits) + 15) & ~15;       // slices are whole tiles
-            const int c0 = blockIdx.x * per, c1 = min(m, c0 + per);
-            auto exact_row = [&](int row) {                                  // exact D2 of one flagged row, by the warp
-                unsigned long long acc = 0;
-                if (lane < LPR) {
-                    float xf[8], kf[8];
-                    Elem<T>::unpack(*reinterpret_cast<const uint4*>(Xu + (size_t)row * D + lane * 8), xf);
-                    Elem<T>::unpack(krow[lane], kf);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) acc += fx_sqdiff(xf[j], kf[j]);
-                }
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-                if (better(acc, row, bst)) { bst.d2 = acc; bst.idx = row; }
-            };
-            constexpr int kTiles = 2;
-            for (int base = c0 + warp * 16 * kTiles; base < c1; base += NW * 16 * kTiles) {
-                uint4 ha[kTiles], hc[kTiles];
-                float xa[kTiles], xb[kTiles];
-#pragma unroll
-                for (int i = 0; i < kTiles; ++i) {
-                    const int ra = base + i * 16 + g, rb = ra + 8;
-                    const bool va = ra < c1, vb = rb < c1;
-                    ha[i] = ldg16(Xhu + (size_t)(va ? ra : c1 - 1) * kHeadDims + tq * 8);
-                    hc[i] = ldg16(Xhu + (size_t)(vb ? rb : c1 - 1) * kHeadDims + tq * 8);
-                    xa[i] = va ? xhnu[ra] : 0.f;
-                    xb[i] = vb ? xhnu[rb] : 0.f;
-                }
-#pragma unroll
-                for (int i = 0; i < kTiles; ++i) {
-                    const int ra = base + i * 16 + g, rb = ra + 8;
-                    float sc[4] = {0.f, 0.f, 0.f, 0.f};
-                    mma_bf16_16816(sc, ha[i].x, hc[i].x, ha[i].y, hc[i].y, kb0[0], kb0[1]);
-                    mma_bf16_16816(sc, ha[i].z, hc[i].z, ha[i].w, hc[i].w, kb0[2], kb0[3]);
-                    const float na = xa[i] + kn, nb = xb[i] + kn;
-                    const bool fa = ra < c1 && tq == 0 && (na - 2.f * sc[0]) <= d2f + 1.220703125e-4f * na;
-                    const bool fb = rb < c1 && tq == 0 && (nb - 2.f * sc[2]) <= d2f + 1.220703125e-4f * nb;
-                    unsigned ma = __ballot_sync(0xffffffffu, fa), mb = __ballot_sync(0xffffffffu, fb);
-                    while (ma) { exact_row(base + i * 16 + ((__ffs(ma) - 1) >> 2)); ma &= ma - 1; }
-                    while (mb) { exact_row(base + i * 16 + 8 + ((__ffs(mb) - 1) >> 2)); mb &= mb - 1; }
-                }
-            }
+            const int c0 = blockIdx.x * per;
+            head_scan_slice<D, 2>(C, u, c0, min(m, c0 + per), krow, NW, bst);
         }
         bst = block_best(bst, smb);
         if (tid == 0) C.part1[(size_t)u * splits + blockIdx.x] = bst;
@@ -176,7 +392,7 @@ __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bf
     int* rix = reinterpret_cast<int*>(scratch + NW * 16 * 64) + warp * kTauRows;
     float* rwt = reinterpret_cast<float*>(scratch + NW * (16 * 64 + kTauRows * 4)) + warp * kTauRows;
     const int wn = min(n + 1, w);
-    const int n_a = (m + 15) >> 4, n_b = (s + 15) >> 4, n_c = (wn + 15) >> 4, n_v = n_b + n_c;
+    const int n_a = (m + 15) >> 4;
     // Roles. The unit's TW warps are dealt to the two queues in proportion to the rows behind them (cluster rows
     // are not counted anywhere: at most t per cluster and at most one per inserted token, at least one per cluster).
     const int TW = splits * NW, gw = blockIdx.x * NW + warp;
@@ -213,104 +429,7 @@ __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bf
     }
 #pragma unroll
     for (int j = 0; j < D / 16; ++j) S.acc[j][0] = S.acc[j][1] = S.acc[j][2] = S.acc[j][3] = 0.f;
-    {
-        const T* Mku = C.Mk + (size_t)u * s * D;
-        const T* Mvu = C.Mv + (size_t)u * s * D;
-        const float* MiWu = C.MinvW + (size_t)u * s;
-        const T* Rk = C.ringK + (size_t)u * w * D;
-        const T* Rv = C.ringV + (size_t)u * w * D;
-        const float mu_over_s = (float)tot / (float)s;
-        const float inv_we = W ? 1.f / (float)W : 0.f;
-        int item = is_v ? vi : __shfl_sync(0xffffffffu, t1, 0);
-        while (item < n_v) {
-            int next = 0;
-            if (lane == 0) next = VW + (int)atomicAdd(&C.qnext2[u], 1u);     // asked for early, needed late
-            // 16 value samples (weight mu/(s W), numerator only) or 16 window rows (weight 1, both sums)
-            const bool isM = item < n_b;
-            const int base = (isM ? item : item - n_b) * 16;
-            const int lim = isM ? s : wn;
-            const T* Kb = isM ? Mku : Rk;
-            const T* Vb = isM ? Mvu : Rv;
-            const int ia = min(base + g, lim - 1), ib = min(base + g + 8, lim - 1);
-            bool va = base + g < lim, vb = base + g + 8 < lim;
-            const int iv[4] = {min(base + 2 * tq, lim - 1), min(base + 2 * tq + 1, lim - 1), min(base + 2 * tq + 8, lim - 1),
-                               min(base + 2 * tq + 9, lim - 1)};
-            const T* pka = Kb + (size_t)ia * D;
-            const T* pkb = Kb + (size_t)ib * D;
-            const T* pv[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) pv[i] = Vb + (size_t)iv[i] * D;
-            float wa_in = 1.f, wb_in = 1.f;
-            unsigned sub = 0;                     // rows of this tile that are scored from another place
-            if (isM) {
-                wa_in = MiWu[ia];                 // 1/W, 0 for a null slot
-                wb_in = MiWu[ib];
-            } else if (w && slot >= base && slot < base + 16) {
-                // the new token's row: not in the ring yet, read from the call's input
-                if (ia == slot) pka = knew_u;
-                if (ib == slot) pkb = knew_u;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) if (iv[i] == slot) pv[i] = vnew_u;
-            }
-            uint4 ka[NC], kb[NC], v[4][D / 64];
-            load_keys_stream<D>(pka, pkb, tq, ka, kb);           // keys and values in flight together
-            load_values_stream<D>(pv, g, v);
-            if (isM && W > 0) {
-                // UpdateMatrixProduct for the 16 slots of this tile: four Philox blocks, flipped while the rows
-                // are on their way; a slot that takes the leaving token is scored from that token's rows
-                unsigned nib = 0;
-                if (lane < 4) {
-                    const int blk = (base >> 2) + lane;
-                    if (blk * 4 < s) {
-                        const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)blk, 1u), C.key0, C.key1);
-                        const uint32_t words[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-                        for (int qq = 0; qq < 4; ++qq)
-                            if (blk * 4 + qq < s && coin_value(words[qq], tot, W)) nib |= 1u << qq;
-                    }
-                }
-                sub = __shfl_sync(0xffffffffu, nib, 0) | (__shfl_sync(0xffffffffu, nib, 1) << 4) |
-                      (__shfl_sync(0xffffffffu, nib, 2) << 8) | (__shfl_sync(0xffffffffu, nib, 3) << 12);
-                if (sub) {                        // rare: about s / (tokens inserted) slots per step
-                    if ((sub >> g) & 1u) { wa_in = inv_we; for (int c = 0; c < NC; ++c) ka[c] = ldg16(kE + c * 32 + tq * 8); }
-                    if ((sub >> (g + 8)) & 1u) { wb_in = inv_we; for (int c = 0; c < NC; ++c) kb[c] = ldg16(kE + c * 32 + tq * 8); }
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int r = 2 * tq + (i & 1) + (i >> 1) * 8;
-                        if ((sub >> r) & 1u)
-                            for (int cc = 0; cc < D / 64; ++cc) v[i][cc] = ldg16(vE + cc * 64 + g * 8);
-                    }
-                }
-            }
-            float wza = 1.f, wzb = 1.f;
-            if (isM) {
-                va = va && wa_in != 0.f;
-                vb = vb && wb_in != 0.f;
-                wza = va ? mu_over_s * wa_in : 0.f;
-                wzb = vb ? mu_over_s * wb_in : 0.f;
-            }
-            float p[4];
-            tile_scores<D, D>(S, ka, kb, va, vb, qb, p);
-            if (!isM) {
-                S.tau0 += p[0] + p[2];
-                S.tau1 += p[1] + p[3];
-            }
-            const float pz[4] = {wza * p[0], wza * p[1], wzb * p[2], wzb * p[3]};
-            tile_values<D>(S, pz, v, g, tq);
-            while (sub) {                         // the replaced slots take (k_e, v_e): half a warp per row
-                const int i = base + __ffs(sub) - 1;
-                sub &= sub - 1;
-                if (lane < LPR) reinterpret_cast<uint4*>(C.Mk + ((size_t)u * s + i) * D)[lane] = krow[lane];
-                else if (lane < 2 * LPR) reinterpret_cast<uint4*>(C.Mv + ((size_t)u * s + i) * D)[lane - LPR] = vrow[lane - LPR];
-                if (lane == 31) {
-                    C.MW[(size_t)u * s + i] = W;
-                    C.MinvW[(size_t)u * s + i] = inv_we;
-                    C.Mtok[(size_t)u * s + i] = e;
-                }
-            }
-            item = __shfl_sync(0xffffffffu, next, 0);
-        }
-    }
+    value_scan<D>(S, qb, C, u, tk, krow, vrow, is_v ? vi : __shfl_sync(0xffffffffu, t1, 0), &C.qnext2[u], VW);
     // value warps that are done help with whatever clusters are left (one tile in flight: the accumulators are live)
     if (is_v) cluster_scan<D, D, 1>(S, qb, C, u, m, __shfl_sync(0xffffffffu, t1, 0), __shfl_sync(0xffffffffu, t2, 0), &C.qnext[u],
                                     2 * CW, als, rix, rwt);
@@ -373,70 +492,7 @@ __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bf
     const bool patched = has_ins && !is_full;
     float* pmx = sred;                                // [G] maximum the correction is relative to
     float* pdl = sred + 8;                            // [G] the correction
-    if (warp == 0) {
-        if (patched) {
-            const int c = joins ? bb.idx : 0;
-            const int n_old = joins ? cntu[c] : 0;
-            const int nrow_old = !joins ? 0 : (n_old >= 2 ? t : 1);
-            const int R = nrow_old + 1;
-            auto rowptr = [&](int r) -> const T* {
-                if (r >= nrow_old) return kE;
-                return n_old >= 2 ? Su + ((size_t)c * t + r) * D : Xu + (size_t)c * D;
-            };
-            for (int r0 = 0; r0 < R; r0 += 16) {
-                const int ra = r0 + g, rb = r0 + g + 8;
-                uint4 ka[NC], kb[NC];
-                load_keys<D>(rowptr(min(ra, R - 1)), rowptr(min(rb, R - 1)), tq, ka, kb);
-                float sc[4];
-                tile_raw_scores<D>(ka, kb, qb, sc);
-                if (ra < R) { psc[ra][2 * tq] = sc[0]; psc[ra][2 * tq + 1] = sc[1]; }
-                if (rb < R) { psc[rb][2 * tq] = sc[2]; psc[rb][2 * tq + 1] = sc[3]; }
-            }
-            // the cluster coins of e (the same draws apply_cluster takes)
-            unsigned long long coins = 0;
-            if (joins) {
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const int j = half * 32 + lane;
-                    bool hit = false;
-                    if (j < t) {
-                        const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)(j >> 2), 0u), C.key0, C.key1);
-                        const uint32_t word = (j & 3) == 0 ? r.x : (j & 3) == 1 ? r.y : (j & 3) == 2 ? r.z : r.w;
-                        hit = coin_cluster(word, (uint32_t)n_old + 1u);
-                    }
-                    coins |= (unsigned long long)__ballot_sync(0xffffffffu, hit) << (32 * half);
-                }
-            }
-            __syncwarp();
-            if (lane < G) {
-                const float se = psc[nrow_old][lane];
-                float mx = se;
-                for (int r = 0; r < nrow_old; ++r) mx = fmaxf(mx, psc[r][lane]);
-                const float ee = __expf(se - mx);
-                float delta;
-                if (!joins) {
-                    delta = ee;                                   // a new singleton cluster: weight 1
-                } else if (n_old >= 2) {
-                    float so = 0.f, sn = 0.f;
-                    for (int j = 0; j < t; ++j) {
-                        const float ej = __expf(psc[j][lane] - mx);
-                        so += ej;
-                        sn += ((coins >> j) & 1ull) ? ee : ej;
-                    }
-                    delta = ((float)(n_old + 1) * sn - (float)n_old * so) / (float)t;
-                } else {
-                    const float ex = __expf(psc[0][lane] - mx);
-                    const int ne = __popcll(coins);
-                    delta = 2.f * ((float)ne * ee + (float)(t - ne) * ex) / (float)t - ex;
-                }
-                pmx[lane] = mx;
-                pdl[lane] = delta;
-            }
-        } else if (lane < G) {
-            pmx[lane] = -INFINITY;
-            pdl[lane] = 0.f;
-        }
-    }
+    if (warp == 0) tau_correction<D, G>(C, u, tk, qb, patched, joins, bb.idx, psc, pmx, pdl);
     // Merge of the blocks' partials {max, tau, z[D]}, first half: per head the maximum over the partials, the
     // partition sum under it and every partial's factor exp(max_i - max) (warps 1.. while warp 0 is busy above).
     float* fac = smp;                                 // [splits][8]
