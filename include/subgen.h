@@ -84,6 +84,12 @@ typedef struct subgen_config {
     int step_mode;          /* how subgen_step runs on bf16 handles: SUBGEN_STEP_AUTO (0) picks by the number of
                              * units, SUBGEN_STEP_FUSED one kernel per step, SUBGEN_STEP_SPLIT three kernels
                              * (insertion, cluster scan, value scan). Same results either way. */
+    int unit_stride;        /* Sharding: a handle that serves part of a larger job (some KV heads of every sequence, or */
+    int unit_offset;        /* some sequences) should draw exactly the coins the whole job would. The Philox counter's
+                             * unit index of this handle's (seq, kvhead) is seq * unit_stride + unit_offset + kvhead;
+                             * unit_stride = 0 means Hkv (with unit_offset = 0: the plain numbering seq * Hkv + kvhead).
+                             * A shard holding KV heads [h0, h1) of a job with HKV heads: unit_stride = HKV,
+                             * unit_offset = h0; a shard holding sequences [b0, b1): unit_offset = b0 * Hkv. */
 } subgen_config;
 
 #define SUBGEN_STEP_AUTO 0
@@ -222,7 +228,7 @@ int subgen_step_kernels(const subgen_t* h);
  * conversation between GPUs or survive a restart, so the state between two calls (D with its samples and counts, M
  * with its weights, mu, the window ring, the per-unit counters and status bits) can be written to one host blob and
  * loaded into another handle. The blob stores cluster arrays only up to the largest cluster count of any unit.
- * Loading needs a handle created with the same B, H, Hkv, d, t, s, window, dtype, delta and seed (the Philox
+ * Loading needs a handle created with the same B, H, Hkv, d, t, s, window, dtype, delta, seed and unit numbering (the Philox
  * draws of later tokens depend on the seed and on the token index, which the blob carries); m_max may differ as
  * long as it holds the stored clusters, which is also the way to continue a stream with a larger capacity.
  * Everything the handle held before is discarded. After a load the handle continues the stream exactly as the

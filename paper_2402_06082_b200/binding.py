@@ -35,7 +35,8 @@ class SubgenConfig(C.Structure):
     _fields_ = [("B", C.c_int), ("H", C.c_int), ("Hkv", C.c_int), ("d", C.c_int), ("delta", C.c_float),
                 ("t", C.c_int), ("s", C.c_int), ("window", C.c_int), ("seed", C.c_uint64), ("dtype", C.c_int),
                 ("m_max", C.c_int), ("splits", C.c_int), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-                ("stream", C.c_void_p), ("nq_max", C.c_int), ("bounded", C.c_int), ("step_mode", C.c_int)]
+                ("stream", C.c_void_p), ("nq_max", C.c_int), ("bounded", C.c_int), ("step_mode", C.c_int),
+                ("unit_stride", C.c_int), ("unit_offset", C.c_int)]
 
 
 class StateView(C.Structure):
@@ -139,7 +140,7 @@ class SubGen:
 
     def __init__(self, B, H, d, delta, t, s, window, seed=0, *, Hkv=None, dtype=torch.bfloat16, m_max=0, splits=0,
                  stream: Optional[torch.cuda.Stream] = None, bounded: bool = False, nq_max: int = 1,
-                 step_mode: str = "auto"):
+                 step_mode: str = "auto", unit_stride: int = 0, unit_offset: int = 0):
         self._L = load()
         self._h = None
         if not torch.cuda.is_available():
@@ -150,7 +151,7 @@ class SubGen:
         self.stream = stream or torch.cuda.current_stream()
         cfg = SubgenConfig(self.B, self.H, self.Hkv, self.d, float(delta), self.t, self.s, self.window, int(seed),
                            _dtype_code(dtype), int(m_max), int(splits), None, 0, self.stream.cuda_stream, int(nq_max), int(bool(bounded)),
-                           STEP_MODES[step_mode])
+                           STEP_MODES[step_mode], int(unit_stride), int(unit_offset))
         nbytes = self._L.subgen_workspace_bytes(C.byref(cfg))
         if nbytes == 0:
             raise SubgenError(self._L.subgen_last_error().decode())

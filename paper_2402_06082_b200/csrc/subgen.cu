@@ -81,6 +81,11 @@ bool resolve(const subgen_config* c, Dims* o, const char** why) {
     if (d.m_max < 1) { *why = "m_max must be positive"; return false; }
     if (!(c->delta >= 0.f) || !isfinite(c->delta) || c->delta > 32768.f) { *why = "delta must be finite, in [0, 32768]"; return false; }
     if (c->dtype != SUBGEN_DTYPE_FP32 && c->dtype != SUBGEN_DTYPE_BF16) { *why = "unknown dtype"; return false; }
+    if (c->unit_stride < 0 || (c->unit_stride && c->unit_stride < d.Hkv) || c->unit_offset < 0 ||
+        (long long)(d.B - 1) * (c->unit_stride ? c->unit_stride : d.Hkv) + c->unit_offset + d.Hkv - 1 > 0x7fffffffLL) {
+        *why = "unit_stride must be 0 or >= Hkv, unit_offset >= 0, and the largest unit index must fit 31 bits";
+        return false;
+    }
     if (c->step_mode < SUBGEN_STEP_AUTO || c->step_mode > SUBGEN_STEP_SPLIT) { *why = "unknown step_mode"; return false; }
     if ((long long)d.B * d.Hkv > 65535) { *why = "B * Hkv must be <= 65535"; return false; }
     d.E = c->dtype == SUBGEN_DTYPE_FP32 ? 4 : 2;
@@ -237,6 +242,8 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
     C.part_tau = (float*)(w + L.part_tau); C.MinvW = (float*)(w + L.MinvW);
     C.pairs = (unsigned long long*)(w + L.pairs);
     C.bounded = h->cfg.bounded ? 1 : 0;
+    C.uid_stride = h->cfg.unit_stride ? h->cfg.unit_stride : d.Hkv;
+    C.uid_off = h->cfg.unit_offset;
     C.thr2 = (unsigned long long*)(w + L.thr2); C.level = (int*)(w + L.level);
     return C;
 }
@@ -491,11 +498,14 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         // Key phase. Many units with few representatives each: one persistent block per unit walks its chunks
         // (subgen_prefill_persist.cuh). Few units: a score and a resolve kernel per chunk, the representatives of a
         // unit spread over many blocks.
-        const bool persist = tc && (h->persist >= 0 ? h->persist == 1 : d.U >= 24);
+        // Bounded handles always walk their chunks in the persistent kernel: it is the one that can end a chunk at
+        // the key that finds the budget used up and insert that key on its own.
+        const bool persist = tc && (C.bounded || (h->persist >= 0 ? h->persist == 1 : d.U >= 24));
         h->pf_persist = persist && h->prof;
         if (persist) {
             h->pf_phase_dev = phase_ns;
-            prefill_keys_persist_kernel<<<d.U, kPpThreads, kPpSmemBytes, h->st>>>(C, a, h->prof ? phase_ns : nullptr);
+            if (C.bounded) prefill_keys_persist_kernel<true><<<d.U, kPpThreads, kPpSmemBytes, h->st>>>(C, a, h->prof ? phase_ns : nullptr);
+            else prefill_keys_persist_kernel<false><<<d.U, kPpThreads, kPpSmemBytes, h->st>>>(C, a, h->prof ? phase_ns : nullptr);
             launches += 1;
             if (int rc = mark()) return rc;
         } else {
@@ -603,7 +613,8 @@ subgen_t* subgen_create_ex(const subgen_config* cfg) {
     // so it is set for the device of every handle that can launch the kernel
     if (cfg->dtype == SUBGEN_DTYPE_BF16 && d.D == 128 &&
         (cudaFuncSetAttribute(prefill_score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) != cudaSuccess ||
-         cudaFuncSetAttribute(prefill_keys_persist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPpSmemBytes) != cudaSuccess)) {
+         cudaFuncSetAttribute(prefill_keys_persist_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPpSmemBytes) != cudaSuccess ||
+         cudaFuncSetAttribute(prefill_keys_persist_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPpSmemBytes) != cudaSuccess)) {
         fail(SUBGEN_ECUDA, "subgen_create: cudaFuncSetAttribute failed: %s", cudaGetErrorString(cudaGetLastError()));
         if (h->owns) cudaFree(h->ws);
         delete h;
@@ -625,9 +636,9 @@ subgen_t* subgen_create_ex(const subgen_config* cfg) {
         if (strcmp(env, "split") == 0) h->fused = false;
     }
     if (h->cfg.bounded) {
-        // merges renumber the clusters in the middle of a chunk, which the chunked prefill does not handle:
-        // bounded handles insert their prompts token by token
-        h->seq_prefill = true;
+        // merges renumber the clusters in the middle of a chunk; only the persistent key kernel (bf16, d = 128) ends
+        // a chunk at such a key. Other bounded handles insert their prompts token by token.
+        if (!(cfg->dtype == SUBGEN_DTYPE_BF16 && d.D == 128) || h->mma_score) h->seq_prefill = true;
         if (reset_thresholds(h) != cudaSuccess) {
             fail(SUBGEN_ECUDA, "subgen_create: threshold initialisation failed");
             if (h->owns) cudaFree(h->ws);
@@ -936,6 +947,7 @@ struct CkptHeader {
     float delta;
     uint32_t pad;
     uint64_t seed, payload_bytes;
+    int32_t unit_stride, unit_offset;      // numbering of the units in the Philox counter (resolved: stride >= Hkv)
 };
 
 struct CkptArray {
@@ -998,10 +1010,11 @@ int subgen_checkpoint_save(subgen_t* h, void* host, size_t bytes, size_t* writte
     if (bytes < need) return fail(SUBGEN_EINVAL, "subgen_checkpoint_save: buffer needs %zu bytes", need);
     CkptHeader hd;
     memset(&hd, 0, sizeof hd);
-    hd.magic = kCkptMagic; hd.version = 1; hd.dtype = (uint32_t)h->cfg.dtype;
+    hd.magic = kCkptMagic; hd.version = 2; hd.dtype = (uint32_t)h->cfg.dtype;
     hd.B = h->d.B; hd.H = h->d.H; hd.Hkv = h->d.Hkv; hd.d = h->d.D; hd.t = h->d.t; hd.s = h->d.s; hd.window = h->d.w;
     hd.m_rows = m_rows; hd.delta = h->cfg.delta; hd.seed = h->cfg.seed; hd.payload_bytes = payload;
     hd.pad = h->cfg.bounded ? 1u : 0u;
+    hd.unit_stride = h->cfg.unit_stride ? h->cfg.unit_stride : h->d.Hkv; hd.unit_offset = h->cfg.unit_offset;
     memcpy(host, &hd, sizeof hd);
     char* dst = (char*)host + sizeof hd;
     for (const CkptArray& a : ckpt_arrays(h, m_rows)) {
@@ -1018,13 +1031,15 @@ int subgen_checkpoint_load(subgen_t* h, const void* host, size_t bytes) {
     if (bytes < sizeof(CkptHeader)) return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: blob shorter than its header");
     CkptHeader hd;
     memcpy(&hd, host, sizeof hd);
-    if (hd.magic != kCkptMagic || hd.version != 1) return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: not a checkpoint of this library version");
+    if (hd.magic != kCkptMagic || hd.version != 2) return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: not a checkpoint of this library version");
     const Dims& d = h->d;
     if (hd.B != d.B || hd.H != d.H || hd.Hkv != d.Hkv || hd.d != d.D || hd.t != d.t || hd.s != d.s || hd.window != d.w ||
         (int)hd.dtype != h->cfg.dtype || hd.seed != h->cfg.seed || memcmp(&hd.delta, &h->cfg.delta, sizeof(float)) != 0 ||
-        hd.pad != (h->cfg.bounded ? 1u : 0u))
+        hd.pad != (h->cfg.bounded ? 1u : 0u) || hd.unit_stride != (h->cfg.unit_stride ? h->cfg.unit_stride : d.Hkv) ||
+        hd.unit_offset != h->cfg.unit_offset)
         return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: the checkpoint was written with another configuration "
-                    "(B, H, Hkv, d, t, s, window, dtype, delta, seed and the bounded flag must match; only m_max may differ)");
+                    "(B, H, Hkv, d, t, s, window, dtype, delta, seed, the bounded flag and the unit numbering must match; "
+                    "only m_max may differ)");
     if (hd.m_rows < 0 || hd.m_rows > d.m_max)
         return fail(SUBGEN_EINVAL, "subgen_checkpoint_load: the checkpoint holds %d clusters per unit, this handle's m_max is %d", hd.m_rows, d.m_max);
     const size_t payload = ckpt_payload(h, hd.m_rows);

@@ -130,11 +130,20 @@ template <typename T> struct Cache {
     unsigned* qnext;     // [U] next work item of the cluster scan's per-unit queue
     unsigned* qnext2;    // [U] same for the scan of M and the window
     unsigned long long* pairs;   // [U] (key, representative) pairs scored by the chunked prefill so far
+    int uid_stride, uid_off;     // numbering of the units in the Philox counter, see unit_id()
     // bounded-m variant: m_max is a budget, the threshold doubles and clusters merge when it is exhausted
     int bounded;
     unsigned long long* thr2;    // [U] threshold in force (fixed point), starts as delta2_fx
     int* level;                  // [U] doublings so far
 };
+
+// The unit index that keys the Philox draws of unit u = seq * Hkv + kvhead of this handle. A handle that serves a
+// shard of a larger job (some of its KV heads, or some of its sequences) numbers its units as the whole job would,
+// seq * uid_stride + uid_off + kvhead, so that sharding does not change a single draw.
+template <typename T>
+__device__ __forceinline__ uint32_t unit_id(const Cache<T>& C, int u) {
+    return (uint32_t)((u / C.Hkv) * C.uid_stride + C.uid_off + (u % C.Hkv));
+}
 
 // The squared threshold a key of unit u is tested against. BND: the handle runs the bounded-m variant; it is a
 // template parameter of the insertion kernels so that the plain path carries none of the variant's code.
@@ -280,7 +289,7 @@ __device__ void make_room(const Cache<T>& C, int u, int e, const uint4* krow, Be
                 const unsigned long long n_new = (unsigned long long)n_i + (unsigned long long)n_j;
                 for (int p = tid; p < t * LPR; p += nt) {
                     const int q = p / LPR, part = p % LPR;
-                    const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)(q >> 2) + 256u * (uint32_t)i,
+                    const uint4 r = philox4x32_10(make_uint4((uint32_t)e, unit_id(C, u), (uint32_t)(q >> 2) + 256u * (uint32_t)i,
                                                              2u + 4u * (uint32_t)level), C.key0, C.key1);
                     const uint32_t word = (q & 3) == 0 ? r.x : (q & 3) == 1 ? r.y : (q & 3) == 2 ? r.z : r.w;
                     uint4* dst = reinterpret_cast<uint4*>(Su + ((size_t)j * t + q) * D) + part;
@@ -399,7 +408,7 @@ __device__ int apply_cluster(const Cache<T>& C, int u, int e, Best& best, int& m
         // slot j is written by LPR threads, one 16-byte piece each
         for (int p = tid; p < t * LPR; p += nt) {
             const int j = p / LPR, part = p % LPR;
-            const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)(j >> 2), 0u), C.key0, C.key1);
+            const uint4 r = philox4x32_10(make_uint4((uint32_t)e, unit_id(C, u), (uint32_t)(j >> 2), 0u), C.key0, C.key1);
             const uint32_t word = (j & 3) == 0 ? r.x : (j & 3) == 1 ? r.y : (j & 3) == 2 ? r.z : r.w;
             uint4* dst = reinterpret_cast<uint4*>(Su + ((size_t)c * t + j) * D) + part;
             if (coin_cluster(word, n_new)) {
@@ -463,7 +472,7 @@ __device__ int apply_insert(const Cache<T>& C, int u, int e, Best best, int m, c
     if (W > 0) {
         const unsigned long long tot = mu_old + W;
         for (int blk = tid; blk * 4 < s; blk += nt) {
-            const uint4 r = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)blk, 1u), C.key0, C.key1);
+            const uint4 r = philox4x32_10(make_uint4((uint32_t)e, unit_id(C, u), (uint32_t)blk, 1u), C.key0, C.key1);
             const uint32_t words[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
             for (int q = 0; q < 4; ++q) {

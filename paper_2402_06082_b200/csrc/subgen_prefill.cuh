@@ -170,7 +170,7 @@ __global__ void prefill_coin_kernel(Cache<__nv_bfloat16> C, PrefillArgs a, int s
         const unsigned long long thr = Tb[i];
         if (thr == 0ull) continue;                          // W = 0: never sampled
         const int e = r.ins_lo + i;
-        const uint4 rr = philox4x32_10(make_uint4((uint32_t)e, (uint32_t)u, (uint32_t)blk, 1u), C.key0, C.key1);
+        const uint4 rr = philox4x32_10(make_uint4((uint32_t)e, unit_id(C, u), (uint32_t)blk, 1u), C.key0, C.key1);
         if ((unsigned long long)rr.x < thr) win[0] = e;
         if ((unsigned long long)rr.y < thr) win[1] = e;
         if ((unsigned long long)rr.z < thr) win[2] = e;
@@ -436,7 +436,7 @@ __global__ void __launch_bounds__(kResolveThreads) prefill_resolve_kernel(Cache<
     for (int p = tid; p < cl * nblk; p += kResolveThreads) {
         const int j = p / nblk, blk = p % nblk;
         if (cid[j] < 0) continue;
-        const uint4 rr = philox4x32_10(make_uint4((uint32_t)(e0 + j), (uint32_t)u, (uint32_t)blk, 0u), C.key0, C.key1);
+        const uint4 rr = philox4x32_10(make_uint4((uint32_t)(e0 + j), unit_id(C, u), (uint32_t)blk, 0u), C.key0, C.key1);
         const uint32_t words[4] = {rr.x, rr.y, rr.z, rr.w};
         unsigned long long bits = 0;
 #pragma unroll

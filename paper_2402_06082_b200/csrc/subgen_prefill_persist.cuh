@@ -39,6 +39,7 @@ struct PpSmem {                                   // after a 1024-byte aligned b
     unsigned cand[kPpCand];                       // key | representative << 7
     unsigned char is_open[kChunk], has_later[kChunk], dropped[kChunk];
     unsigned long long mbar[2];
+    unsigned long long sm_w[2];                   // bounded handles: {unused, ||k||^2 | ||k head||^2 << 32} of the key inserted on its own
     unsigned tmem_base, ncand, failed, far_mask[4]; // far_mask: keys with no old representative within delta
     int opened, full;
 };
@@ -47,6 +48,10 @@ constexpr size_t kPpSmemBytes = sizeof(PpSmem) + 1024;
 constexpr int kPpPhases = 8;   // staging, MMA wait, read-back, tile store + issue, exact follow-up | openings, ranks + coins, writes
 
 // phase_ns: NULL, or [U][kPpPhases] SM cycles thread 0 of the unit's block spent in each phase (profiling).
+// BND: the handle runs the bounded-m variant. A key that needs a cluster when the budget is used up ends its chunk
+// early: the keys before it are resolved as a shorter chunk, the key itself is inserted on its own (threshold
+// doubling and merge sweep, make_room), and the walk resumes behind it under the new threshold and cluster numbering.
+template <bool BND>
 __global__ void __launch_bounds__(kPpThreads, 2) prefill_keys_persist_kernel(Cache<__nv_bfloat16> C, PrefillArgs a,
                                                                             unsigned long long* phase_ns) {
     typedef __nv_bfloat16 T;
@@ -57,14 +62,13 @@ __global__ void __launch_bounds__(kPpThreads, 2) prefill_keys_persist_kernel(Cac
     const Range r = unit_range(C, a, u);
     const int len = r.ins_hi - r.ins_lo;
     if (len <= 0) return;
-    const int nchunks = (len + kChunk - 1) / kChunk;
     const int t = C.t;
-    const unsigned long long thr = C.delta2_fx;
+    unsigned long long thr = BND ? C.thr2[u] : C.delta2_fx;       // bounded handles: the threshold in force
     T* Xu = C.X + (size_t)u * C.m_max * D;
     T* Su = C.S + (size_t)u * C.m_max * t * D;
     int* cntu = C.cnt + (size_t)u * C.m_max;
     int* stoku = C.stok + (size_t)u * C.m_max * t;
-    const float d2f = (float)((double)C.delta2_fx * (1.0 / 4294967296.0));
+    float d2f = (float)((double)thr * (1.0 / 4294967296.0));
     constexpr float kOneMinusG = 1.f - 1.220703125e-4f;
     const uint32_t sA = (uint32_t)__cvta_generic_to_shared(sm.A);
     const uint32_t sB = (uint32_t)__cvta_generic_to_shared(sm.B[0]);
@@ -143,8 +147,8 @@ __global__ void __launch_bounds__(kPpThreads, 2) prefill_keys_persist_kernel(Cac
     };
     const uint4* keys4 = reinterpret_cast<const uint4*>(sm.keys);
 
-    for (int chunk = 0; chunk < nchunks && ok; ++chunk) {
-        const int e0 = r.ins_lo + chunk * kChunk, cl = min(kChunk, r.ins_hi - e0);
+    for (int pos = 0; pos < len && ok;) {
+        const int e0 = r.ins_lo + pos, cl = min(kChunk, r.ins_hi - e0);
         if (timing) tick = clock64();
         // ---- stage the chunk: full rows, heads as operand A (rows beyond cl are zero), per-key bookkeeping ----
         for (int p = tid; p < kChunk * LPR; p += kPpThreads) {
@@ -161,7 +165,7 @@ __global__ void __launch_bounds__(kPpThreads, 2) prefill_keys_persist_kernel(Cac
         }
         if (tid == 0) { sm.opened = 0; sm.full = 0; sm.ncand = 0; }
         // the next chunk's rows are wanted in about one chunk's time: ask for them now (one 128-byte line per thread)
-        if (chunk + 1 < nchunks) {
+        {
             const int j = tid >> 1, en = e0 + kChunk + j;
             if (en < r.ins_hi) {
                 const char* nx = reinterpret_cast<const char*>(key_row<D>(C, a, r, u, en)) + (tid & 1) * 128;
@@ -373,17 +377,18 @@ __global__ void __launch_bounds__(kPpThreads, 2) prefill_keys_persist_kernel(Cac
             if (lane == 0) sm.far_mask[warp] = fm;
         }
         __syncthreads();
-        int n_open = 0;
+        int n_open = 0, stop = -1;                                     // stop: the key that found the budget used up (BND)
         const uint32_t gaddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((JT & 1) * 128);
-        for (int wd = 0; wd < 4; ++wd) {
+        for (int wd = 0; wd < 4 && stop < 0; ++wd) {
             unsigned fm = sm.far_mask[wd];                             // uniform
             while (fm) {
                 const int j = wd * 32 + __ffs(fm) - 1;
                 fm &= fm - 1;
                 if (!(sm.new_d2[j] > thr)) continue;                   // uniform: written before the last barrier
                 const int cidx = m_old + n_open;
-                if (cidx >= C.m_max) {                                 // capacity: the key is dropped from D
-                    if (tid == 0) { sm.dropped[j] = 1; sm.full = 1; }
+                if (cidx >= C.m_max) {
+                    if (BND) { stop = j; break; }                      // the chunk ends before this key
+                    if (tid == 0) { sm.dropped[j] = 1; sm.full = 1; }  // capacity: the key is dropped from D
                     continue;
                 }
                 if (col_half == 0) {
@@ -422,10 +427,11 @@ __global__ void __launch_bounds__(kPpThreads, 2) prefill_keys_persist_kernel(Cac
             }
         }
         if (tid == 0) sm.opened = n_open;
+        const int ce = stop >= 0 ? stop : cl;                          // keys resolved in this turn
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
         lap(5);
-        if (tid < cl) {
+        if (tid < ce) {
             const int j = tid;
             int c;
             if (sm.is_open[j]) c = sm.opened_at[j];
@@ -435,11 +441,11 @@ __global__ void __launch_bounds__(kPpThreads, 2) prefill_keys_persist_kernel(Cac
             sm.cid[j] = c;
         }
         __syncthreads();
-        if (tid < cl) {
+        if (tid < ce) {
             const int j = tid, c = sm.cid[j];
             int rank = 1;
             bool lat = false;
-            for (int i = 0; i < cl; ++i) {
+            for (int i = 0; i < ce; ++i) {
                 if (i < j && sm.cid[i] == c) ++rank;
                 if (i > j && sm.cid[i] == c) lat = true;
             }
@@ -448,10 +454,10 @@ __global__ void __launch_bounds__(kPpThreads, 2) prefill_keys_persist_kernel(Cac
         }
         __syncthreads();
         const int nblk = (t + 3) >> 2;
-        for (int p = tid; p < cl * nblk; p += kPpThreads) {
+        for (int p = tid; p < ce * nblk; p += kPpThreads) {
             const int j = p / nblk, blk = p % nblk;
             if (sm.cid[j] < 0) continue;
-            const uint4 rr = philox4x32_10(make_uint4((uint32_t)(e0 + j), (uint32_t)u, (uint32_t)blk, 0u), C.key0, C.key1);
+            const uint4 rr = philox4x32_10(make_uint4((uint32_t)(e0 + j), unit_id(C, u), (uint32_t)blk, 0u), C.key0, C.key1);
             const uint32_t words[4] = {rr.x, rr.y, rr.z, rr.w};
             unsigned long long bits = 0;
 #pragma unroll
@@ -460,16 +466,16 @@ __global__ void __launch_bounds__(kPpThreads, 2) prefill_keys_persist_kernel(Cac
             if (bits) atomicOr(&sm.succ[j], bits);
         }
         __syncthreads();
-        if (tid < cl) {
+        if (tid < ce) {
             const int j = tid;
             unsigned long long lm = 0;
-            for (int i = j + 1; i < cl; ++i) if (sm.cid[i] == sm.cid[j]) lm |= sm.succ[i];
+            for (int i = j + 1; i < ce; ++i) if (sm.cid[i] == sm.cid[j]) lm |= sm.succ[i];
             sm.later[j] = lm;
         }
         __syncthreads();
         lap(6);
         const unsigned long long tmask = t == 64 ? ~0ull : ((1ull << t) - 1ull);
-        for (int j = warp; j < cl; j += kPpWarps) {                    // writes: a warp per key
+        for (int j = warp; j < ce; j += kPpWarps) {                    // writes: a warp per key
             const int c = sm.cid[j];
             if (c < 0) continue;
             const int e = e0 + j;
@@ -519,12 +525,13 @@ __global__ void __launch_bounds__(kPpThreads, 2) prefill_keys_persist_kernel(Cac
             if (!sm.has_later[j] && lane == 0) cntu[c] = sm.nnew[j];   // last key of its cluster in this chunk
         }
         __syncthreads();                                               // the writes above are read by the next chunk
-        pairs += (unsigned long long)cl * (unsigned long long)m_old;
+        pairs += (unsigned long long)ce * (unsigned long long)m_old;
         m = m_old + sm.opened;
+        const bool last_turn = stop < 0 && pos + ce == len;
         if (tid == 0) {
             if (sm.full) atomicOr(&C.status[u], 1);
-            if (chunk == nchunks - 1) {                                // the most recent insertion of this unit
-                const int j = cl - 1;
+            if (last_turn && ce > 0) {                                 // the most recent insertion of this unit
+                const int j = ce - 1;
                 C.last_cid[u] = sm.cid[j];
                 C.last_open[u] = sm.is_open[j] || sm.dropped[j];
                 C.last_d2[u] = (sm.new_d2[j] <= thr && (sm.old_d2[j] > thr || sm.new_d2[j] < sm.old_d2[j])) ? sm.new_d2[j] : sm.old_d2[j];
@@ -532,6 +539,43 @@ __global__ void __launch_bounds__(kPpThreads, 2) prefill_keys_persist_kernel(Cac
         }
         __syncthreads();                                               // sm.opened is reset by the next chunk's staging
         lap(7);
+        pos += ce;
+        if constexpr (BND) {
+            if (stop >= 0) {
+                // The key at `stop` is farther than the threshold from every representative and no cluster is free:
+                // the cluster half of its insertion on its own (make_room doubles the threshold and sweeps, then the
+                // key joins or opens under the new threshold).
+                const int e = e0 + stop;
+                if (tid == 0) {
+                    float kh = 0.f;
+                    for (int p = 0; p < kHeadDims / 8; ++p) {
+                        float f[8];
+                        Elem<T>::unpack(keys4[stop * LPR + p], f);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) kh = fmaf(f[q], f[q], kh);
+                    }
+                    sm.sm_w[0] = 0ull;
+                    sm.sm_w[1] = (unsigned long long)__float_as_uint(sm.kn_full[stop]) | ((unsigned long long)__float_as_uint(kh) << 32);
+                }
+                __syncthreads();
+                Best far;
+                far.d2 = ~0ull; far.idx = INT_MAX; far.pad = 0;
+                bool joined, full;
+                int m_ref = m;
+                const int m_new = apply_cluster<T, D, true>(C, u, e, far, m_ref, keys4 + stop * LPR, sm.sm_w, joined, full);
+                __syncthreads();
+                if (tid == 0 && pos + 1 == len) {
+                    C.last_cid[u] = joined ? far.idx : (full ? -1 : m_ref);
+                    C.last_open[u] = joined ? 0 : 1;
+                    C.last_d2[u] = far.d2;
+                }
+                m = m_new;
+                thr = C.thr2[u];
+                d2f = (float)((double)thr * (1.0 / 4294967296.0));
+                pos += 1;
+                __syncthreads();
+            }
+        }
     }
     if (tid == 0) {
         if (ok) {

@@ -188,7 +188,7 @@ __device__ __forceinline__ void value_scan(MmaState<D>& S, const uint32_t (&qb)[
             if (lane < 4) {
                 const int blk = (base >> 2) + lane;
                 if (blk * 4 < s) {
-                    const uint4 r = philox4x32_10(make_uint4((uint32_t)tk.e, (uint32_t)u, (uint32_t)blk, 1u), C.key0, C.key1);
+                    const uint4 r = philox4x32_10(make_uint4((uint32_t)tk.e, unit_id(C, u), (uint32_t)blk, 1u), C.key0, C.key1);
                     const uint32_t words[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
                     for (int qq = 0; qq < 4; ++qq)
@@ -282,7 +282,7 @@ __device__ __forceinline__ void tau_correction(const Cache<__nv_bfloat16>& C, in
             const int j = half * 32 + lane;
             bool hit = false;
             if (j < t) {
-                const uint4 r = philox4x32_10(make_uint4((uint32_t)tk.e, (uint32_t)u, (uint32_t)(j >> 2), 0u), C.key0, C.key1);
+                const uint4 r = philox4x32_10(make_uint4((uint32_t)tk.e, unit_id(C, u), (uint32_t)(j >> 2), 0u), C.key0, C.key1);
                 const uint32_t word = (j & 3) == 0 ? r.x : (j & 3) == 1 ? r.y : (j & 3) == 2 ? r.z : r.w;
                 hit = coin_cluster(word, (uint32_t)n_old + 1u);
             }

@@ -139,3 +139,39 @@ def test_bounded_checkpoint_resume():
         o.push_many(f32(K)[0, h], f32(V)[0, h])
         _same(b, o, 0, h, "resumed bounded handle")
         assert o.level >= 2
+
+
+def test_chunked_prefill_of_a_bounded_handle(monkeypatch):
+    """bf16 handles with d = 128 prefill chunk by chunk also when they are bounded: a chunk ends at the key that finds
+    the budget used up, that key is inserted on its own (doubling, merge sweep) and the walk resumes behind it. A long
+    prompt with several doublings, cut at awkward places, against the oracle and against the token-by-token kernel."""
+    w = synth.CFG3.scaled(B=2, H=4, Hkv=2, n_prompt=2600, ncomp=300, s=64, window=24, m_max=48, delta=0.5)
+    K, V, Q = synth.batch_stream(w, w.n_prompt + 6, "cuda")
+    Kn, Vn, Qn = f32(K), f32(V), f32(Q)
+    a = _sg(w)
+    cuts = [0, 1, 129, 130, 1000, 2600]
+    orcs = {(b, h): _oracle(w, b, h) for b in range(w.B) for h in range(w.Hkv)}
+    launches = a.launch_count
+    for lo, hi in zip(cuts[:-1], cuts[1:]):
+        a.prefill(K[:, :, lo:hi].contiguous(), V[:, :, lo:hi].contiguous())
+        for (b, h), o in orcs.items():
+            o.push_many(Kn[b, h, lo:hi], Vn[b, h, lo:hi])
+            _same(a, o, b, h, "chunked, after prefill to %d, unit %s" % (hi, (b, h)))
+    assert a.launch_count - launches < 80                 # a handful of kernels per call, not one pass per token
+    assert min(o.level for o in orcs.values()) >= 2        # the budget was exhausted more than once
+    monkeypatch.setenv("SUBGEN_PREFILL", "seq")
+    s = _sg(w)
+    s.prefill(K[:, :, :w.n_prompt].contiguous(), V[:, :, :w.n_prompt].contiguous())
+    for (b, h), o in orcs.items():
+        _same(s, o, b, h, "token by token, unit %s" % ((b, h),))
+    G = w.H // w.Hkv
+    for i in range(w.n_prompt, w.n_prompt + 6):
+        out = f32(a.step(Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous()))
+        for (b, h), o in orcs.items():
+            o.push(Kn[b, h, i], Vn[b, h, i])
+            for g in range(G):
+                hp.assert_output(out[b, h * G + g], o.query(Qn[b, h * G + g, i]), w.torch_dtype, "step %d" % i)
+    for (b, h), o in orcs.items():
+        st = _same(a, o, b, h, "end, unit %s" % ((b, h),))
+        hp.assert_rows_match_tokens(a, b, h, st, K[b, h], V[b, h])
+    assert a.status() == 0

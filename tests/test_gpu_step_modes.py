@@ -149,3 +149,47 @@ def test_fused_capacity_overflow_sets_status():
         out = sg.step(Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous())
     assert sg.status() & 1
     assert torch.isnan(out.float()).all()
+
+
+@pytest.mark.parametrize("mode", ["sequence", "head"])
+def test_sharded_handles_reproduce_the_whole_job(mode):
+    """A job cut in two shards (by sequence: 2 + 1 sequences; by KV head: 2 + 2 heads), each shard on a handle of its
+    own with the whole job's unit numbering: every shard ends in exactly the state the unsharded handle has for those
+    units (same Philox draws), and the outputs put back in place agree with the unsharded outputs up to rounding."""
+    from paper_2402_06082_b200 import sharding
+    from paper_2402_06082_b200.binding import SubGen
+    w = synth.CFG3.scaled(B=3, H=8, Hkv=4, n_prompt=500, ncomp=12, s=64, window=16, m_max=256)
+    n0, nd = w.n_prompt, 10
+    K, V, Q = synth.batch_stream(w, n0 + nd, "cuda")
+    whole = _sg(w)
+    whole.prefill(K[:, :, :n0].contiguous(), V[:, :, :n0].contiguous())
+    shards = sharding.partition(w.B, w.H, w.Hkv, 2, mode)
+    handles = []
+    for sh in shards:
+        kw = sh.handle_kwargs()
+        sg = SubGen(kw.pop("B"), kw.pop("H"), w.d, w.delta, w.t, w.s, w.window, w.philox_seed, dtype=w.torch_dtype,
+                    m_max=w.m_max, **kw)
+        sg.prefill(sh.kv_rows(K[:, :, :n0]), sh.kv_rows(V[:, :, :n0]))
+        handles.append(sg)
+    for i in range(n0, n0 + nd):
+        q, k, v = Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous()
+        ref = f32(whole.step(q, k, v))
+        full = torch.zeros(w.B, w.H, w.d, dtype=w.torch_dtype, device="cuda")
+        for sh, sg in zip(shards, handles):
+            sharding.scatter_outputs(full, sh, sg.step(sh.q_rows(q), sh.kv_rows(k), sh.kv_rows(v)))
+        got = f32(full)
+        for b in range(w.B):
+            for h in range(w.H):
+                hp.assert_output(got[b, h], ref[b, h], w.torch_dtype, "step %d seq %d head %d" % (i, b, h))
+    for sh, sg in zip(shards, handles):
+        for lb in range(sh.B_local):
+            for lh in range(sh.Hkv_local):
+                a, c = sg.export_state(lb, lh), whole.export_state(sh.b0 + lb, sh.h0 + lh)
+                for key in ("n", "m", "mu", "last_cluster", "last_opened", "last_d2"):
+                    assert a[key] == c[key], key
+                for key in ("counts", "centre_tok", "slot_tok", "m_tok", "m_w"):
+                    np.testing.assert_array_equal(a[key], c[key], err_msg=key)
+    o = hp.oracle_unit(w, 2, 3)
+    o.push_many(f32(K[2, 3]), f32(V[2, 3]))
+    last = handles[1]
+    hp.assert_state_equal(last.export_state(last.B - 1, last.Hkv - 1), o, "last unit of the job, on its shard")
