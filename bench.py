@@ -409,7 +409,7 @@ def measure(wr, args, K_steps, W_steps, world, rank, local, dist, headline):
                 "step_kernels": nk, "prefill_ms": prefill_ms, "prefill_tokens_per_s": sum(lens) / (prefill_ms * 1e-3) if sum(lens) else None,
                 "e2e_steps_per_s": e2e["value"], "gpu_launches_per_region": int(launches), "clocks": clocks,
                 "clusters_per_unit": stats1["clusters"] / wr.units}
-    traffic = ncu_traffic(dom[0], wr) if not args.prompt else None
+    traffic = ncu_traffic(dom[0], wr, dom[1])
     roofline = {"bound": "hbm", "kernel": dom[0], "achieved": achieved, "peak": peak, "peak_source": which,
                 "unit": "GB/s", "frac": achieved / peak if achieved else None, "traffic": traffic,
                 "algorithmic_bytes_per_launch": dom[1], "ms_per_launch": dom[2],
@@ -473,13 +473,14 @@ def measure(wr, args, K_steps, W_steps, world, rank, local, dist, headline):
             "launches": int(launches), "roofline": roofline, "extra": extra, "lens": lens, "varlen": varlen}
 
 
-def ncu_traffic(kernel, wr):
-    """DRAM bytes of one launch of `kernel` from the tracked record of an ncu capture (profiles/ncu_traffic.json),
-    scaled by the units processed (units share nothing, so traffic grows in proportion). None when there is no
-    record for this kernel and workload, or when the kernel's source file has changed since the capture."""
+def ncu_traffic(kernel, wr, alg_bytes):
+    """DRAM bytes of one launch of `kernel` from the tracked record of an ncu capture (profiles/ncu_traffic.json). The
+    capture is of a smaller case of the same workload, so its DRAM bytes are scaled by the algorithmic bytes of this
+    launch over those of the captured one (units share nothing; both grow with units x rows per unit). None when there
+    is no record for this kernel and workload, or when the kernel's source file has changed since the capture."""
     import hashlib
     path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
-    if not os.path.exists(path):
+    if not os.path.exists(path) or not alg_bytes:
         return None
     with open(path) as f:
         rec = json.load(f).get(kernel)
@@ -493,7 +494,7 @@ def ncu_traffic(kernel, wr):
     blob = hashlib.sha1(b"blob %d\0" % len(data) + data).hexdigest()      # what `git hash-object` prints
     if blob != rec.get("source_blob"):
         return None
-    return rec["dram_bytes"] * wr.units / rec["units"]
+    return rec["dram_bytes"] * alg_bytes / rec["algorithmic_bytes"]
 
 
 def run_subgen(args, w):

@@ -55,7 +55,8 @@ extern "C" {
 #define SUBGEN_DTYPE_BF16 1
 
 /* sticky per-unit status bits */
-#define SUBGEN_ST_CAPACITY 1 /* a key had to open a cluster but m_max clusters exist */
+#define SUBGEN_ST_CAPACITY 1 /* a key had to open a cluster but m_max clusters exist; the key is dropped from D, the
+                              * unit's outputs are NaN from then on and its M and mu are unspecified */
 #define SUBGEN_ST_RANGE 2    /* non-finite input, or |x| > 32768 */
 #define SUBGEN_ST_TIMEOUT 4  /* a bounded wait inside a kernel ran out (not expected; the state is unusable) */
 
