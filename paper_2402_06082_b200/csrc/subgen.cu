@@ -1,6 +1,7 @@
 // Host side of the SubGen library: handles, memory layout, launches, C ABI (see include/subgen.h).
 #include "../../include/subgen.h"
 
+#include <cuda.h>
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
@@ -203,6 +204,9 @@ struct subgen {
     int persist = -1;             // key phase as one persistent kernel (d = 128): -1 chosen from the unit count,
                                   // 0 / 1 forced by SUBGEN_PREFILL=chunk / persist
     bool pf_persist = false;      // the most recent profiled prefill used the persistent kernel
+    volatile unsigned* done_host = nullptr;   // subgen_step_host: a pinned word the stream writes after each step
+    CUdeviceptr done_dev = 0;
+    unsigned done_seq = 0;
     bool fused = false;           // stream steps run as one kernel (bf16, not bounded): few units, or SUBGEN_STEP=fused
     unsigned long long* pf_phase_dev = nullptr;   // its per-unit phase times (inside scratch)
 };
@@ -664,6 +668,7 @@ void subgen_destroy(subgen_t* h) {
     for (cudaEvent_t e : h->pev) cudaEventDestroy(e);
     if (h->owns) cudaFree(h->ws);
     if (h->scratch) cudaFree(h->scratch);
+    if (h->done_host) cudaFreeHost((void*)h->done_host);
     delete h;
 }
 
@@ -742,6 +747,51 @@ static bool pinned_alias(const void* host, void** dev) {
     return true;
 }
 
+// cuStreamWriteValue32 of the driver, looked up once (NULL if this driver does not offer it).
+typedef CUresult (*stream_write32_fn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
+static stream_write32_fn stream_write32() {
+    static stream_write32_fn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuStreamWriteValue32", &p, cudaEnableDefault, &qr) != cudaSuccess || qr != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            p = nullptr;
+        }
+        return (stream_write32_fn)p;
+    }();
+    return fn;
+}
+
+// Wait until the stream has finished the step just enqueued. Instead of a stream synchronisation the stream itself
+// writes a sequence number into a pinned word once the step's kernels are done (a stream memory operation), and the
+// host spins on that word: the result is seen a few microseconds earlier. Falls back to cudaStreamSynchronize when the
+// driver has no such operation, and after a bounded spin.
+static cudaError_t wait_step_done(subgen* h) {
+    stream_write32_fn wr = stream_write32();
+    if (wr && !h->done_host) {
+        void* p = nullptr;
+        if (cudaHostAlloc(&p, 64, cudaHostAllocMapped) == cudaSuccess) {
+            void* dp = nullptr;
+            if (cudaHostGetDevicePointer(&dp, p, 0) == cudaSuccess) {
+                h->done_host = (volatile unsigned*)p;
+                h->done_host[0] = 0;
+                h->done_dev = (CUdeviceptr)(uintptr_t)dp;
+            } else {
+                cudaFreeHost(p);
+            }
+        }
+        cudaGetLastError();
+    }
+    if (wr && h->done_host) {
+        const unsigned seq = ++h->done_seq;
+        if (wr((CUstream)h->st, h->done_dev, seq, 0) == CUDA_SUCCESS) {
+            for (long long spin = 0; spin < (1ll << 27); ++spin)
+                if (h->done_host[0] == seq) return cudaGetLastError();
+        }
+    }
+    return cudaStreamSynchronize(h->st);
+}
+
 int subgen_step_host(subgen_t* h, const void* q, const void* k, const void* v, void* out) {
     if (!h) return fail(SUBGEN_EINVAL, "subgen_step_host: handle is NULL");
     if (!q || !k || !v || !out) return fail(SUBGEN_EINVAL, "subgen_step_host: q, k, v, out must not be NULL");
@@ -754,7 +804,7 @@ int subgen_step_host(subgen_t* h, const void* q, const void* k, const void* v, v
         // (each input row is read by the few blocks of its unit, the result is written once)
         int rc = subgen_step(h, dq, dk, dv, dout);
         if (rc) return rc;
-        CUDA_TRY(cudaStreamSynchronize(h->st));
+        CUDA_TRY(wait_step_done(h));
         return SUBGEN_OK;
     }
     char* w = h->ws;
