@@ -19,6 +19,12 @@
  *    outputs.
  *  - Calls are asynchronous on the handle's stream unless stated otherwise. One handle is used by
  *    one host thread at a time.
+ *  - Inputs are consumed in stream order: q, k, v, K, V may be written by earlier work on the same
+ *    stream (the kernel that produced them), also when that work signals early completion to its
+ *    successors (programmatic dependent launch). The first kernel of every call orders itself after
+ *    everything earlier in the stream before it reads any input or any state; only the kernels a
+ *    call launches after its first one overlap their predecessor's tail. Inputs produced on ANOTHER
+ *    stream need an event, as usual.
  *  - Return value: 0 (SUBGEN_OK) or a negative SUBGEN_E* code for a host-side error;
  *    subgen_last_error() then gives a text. Problems found on the device (cluster capacity
  *    exhausted, non-finite or out-of-range input) never trap: they set sticky per-unit status
