@@ -50,7 +50,7 @@ size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
     size_t X, S, xn, cnt, ctok, stok, Mk, Mv, MW, Mtok, ringK, ringV;
     size_t n_unit, m_unit, mu, status, last_cid, last_open, last_d2, part1, part2, ticket1, ticket2, qnext, qnext2, part_tau, MinvW, pairs;
-    size_t thr2, level, Xh, xhn, alias, ndist;
+    size_t thr2, level, Xh, xhn, alias, ndist, epoch;
     size_t stage_q, stage_k, stage_v, stage_out, cu, stats;
     size_t book_begin, book_end;   // bookkeeping region cleared at creation
     size_t total;
@@ -165,6 +165,7 @@ Layout make_layout(const Dims& d) {
     L.qnext = take(U * sizeof(unsigned));
     L.qnext2 = take(U * sizeof(unsigned));
     L.pairs = take(U * sizeof(uint64_t));
+    L.epoch = take(U * sizeof(int));
     L.thr2 = take(U * sizeof(uint64_t));
     L.level = take(U * sizeof(int));
     L.MinvW = take(U * d.s * sizeof(float));
@@ -245,6 +246,7 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
     C.qnext = (unsigned*)(w + L.qnext); C.qnext2 = (unsigned*)(w + L.qnext2);
     C.part_tau = (float*)(w + L.part_tau); C.MinvW = (float*)(w + L.MinvW);
     C.pairs = (unsigned long long*)(w + L.pairs);
+    C.epoch = (int*)(w + L.epoch);
     C.bounded = h->cfg.bounded ? 1 : 0;
     C.uid_stride = h->cfg.unit_stride ? h->cfg.unit_stride : d.Hkv;
     C.uid_off = h->cfg.unit_offset;

@@ -47,6 +47,8 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
         if (blockIdx.x == 0) {
             if (tid < LPR) ringk[tid] = knew_u[tid];
             else if (tid < 2 * LPR) ringv[tid - LPR] = vnew_u[tid - LPR];
+            __syncthreads();
+            if (tid == 0) release_unit(C, u, n + 1);          // the value scan of this step may read the window now
         }
         return;
     }
@@ -152,6 +154,9 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
         if (tid < LPR) ringk[tid] = knew_u[tid];
         else if (tid < 2 * LPR) ringv[tid - LPR] = vnew_u[tid - LPR];
     }
+    // everything the value scan of this step reads (M, the window row, mu) has been written by this block
+    __syncthreads();
+    if (tid == 0) release_unit(C, u, n + 1);
 }
 
 }  // namespace sgk

@@ -172,6 +172,24 @@ __device__ __forceinline__ void tile_values(MmaState<D>& S, const float (&pz)[4]
     }
 }
 
+// What the insertion of a step wrote (M, the window row, mu) made visible to a block of the value scan, which does
+// not wait for the whole stream (see query_z_kernel): the insertion kernel ends a unit's update with a release store
+// of the unit's epoch, the value scan begins the unit with an acquire load of it. Called by a whole block; ends with
+// a __syncthreads().
+template <typename T>
+__device__ __forceinline__ void acquire_unit(const Cache<T>& C, int u) {
+    if (threadIdx.x == 0) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(C.epoch + u) : "memory");
+        (void)v;
+    }
+    __syncthreads();
+}
+template <typename T>
+__device__ __forceinline__ void release_unit(const Cache<T>& C, int u, int value) {
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(C.epoch + u), "r"(value) : "memory");
+}
+
 constexpr int kTauRows = 256 + 16;   // rows of one pass of the cluster scan: at most 256 sample rows and 16 singletons
 
 // floor(r / t) for small r by one multiply-high (t = 1 handled by the caller's magic = 0)
@@ -418,7 +436,6 @@ __global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfl
     const int lane = tid & 31, warp = tid >> 5, g = lane >> 2, tq = lane & 3;
     const int b = u / C.Hkv, kvh = u % C.Hkv;
     const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;
-    pdl_trigger();
 
     uint32_t qb[NC][4];                   // the queries are an input of the call, not a predecessor's output
 #pragma unroll
@@ -428,6 +445,9 @@ __global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfl
         qb[c][0] = r.x; qb[c][1] = r.y; qb[c][2] = r.z; qb[c][3] = r.w;
     }
     pdl_wait();
+    // The value scan may be scheduled from here on: it starts without waiting for this kernel, so the insertion (this
+    // kernel's predecessor) must be complete before it is let go.
+    pdl_trigger();
     const int m = C.m_unit[u];
     MmaState<16> S;                       // the accumulators stay untouched here and cost no registers
     S.m0 = S.m1 = -INFINITY;
@@ -480,7 +500,11 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_kernel(Cache<__nv_bfloa
         if (g < G) r = ldg16(q + (qrow0 + g) * D + c * 32 + tq * 8);
         qb[c][0] = r.x; qb[c][1] = r.y; qb[c][2] = r.z; qb[c][3] = r.w;
     }
-    pdl_wait();
+    // No wait for the cluster scan here. This kernel is scheduled once every block of the cluster scan has passed ITS
+    // wait for the insertion, so what the scan below reads (M, the window, mu, n: left by the insertion and by earlier
+    // steps) is complete; the acquire makes it visible. The cluster scan's partials are needed only by the final merge,
+    // and the wait stands before this block delivers its partial.
+    acquire_unit(C, u);
     // advance = 1: the query of a stream step, the step's token is in the ring but not counted yet;
     // advance = 0: a read-only query of the state as it stands
     const int n = C.n_unit[u] - (advance ? 0 : 1), w = C.w, s = C.s;
@@ -562,6 +586,7 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_kernel(Cache<__nv_bfloa
     }
     float* part_u = C.part2 + (size_t)u * splits * G * STR;
     block_combine<D, G>(sm, part_u + (size_t)blockIdx.x * G * STR);
+    pdl_wait();                     // the cluster scan is complete: its partials, its work queue
     __threadfence();
     __syncthreads();
     if (splits > 1) {
@@ -602,7 +627,6 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_flat_kernel(Cache<__nv_
     const long long NB = gridDim.x, Ttot = (long long)C.B * C.Hkv * ipu;
     const long long i0 = (long long)blockIdx.x * Ttot / NB, i1 = ((long long)blockIdx.x + 1) * Ttot / NB;
     pdl_trigger();
-    pdl_wait();
     if (i0 >= i1) return;
     const int w = C.w, s = C.s;
     const int u_first = (int)(i0 / ipu), u_last = (int)((i1 - 1) / ipu);
@@ -611,6 +635,7 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_flat_kernel(Cache<__nv_
         const int lo = (int)(max(i0, ulo) - ulo), hi = (int)(min(i1, ulo + ipu) - ulo);
         const int b = u / C.Hkv, kvh = u % C.Hkv;
         const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;
+        acquire_unit(C, u);         // no wait for the cluster scan before the scan of M and the window (see query_z_kernel)
         uint32_t qb[NC][4];
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
@@ -692,6 +717,7 @@ __global__ void __launch_bounds__(kQmThreads, 4) query_z_flat_kernel(Cache<__nv_
         const int np = b_last - b_first + 1;
         float* part_u = C.part2 + (size_t)u * slots * G * STR;
         block_combine<D, G>(sm, part_u + (size_t)((int)blockIdx.x - b_first) * G * STR);
+        pdl_wait();                 // the cluster scan is complete (returns at once after the first time)
         __threadfence();
         __syncthreads();
         bool last = true;
