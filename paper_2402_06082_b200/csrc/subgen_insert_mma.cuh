@@ -133,12 +133,14 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
     if (splits > 1) {
         if (tid == 0) {
             C.part1[(size_t)u * splits + blockIdx.x] = b;
-            __threadfence();
-            sm_last = (atomicAdd(&C.ticket1[u], 1u) == (unsigned)splits - 1u);
+            // arrival ticket: the release half publishes this block's candidate, the acquire half lets the last block
+            // read everybody else's
+            unsigned old;
+            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(&C.ticket1[u]) : "memory");
+            sm_last = (old == (unsigned)splits - 1u);
         }
         __syncthreads();
         if (!sm_last) return;
-        __threadfence();
         Best bb;
         bb.d2 = ~0ull; bb.idx = INT_MAX; bb.pad = 0;
         for (int i = tid; i < splits; i += nt) {
@@ -149,10 +151,16 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
         b = block_best(bb, smb);
         if (tid == 0) C.ticket1[u] = 0;
     }
+    // the new token's rows are asked for now and stored after the insertion (one round trip less at the end)
+    uint4 fresh = make_uint4(0, 0, 0, 0);
+    if (w) {
+        if (tid < LPR) fresh = knew_u[tid];
+        else if (tid < 2 * LPR) fresh = vnew_u[tid - LPR];
+    }
     apply_insert<T, D, BND>(C, u, e, b, m, krow, vrow, sm_w);
     if (w) {
-        if (tid < LPR) ringk[tid] = knew_u[tid];
-        else if (tid < 2 * LPR) ringv[tid - LPR] = vnew_u[tid - LPR];
+        if (tid < LPR) ringk[tid] = fresh;
+        else if (tid < 2 * LPR) ringv[tid - LPR] = fresh;
     }
     // everything the value scan of this step reads (M, the window row, mu) has been written by this block
     __syncthreads();
