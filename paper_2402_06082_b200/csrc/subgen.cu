@@ -208,6 +208,7 @@ struct subgen {
     volatile unsigned* done_host = nullptr;   // subgen_step_host: a pinned word the stream writes after each step
     CUdeviceptr done_dev = 0;
     unsigned done_seq = 0;
+    bool epoch_stale = true;      // the units' epochs may lag their token counts (creation, prefill, checkpoint load)
     bool fused = false;           // stream steps run as one kernel (bf16, not bounded): few units, or SUBGEN_STEP=fused
     unsigned long long* pf_phase_dev = nullptr;   // its per-unit phase times (inside scratch)
 };
@@ -384,6 +385,11 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
             CUDA_TRY(take_launch_error());
             h->launches += 1;
             return SUBGEN_OK;
+        }
+        if (h->epoch_stale) {            // ordinary launch: a full dependency on the prefill (or load) before it
+            epoch_sync_kernel<<<(h->d.U + 255) / 256, 256, 0, h->st>>>(C, h->d.U);
+            h->epoch_stale = false;
+            h->launches += 1;
         }
         if (C.bounded) launch_pdl(insert_mma_kernel<D, true>, grid_i, dim3(kInsertMmaThreads), h->st, C, (const T*)k, (const T*)v);
         else launch_pdl(insert_mma_kernel<D, false>, grid_i, dim3(kInsertMmaThreads), h->st, C, (const T*)k, (const T*)v);
@@ -684,6 +690,7 @@ int subgen_prefill(subgen_t* h, const void* K, const void* V, int n) {
     std::vector<int> add(h->d.B, n);
     int rc = launch_prefill(h, K, V, n, nullptr, 0, add.data());
     if (rc) return rc;
+    h->epoch_stale = true;
     for (int b = 0; b < h->d.B; ++b) h->n_host[b] += n;
     return SUBGEN_OK;
 }
@@ -708,6 +715,7 @@ int subgen_prefill_varlen(subgen_t* h, const void* K, const void* V, const int* 
     for (int b = 0; b < h->d.B; ++b) add[b] = cu[b + 1] - cu[b];
     int rc = launch_prefill(h, K, V, 0, cu_dev, total, add.data());
     if (rc) return rc;
+    h->epoch_stale = true;
     for (int b = 0; b < h->d.B; ++b) h->n_host[b] += cu[b + 1] - cu[b];
     return SUBGEN_OK;
 }
@@ -1109,6 +1117,7 @@ int subgen_checkpoint_load(subgen_t* h, const void* host, size_t bytes) {
     std::vector<int> n(d.U);
     CUDA_TRY(cudaMemcpy(n.data(), h->ws + h->L.n_unit, (size_t)d.U * 4, cudaMemcpyDeviceToHost));
     for (int b = 0; b < d.B; ++b) h->n_host[b] = n[(size_t)b * d.Hkv];
+    h->epoch_stale = true;
     return SUBGEN_OK;
 }
 

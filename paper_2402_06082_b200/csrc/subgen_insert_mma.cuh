@@ -33,11 +33,24 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
     __shared__ int sm_last;
     const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, nw = nt >> 5, g = lane >> 2, tq = lane & 3;
-    // The successor (the cluster scan) loads the call's queries before its own dependency wait, so it may only be
-    // scheduled once everything that precedes this call in the stream has completed: wait first, then trigger.
-    pdl_wait();
-    pdl_trigger();
-    const int n = C.n_unit[u], w = C.w;
+    // The search for the nearest representative needs nothing that the previous step's scans write and nothing of
+    // this call's inputs (the token that leaves the window has been in the ring since an earlier insertion), so it
+    // runs before the wait for the rest of the stream, under the tail of the previous step's value scan. What it reads
+    // was written by earlier insertion kernels, the latest of which released the unit's epoch = tokens seen: the
+    // acquire load makes all of it visible and replaces the token counter, which the previous step's value scan may
+    // still be about to advance. The wait comes before the first touch of an input (window 0: right here) and before
+    // the insertion is applied; the successor (the cluster scan, which loads the call's queries before its own wait)
+    // is let go only after the wait, i.e. once everything that precedes this call in the stream has completed.
+    const int w = C.w;
+    if (w == 0) pdl_wait();
+    __shared__ int sm_n;
+    if (tid == 0) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(C.epoch + u) : "memory");
+        sm_n = v;
+    }
+    __syncthreads();
+    const int n = sm_n;
     const uint4* knew_u = reinterpret_cast<const uint4*>(k_new + (size_t)u * D);
     const uint4* vnew_u = reinterpret_cast<const uint4*>(v_new + (size_t)u * D);
     const int slot = w ? n % w : 0;
@@ -45,6 +58,8 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
     uint4* ringv = w ? reinterpret_cast<uint4*>(C.ringV + ((size_t)u * w + slot) * D) : nullptr;
     if (w && n < w) {                       // window not full yet: nothing leaves it
         if (blockIdx.x == 0) {
+            pdl_wait();
+            pdl_trigger();
             if (tid < LPR) ringk[tid] = knew_u[tid];
             else if (tid < 2 * LPR) ringv[tid - LPR] = vnew_u[tid - LPR];
             __syncthreads();
@@ -151,6 +166,9 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
         b = block_best(bb, smb);
         if (tid == 0) C.ticket1[u] = 0;
     }
+    // From here on the state that the previous step's scans read is overwritten, and the call's inputs are read.
+    pdl_wait();
+    pdl_trigger();
     // the new token's rows are asked for now and stored after the insertion (one round trip less at the end)
     uint4 fresh = make_uint4(0, 0, 0, 0);
     if (w) {
@@ -165,6 +183,13 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
     // everything the value scan of this step reads (M, the window row, mu) has been written by this block
     __syncthreads();
     if (tid == 0) release_unit(C, u, n + 1);
+}
+
+// The units' epochs (see acquire_unit) set to their token counts: launched before the first stream step that follows
+// a prefill, a checkpoint load or the handle's creation, whose kernels advance the counts without touching the epochs.
+__global__ void epoch_sync_kernel(Cache<__nv_bfloat16> C, int U) {
+    const int u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u < U) C.epoch[u] = C.n_unit[u];
 }
 
 }  // namespace sgk
