@@ -24,7 +24,11 @@
  *    successors (programmatic dependent launch). The first kernel of every call orders itself after
  *    everything earlier in the stream before it reads any input or any state; only the kernels a
  *    call launches after its first one overlap their predecessor's tail. Inputs produced on ANOTHER
- *    stream need an event, as usual.
+ *    stream need an event, as usual. One thing is asked of work that the caller enqueues on the
+ *    handle's stream BETWEEN two calls: if it is itself launched with programmatic dependent launch, it
+ *    must wait for its predecessors (cudaGridDependencySynchronize) before it completes, as ordinary
+ *    kernels do implicitly; a call relies on "my predecessor has completed" implying "everything
+ *    before it has completed".
  *  - Return value: 0 (SUBGEN_OK) or a negative SUBGEN_E* code for a host-side error;
  *    subgen_last_error() then gives a text. Problems found on the device (cluster capacity
  *    exhausted, non-finite or out-of-range input) never trap: they set sticky per-unit status
