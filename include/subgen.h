@@ -22,8 +22,9 @@
  *  - Inputs are consumed in stream order: q, k, v, K, V may be written by earlier work on the same
  *    stream (the kernel that produced them), also when that work signals early completion to its
  *    successors (programmatic dependent launch). The first kernel of every call orders itself after
- *    everything earlier in the stream before it reads any input or any state; only the kernels a
- *    call launches after its first one overlap their predecessor's tail. Inputs produced on ANOTHER
+ *    everything earlier in the stream before it reads any input and before it touches anything that
+ *    earlier work may still be using (what it does before that point reads only cache arrays that
+ *    no kernel in flight writes). Inputs produced on ANOTHER
  *    stream need an event, as usual. One thing is asked of work that the caller enqueues on the
  *    handle's stream BETWEEN two calls: if it is itself launched with programmatic dependent launch, it
  *    must wait for its predecessors (cudaGridDependencySynchronize) before it completes, as ordinary
