@@ -50,7 +50,7 @@ size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
     size_t X, S, xn, cnt, ctok, stok, Mk, Mv, MW, Mtok, ringK, ringV;
     size_t n_unit, m_unit, mu, status, last_cid, last_open, last_d2, part1, part2, ticket1, ticket2, qnext, qnext2, part_tau, MinvW, pairs;
-    size_t thr2, level, Xh, xhn, alias, ndist, epoch;
+    size_t thr2, level, Xh, xhn, alias, ndist, epoch, order;
     size_t stage_q, stage_k, stage_v, stage_out, cu, stats;
     size_t book_begin, book_end;   // bookkeeping region cleared at creation
     size_t total;
@@ -166,6 +166,7 @@ Layout make_layout(const Dims& d) {
     L.qnext2 = take(U * sizeof(unsigned));
     L.pairs = take(U * sizeof(uint64_t));
     L.epoch = take(U * sizeof(int));
+    L.order = take(U * sizeof(int));
     L.thr2 = take(U * sizeof(uint64_t));
     L.level = take(U * sizeof(int));
     L.MinvW = take(U * d.s * sizeof(float));
@@ -208,6 +209,7 @@ struct subgen {
     volatile unsigned* done_host = nullptr;   // subgen_step_host: a pinned word the stream writes after each step
     CUdeviceptr done_dev = 0;
     unsigned done_seq = 0;
+    bool order_ready = false;     // the units are ranked by cluster count (set by a prefill of a many-unit handle)
     bool epoch_stale = true;      // the units' epochs may lag their token counts (creation, prefill, checkpoint load)
     bool fused = false;           // stream steps run as one kernel (bf16, not bounded): few units, or SUBGEN_STEP=fused
     unsigned long long* pf_phase_dev = nullptr;   // its per-unit phase times (inside scratch)
@@ -248,6 +250,7 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
     C.part_tau = (float*)(w + L.part_tau); C.MinvW = (float*)(w + L.MinvW);
     C.pairs = (unsigned long long*)(w + L.pairs);
     C.epoch = (int*)(w + L.epoch);
+    C.order = h->order_ready ? (const int*)(w + L.order) : nullptr;
     C.bounded = h->cfg.bounded ? 1 : 0;
     C.uid_stride = h->cfg.unit_stride ? h->cfg.unit_stride : d.Hkv;
     C.uid_off = h->cfg.unit_offset;
@@ -561,6 +564,18 @@ int launch_prefill(subgen* h, const void* K, const void* V, int n, const int* cu
                : launch_prefill_td<__nv_bfloat16, 128>(h, K, V, n, cu_dev, total);
 }
 
+// After a prefill of a bf16 handle that steps with one grid row per unit (three-kernel step): rank the units by
+// cluster count, for the block order of the step's insertion kernel and cluster scan.
+void rank_units(subgen* h) {
+    static const bool off = [] { const char* e = getenv("SUBGEN_ORDER"); return e && e[0] == '0'; }();
+    h->order_ready = false;
+    if (off || h->cfg.dtype != SUBGEN_DTYPE_BF16 || h->fused) return;
+    Cache<__nv_bfloat16> C = make_cache<__nv_bfloat16>(h);
+    unit_order_kernel<<<(h->d.U + 255) / 256, 256, 0, h->st>>>(C, h->d.U, (int*)(h->ws + h->L.order));
+    h->launches += 1;
+    h->order_ready = true;
+}
+
 int check_device() {
     int n = 0;
     cudaError_t e = cudaGetDeviceCount(&n);
@@ -691,6 +706,7 @@ int subgen_prefill(subgen_t* h, const void* K, const void* V, int n) {
     int rc = launch_prefill(h, K, V, n, nullptr, 0, add.data());
     if (rc) return rc;
     h->epoch_stale = true;
+    rank_units(h);
     for (int b = 0; b < h->d.B; ++b) h->n_host[b] += n;
     return SUBGEN_OK;
 }
@@ -716,6 +732,7 @@ int subgen_prefill_varlen(subgen_t* h, const void* K, const void* V, const int* 
     int rc = launch_prefill(h, K, V, 0, cu_dev, total, add.data());
     if (rc) return rc;
     h->epoch_stale = true;
+    rank_units(h);
     for (int b = 0; b < h->d.B; ++b) h->n_host[b] += cu[b + 1] - cu[b];
     return SUBGEN_OK;
 }
@@ -1118,6 +1135,7 @@ int subgen_checkpoint_load(subgen_t* h, const void* host, size_t bytes) {
     CUDA_TRY(cudaMemcpy(n.data(), h->ws + h->L.n_unit, (size_t)d.U * 4, cudaMemcpyDeviceToHost));
     for (int b = 0; b < d.B; ++b) h->n_host[b] = n[(size_t)b * d.Hkv];
     h->epoch_stale = true;
+    h->order_ready = false;
     return SUBGEN_OK;
 }
 

@@ -131,6 +131,8 @@ template <typename T> struct Cache {
     unsigned* qnext2;    // [U] same for the scan of M and the window
     unsigned long long* pairs;   // [U] (key, representative) pairs scored by the chunked prefill so far
     int* epoch;                  // [U] tokens seen, as released by the step's insertion kernel (see acquire_unit)
+    const int* order;            // [U] or NULL: the unit that the blocks with blockIdx.y = i serve, units with many
+                                 //     clusters first (handles whose per-unit grids need several waves of blocks)
     int uid_stride, uid_off;     // numbering of the units in the Philox counter, see unit_id()
     // bounded-m variant: m_max is a budget, the threshold doubles and clusters merge when it is exhausted
     int bounded;

@@ -31,7 +31,7 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
     __shared__ Best smb[32];
     __shared__ unsigned long long sm_w[2];
     __shared__ int sm_last;
-    const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x, nt = blockDim.x;
+    const int u = C.order ? C.order[blockIdx.y] : (int)blockIdx.y, splits = gridDim.x, tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, nw = nt >> 5, g = lane >> 2, tq = lane & 3;
     // The search for the nearest representative needs nothing that the previous step's scans write and nothing of
     // this call's inputs (the token that leaves the window has been in the ring since an earlier insertion), so it
@@ -183,6 +183,25 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
     // everything the value scan of this step reads (M, the window row, mu) has been written by this block
     __syncthreads();
     if (tid == 0) release_unit(C, u, n + 1);
+}
+
+// Units ranked by their cluster count, largest first (ties: lower unit first): order[rank] = unit. Blocks are handed
+// to the SMs in grid order, so with several waves of one block per unit the long units start first and the short ones
+// fill the end. Units of about one size (largest count within 5/4 of the smallest) keep their own order: nothing is
+// gained there, and neighbouring units share a sequence's rows. One thread per unit, O(U) each; launched after a prefill.
+__global__ void unit_order_kernel(Cache<__nv_bfloat16> C, int U, int* order) {
+    const int u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= U) return;
+    const int mu = C.m_unit[u];
+    int rank = 0, mn = mu, mx = mu;
+    for (int v = 0; v < U; ++v) {
+        const int mv = __ldg(C.m_unit + v);
+        rank += (mv > mu) || (mv == mu && v < u);
+        mn = min(mn, mv);
+        mx = max(mx, mv);
+    }
+    if ((long long)mx * 4 <= (long long)mn * 5) order[u] = u;
+    else order[rank] = u;
 }
 
 // The units' epochs (see acquire_unit) set to their token counts: launched before the first stream step that follows

@@ -432,7 +432,7 @@ __global__ void __launch_bounds__(kQmThreads, 6) query_tau_kernel(Cache<__nv_bfl
     __shared__ unsigned als[NW][16 * 64 / 4];          // alias rows of the item's 16 clusters, t <= 64 bytes each
     __shared__ int rix[NW][kTauRows];                  // row list of a pass: sample row index, or representative | 2^31
     __shared__ float rwt[NW][kTauRows];
-    const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
+    const int u = C.order ? C.order[blockIdx.y] : (int)blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5, g = lane >> 2, tq = lane & 3;
     const int b = u / C.Hkv, kvh = u % C.Hkv;
     const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;

@@ -193,3 +193,38 @@ def test_sharded_handles_reproduce_the_whole_job(mode):
     o.push_many(f32(K[2, 3]), f32(V[2, 3]))
     last = handles[1]
     hp.assert_state_equal(last.export_state(last.B - 1, last.Hkv - 1), o, "last unit of the job, on its shard")
+
+
+def test_ragged_prompts_many_units():
+    """Prompts of very different lengths on a handle with more units than SMs: the three-kernel step serves the units
+    largest first (an order built after the prefill); every unit must still be served exactly once per step."""
+    w = synth.CFG5.scaled(B=6, H=32, Hkv=32, ncomp=16, s=64, window=16, m_max=512)
+    lens = [40, 700, 120, 350, 17, 500]
+    n_dec = 5
+    streams = [synth.sequence_stream(w, b, lens[b] + n_dec, "cuda") for b in range(w.B)]
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    Kp = torch.cat([streams[b][0][:, :lens[b]] for b in range(w.B)], dim=1).contiguous()
+    Vp = torch.cat([streams[b][1][:, :lens[b]] for b in range(w.B)], dim=1).contiguous()
+    sg = _sg(w)
+    assert sg.step_kernels == 3
+    sg.prefill_varlen(Kp, Vp, cu)
+    orcs = {}
+    for b in range(w.B):
+        for h in range(w.Hkv):
+            o = hp.oracle_unit(w, b, h)
+            o.push_many(f32(streams[b][0][h, :lens[b]]), f32(streams[b][1][h, :lens[b]]))
+            orcs[(b, h)] = o
+    ms = [o.m for o in orcs.values()]
+    assert max(ms) > 2 * max(min(ms), 1)
+    for i in range(n_dec):
+        q = torch.stack([streams[b][2][:, lens[b] + i] for b in range(w.B)]).contiguous()
+        k = torch.stack([streams[b][0][:, lens[b] + i] for b in range(w.B)]).contiguous()
+        v = torch.stack([streams[b][1][:, lens[b] + i] for b in range(w.B)]).contiguous()
+        out = f32(sg.step(q, k, v))
+        kn, vn, qn = f32(k), f32(v), f32(q)
+        for (b, h), o in orcs.items():
+            o.push(kn[b, h], vn[b, h])
+            hp.assert_output(out[b, h], o.query(qn[b, h]), torch.bfloat16, "step %d unit %s" % (i, (b, h)))
+    for (b, h), o in orcs.items():
+        hp.assert_state_equal(sg.export_state(b, h), o, "ragged, ordered units %s" % ((b, h),))
+    assert sg.status() == 0
