@@ -209,6 +209,8 @@ struct subgen {
     volatile unsigned* done_host = nullptr;   // subgen_step_host: a pinned word the stream writes after each step
     CUdeviceptr done_dev = 0;
     unsigned done_seq = 0;
+    cudaStream_t st2 = nullptr;   // prefill: the key phase runs here, beside the value phase on st (fork / join by events)
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     bool order_ready = false;     // the units are ranked by cluster count (set by a prefill of a many-unit handle)
     bool epoch_stale = true;      // the units' epochs may lag their token counts (creation, prefill, checkpoint load)
     bool fused = false;           // stream steps run as one kernel (bf16, not bounded): few units, or SUBGEN_STEP=fused
@@ -461,6 +463,7 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
     a.K = (const T*)K; a.V = (const T*)V; a.n_uniform = n; a.cu = cu_dev; a.total = total; a.Lmax = Lmax; a.slices = slices;
     a.Wbuf = nullptr; a.Tot = nullptr; a.Thr = nullptr; a.Mwin = nullptr; a.pbest = nullptr; a.mhist = nullptr;
     int launches = 0;
+    bool join = false;
     if (Lmax > 0) {
         const size_t b_w = align_up((size_t)d.U * Lmax * 8), b_m = align_up((size_t)d.U * d.s * 4);
         const size_t b_p = align_up((size_t)d.U * slices * kChunk * sizeof(Best));
@@ -492,24 +495,37 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         };
         h->pev_used = 0;
         if (int rc = mark()) return rc;
-        CUDA_TRY(cudaMemsetAsync(a.Mwin, 0xFF, (size_t)d.U * d.s * 4, h->st));
-        constexpr int RPW = 32 / (D / 8);
-        int bx = (Lmax + 8 * RPW - 1) / (8 * RPW);
-        bx = bx > 64 ? 64 : bx;
-        prefill_w_kernel<D><<<dim3(bx, d.U), 256, 0, h->st>>>(C, a);
-        prefill_scan_kernel<<<d.U, 1024, 0, h->st>>>(C, a);
-        const int cbx = ((d.s + 3) / 4 + 127) / 128;
-        long long want = (300000LL + (long long)d.U * cbx * 128 - 1) / ((long long)d.U * cbx * 128);   // fill the GPU about once
-        int segs = (int)(want < 1 ? 1 : want);
-        int seg_len = (Lmax + segs - 1) / segs;
-        seg_len = seg_len < 256 ? 256 : seg_len;
-        segs = (Lmax + seg_len - 1) / seg_len;
-        prefill_coin_kernel<<<dim3(cbx, segs, d.U), 128, 0, h->st>>>(C, a, seg_len);
-        int gx = (d.s + 8 * RPW - 1) / (8 * RPW);
-        gx = gx > 32 ? 32 : gx;
-        prefill_gather_kernel<D><<<dim3(gx, d.U), 256, 0, h->st>>>(C, a);
-        launches += 4;
-        if (int rc = mark()) return rc;
+        // The value phase (weights, running sums, coins, gather into M) and the key phase (clusters) share nothing
+        // until the commit. The key phase is a chain of short dependent stages per unit and leaves most issue slots
+        // idle; the value phase's coin kernel is integer arithmetic that fills them. So the key phase goes to the
+        // handle's second stream (higher priority: its few long-lived blocks take their places first), forked from
+        // and joined back into the caller's stream by events, while the value phase stays on the caller's stream.
+        // With profiling on, both stay in one stream so that each can be timed.
+        static const bool no_overlap = [] { const char* e = getenv("SUBGEN_PREFILL_OVERLAP"); return e && e[0] == '0'; }();
+        const bool overlap = !h->prof && h->st2 && !no_overlap;
+        auto value_phase = [&](cudaStream_t sv) -> int {
+            CUDA_TRY(cudaMemsetAsync(a.Mwin, 0xFF, (size_t)d.U * d.s * 4, sv));
+            constexpr int RPW = 32 / (D / 8);
+            int bx = (Lmax + 8 * RPW - 1) / (8 * RPW);
+            bx = bx > 64 ? 64 : bx;
+            prefill_w_kernel<D><<<dim3(bx, d.U), 256, 0, sv>>>(C, a);
+            prefill_scan_kernel<<<d.U, 1024, 0, sv>>>(C, a);
+            // a warp per group of four slots and segment; one segment when the groups alone give enough warps (a scan
+            // that ends early saves most over a whole prompt), more for handles with few units
+            const int groups = (d.s + 3) / 4;
+            long long want = (20000LL + (long long)d.U * groups - 1) / ((long long)d.U * groups);
+            int segs = (int)(want < 1 ? 1 : want);
+            int seg_len = (Lmax + segs - 1) / segs;
+            seg_len = seg_len < 1024 ? 1024 : seg_len;
+            seg_len = (seg_len + 31) / 32 * 32;
+            segs = (Lmax + seg_len - 1) / seg_len;
+            prefill_coin_kernel<<<dim3((groups + 3) / 4, segs, d.U), 128, 0, sv>>>(C, a, seg_len);
+            int gx = (d.s + 8 * RPW - 1) / (8 * RPW);
+            gx = gx > 32 ? 32 : gx;
+            prefill_gather_kernel<D><<<dim3(gx, d.U), 256, 0, sv>>>(C, a);
+            launches += 4;
+            return SUBGEN_OK;
+        };
         // Key phase. Many units with few representatives each: one persistent block per unit walks its chunks
         // (subgen_prefill_persist.cuh). Few units: a score and a resolve kernel per chunk, the representatives of a
         // unit spread over many blocks.
@@ -517,28 +533,44 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         // the key that finds the budget used up and insert that key on its own.
         const bool persist = tc && (C.bounded || (h->persist >= 0 ? h->persist == 1 : d.U >= 24));
         h->pf_persist = persist && h->prof;
-        if (persist) {
-            h->pf_phase_dev = phase_ns;
-            if (C.bounded) prefill_keys_persist_kernel<true><<<d.U, kPpThreads, kPpSmemBytes, h->st>>>(C, a, h->prof ? phase_ns : nullptr);
-            else prefill_keys_persist_kernel<false><<<d.U, kPpThreads, kPpSmemBytes, h->st>>>(C, a, h->prof ? phase_ns : nullptr);
-            launches += 1;
-            if (int rc = mark()) return rc;
-        } else {
+        auto key_phase = [&](cudaStream_t sk) -> int {
+            if (persist) {
+                h->pf_phase_dev = phase_ns;
+                if (C.bounded) prefill_keys_persist_kernel<true><<<d.U, kPpThreads, kPpSmemBytes, sk>>>(C, a, h->prof ? phase_ns : nullptr);
+                else prefill_keys_persist_kernel<false><<<d.U, kPpThreads, kPpSmemBytes, sk>>>(C, a, h->prof ? phase_ns : nullptr);
+                launches += 1;
+                if (int rc = mark()) return rc;
+                return SUBGEN_OK;
+            }
             const int nchunks = (Lmax + kChunk - 1) / kChunk;
-            prefill_mhist_kernel<<<(d.U + 255) / 256, 256, 0, h->st>>>(C, a, d.U);
+            prefill_mhist_kernel<<<(d.U + 255) / 256, 256, 0, sk>>>(C, a, d.U);
             launches += 1;
             for (int c = 0; c < nchunks; ++c) {
                 // both kernels stage their chunk keys before they wait for their predecessor in the stream;
                 // chunk 0 reads the cluster-count history its immediate predecessor wrote before it waits: ordinary launch
-                if (tc) launch_pdl_opt(c == 0, prefill_score_tc_kernel, dim3(slices, d.U), dim3(kTcThreads), kTcSmemBytes, h->st, C, a, c);
-                else prefill_score_kernel<D><<<dim3(slices, d.U), kScoreThreads, 0, h->st>>>(C, a, c);
+                if (tc) launch_pdl_opt(c == 0, prefill_score_tc_kernel, dim3(slices, d.U), dim3(kTcThreads), kTcSmemBytes, sk, C, a, c);
+                else prefill_score_kernel<D><<<dim3(slices, d.U), kScoreThreads, 0, sk>>>(C, a, c);
                 if (int rc = mark()) return rc;
-                launch_pdl(prefill_resolve_kernel<D>, dim3(d.U), dim3(kResolveThreads), h->st, C, a, c);
+                launch_pdl(prefill_resolve_kernel<D>, dim3(d.U), dim3(kResolveThreads), sk, C, a, c);
                 if (int rc = mark()) return rc;
             }
             launches += 2 * nchunks;
+            return SUBGEN_OK;
+        };
+        if (overlap) {
+            CUDA_TRY(cudaEventRecord(h->ev_fork, h->st));
+            CUDA_TRY(cudaStreamWaitEvent(h->st2, h->ev_fork, 0));
+            if (int rc = key_phase(h->st2)) return rc;
+            CUDA_TRY(cudaEventRecord(h->ev_join, h->st2));
+            join = true;
+            if (int rc = value_phase(h->st)) return rc;
+        } else {
+            if (int rc = value_phase(h->st)) return rc;
+            if (int rc = mark()) return rc;
+            if (int rc = key_phase(h->st)) return rc;
         }
     }
+    if (join) CUDA_TRY(cudaStreamWaitEvent(h->st, h->ev_join, 0));   // the clusters are complete
     int longest = 0;
     for (int b = 0; b < d.B; ++b) longest = add[b] > longest ? add[b] : longest;
     int fx = (int)(((size_t)(longest < d.w ? longest : d.w) * (D / 8) + 255) / 256);
@@ -574,6 +606,12 @@ void rank_units(subgen* h) {
     unit_order_kernel<<<(h->d.U + 255) / 256, 256, 0, h->st>>>(C, h->d.U, (int*)(h->ws + h->L.order));
     h->launches += 1;
     h->order_ready = true;
+}
+
+void destroy_side_stream(subgen* h) {
+    if (h->st2) { cudaStreamSynchronize(h->st2); cudaStreamDestroy(h->st2); h->st2 = nullptr; }
+    if (h->ev_fork) { cudaEventDestroy(h->ev_fork); h->ev_fork = nullptr; }
+    if (h->ev_join) { cudaEventDestroy(h->ev_join); h->ev_join = nullptr; }
 }
 
 int check_device() {
@@ -636,6 +674,18 @@ subgen_t* subgen_create_ex(const subgen_config* cfg) {
         return nullptr;
     }
     h->n_host.assign(d.B, 0);
+    int prio_lo = 0, prio_hi = 0;
+    if (cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) != cudaSuccess) { cudaGetLastError(); prio_hi = 0; }
+    if (cfg->dtype == SUBGEN_DTYPE_BF16 &&
+        (cudaStreamCreateWithPriority(&h->st2, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+         cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+         cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess)) {
+        fail(SUBGEN_ECUDA, "subgen_create: second stream: %s", cudaGetErrorString(cudaGetLastError()));
+        destroy_side_stream(h);
+        if (h->owns) cudaFree(h->ws);
+        delete h;
+        return nullptr;
+    }
     // the tcgen05 score kernel needs more dynamic shared memory than the default limit; the attribute is per device,
     // so it is set for the device of every handle that can launch the kernel
     if (cfg->dtype == SUBGEN_DTYPE_BF16 && d.D == 128 &&
@@ -643,6 +693,7 @@ subgen_t* subgen_create_ex(const subgen_config* cfg) {
          cudaFuncSetAttribute(prefill_keys_persist_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPpSmemBytes) != cudaSuccess ||
          cudaFuncSetAttribute(prefill_keys_persist_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPpSmemBytes) != cudaSuccess)) {
         fail(SUBGEN_ECUDA, "subgen_create: cudaFuncSetAttribute failed: %s", cudaGetErrorString(cudaGetLastError()));
+        destroy_side_stream(h);
         if (h->owns) cudaFree(h->ws);
         delete h;
         return nullptr;
@@ -668,6 +719,7 @@ subgen_t* subgen_create_ex(const subgen_config* cfg) {
         if (!(cfg->dtype == SUBGEN_DTYPE_BF16 && d.D == 128) || h->mma_score) h->seq_prefill = true;
         if (reset_thresholds(h) != cudaSuccess) {
             fail(SUBGEN_ECUDA, "subgen_create: threshold initialisation failed");
+            destroy_side_stream(h);
             if (h->owns) cudaFree(h->ws);
             delete h;
             return nullptr;
@@ -689,6 +741,7 @@ void subgen_destroy(subgen_t* h) {
     cudaStreamSynchronize(h->st);
     for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
     for (cudaEvent_t e : h->pev) cudaEventDestroy(e);
+    destroy_side_stream(h);
     if (h->owns) cudaFree(h->ws);
     if (h->scratch) cudaFree(h->scratch);
     if (h->done_host) cudaFreeHost((void*)h->done_host);

@@ -156,29 +156,44 @@ __global__ void prefill_scan_kernel(Cache<__nv_bfloat16> C, PrefillArgs a) {
     }
 }
 
-// Value coins. grid (ceil(s/4 / threads), segments, U): a thread owns one block of four slots over one
-// segment of tokens and reports the last token whose coin succeeded.
+// Value coins: for every slot of M the last token of the call whose coin succeeded. One Philox block serves the
+// four slots of a group, so a warp takes one group over one segment of tokens, 32 consecutive tokens per pass, the
+// latest first, and stops once all four slots have their winner: the position of a slot's last success is uniform in
+// the cumulative weight, so a group's scan ends after four fifths of the tokens on average, and the common pass (no
+// coin of the 128 succeeds) costs one minimum and one comparison after the Philox block.
+// grid (ceil(groups / warps per block), segments, U); segments are a multiple of 32 tokens long.
 __global__ void prefill_coin_kernel(Cache<__nv_bfloat16> C, PrefillArgs a, int seg_len) {
-    const int u = blockIdx.z, blk = blockIdx.x * blockDim.x + threadIdx.x;
+    const int u = blockIdx.z, lane = threadIdx.x & 31, blk = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const Range r = unit_range(C, a, u);
     const int len = r.ins_hi - r.ins_lo;
     const int i0 = blockIdx.y * seg_len, i1 = min(len, i0 + seg_len);
     if (blk * 4 >= C.s || i0 >= i1) return;
     const unsigned long long* Tb = a.Thr + (size_t)u * a.Lmax;
+    const uint32_t uid = unit_id(C, u);
     int win[4] = {-1, -1, -1, -1};
-    for (int i = i0; i < i1; ++i) {
-        const unsigned long long thr = Tb[i];
-        if (thr == 0ull) continue;                          // W = 0: never sampled
-        const int e = r.ins_lo + i;
-        const uint4 rr = philox4x32_10(make_uint4((uint32_t)e, unit_id(C, u), (uint32_t)blk, 1u), C.key0, C.key1);
-        if ((unsigned long long)rr.x < thr) win[0] = e;
-        if ((unsigned long long)rr.y < thr) win[1] = e;
-        if ((unsigned long long)rr.z < thr) win[2] = e;
-        if ((unsigned long long)rr.w < thr) win[3] = e;
-    }
+    unsigned found = 0;
+    for (int top = i1; top > i0 && found != 15u; top -= 32) {
+        const int i = top - 1 - lane;
+        const unsigned long long thr = i >= i0 ? Tb[i] : 0ull;            // 0 (also for W = 0): never sampled
+        const uint4 rr = philox4x32_10(make_uint4((uint32_t)(r.ins_lo + i), uid, (uint32_t)blk, 1u), C.key0, C.key1);
+        const uint32_t mn = min(min(rr.x, rr.y), min(rr.z, rr.w));
+        if (__any_sync(0xffffffffu, (unsigned long long)mn < thr)) {
+            const uint32_t wd[4] = {rr.x, rr.y, rr.z, rr.w};
 #pragma unroll
-    for (int q = 0; q < 4; ++q)
-        if (win[q] >= 0 && blk * 4 + q < C.s) atomicMax(&a.Mwin[(size_t)u * C.s + blk * 4 + q], win[q]);
+            for (int q = 0; q < 4; ++q) {
+                const unsigned hit = __ballot_sync(0xffffffffu, (unsigned long long)wd[q] < thr);
+                if (hit && !(found >> q & 1u)) {                           // lowest lane = latest token
+                    win[q] = r.ins_lo + top - 1 - (__ffs(hit) - 1);
+                    found |= 1u << q;
+                }
+            }
+        }
+    }
+    if (lane == 0) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            if (win[q] >= 0 && blk * 4 + q < C.s) atomicMax(&a.Mwin[(size_t)u * C.s + blk * 4 + q], win[q]);
+    }
 }
 
 // Copies the winners into M. grid (blocks, U); a row group per slot.
