@@ -504,10 +504,12 @@ int launch_prefill_chunked(subgen* h, const void* K, const void* V, int n, const
         h->pev_used = 0;
         if (int rc = mark()) return rc;
         // The value phase (weights, running sums, coins, gather into M) and the key phase (clusters) share nothing
-        // until the commit. The key phase is a chain of short dependent stages per unit and leaves most issue slots
-        // idle; the value phase's coin kernel is integer arithmetic that fills them. So the key phase goes to the
-        // handle's second stream (higher priority: its few long-lived blocks take their places first), forked from
-        // and joined back into the caller's stream by events, while the value phase stays on the caller's stream.
+        // until the commit, so the key phase goes to the handle's second stream (higher priority: its few long-lived
+        // blocks take their places first), forked from and joined back into the caller's stream by events, while the
+        // value phase stays on the caller's stream. Two blocks of the persistent key kernel hold all registers of
+        // their SM, so the coin kernel runs on the SMs that the key kernel leaves free or half used and on the
+        // others once their units are done (256 units: 28.3 -> 26.4 ms; capping the key kernel's registers to let
+        // both share every SM cost more in its read-back than the sharing returned).
         // With profiling on, both stay in one stream so that each can be timed.
         static const bool no_overlap = [] { const char* e = getenv("SUBGEN_PREFILL_OVERLAP"); return e && e[0] == '0'; }();
         const bool overlap = !h->prof && h->st2 && !no_overlap;
