@@ -161,7 +161,8 @@ int subgen_step(subgen_t* h, const void* q, const void* k, const void* v, void* 
 int subgen_query(subgen_t* h, const void* q, int nq, void* out);
 
 /* subgen_step with HOST buffers, returning when out is filled. With page-locked (pinned, mapped) buffers the
- * step's kernels read q, k, v and write out across the bus themselves: no staging copies, one wait. With pageable
+ * step's kernels write out across the bus themselves and read q, k, v the same way (handles whose one-kernel step
+ * runs many blocks per unit let one small kernel bring q, k, v over first): no copy engine, one wait. With pageable
  * buffers q, k, v are copied to the device first and out is copied back. */
 int subgen_step_host(subgen_t* h, const void* q, const void* k, const void* v, void* out);
 

@@ -827,6 +827,15 @@ int subgen_query(subgen_t* h, const void* q, int nq, void* out) {
     return f32 ? launch_query_only_td<float, 128>(h, q, nq, out) : launch_query_only_td<__nv_bfloat16, 128>(h, q, nq, out);
 }
 
+// q, k, v from mapped host memory into the handle's staging buffers, 16 bytes per thread.
+__global__ void stage_inputs_kernel(const uint4* __restrict__ q, const uint4* __restrict__ k, const uint4* __restrict__ v,
+                                    uint4* dq, uint4* dk, uint4* dv, size_t nq, size_t nk) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < nq) dq[i] = q[i];
+    else if (i < nq + nk) dk[i - nq] = k[i - nq];
+    else if (i < nq + 2 * nk) dv[i - nq - nk] = v[i - nq - nk];
+}
+
 // Device-side alias of a page-locked, mapped host buffer (what cudaHostAlloc / cudaHostRegister hand out under unified
 // addressing); false for pageable memory.
 static bool pinned_alias(const void* host, void** dev) {
@@ -892,6 +901,25 @@ int subgen_step_host(subgen_t* h, const void* q, const void* k, const void* v, v
         !(((uintptr_t)dq | (uintptr_t)dk | (uintptr_t)dv | (uintptr_t)dout) & 15)) {
         // pinned buffers: the step's kernels read the inputs and write the result across the bus themselves
         // (each input row is read by the few blocks of its unit, the result is written once)
+        // A one-kernel step with many blocks per unit would fetch every input row across the bus once per block
+        // (8 units, 37 blocks each: 88 -> 65 us per call with staging); then one small kernel brings q, k, v over
+        // first, every 16-byte piece once, and the step reads device memory. The result is still written into the
+        // caller's buffer by the step itself. With few blocks per unit the direct reads are as fast (measured at 256
+        // units x 3 blocks and 32 units x 9 blocks). SUBGEN_E2E_STAGE=0 / 1 forces either way.
+        static const int stage_env = [] { const char* e = getenv("SUBGEN_E2E_STAGE"); return e ? atoi(e) : -1; }();
+        const bool stage = stage_env >= 0 ? stage_env != 0 : (h->fused && h->d.sp_fused > 16);
+        if (stage) {
+            char* w = h->ws;
+            const size_t nq = qb / 16, nk = kb / 16, total = nq + 2 * nk;
+            stage_inputs_kernel<<<(unsigned)((total + 255) / 256), 256, 0, h->st>>>(
+                (const uint4*)dq, (const uint4*)dk, (const uint4*)dv, (uint4*)(w + h->L.stage_q), (uint4*)(w + h->L.stage_k),
+                (uint4*)(w + h->L.stage_v), nq, nk);
+            h->launches += 1;
+            int rc = subgen_step(h, w + h->L.stage_q, w + h->L.stage_k, w + h->L.stage_v, dout);
+            if (rc) return rc;
+            CUDA_TRY(wait_step_done(h));
+            return SUBGEN_OK;
+        }
         int rc = subgen_step(h, dq, dk, dv, dout);
         if (rc) return rc;
         CUDA_TRY(wait_step_done(h));

@@ -233,15 +233,18 @@ def test_host_argument_errors():
     L.subgen_destroy(None)
 
 
-@pytest.mark.parametrize("pinned", [True, False])
-def test_step_host_matches_step(pinned):
-    """Pinned buffers are read and written by the kernels directly, pageable ones go through staging copies."""
+@pytest.mark.parametrize("how", ["pinned_staged", "pinned_direct", "pageable"])
+def test_step_host_matches_step(how):
+    """Pinned buffers: the result is written by the kernels directly; the inputs are read by them directly (few blocks
+    per unit) or brought over by one staging kernel first (many blocks per unit). Pageable buffers go through staging
+    copies."""
     w = synth.CFG2.scaled(B=2, H=4, Hkv=2, n_prompt=100, ncomp=8, s=32, window=16, m_max=64)
     K, V, Q = synth.batch_stream(w, 110, "cuda")
-    a, b = _sg(w), _sg(w)
+    kw = dict(splits=2) if how == "pinned_direct" else {}
+    a, b = _sg(w, **kw), _sg(w, **kw)
     a.prefill(K[:, :, :100].contiguous(), V[:, :, :100].contiguous())
     b.prefill(K[:, :, :100].contiguous(), V[:, :, :100].contiguous())
-    host = (lambda x: x.cpu().pin_memory()) if pinned else (lambda x: x.cpu())
+    host = (lambda x: x.cpu()) if how == "pageable" else (lambda x: x.cpu().pin_memory())
     for i in range(100, 110):
         q, k, v = Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous()
         o1 = a.step(q, k, v)
