@@ -207,7 +207,7 @@ def measure(wr, args, K_steps, W_steps, world, rank, local, dist, headline):
     """Prefill + decode of one workload on this rank's GPU. headline = True adds the prefill phase profile, the exact
     comparison, the per-kernel roofline block; False gives the compact entry of the per-config table."""
     from paper_2402_06082_b200 import binding
-    n_e2e = args.e2e_steps if headline else min(args.e2e_steps, 16)
+    n_e2e = args.e2e_steps if headline else min(args.e2e_steps, 80)
     P_steps = min(K_steps, 256 if headline else 64)          # second, shorter pass with CUDA events between the kernels
     lens = wr.prompt_lens()
     varlen = wr.varlen is not None
@@ -353,17 +353,20 @@ def measure(wr, args, K_steps, W_steps, world, rank, local, dist, headline):
     hk = ks[pos:pos + n_e2e].cpu().pin_memory()
     hv = vs[pos:pos + n_e2e].cpu().pin_memory()
     hout = torch.empty(wr.B, wr.H, wr.d, dtype=dt).pin_memory()
-    for i in range(min(2, n_e2e)):        # the first host-buffer call resolves the pinned mappings
+    # untimed calls first: the first one resolves the pinned mappings, and the calls after an idle gap (the host copies
+    # above) run slower than the steady state (cfg3: 219 us per call over the first 30, 195 us over 254)
+    e2e_warm = min(16, n_e2e // 4) if n_e2e >= 8 else min(2, n_e2e)
+    for i in range(e2e_warm):
         sg.step_host(hq[i], hk[i], hv[i], hout)
     if dist:
         dist.barrier()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
-    for i in range(min(2, n_e2e), n_e2e):
+    for i in range(e2e_warm, n_e2e):
         sg.step_host(hq[i], hk[i], hv[i], hout)
     t_e2e = time.perf_counter() - t0
     t_e2e = sharding.max_over_ranks(t_e2e, dist, dev)
-    n_timed_e2e = max(1, n_e2e - min(2, n_e2e))
+    n_timed_e2e = max(1, n_e2e - e2e_warm)
     esz = 2 if dt == torch.bfloat16 else 4
     h2d = (wr.B * wr.H + 2 * wr.B * wr.Hkv) * wr.d * esz
     d2h = wr.B * wr.H * wr.d * esz
@@ -648,7 +651,7 @@ def main():
     ap.add_argument("--impl", default="subgen", choices=["subgen", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=sorted(synth.CONFIGS))
     ap.add_argument("--splits", type=int, default=0)
-    ap.add_argument("--e2e-steps", type=int, default=32)
+    ap.add_argument("--e2e-steps", type=int, default=272, help="host-buffer calls, the first 16 untimed")
     ap.add_argument("--no-exact", dest="exact", action="store_false")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--no-configs", dest="configs", action="store_false",

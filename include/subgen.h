@@ -251,6 +251,19 @@ int subgen_checkpoint_bytes(subgen_t* h, size_t* bytes);
 int subgen_checkpoint_save(subgen_t* h, void* host, size_t bytes, size_t* written);
 int subgen_checkpoint_load(subgen_t* h, const void* host, size_t bytes);
 
+/* Growth of the cluster arrays. Algorithm 1 puts no bound on the number of clusters (Section 2.3: m depends on how
+ * clusterable the keys are), while a handle's arrays hold m_max clusters per unit. subgen_grow re-lays the handle's
+ * state out for a larger m_max on the device (one strided device copy per state array into a new workspace) and
+ * leaves the stream exactly where it was: later steps and prefills give the integer state and the outputs that a
+ * handle created with the larger m_max would give. Call it before a unit runs out of room (subgen_cache_stats and
+ * subgen_export_state report the cluster counts); a SUBGEN_ST_CAPACITY bit that is already set stays set.
+ * workspace: device memory owned by the caller for the new layout (subgen_workspace_bytes of the configuration
+ * with the new m_max; 256-byte aligned, not overlapping the old one), or NULL: the library allocates it. The old
+ * workspace is freed if the library had allocated it, else it is the caller's again once the call has returned.
+ * Synchronous. m_max must exceed the current value (SUBGEN_EINVAL); bounded handles are refused (SUBGEN_ESTATE:
+ * there m_max is the budget of the variant). Old and new workspace are both held until the copy is done. */
+int subgen_grow(subgen_t* h, int m_max, void* workspace, size_t workspace_bytes);
+
 /* Text of the calling thread's most recent error. */
 const char* subgen_last_error(void);
 

@@ -24,7 +24,7 @@ EXPORTS = [
     "subgen_workspace_bytes", "subgen_create", "subgen_create_ex", "subgen_destroy", "subgen_prefill",
     "subgen_prefill_varlen", "subgen_step", "subgen_step_host", "subgen_status", "subgen_export_state",
     "subgen_export_rows", "subgen_cache_stats", "subgen_profile_enable", "subgen_profile_read", "subgen_profile_prefill_read",
-    "subgen_query", "subgen_launch_count", "subgen_step_kernels", "subgen_last_error", "subgen_checkpoint_bytes", "subgen_checkpoint_save", "subgen_checkpoint_load", "subgen_exact_create", "subgen_exact_destroy",
+    "subgen_query", "subgen_launch_count", "subgen_step_kernels", "subgen_last_error", "subgen_checkpoint_bytes", "subgen_checkpoint_save", "subgen_checkpoint_load", "subgen_grow", "subgen_exact_create", "subgen_exact_destroy",
     "subgen_exact_append", "subgen_exact_append_varlen", "subgen_exact_step", "subgen_exact_bytes",
     "subgen_exact_launch_count", "subgen_exact_attention_noalloc",
     "subgen_exact_kcenter_compress", "subgen_exact_kcenter_counters", "subgen_exact_export_tokens",
@@ -90,6 +90,7 @@ def load():
     L.subgen_checkpoint_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
     L.subgen_checkpoint_save.argtypes = [vp, vp, C.c_size_t, C.POINTER(C.c_size_t)]
     L.subgen_checkpoint_load.argtypes = [vp, vp, C.c_size_t]
+    L.subgen_grow.argtypes = [vp, C.c_int, vp, C.c_size_t]
     L.subgen_launch_count.restype = C.c_uint64
     L.subgen_last_error.restype = C.c_char_p
     L.subgen_exact_create.restype = vp
@@ -155,6 +156,7 @@ class SubGen:
         nbytes = self._L.subgen_workspace_bytes(C.byref(cfg))
         if nbytes == 0:
             raise SubgenError(self._L.subgen_last_error().decode())
+        self._cfg = cfg
         self.m_max = int(m_max) if m_max else 8192
         self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")   # torch owns the memory
         base = (self.workspace.data_ptr() + 255) // 256 * 256
@@ -280,6 +282,21 @@ class SubGen:
         if blob.dtype != torch.uint8 or blob.device.type != "cpu" or not blob.is_contiguous():
             raise ValueError("blob must be a contiguous uint8 host tensor")
         _check(self._L.subgen_checkpoint_load(self._h, blob.data_ptr(), blob.numel()))
+
+    def grow(self, m_max: int):
+        """Re-lay the state out for a larger cluster capacity per unit (see subgen_grow); the stream continues unchanged."""
+        cfg = SubgenConfig.from_buffer_copy(self._cfg)
+        cfg.m_max = int(m_max)
+        cfg.workspace, cfg.workspace_bytes = None, 0
+        nbytes = self._L.subgen_workspace_bytes(C.byref(cfg))
+        if nbytes == 0:
+            raise SubgenError(self._L.subgen_last_error().decode())
+        ws = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+        base = (ws.data_ptr() + 255) // 256 * 256
+        _check(self._L.subgen_grow(self._h, int(m_max), base, nbytes))
+        self.workspace, self.workspace_bytes = ws, nbytes            # the old tensor is released here
+        self._cfg.m_max = int(m_max)
+        self.m_max = int(m_max)
 
 
 class ExactAttention:

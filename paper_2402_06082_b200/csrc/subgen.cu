@@ -1126,9 +1126,7 @@ struct CkptArray {
 
 // The arrays that make up the state between two calls, in blob order. Cluster arrays are stored up to m_rows
 // clusters per unit; partials, tickets and work queues are scratch of a single call and are not part of it.
-std::vector<CkptArray> ckpt_arrays(const subgen* h, int m_rows) {
-    const Dims& d = h->d;
-    const Layout& L = h->L;
+std::vector<CkptArray> ckpt_arrays(const Dims& d, const Layout& L, int m_rows) {
     const size_t row = (size_t)d.D * d.E, mm = (size_t)d.m_max, mr = (size_t)m_rows, s = (size_t)d.s, w = (size_t)d.w, t = (size_t)d.t;
     return {
         {L.X, mm * row, mr * row}, {L.S, mm * t * row, mr * t * row}, {L.xn, mm * 4, mr * 4}, {L.cnt, mm * 4, mr * 4},
@@ -1140,6 +1138,8 @@ std::vector<CkptArray> ckpt_arrays(const subgen* h, int m_rows) {
         {L.last_d2, 8, 8}, {L.pairs, 8, 8}, {L.thr2, 8, 8}, {L.level, 4, 4},
     };
 }
+
+std::vector<CkptArray> ckpt_arrays(const subgen* h, int m_rows) { return ckpt_arrays(h->d, h->L, m_rows); }
 
 size_t ckpt_payload(const subgen* h, int m_rows) {
     size_t n = 0;
@@ -1225,6 +1225,52 @@ int subgen_checkpoint_load(subgen_t* h, const void* host, size_t bytes) {
     std::vector<int> n(d.U);
     CUDA_TRY(cudaMemcpy(n.data(), h->ws + h->L.n_unit, (size_t)d.U * 4, cudaMemcpyDeviceToHost));
     for (int b = 0; b < d.B; ++b) h->n_host[b] = n[(size_t)b * d.Hkv];
+    h->epoch_stale = true;
+    h->order_ready = false;
+    return SUBGEN_OK;
+}
+
+int subgen_grow(subgen_t* h, int m_max, void* workspace, size_t workspace_bytes) {
+    if (!h) return fail(SUBGEN_EINVAL, "subgen_grow: handle is NULL");
+    if (h->cfg.bounded) return fail(SUBGEN_ESTATE, "subgen_grow: m_max of a bounded handle is its budget and stays as created");
+    if (m_max <= h->d.m_max) return fail(SUBGEN_EINVAL, "subgen_grow: m_max must exceed the current %d", h->d.m_max);
+    Dims d2 = h->d;
+    d2.m_max = m_max;
+    const Layout L2 = make_layout(d2);
+    int m_rows = 0;
+    if (int rc = ckpt_m_rows(h, &m_rows)) return rc;                 // synchronises the stream
+    char* ws2 = (char*)workspace;
+    cudaError_t e = cudaSuccess;
+    if (workspace) {
+        if (workspace_bytes < L2.total || ((uintptr_t)workspace % kAlign))
+            return fail(SUBGEN_ENOMEM, "subgen_grow: workspace needs %zu bytes, 256-byte aligned (got %zu)", L2.total, workspace_bytes);
+        if (ws2 < h->ws + h->L.total && h->ws < ws2 + L2.total) return fail(SUBGEN_EINVAL, "subgen_grow: the new workspace overlaps the old one");
+    } else {
+        e = cudaMalloc((void**)&ws2, L2.total);
+        if (e != cudaSuccess) return fail(SUBGEN_ENOMEM, "subgen_grow: cudaMalloc(%zu) failed: %s", L2.total, cudaGetErrorString(e));
+    }
+    // a new handle's workspace, then the state arrays on top: every array keeps its per-unit layout, only the room
+    // per unit changes, so each is one strided device copy
+    e = cudaMemsetAsync(ws2 + L2.book_begin, 0, L2.book_end - L2.book_begin, h->st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ws2 + L2.book_end, 0xFF, L2.total - L2.book_end, h->st);
+    const std::vector<CkptArray> from = ckpt_arrays(h->d, h->L, m_rows), to = ckpt_arrays(d2, L2, m_rows);
+    for (size_t i = 0; i < from.size() && e == cudaSuccess; ++i)
+        if (from[i].unit_live)
+            e = cudaMemcpy2DAsync(ws2 + to[i].off, to[i].unit_cap, h->ws + from[i].off, from[i].unit_cap, from[i].unit_live,
+                                  (size_t)h->d.U, cudaMemcpyDeviceToDevice, h->st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->st);
+    if (e != cudaSuccess) {
+        if (!workspace) cudaFree(ws2);
+        return fail(SUBGEN_ECUDA, "subgen_grow: %s", cudaGetErrorString(e));
+    }
+    if (h->owns) cudaFree(h->ws);
+    h->owns = workspace == nullptr;
+    h->cfg.workspace = workspace;
+    h->cfg.workspace_bytes = workspace ? workspace_bytes : 0;
+    h->ws = ws2;
+    h->L = L2;
+    h->d = d2;
+    h->cfg.m_max = m_max;
     h->epoch_stale = true;
     h->order_ready = false;
     return SUBGEN_OK;

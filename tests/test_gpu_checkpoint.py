@@ -99,3 +99,115 @@ def test_checkpoint_of_an_empty_handle_and_rejections():
     # the handle is still usable after a rejected load
     out = a.step(Q[:, :, 60].contiguous(), K[:, :, 60].contiguous(), V[:, :, 60].contiguous())
     assert torch.isfinite(out.float()).all()
+
+
+@pytest.mark.parametrize("dtype,d,mode", [("bf16", 128, "fused"), ("bf16", 128, "split"), ("bf16", 64, "auto"), ("fp32", 64, "auto")])
+def test_grow_keeps_the_stream(dtype, d, mode):
+    """A handle created with room for few clusters is grown twice while outliers keep opening clusters (delta small
+    enough that the first capacity would overflow): prefill, steps, grow, prefill again, steps, grow, steps. State and
+    outputs must be those of the oracle, which never had a bound; the rows stored before a growth must still be the
+    tokens' rows after it."""
+    big = 1024
+    w = synth.CFG3.scaled(B=2, H=4, Hkv=2, d=d, dtype=dtype, n_prompt=300, ncomp=24, s=64, window=16, m_max=big,
+                          outlier_frac=0.15)
+    n0, n1, n2, n3, n4 = 300, 20, 200, 20, 30
+    n = n0 + n1 + n2 + n3 + n4
+    K, V, Q = synth.batch_stream(w, n, "cuda")
+    Kn, Vn, Qn = f32(K), f32(V), f32(Q)
+    units = [(b, h) for b in range(w.B) for h in range(w.Hkv)]
+    orcs = {bh: hp.oracle_unit(w, *bh) for bh in units}
+    G = w.H // w.Hkv
+    for (b, h), o in orcs.items():
+        o.push_many(Kn[b, h, :n0 + n1], Vn[b, h, :n0 + n1])
+    m1 = max(o.m for o in orcs.values())
+    for (b, h), o in orcs.items():
+        o.push_many(Kn[b, h, n0 + n1:n0 + n1 + n2 + n3], Vn[b, h, n0 + n1:n0 + n1 + n2 + n3])
+    m2 = max(o.m for o in orcs.values())
+    cap0, cap1 = m1 + 2, m2 + 2
+    assert m1 < m2 and cap0 < m2, "the first capacity must be too small for the second phase"
+    orcs = {bh: hp.oracle_unit(w, *bh) for bh in units}
+
+    def steps(sg, lo, hi):
+        for i in range(lo, hi):
+            out = f32(sg.step(Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous()))
+            for (b, h), o in orcs.items():
+                o.push(Kn[b, h, i], Vn[b, h, i])
+                for g in range(G):
+                    hp.assert_output(out[b, h * G + g], o.query(Qn[b, h * G + g, i]), w.torch_dtype,
+                                     "step %d unit %s head %d" % (i, (b, h), g))
+
+    kw = dict(step_mode=mode) if mode != "auto" else {}
+    sg = _sg(w, m_max=cap0, **kw)
+    sg.prefill(K[:, :, :n0].contiguous(), V[:, :, :n0].contiguous())
+    for (b, h), o in orcs.items():
+        o.push_many(Kn[b, h, :n0], Vn[b, h, :n0])
+    steps(sg, n0, n0 + n1)
+    with pytest.raises(Exception):
+        sg.grow(cap0)                                   # not larger
+    sg.grow(cap1)
+    assert sg.m_max == cap1
+    for (b, h), o in orcs.items():
+        st = sg.export_state(b, h)
+        hp.assert_state_equal(st, o, "right after the first growth, unit %s" % ((b, h),))
+        hp.assert_rows_match_tokens(sg, b, h, st, K[b, h], V[b, h])
+    lo = n0 + n1
+    sg.prefill(K[:, :, lo:lo + n2].contiguous(), V[:, :, lo:lo + n2].contiguous())
+    for (b, h), o in orcs.items():
+        o.push_many(Kn[b, h, lo:lo + n2], Vn[b, h, lo:lo + n2])
+    steps(sg, lo + n2, lo + n2 + n3)
+    sg.grow(big)
+    steps(sg, lo + n2 + n3, n)
+    for (b, h), o in orcs.items():
+        st = sg.export_state(b, h)
+        hp.assert_state_equal(st, o, "end, unit %s" % ((b, h),))
+        hp.assert_rows_match_tokens(sg, b, h, st, K[b, h], V[b, h])
+    assert sg.status() == 0
+
+
+def test_grow_is_refused_where_it_does_not_apply():
+    from paper_2402_06082_b200.binding import SubGen
+    w = synth.CFG2.scaled(B=1, H=2, Hkv=2, s=32, window=8, m_max=64)
+    bounded = SubGen(w.B, w.H, w.d, w.delta, w.t, w.s, w.window, w.philox_seed, Hkv=w.Hkv, dtype=w.torch_dtype,
+                     m_max=64, bounded=True)
+    with pytest.raises(Exception):
+        bounded.grow(128)
+
+
+def test_grow_with_a_library_owned_workspace():
+    """The C call with workspace = NULL (the library allocates and frees) on a handle created without a workspace."""
+    import ctypes as C
+    from paper_2402_06082_b200 import binding
+    L = binding.load()
+    w = synth.CFG3.scaled(B=1, H=2, Hkv=2, n_prompt=200, ncomp=12, s=32, window=8, m_max=512, outlier_frac=0.15)
+    K, V, Q = synth.batch_stream(w, 260, "cuda")
+    m_prompt = 0
+    for hh in range(w.Hkv):
+        o = hp.oracle_unit(w, 0, hh)
+        o.push_many(f32(K)[0, hh, :200], f32(V)[0, hh, :200])
+        m_prompt = max(m_prompt, o.m)
+    cap0 = m_prompt + 1
+    cfg = binding.SubgenConfig(w.B, w.H, w.Hkv, w.d, float(w.delta), w.t, w.s, w.window, int(w.philox_seed), 1, cap0, 0, None, 0,
+                               torch.cuda.current_stream().cuda_stream, 1, 0, 0, 0, 0)
+    h = L.subgen_create_ex(C.byref(cfg))
+    assert h
+    try:
+        k0, v0 = K[:, :, :200].contiguous(), V[:, :, :200].contiguous()
+        assert L.subgen_prefill(h, k0.data_ptr(), v0.data_ptr(), 200) == 0
+        assert L.subgen_grow(h, 512, None, 0) == 0
+        out = torch.empty(w.B, w.H, w.d, dtype=torch.bfloat16, device="cuda")
+        for i in range(200, 260):
+            q, k, v = Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous()
+            assert L.subgen_step(h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr()) == 0
+        assert L.subgen_status(h) == 0
+        ref = _sg(w)
+        ref.prefill(k0, v0)
+        for i in range(200, 260):
+            o2 = ref.step(Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous())
+        torch.cuda.synchronize()
+        assert hp.rel_err(f32(out).reshape(-1, w.d), f32(o2).reshape(-1, w.d)) <= 1e-2
+        o = hp.oracle_unit(w, 0, 1)
+        o.push_many(f32(K)[0, 1], f32(V)[0, 1])
+        assert o.m > cap0, "the first capacity must have been too small"
+        assert ref.export_state(0, 1)["m"] == o.m
+    finally:
+        L.subgen_destroy(h)
