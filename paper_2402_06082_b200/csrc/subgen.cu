@@ -50,7 +50,7 @@ size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
     size_t X, S, xn, cnt, ctok, stok, Mk, Mv, MW, Mtok, ringK, ringV;
     size_t n_unit, m_unit, mu, status, last_cid, last_open, last_d2, part1, part2, ticket1, ticket2, qnext, qnext2, part_tau, MinvW, pairs;
-    size_t thr2, level, Xh, xhn, alias, ndist, epoch, order;
+    size_t thr2, level, Xh, xhn, alias, ndist, epoch, order, m_hist;
     size_t stage_q, stage_k, stage_v, stage_out, cu, stats;
     size_t book_begin, book_end;   // bookkeeping region cleared at creation
     size_t total;
@@ -175,6 +175,7 @@ Layout make_layout(const Dims& d) {
     L.pairs = take(U * sizeof(uint64_t));
     L.epoch = take(U * sizeof(int));
     L.order = take(U * sizeof(int));
+    L.m_hist = take(2 * U * sizeof(int));
     L.thr2 = take(U * sizeof(uint64_t));
     L.level = take(U * sizeof(int));
     L.MinvW = take(U * d.s * sizeof(float));
@@ -220,6 +221,7 @@ struct subgen {
     cudaStream_t st2 = nullptr;   // prefill: the key phase runs here, beside the value phase on st (fork / join by events)
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     bool order_ready = false;     // the units are ranked by cluster count (set by a prefill of a many-unit handle)
+    int step_seq = 0;             // one-kernel steps since the epochs were last set
     bool epoch_stale = true;      // the units' epochs may lag their token counts (creation, prefill, checkpoint load)
     bool fused = false;           // stream steps run as one kernel (bf16, not bounded): few units, or SUBGEN_STEP=fused
     unsigned long long* pf_phase_dev = nullptr;   // its per-unit phase times (inside scratch)
@@ -260,6 +262,7 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
     C.part_tau = (float*)(w + L.part_tau); C.MinvW = (float*)(w + L.MinvW);
     C.pairs = (unsigned long long*)(w + L.pairs);
     C.epoch = (int*)(w + L.epoch);
+    C.m_hist = (int*)(w + L.m_hist);
     C.order = h->order_ready ? (const int*)(w + L.order) : nullptr;
     C.bounded = h->cfg.bounded ? 1 : 0;
     C.uid_stride = h->cfg.unit_stride ? h->cfg.unit_stride : d.Hkv;
@@ -387,12 +390,23 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
         if (h->fused) {
             const dim3 grid_f(h->d.sp_fused, h->d.U);
+            // The kernel works on the token that leaves the window before its dependency wait; it takes the token
+            // count from the unit's epoch plus the number of steps since the epochs were set. The first step after
+            // that is launched the ordinary way: it reads what the epoch kernel, its direct predecessor, wrote.
+            const bool first = h->epoch_stale;
+            if (first) {
+                epoch_sync_kernel<<<(h->d.U + 255) / 256, 256, 0, h->st>>>(C, h->d.U);
+                h->epoch_stale = false;
+                h->step_seq = 0;
+                h->launches += 1;
+            }
+            const int seq = h->step_seq++;
             if (e) CUDA_TRY(cudaEventRecord(e[1], h->st));          // the whole step is reported as the middle interval
             switch (h->d.G) {
-                case 1: launch_pdl(step_fused_kernel<D, 1>, grid_f, dim3(kFsThreads), h->st, C, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
-                case 2: launch_pdl(step_fused_kernel<D, 2>, grid_f, dim3(kFsThreads), h->st, C, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
-                case 4: launch_pdl(step_fused_kernel<D, 4>, grid_f, dim3(kFsThreads), h->st, C, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
-                default: launch_pdl(step_fused_kernel<D, 8>, grid_f, dim3(kFsThreads), h->st, C, (const T*)q, (const T*)k, (const T*)v, (T*)out); break;
+                case 1: launch_pdl_opt(first, step_fused_kernel<D, 1>, grid_f, dim3(kFsThreads), 0, h->st, C, (const T*)q, (const T*)k, (const T*)v, (T*)out, seq); break;
+                case 2: launch_pdl_opt(first, step_fused_kernel<D, 2>, grid_f, dim3(kFsThreads), 0, h->st, C, (const T*)q, (const T*)k, (const T*)v, (T*)out, seq); break;
+                case 4: launch_pdl_opt(first, step_fused_kernel<D, 4>, grid_f, dim3(kFsThreads), 0, h->st, C, (const T*)q, (const T*)k, (const T*)v, (T*)out, seq); break;
+                default: launch_pdl_opt(first, step_fused_kernel<D, 8>, grid_f, dim3(kFsThreads), 0, h->st, C, (const T*)q, (const T*)k, (const T*)v, (T*)out, seq); break;
             }
             if (e) { CUDA_TRY(cudaEventRecord(e[2], h->st)); CUDA_TRY(cudaEventRecord(e[3], h->st)); }
             CUDA_TRY(take_launch_error());

@@ -131,6 +131,7 @@ template <typename T> struct Cache {
     unsigned* qnext2;    // [U] same for the scan of M and the window
     unsigned long long* pairs;   // [U] (key, representative) pairs scored by the chunked prefill so far
     int* epoch;                  // [U] tokens seen, as released by the step's insertion kernel (see acquire_unit)
+    int* m_hist;                 // [2][U] one-kernel step: cluster count left by the step before the previous one (see step_fused_kernel)
     const int* order;            // [U] or NULL: the unit that the blocks with blockIdx.y = i serve, units with many
                                  //     clusters first (handles whose per-unit grids need several waves of blocks)
     int uid_stride, uid_off;     // numbering of the units in the Philox counter, see unit_id()
@@ -347,9 +348,10 @@ __device__ void make_room(const Cache<T>& C, int u, int e, const uint4* krow, Be
 
 // W(v_e), ||k_e||^2 (whole row and packed head, fp32) and the input range check. Called by ONE warp; leaves
 // sm_w[0] = W and sm_w[1] = {||k||^2, ||k head||^2} in shared memory (visible to the block after a barrier).
+// token_weights_rows reports a failed range check through bad_out (written by lane 0); token_weights sets the unit's
+// status bit 2 itself.
 template <typename T, int D>
-__device__ __forceinline__ void token_weights(const Cache<T>& C, int u, const uint4* krow, const uint4* vrow,
-                                              unsigned long long* sm_w) {
+__device__ __forceinline__ void token_weights_rows(const uint4* krow, const uint4* vrow, unsigned long long* sm_w, int* bad_out) {
     constexpr int EPL = Elem<T>::EPL, LPR = D / EPL;
     const int lane = threadIdx.x & 31;
     unsigned long long acc = 0;
@@ -379,8 +381,15 @@ __device__ __forceinline__ void token_weights(const Cache<T>& C, int u, const ui
     if (lane == 0) {
         sm_w[0] = acc;
         sm_w[1] = (unsigned long long)__float_as_uint(kk) | ((unsigned long long)__float_as_uint(kh) << 32);
-        if (bad) atomicOr(&C.status[u], 2);
+        *bad_out = bad ? 1 : 0;
     }
+}
+template <typename T, int D>
+__device__ __forceinline__ void token_weights(const Cache<T>& C, int u, const uint4* krow, const uint4* vrow,
+                                              unsigned long long* sm_w) {
+    int bad = 0;                                       // lane 0's copy is the one that is written
+    token_weights_rows<T, D>(krow, vrow, sm_w, &bad);
+    if ((threadIdx.x & 31) == 0 && bad) atomicOr(&C.status[u], 2);
 }
 
 // UpdateSoftmaxNormalizer for token e given its nearest representative: join (count, t coins) or open

@@ -208,7 +208,10 @@ __global__ void unit_order_kernel(Cache<__nv_bfloat16> C, int U, int* order) {
 // a prefill, a checkpoint load or the handle's creation, whose kernels advance the counts without touching the epochs.
 __global__ void epoch_sync_kernel(Cache<__nv_bfloat16> C, int U) {
     const int u = blockIdx.x * blockDim.x + threadIdx.x;
-    if (u < U) C.epoch[u] = C.n_unit[u];
+    if (u < U) {
+        C.epoch[u] = C.n_unit[u];
+        C.m_hist[u] = C.m_hist[U + u] = C.m_unit[u];
+    }
 }
 
 }  // namespace sgk

@@ -57,18 +57,17 @@ struct StepToken {
     const __nv_bfloat16 *knew, *vnew; // rows of the new token (the call's input)
 };
 
-// Nearest representative of the key in krow over rows [c0, c1) of the unit's packed heads: the tensor-core filter
+// Nearest representative of the key in krow over rows [c0, c1) of the unit's packed heads (Xu, Xhu, xhnu: the unit's
+// representatives, their packed heads and the heads' squared norms): the tensor-core filter
 // and exact follow-up of insert_mma_kernel. Warps take KT tiles of 16 heads per turn; every thread ends with the
 // best (D2, index) its warp has seen (bst is updated, not reset).
 template <int D, int KT>
-__device__ __forceinline__ void head_scan_slice(const Cache<__nv_bfloat16>& C, int u, int c0, int c1, const uint4* krow, int nwarps,
+__device__ __forceinline__ void head_scan_slice(const __nv_bfloat16* Xu, const __nv_bfloat16* Xhu, const float* xhnu,
+                                                unsigned long long delta2_fx, int c0, int c1, const uint4* krow, int nwarps,
                                                 Best& bst) {
     typedef __nv_bfloat16 T;
     constexpr int LPR = D / 8;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, tq = lane & 3;
-    const T* Xu = C.X + (size_t)u * C.m_max * D;
-    const T* Xhu = C.Xh + (size_t)u * C.m_max * kHeadDims;
-    const float* xhnu = C.xhn + (size_t)u * C.m_max;
     uint32_t kb0[4];
     float kn = 0.f;
     {
@@ -82,7 +81,7 @@ __device__ __forceinline__ void head_scan_slice(const Cache<__nv_bfloat16>& C, i
     }
     kn += __shfl_xor_sync(0xffffffffu, kn, 1);
     kn += __shfl_xor_sync(0xffffffffu, kn, 2);
-    const float d2f = (float)((double)C.delta2_fx * (1.0 / 4294967296.0));
+    const float d2f = (float)((double)delta2_fx * (1.0 / 4294967296.0));
     auto exact_row = [&](int row) {                                  // exact D2 of one flagged row, by the warp
         unsigned long long acc = 0;
         if (lane < LPR) {
@@ -316,11 +315,46 @@ __device__ __forceinline__ void tau_correction(const Cache<__nv_bfloat16>& C, in
     }
 }
 
+// The token that leaves the window (kE, vE: its rows; has_ins = false: none leaves yet): its rows into krow / vrow,
+// its weights into sm_w (range check reported through sm_bad), and the nearest representative of its key over this
+// block's slice of the unit's representatives [0, m_scan) into sm_best. Called by the whole block; ends with a
+// barrier. Kept out of line, with plain pointers as arguments, so that the kernel's two call sites share one copy
+// and its registers do not weigh on the scans.
+template <int D>
+__device__ __noinline__ void leaving_token(const __nv_bfloat16* Xu, const __nv_bfloat16* Xhu, const float* xhnu,
+                                           unsigned long long delta2_fx, const __nv_bfloat16* kE, const __nv_bfloat16* vE,
+                                           bool has_ins, int m_scan, uint4* krow, uint4* vrow, unsigned long long* sm_w,
+                                           int* sm_bad, Best* smb, Best* sm_best) {
+    typedef __nv_bfloat16 T;
+    constexpr int LPR = D / 8;
+    const int tid = threadIdx.x, warp = tid >> 5, splits = gridDim.x;
+    if (tid == 0) *sm_bad = 0;
+    if (has_ins) {
+        if (tid < LPR) krow[tid] = reinterpret_cast<const uint4*>(kE)[tid];
+        else if (tid < 2 * LPR) vrow[tid - LPR] = reinterpret_cast<const uint4*>(vE)[tid - LPR];
+    }
+    __syncthreads();
+    if (has_ins && warp == 0) token_weights_rows<T, D>(krow, vrow, sm_w, sm_bad);
+    __syncthreads();
+    Best bst;
+    bst.d2 = ~0ull; bst.idx = INT_MAX; bst.pad = 0;
+    if (has_ins) {
+        if (m_scan > 0) {
+            const int per = (((m_scan + splits - 1) / splits) + 15) & ~15;       // slices are whole tiles
+            const int c0 = blockIdx.x * per;
+            head_scan_slice<D, 2>(Xu, Xhu, xhnu, delta2_fx, c0, min(m_scan, c0 + per), krow, kFsWarps, bst);
+        }
+        bst = block_best(bst, smb);
+        if (tid == 0) *sm_best = bst;
+    }
+    __syncthreads();
+}
+
 template <int D, int G>
 __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ q,
                                                                   const __nv_bfloat16* __restrict__ k_new,
                                                                   const __nv_bfloat16* __restrict__ v_new,
-                                                                  __nv_bfloat16* __restrict__ out) {
+                                                                  __nv_bfloat16* __restrict__ out, int step_k) {
     typedef __nv_bfloat16 T;
     constexpr int NC = D / 32, LPR = D / 8, STR = D + 2, NW = kFsWarps;
     // During the scan every warp keeps the row list of its item here; afterwards the same bytes hold the warps'
@@ -339,7 +373,34 @@ __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bf
     const int lane = tid & 31, warp = tid >> 5, g = lane >> 2, tq = lane & 3;
     const int b = u / C.Hkv, kvh = u % C.Hkv;
     const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;
-    // The call's inputs may come from the kernel that precedes this one in the stream: everything waits for it.
+    const int w = C.w, s = C.s, t = C.t, U = C.B * C.Hkv;
+    const T* knew_u = k_new + (size_t)u * D;
+    const T* vnew_u = v_new + (size_t)u * D;
+    __shared__ int sm_bad;
+    __shared__ Best sm_best;
+
+    // ---- the token that leaves the window: its rows, its weights, its nearest representative ----
+    // With a window of two rows or more none of this depends on the call's inputs or on the previous step: the
+    // leaving token has been in the ring since an earlier step, the previous step writes another ring row, and
+    // representatives never change once written. So it runs BEFORE the dependency wait, while the previous step's
+    // last blocks finish: on the token count epoch + step_k (the epochs were set by a kernel that completed before
+    // this one was launched) and on the representatives [0, m_hist): the cluster count left by the step before
+    // the previous one, which has completed (the previous step passed its own wait before it let this kernel be
+    // scheduled). The previous step can have opened at most one cluster beyond that; it is looked at after the wait.
+    // Shorter windows (the leaving token is the previous step's, or the call's own) do all of it after the wait.
+    const bool early = w >= 2;
+    const T* Xu = C.X + (size_t)u * C.m_max * D;
+    const T* Xhu = C.Xh + (size_t)u * C.m_max * kHeadDims;
+    const float* xhnu = C.xhn + (size_t)u * C.m_max;
+    int n_pre = -1, m_scan = 0;
+    if (early) {
+        n_pre = C.epoch[u] + step_k;
+        m_scan = C.m_hist[(size_t)(step_k & 1) * U + u];
+        const int slot_pre = n_pre % w;
+        leaving_token<D>(Xu, Xhu, xhnu, C.delta2_fx, C.ringK + ((size_t)u * w + slot_pre) * D, C.ringV + ((size_t)u * w + slot_pre) * D,
+                         n_pre >= w, m_scan, krow, vrow, sm_w, &sm_bad, smb, &sm_best);
+    }
+    // The call's inputs may come from the kernel that precedes this one in the stream: the rest waits for it.
     pdl_wait();
     pdl_trigger();
 
@@ -352,40 +413,43 @@ __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bf
     }
     const int n = C.n_unit[u], m = C.m_unit[u];
     const unsigned long long mu_old = C.mu[u];
-    const int w = C.w, s = C.s, t = C.t;
     const bool has_ins = n >= w;                     // a token leaves the window (w = 0: the new token itself)
     const int e = n - w;
     const int slot = w ? n % w : 0;
-    const T* knew_u = k_new + (size_t)u * D;
-    const T* vnew_u = v_new + (size_t)u * D;
     const T* kE = w ? C.ringK + ((size_t)u * w + slot) * D : knew_u;      // rows of the token that leaves
     const T* vE = w ? C.ringV + ((size_t)u * w + slot) * D : vnew_u;
-    if (has_ins) {
-        if (tid < LPR) krow[tid] = reinterpret_cast<const uint4*>(kE)[tid];
-        else if (tid < 2 * LPR) vrow[tid - LPR] = reinterpret_cast<const uint4*>(vE)[tid - LPR];
+    if (n != n_pre) {                                 // short window, or nothing prepared for this count
+        m_scan = m;
+        leaving_token<D>(Xu, Xhu, xhnu, C.delta2_fx, kE, vE, has_ins, m, krow, vrow, sm_w, &sm_bad, smb, &sm_best);
     }
-    __syncthreads();
-    if (has_ins && warp == 0) token_weights<T, D>(C, u, krow, vrow, sm_w);
-    __syncthreads();
     const unsigned long long W = has_ins ? sm_w[0] : 0ull;
     const unsigned long long tot = mu_old + W;       // mu after this step's insertion
     StepToken tk;
     tk.n = n; tk.e = e; tk.slot = slot; tk.has_ins = has_ins; tk.W = W; tk.tot = tot;
     tk.kE = kE; tk.vE = vE; tk.knew = knew_u; tk.vnew = vnew_u;
-
-    // ---- nearest representative of k_e over this block's slice of the packed heads ----
-    Best bst;
-    bst.d2 = ~0ull; bst.idx = INT_MAX; bst.pad = 0;
-    if (has_ins) {
-        if (m > 0) {
-            const int per = (((m + splits - 1) / splits) + 15) & ~15;       // slices are whole tiles
-            const int c0 = blockIdx.x * per;
-            head_scan_slice<D, 2>(C, u, c0, min(m, c0 + per), krow, NW, bst);
+    if (has_ins && tid < 32) {
+        Best bst = sm_best;
+        // the cluster the previous step may have opened since the early scan: exact distance, read past the L1
+        if (blockIdx.x == 0) {
+            for (int row = m_scan; row < m; ++row) {
+                unsigned long long acc = 0;
+                if (lane < LPR) {
+                    float xf[8], kf[8];
+                    Elem<T>::unpack(__ldcg(reinterpret_cast<const uint4*>(Xu + (size_t)row * D + lane * 8)), xf);
+                    Elem<T>::unpack(krow[lane], kf);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc += fx_sqdiff(xf[j], kf[j]);
+                }
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+                if (better(acc, row, bst)) { bst.d2 = acc; bst.idx = row; }
+            }
         }
-        bst = block_best(bst, smb);
-        if (tid == 0) C.part1[(size_t)u * splits + blockIdx.x] = bst;
+        if (tid == 0) {
+            C.part1[(size_t)u * splits + blockIdx.x] = bst;
+            if (sm_bad && blockIdx.x == 0) atomicOr(&C.status[u], 2);
+        }
     }
-
 
     // ---- scan of the state as it stands before the insertion ----
     unsigned* als = reinterpret_cast<unsigned*>(scratch) + warp * (16 * 64 / 4);
@@ -526,10 +590,12 @@ __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bf
         }
     }
     __syncthreads();                                  // the correction is in shared memory; the old sample rows were read
+    int m_after = m;
     if (has_ins) {
         bool join2, full2;
         int m_ref = m;
         const int m_new = apply_cluster<T, D, false>(C, u, e, bb, m_ref, krow, sm_w, join2, full2);
+        m_after = m_new;
         if (tid == 0) {
             C.mu[u] = tot;
             C.m_unit[u] = m_new;
@@ -595,6 +661,7 @@ __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bf
     }
     if (tid == 0) {
         C.n_unit[u] = n + 1;
+        C.m_hist[(size_t)(step_k & 1) * U + u] = m_after;     // read by the step after the next one, before its wait
         C.ticket2[u] = 0;
         C.qnext[u] = 0;
         C.qnext2[u] = 0;

@@ -228,3 +228,39 @@ def test_ragged_prompts_many_units():
     for (b, h), o in orcs.items():
         hp.assert_state_equal(sg.export_state(b, h), o, "ragged, ordered units %s" % ((b, h),))
     assert sg.status() == 0
+
+
+@pytest.mark.parametrize("window", [2, 3, 64])
+def test_long_fused_stream_with_frequent_openings(window):
+    """The one-kernel step works on the leaving token before it waits for the previous step (windows of two rows or
+    more), from a cluster count that is two steps old, and looks at the cluster the previous step may have opened
+    afterwards. A long back-to-back stream in which many steps open a cluster (so that the nearest representative is
+    often the one opened by the step before) must end in the oracle's state; every 50th step's outputs are checked."""
+    w = synth.CFG3.scaled(B=2, H=8, Hkv=4, n_prompt=64, ncomp=10, s=48, t=4, window=window, m_max=2048, outlier_frac=0.3)
+    n0, nd = 64, 1500
+    K, V, Q = synth.batch_stream(w, n0 + nd, "cuda")
+    sg = _sg(w, step_mode="fused")
+    sg.prefill(K[:, :, :n0].contiguous(), V[:, :, :n0].contiguous())
+    outs = {}
+    for i in range(n0, n0 + nd):
+        o = sg.step(Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous())
+        if i % 50 == 0:
+            outs[i] = f32(o)
+    Kn, Vn, Qn = f32(K), f32(V), f32(Q)
+    G = w.H // w.Hkv
+    opened = 0
+    for b in range(w.B):
+        for h in range(w.Hkv):
+            o = hp.oracle_unit(w, b, h)
+            o.push_many(Kn[b, h, :n0], Vn[b, h, :n0])
+            m0 = o.m
+            for i in range(n0, n0 + nd):
+                o.push(Kn[b, h, i], Vn[b, h, i])
+                if i in outs:
+                    for g in range(G):
+                        hp.assert_output(outs[i][b, h * G + g], o.query(Qn[b, h * G + g, i]), w.torch_dtype,
+                                         "step %d unit %s head %d" % (i, (b, h), g))
+            opened += o.m - m0
+            hp.assert_state_equal(sg.export_state(b, h), o, "window %d, unit %s" % (window, (b, h)))
+    assert opened > 200
+    assert sg.status() == 0
