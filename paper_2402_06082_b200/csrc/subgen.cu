@@ -50,7 +50,7 @@ size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
     size_t X, S, xn, cnt, ctok, stok, Mk, Mv, MW, Mtok, ringK, ringV;
     size_t n_unit, m_unit, mu, status, last_cid, last_open, last_d2, part1, part2, ticket1, ticket2, qnext, qnext2, part_tau, MinvW, pairs;
-    size_t thr2, level, Xh, xhn, alias, ndist, epoch, order, m_hist;
+    size_t thr2, level, Xh, xhn, alias, ndist, epoch, order, m_hist, next_best;
     size_t stage_q, stage_k, stage_v, stage_out, cu, stats;
     size_t book_begin, book_end;   // bookkeeping region cleared at creation
     size_t total;
@@ -176,6 +176,7 @@ Layout make_layout(const Dims& d) {
     L.epoch = take(U * sizeof(int));
     L.order = take(U * sizeof(int));
     L.m_hist = take(2 * U * sizeof(int));
+    L.next_best = take(U * sizeof(Best));
     L.thr2 = take(U * sizeof(uint64_t));
     L.level = take(U * sizeof(int));
     L.MinvW = take(U * d.s * sizeof(float));
@@ -221,6 +222,7 @@ struct subgen {
     cudaStream_t st2 = nullptr;   // prefill: the key phase runs here, beside the value phase on st (fork / join by events)
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     bool order_ready = false;     // the units are ranked by cluster count (set by a prefill of a many-unit handle)
+    bool search_ready = false;    // next_best holds the search for the next step's leaving token (host-buffer steps)
     int step_seq = 0;             // one-kernel steps since the epochs were last set
     bool epoch_stale = true;      // the units' epochs may lag their token counts (creation, prefill, checkpoint load)
     bool fused = false;           // stream steps run as one kernel (bf16, not bounded): few units, or SUBGEN_STEP=fused
@@ -263,6 +265,7 @@ template <typename T> Cache<T> make_cache(const subgen* h) {
     C.pairs = (unsigned long long*)(w + L.pairs);
     C.epoch = (int*)(w + L.epoch);
     C.m_hist = (int*)(w + L.m_hist);
+    C.next_best = (Best*)(w + L.next_best);
     C.order = h->order_ready ? (const int*)(w + L.order) : nullptr;
     C.bounded = h->cfg.bounded ? 1 : 0;
     C.uid_stride = h->cfg.unit_stride ? h->cfg.unit_stride : d.Hkv;
@@ -419,7 +422,9 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
             h->launches += 1;
         }
         if (C.bounded) launch_pdl(insert_mma_kernel<D, true>, grid_i, dim3(kInsertMmaThreads), h->st, C, (const T*)k, (const T*)v);
+        else if (h->search_ready) launch_pdl(insert_mma_kernel<D, false, 2>, dim3(1, h->d.U), dim3(kInsertMmaThreads), h->st, C, (const T*)k, (const T*)v);
         else launch_pdl(insert_mma_kernel<D, false>, grid_i, dim3(kInsertMmaThreads), h->st, C, (const T*)k, (const T*)v);
+        h->search_ready = false;
     } else {
         if (C.bounded) insert_kernel<T, D, true><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
         else insert_kernel<T, D, false><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
@@ -783,6 +788,7 @@ int subgen_prefill(subgen_t* h, const void* K, const void* V, int n) {
     int rc = launch_prefill(h, K, V, n, nullptr, 0, add.data());
     if (rc) return rc;
     h->epoch_stale = true;
+    h->search_ready = false;
     rank_units(h);
     for (int b = 0; b < h->d.B; ++b) h->n_host[b] += n;
     return SUBGEN_OK;
@@ -809,6 +815,7 @@ int subgen_prefill_varlen(subgen_t* h, const void* K, const void* V, const int* 
     int rc = launch_prefill(h, K, V, 0, cu_dev, total, add.data());
     if (rc) return rc;
     h->epoch_stale = true;
+    h->search_ready = false;
     rank_units(h);
     for (int b = 0; b < h->d.B; ++b) h->n_host[b] += cu[b + 1] - cu[b];
     return SUBGEN_OK;
@@ -879,7 +886,9 @@ static stream_write32_fn stream_write32() {
 // writes a sequence number into a pinned word once the step's kernels are done (a stream memory operation), and the
 // host spins on that word: the result is seen a few microseconds earlier. Falls back to cudaStreamSynchronize when the
 // driver has no such operation, and after a bounded spin.
-static cudaError_t wait_step_done(subgen* h) {
+// behind: called once the completion word has been enqueued (or, without one, after the synchronisation): work for
+// the stream that the host does not wait for.
+static cudaError_t wait_step_done(subgen* h, void (*behind)(subgen*) = nullptr) {
     stream_write32_fn wr = stream_write32();
     if (wr && !h->done_host) {
         void* p = nullptr;
@@ -898,11 +907,35 @@ static cudaError_t wait_step_done(subgen* h) {
     if (wr && h->done_host) {
         const unsigned seq = ++h->done_seq;
         if (wr((CUstream)h->st, h->done_dev, seq, 0) == CUDA_SUCCESS) {
+            if (behind) behind(h);
             for (long long spin = 0; spin < (1ll << 27); ++spin)
                 if (h->done_host[0] == seq) return cudaGetLastError();
+            return cudaStreamSynchronize(h->st);
         }
     }
-    return cudaStreamSynchronize(h->st);
+    const cudaError_t e = cudaStreamSynchronize(h->st);
+    if (behind && e == cudaSuccess) behind(h);
+    return e;
+}
+
+// Three-kernel steps of bf16 handles (not bounded, window of one row or more): the search for the nearest
+// representative of the token that the NEXT step takes out of the window, enqueued behind a host-buffer step and its
+// completion word, where it runs while the host has the result and prepares its next call; that step then launches
+// the insertion kernel in its apply-only mode. A host-buffer step cannot overlap with its successor, so without this
+// the whole search stands in front of every step's scans (256 units: 2 to 5 % more calls per second, depending on how
+// long the host takes between calls; launched in front of the completion word, beside the value scan, it delayed the
+// word by its own completion and gained 1 %).
+static void search_ahead(subgen* h) {
+    static const bool off = [] { const char* e = getenv("SUBGEN_SEARCH_AHEAD"); return e && e[0] == '0'; }();
+    if (off || h->cfg.dtype != SUBGEN_DTYPE_BF16 || h->fused || h->cfg.bounded || h->d.w < 1 || h->epoch_stale) return;
+    Cache<__nv_bfloat16> C = make_cache<__nv_bfloat16>(h);
+    const dim3 grid(h->d.sp_insert, h->d.U);
+    const __nv_bfloat16* none = nullptr;
+    if (h->d.D == 64) launch_pdl(insert_mma_kernel<64, false, 1>, grid, dim3(kInsertMmaThreads), h->st, C, none, none);
+    else launch_pdl(insert_mma_kernel<128, false, 1>, grid, dim3(kInsertMmaThreads), h->st, C, none, none);
+    if (take_launch_error() != cudaSuccess) return;
+    h->launches += 1;
+    h->search_ready = true;
 }
 
 int subgen_step_host(subgen_t* h, const void* q, const void* k, const void* v, void* out) {
@@ -936,7 +969,7 @@ int subgen_step_host(subgen_t* h, const void* q, const void* k, const void* v, v
         }
         int rc = subgen_step(h, dq, dk, dv, dout);
         if (rc) return rc;
-        CUDA_TRY(wait_step_done(h));
+        CUDA_TRY(wait_step_done(h, search_ahead));
         return SUBGEN_OK;
     }
     char* w = h->ws;
@@ -1240,6 +1273,7 @@ int subgen_checkpoint_load(subgen_t* h, const void* host, size_t bytes) {
     CUDA_TRY(cudaMemcpy(n.data(), h->ws + h->L.n_unit, (size_t)d.U * 4, cudaMemcpyDeviceToHost));
     for (int b = 0; b < d.B; ++b) h->n_host[b] = n[(size_t)b * d.Hkv];
     h->epoch_stale = true;
+    h->search_ready = false;
     h->order_ready = false;
     return SUBGEN_OK;
 }
@@ -1286,6 +1320,7 @@ int subgen_grow(subgen_t* h, int m_max, void* workspace, size_t workspace_bytes)
     h->d = d2;
     h->cfg.m_max = m_max;
     h->epoch_stale = true;
+    h->search_ready = false;
     h->order_ready = false;
     return SUBGEN_OK;
 }

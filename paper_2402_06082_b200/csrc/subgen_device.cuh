@@ -131,6 +131,7 @@ template <typename T> struct Cache {
     unsigned* qnext2;    // [U] same for the scan of M and the window
     unsigned long long* pairs;   // [U] (key, representative) pairs scored by the chunked prefill so far
     int* epoch;                  // [U] tokens seen, as released by the step's insertion kernel (see acquire_unit)
+    Best* next_best;             // [U] nearest representative found ahead of the next step (insert_mma_kernel, MODE 1)
     int* m_hist;                 // [2][U] one-kernel step: cluster count left by the step before the previous one (see step_fused_kernel)
     const int* order;            // [U] or NULL: the unit that the blocks with blockIdx.y = i serve, units with many
                                  //     clusters first (handles whose per-unit grids need several waves of blocks)

@@ -22,7 +22,14 @@ namespace sgk {
 
 constexpr int kInsertMmaThreads = 128;
 
-template <int D, bool BND>
+// MODE 0: the whole insertion of a step. A host-buffer step cannot overlap with its successor (the host waits for the
+// result), so there the search for the NEXT step's leaving token is launched behind the step, where it runs while the
+// host is busy, and the next step only applies it:
+// MODE 1: search only, for the token that the next step will take out of the window (windows of one row or more:
+//         that token is in the ring already); leaves the nearest representative in next_best[u]. k_new, v_new unused.
+// MODE 2: apply only (grid.x = 1): takes the nearest representative from next_best[u]. Valid while nothing but that
+//         search has run on the handle since the step before (the host keeps track).
+template <int D, bool BND, int MODE = 0>
 __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<__nv_bfloat16> C, const __nv_bfloat16* __restrict__ k_new,
                                                                     const __nv_bfloat16* __restrict__ v_new) {
     typedef __nv_bfloat16 T;
@@ -57,7 +64,8 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
     uint4* ringk = w ? reinterpret_cast<uint4*>(C.ringK + ((size_t)u * w + slot) * D) : nullptr;
     uint4* ringv = w ? reinterpret_cast<uint4*>(C.ringV + ((size_t)u * w + slot) * D) : nullptr;
     if (w && n < w) {                       // window not full yet: nothing leaves it
-        if (blockIdx.x == 0) {
+        if (MODE == 1) pdl_wait();
+        if (MODE != 1 && blockIdx.x == 0) {
             pdl_wait();
             pdl_trigger();
             if (tid < LPR) ringk[tid] = knew_u[tid];
@@ -98,7 +106,7 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
     const float d2f = (float)((double)threshold2<BND>(C, u) * (1.0 / 4294967296.0));
 
     const int per = (((m + splits - 1) / splits) + 15) & ~15;       // slices are whole tiles
-    const int c0 = blockIdx.x * per, c1 = min(m, c0 + per);
+    const int c0 = blockIdx.x * per, c1 = MODE == 2 ? c0 : min(m, c0 + per);     // MODE 2: nothing to scan
     Best b;
     b.d2 = ~0ull; b.idx = INT_MAX; b.pad = 0;
     // exact D2 of one flagged row, by the whole warp
@@ -144,8 +152,13 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
             while (mb) { exact_row(base + i * 16 + 8 + ((__ffs(mb) - 1) >> 2)); mb &= mb - 1; }
         }
     }
-    b = block_best(b, smb);
-    if (splits > 1) {
+    if (MODE == 2) {
+        const ulonglong2 raw = __ldcg(reinterpret_cast<const ulonglong2*>(C.next_best + u));
+        b.d2 = raw.x; b.idx = (int)(raw.y & 0xffffffffull);
+    } else {
+        b = block_best(b, smb);
+    }
+    if (MODE != 2 && splits > 1) {
         if (tid == 0) {
             C.part1[(size_t)u * splits + blockIdx.x] = b;
             // arrival ticket: the release half publishes this block's candidate, the acquire half lets the last block
@@ -165,6 +178,11 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
         }
         b = block_best(bb, smb);
         if (tid == 0) C.ticket1[u] = 0;
+    }
+    if (MODE == 1) {
+        if (tid == 0) C.next_best[u] = b;
+        pdl_wait();                         // this kernel's completion stands for that of everything before it
+        return;
     }
     // From here on the state that the previous step's scans read is overwritten, and the call's inputs are read.
     pdl_wait();

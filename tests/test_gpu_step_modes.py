@@ -264,3 +264,52 @@ def test_long_fused_stream_with_frequent_openings(window):
             hp.assert_state_equal(sg.export_state(b, h), o, "window %d, unit %s" % (window, (b, h)))
     assert opened > 200
     assert sg.status() == 0
+
+
+@pytest.mark.parametrize("window", [1, 2, 24])
+def test_host_buffer_steps_search_ahead(window):
+    """Host-buffer steps of a three-kernel handle leave the search for the next step's leaving token running behind
+    them; the next step (host or device buffers) only applies it; a prefill in between throws it away. Mixed sequence
+    of calls against the oracle: state bit for bit, every output within tolerance."""
+    w = synth.CFG3.scaled(B=2, H=4, Hkv=2, n_prompt=200, ncomp=12, s=48, t=4, window=window, m_max=1024, outlier_frac=0.2)
+    n0, n = 200, 200 + 90
+    K, V, Q = synth.batch_stream(w, n, "cuda")
+    Kn, Vn, Qn = f32(K), f32(V), f32(Q)
+    units = [(b, h) for b in range(w.B) for h in range(w.Hkv)]
+    orcs = {bh: hp.oracle_unit(w, *bh) for bh in units}
+    G = w.H // w.Hkv
+    sg = _sg(w, step_mode="split")
+    sg.prefill(K[:, :, :n0].contiguous(), V[:, :, :n0].contiguous())
+    for (b, h), o in orcs.items():
+        o.push_many(Kn[b, h, :n0], Vn[b, h, :n0])
+    pin = lambda x: x.contiguous().cpu().pin_memory()
+    hout = torch.empty(w.B, w.H, w.d, dtype=w.torch_dtype).pin_memory()
+    i = n0
+    launches = []
+    while i < n:
+        phase = (i - n0) % 30
+        if phase == 20:                                   # a prefill of 5 tokens between steps
+            sg.prefill(K[:, :, i:i + 5].contiguous(), V[:, :, i:i + 5].contiguous())
+            for (b, h), o in orcs.items():
+                o.push_many(Kn[b, h, i:i + 5], Vn[b, h, i:i + 5])
+            i += 5
+            continue
+        l0 = sg.launch_count
+        if phase % 3 == 2:                                # device buffers
+            out = f32(sg.step(Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous()))
+        else:
+            sg.step_host(pin(Q[:, :, i]), pin(K[:, :, i]), pin(V[:, :, i]), hout)
+            out = f32(hout)
+        launches.append(sg.launch_count - l0)
+        for (b, h), o in orcs.items():
+            o.push(Kn[b, h, i], Vn[b, h, i])
+            for g in range(G):
+                hp.assert_output(out[b, h * G + g], o.query(Qn[b, h * G + g, i]), w.torch_dtype,
+                                 "step %d unit %s head %d" % (i, (b, h), g))
+        i += 1
+    for (b, h), o in orcs.items():
+        st = sg.export_state(b, h)
+        hp.assert_state_equal(st, o, "window %d unit %s" % (window, (b, h)))
+        hp.assert_rows_match_tokens(sg, b, h, st, K[b, h], V[b, h])
+    assert sg.status() == 0
+    assert 4 in launches, "host-buffer steps launch the search for the next step behind their three kernels"
