@@ -163,7 +163,9 @@ int subgen_query(subgen_t* h, const void* q, int nq, void* out);
 /* subgen_step with HOST buffers, returning when out is filled. With page-locked (pinned, mapped) buffers the
  * step's kernels write out across the bus themselves and read q, k, v the same way (handles whose one-kernel step
  * runs many blocks per unit let one small kernel bring q, k, v over first): no copy engine, one wait. With pageable
- * buffers q, k, v are copied to the device first and out is copied back. */
+ * buffers q, k, v are copied to the device first and out is copied back. Three-kernel handles leave one more kernel
+ * on the stream when the call returns: the nearest-representative search for the token that the next step will take
+ * out of the window, which that step then only applies (any other call on the handle discards it). */
 int subgen_step_host(subgen_t* h, const void* q, const void* k, const void* v, void* out);
 
 /* Waits for the stream, returns the OR of all units' status bits (>= 0) or a negative error. */
