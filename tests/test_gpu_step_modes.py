@@ -200,7 +200,7 @@ def test_ragged_prompts_many_units():
     largest first (an order built after the prefill); every unit must still be served exactly once per step."""
     w = synth.CFG5.scaled(B=6, H=32, Hkv=32, ncomp=16, s=64, window=16, m_max=512)
     lens = [40, 700, 120, 350, 17, 500]
-    n_dec = 5
+    n_dec = 6
     streams = [synth.sequence_stream(w, b, lens[b] + n_dec, "cuda") for b in range(w.B)]
     cu = np.concatenate([[0], np.cumsum(lens)])
     Kp = torch.cat([streams[b][0][:, :lens[b]] for b in range(w.B)], dim=1).contiguous()
@@ -220,7 +220,12 @@ def test_ragged_prompts_many_units():
         q = torch.stack([streams[b][2][:, lens[b] + i] for b in range(w.B)]).contiguous()
         k = torch.stack([streams[b][0][:, lens[b] + i] for b in range(w.B)]).contiguous()
         v = torch.stack([streams[b][1][:, lens[b] + i] for b in range(w.B)]).contiguous()
-        out = f32(sg.step(q, k, v))
+        if i % 2:                                         # host buffers: the next step applies a search made ahead
+            hout = torch.empty(w.B, w.H, w.d, dtype=torch.bfloat16).pin_memory()
+            sg.step_host(q.cpu().pin_memory(), k.cpu().pin_memory(), v.cpu().pin_memory(), hout)
+            out = f32(hout)
+        else:
+            out = f32(sg.step(q, k, v))
         kn, vn, qn = f32(k), f32(v), f32(q)
         for (b, h), o in orcs.items():
             o.push(kn[b, h], vn[b, h])
