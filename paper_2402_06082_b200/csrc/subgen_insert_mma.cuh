@@ -78,8 +78,9 @@ __global__ void __launch_bounds__(kInsertMmaThreads, 6) insert_mma_kernel(Cache<
     const int e = n - w;
     // key and value of the token that leaves the window: both fetched now, so that the block that ends up applying
     // the insertion does not wait for the value row after the scan
-    if (tid < LPR) krow[tid] = w ? ringk[tid] : knew_u[tid];
-    else if (tid < 2 * LPR) vrow[tid - LPR] = w ? ringv[tid - LPR] : vnew_u[tid - LPR];
+    // (ring rows past the L1: this runs before the dependency wait)
+    if (tid < LPR) krow[tid] = w ? __ldcg(ringk + tid) : knew_u[tid];
+    else if (tid < 2 * LPR) vrow[tid - LPR] = w ? __ldcg(ringv + (tid - LPR)) : vnew_u[tid - LPR];
     __syncthreads();
     const int m = C.m_unit[u];
     const T* Xu = C.X + (size_t)u * C.m_max * D;

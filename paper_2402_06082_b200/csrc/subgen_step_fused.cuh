@@ -330,8 +330,9 @@ __device__ __noinline__ void leaving_token(const __nv_bfloat16* Xu, const __nv_b
     const int tid = threadIdx.x, warp = tid >> 5, splits = gridDim.x;
     if (tid == 0) *sm_bad = 0;
     if (has_ins) {
-        if (tid < LPR) krow[tid] = reinterpret_cast<const uint4*>(kE)[tid];
-        else if (tid < 2 * LPR) vrow[tid - LPR] = reinterpret_cast<const uint4*>(vE)[tid - LPR];
+        // past the L1: before the kernel's dependency wait nothing has refreshed this SM's view of the ring
+        if (tid < LPR) krow[tid] = __ldcg(reinterpret_cast<const uint4*>(kE) + tid);
+        else if (tid < 2 * LPR) vrow[tid - LPR] = __ldcg(reinterpret_cast<const uint4*>(vE) + (tid - LPR));
     }
     __syncthreads();
     if (has_ins && warp == 0) token_weights_rows<T, D>(krow, vrow, sm_w, sm_bad);
@@ -394,8 +395,8 @@ __global__ void __launch_bounds__(kFsThreads, 2) step_fused_kernel(Cache<__nv_bf
     const float* xhnu = C.xhn + (size_t)u * C.m_max;
     int n_pre = -1, m_scan = 0;
     if (early) {
-        n_pre = C.epoch[u] + step_k;
-        m_scan = C.m_hist[(size_t)(step_k & 1) * U + u];
+        n_pre = __ldcg(C.epoch + u) + step_k;
+        m_scan = __ldcg(C.m_hist + (size_t)(step_k & 1) * U + u);
         const int slot_pre = n_pre % w;
         leaving_token<D>(Xu, Xhu, xhnu, C.delta2_fx, C.ringK + ((size_t)u * w + slot_pre) * D, C.ringV + ((size_t)u * w + slot_pre) * D,
                          n_pre >= w, m_scan, krow, vrow, sm_w, &sm_bad, smb, &sm_best);
