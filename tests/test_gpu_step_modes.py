@@ -235,6 +235,33 @@ def test_ragged_prompts_many_units():
     assert sg.status() == 0
 
 
+@pytest.mark.parametrize("window", [1, 2, 64])
+def test_long_split_stream_many_blocks_per_unit(window):
+    """Three-kernel steps back to back with few units and 64 blocks per unit: every kernel of a step starts work before
+    its dependency wait (the insertion searches under the previous value scan, the value scan runs beside the cluster
+    scan), which rests on the order in which the kernels let each other be scheduled. 1200 steps with frequent
+    openings must end in the oracle's state."""
+    w = synth.CFG3.scaled(B=2, H=8, Hkv=4, n_prompt=64, ncomp=10, s=48, t=4, window=window, m_max=2048, outlier_frac=0.3)
+    n0, nd = 64, 1200
+    K, V, Q = synth.batch_stream(w, n0 + nd, "cuda")
+    sg = _sg(w, step_mode="split", splits=64)
+    sg.prefill(K[:, :, :n0].contiguous(), V[:, :, :n0].contiguous())
+    last = None
+    for i in range(n0, n0 + nd):
+        last = sg.step(Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous())
+    last = f32(last)
+    Kn, Vn, Qn = f32(K), f32(V), f32(Q)
+    G = w.H // w.Hkv
+    for b in range(w.B):
+        for h in range(w.Hkv):
+            o = hp.oracle_unit(w, b, h)
+            o.push_many(Kn[b, h], Vn[b, h])
+            hp.assert_state_equal(sg.export_state(b, h), o, "window %d, unit %s" % (window, (b, h)))
+            for g in range(G):
+                hp.assert_output(last[b, h * G + g], o.query(Qn[b, h * G + g, n0 + nd - 1]), w.torch_dtype, "last step")
+    assert sg.status() == 0
+
+
 @pytest.mark.parametrize("window", [2, 3, 64])
 def test_long_fused_stream_with_frequent_openings(window):
     """The one-kernel step works on the leaving token before it waits for the previous step (windows of two rows or
