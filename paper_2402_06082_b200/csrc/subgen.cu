@@ -337,10 +337,11 @@ void launch_query(const Cache<T>& C, int G, dim3 grid, dim3 grid_z, cudaStream_t
         }
     } else {
         switch (G) {
-            case 1: query_kernel<T, D, 1><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out, advance); break;
-            case 2: query_kernel<T, D, 2><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out, advance); break;
-            case 4: query_kernel<T, D, 4><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out, advance); break;
-            default: query_kernel<T, D, 8><<<grid, kQueryThreads, 0, st>>>(C, (const T*)q, (T*)out, advance); break;
+            // launched the ordinary way when it is the first kernel of its call (it loads q before its dependency wait)
+            case 1: launch_pdl_opt(first_plain, query_kernel<T, D, 1>, grid, dim3(kQueryThreads), 0, st, C, (const T*)q, (T*)out, advance); break;
+            case 2: launch_pdl_opt(first_plain, query_kernel<T, D, 2>, grid, dim3(kQueryThreads), 0, st, C, (const T*)q, (T*)out, advance); break;
+            case 4: launch_pdl_opt(first_plain, query_kernel<T, D, 4>, grid, dim3(kQueryThreads), 0, st, C, (const T*)q, (T*)out, advance); break;
+            default: launch_pdl_opt(first_plain, query_kernel<T, D, 8>, grid, dim3(kQueryThreads), 0, st, C, (const T*)q, (T*)out, advance); break;
         }
         if (mid) cudaEventRecord(mid, st);
     }
@@ -426,8 +427,8 @@ int launch_step_td(subgen* h, const void* q, const void* k, const void* v, void*
         else launch_pdl(insert_mma_kernel<D, false>, grid_i, dim3(kInsertMmaThreads), h->st, C, (const T*)k, (const T*)v);
         h->search_ready = false;
     } else {
-        if (C.bounded) insert_kernel<T, D, true><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
-        else insert_kernel<T, D, false><<<grid_i, kInsertThreads, 0, h->st>>>(C, (const T*)k, (const T*)v);
+        if (C.bounded) launch_pdl(insert_kernel<T, D, true>, grid_i, dim3(kInsertThreads), h->st, C, (const T*)k, (const T*)v);
+        else launch_pdl(insert_kernel<T, D, false>, grid_i, dim3(kInsertThreads), h->st, C, (const T*)k, (const T*)v);
     }
     if (e) CUDA_TRY(cudaEventRecord(e[1], h->st));
     int flat_grid = 0;

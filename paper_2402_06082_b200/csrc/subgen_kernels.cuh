@@ -26,6 +26,10 @@ __global__ void __launch_bounds__(kInsertThreads) insert_kernel(Cache<T> C, cons
     __shared__ int sm_last;
     const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, lr = lane % LPR, sub = lane / LPR;
+    // first kernel of a step: everything earlier in the stream has completed before it reads anything; the query
+    // kernel may be scheduled at once (it loads its queries and then waits for this kernel)
+    pdl_wait();
+    pdl_trigger();
     const int n = C.n_unit[u], w = C.w;
     const uint4* knew_u = reinterpret_cast<const uint4*>(k_new + (size_t)u * D);
     const uint4* vnew_u = reinterpret_cast<const uint4*>(v_new + (size_t)u * D);
@@ -94,17 +98,20 @@ __global__ void __launch_bounds__(kQueryThreads) query_kernel(Cache<T> C, const 
     const int u = blockIdx.y, splits = gridDim.x, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5, lr = lane % LPR, sub = lane / LPR;
     const int b = u / C.Hkv, kvh = u % C.Hkv;
-    // advance = 1: the query of a stream step (its token is in the ring, not counted yet); 0: read-only query
-    const int n = C.n_unit[u] - (advance ? 0 : 1), w = C.w, t = C.t, s = C.s;
-    const int wn = min(n + 1, w), m = C.m_unit[u];
     const size_t qrow0 = (size_t)b * C.H + (size_t)kvh * G;
 
+    // the queries are an input of the call (complete before its first kernel ran); the state is the insertion's
     float qf[G][EPL];
 #pragma unroll
     for (int g = 0; g < G; ++g) {
         const uint4 r = *reinterpret_cast<const uint4*>(q + (qrow0 + g) * D + lr * EPL);
         Elem<T>::unpack(r, qf[g]);
     }
+    pdl_wait();
+    pdl_trigger();
+    // advance = 1: the query of a stream step (its token is in the ring, not counted yet); 0: read-only query
+    const int n = C.n_unit[u] - (advance ? 0 : 1), w = C.w, t = C.t, s = C.s;
+    const int wn = min(n + 1, w), m = C.m_unit[u];
     Acc<G, EPL> A;
     A.init();
     const int gg = (blockIdx.x * (kQueryThreads / 32) + warp) * RPW + sub;
